@@ -1,0 +1,15 @@
+"""TEST INFRASTRUCTURE: CPU oracle for the ConvAttn forward pass (see convattn_ref.c).
+
+Only the test-suite, the smoke check and the benchmark's CPU-baseline leg may use
+this package.  It imports nothing from the CUDA package.
+"""
+from .convattn_oracle import (  # noqa: F401
+    build,
+    forward,
+    gap,
+    dynkernel,
+    stencil,
+    points,
+    set_threads,
+    max_threads,
+)

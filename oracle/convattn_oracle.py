@@ -1,0 +1,167 @@
+"""TEST INFRASTRUCTURE: ctypes loader for the plain-C ConvAttn oracle.
+
+The arithmetic lives in ``convattn_ref.c`` (direct nested loops, fp64
+accumulation, ESC paper Section 3.3, Eq. 4 / Eq. 5).  This module only compiles
+that file with gcc, marshals numpy arrays in and out, and sets the OpenMP thread
+count used by the timing harness.  Logical layout everywhere is dense
+``[B, C, H, W]``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "convattn_ref.c"
+_LIB = _HERE / "libconvattn_ref.so"
+_lib = None
+
+_f32p = ctypes.POINTER(ctypes.c_float)
+_f64p = ctypes.POINTER(ctypes.c_double)
+_i64p = ctypes.POINTER(ctypes.c_int64)
+
+
+def build(force: bool = False) -> Path:
+    """Compile convattn_ref.c into a shared object next to it (gcc -O2 -fopenmp)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(".so.tmp%d" % os.getpid())
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c99", "-o", str(tmp), str(_SRC), "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(str(_LIB))
+        _omp = None
+        for name in ("libgomp.so.1",):
+            try:
+                _omp = ctypes.CDLL(name)
+                break
+            except OSError:
+                pass
+        _lib._omp = _omp
+    return _lib
+
+
+def max_threads() -> int:
+    """Cores this process may run on (what OpenMP would use by default)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def set_threads(n: int) -> None:
+    lib = _load()
+    if lib._omp is not None:
+        lib._omp.omp_set_num_threads(int(n))
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a, a.ctypes.data_as(_f32p)
+
+
+def _f64(a):
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    return a, a.ctypes.data_as(_f64p)
+
+
+def _dims(x, C_a, K):
+    B, C, H, W = (int(v) for v in x.shape)
+    assert 0 < C_a <= C and K % 2 == 1 and K >= 1
+    return B, C, H, W
+
+
+def gap(x, C_a):
+    """g[B,C_a]: per-image, per-channel mean of the first C_a channels."""
+    x, xp = _f32(x)
+    B, C, H, W = (int(v) for v in x.shape)
+    g = np.empty((B, C_a), dtype=np.float64)
+    _load().convattn_ref_gap(xp, B, C, C_a, H, W, g.ctypes.data_as(_f64p))
+    return g
+
+
+def dynkernel(g, w_dyn, b_dyn):
+    """dk[B,C_a,3,3] = W_dyn g + b_dyn, output index o = c*9 + i*3 + j."""
+    g, gp = _f64(g)
+    B, C_a = (int(v) for v in g.shape)
+    w_dyn, wp = _f64(w_dyn)
+    b_dyn, bp = _f64(b_dyn)
+    assert w_dyn.shape == (9 * C_a, C_a) and b_dyn.shape == (9 * C_a,)
+    dk = np.empty((B, C_a, 3, 3), dtype=np.float64)
+    _load().convattn_ref_dynkernel(gp, B, C_a, wp, bp, dk.ctypes.data_as(_f64p))
+    return dk
+
+
+def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
+    """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
+    x, xp = _f32(x)
+    w_large, wp = _f64(w_large)
+    K = int(w_large.shape[-1])
+    B, C, H, W = _dims(x, C_a, K)
+    assert w_large.shape == (C_a, K, K)
+    dk, dp = _f64(dk)
+    assert dk.size == B * C_a * 9
+    y0, y1 = (0, H) if rows is None else (int(rows[0]), int(rows[1]))
+    assert 0 <= y0 <= y1 <= H
+    out = np.empty((B, C, y1 - y0, W), dtype=np.float64)
+    mag = np.empty((B, C_a, y1 - y0, W), dtype=np.float64) if want_mag else None
+    _load().convattn_ref_stencil(
+        xp, B, C, C_a, H, W, K, wp, dp, y0, y1, out.ctypes.data_as(_f64p),
+        mag.ctypes.data_as(_f64p) if want_mag else None,
+    )
+    return (out, mag) if want_mag else out
+
+
+def forward(x, C_a, w_large, w_dyn, b_dyn, want_mag=False, want_dk=False):
+    """Whole ConvAttn forward.  Returns out[B,C,H,W] (fp64) and, on request, mag and dk."""
+    x, xp = _f32(x)
+    w_large, wp = _f64(w_large)
+    K = int(w_large.shape[-1])
+    B, C, H, W = _dims(x, C_a, K)
+    assert w_large.shape == (C_a, K, K)
+    w_dyn, wdp = _f64(w_dyn)
+    b_dyn, bdp = _f64(b_dyn)
+    assert w_dyn.shape == (9 * C_a, C_a) and b_dyn.shape == (9 * C_a,)
+    out = np.empty((B, C, H, W), dtype=np.float64)
+    g = np.empty((B, C_a), dtype=np.float64)
+    dk = np.empty((B, C_a, 3, 3), dtype=np.float64)
+    mag = np.empty((B, C_a, H, W), dtype=np.float64) if want_mag else None
+    _load().convattn_ref_forward(
+        xp, B, C, C_a, H, W, K, wp, wdp, bdp, out.ctypes.data_as(_f64p), g.ctypes.data_as(_f64p),
+        dk.ctypes.data_as(_f64p), mag.ctypes.data_as(_f64p) if want_mag else None,
+    )
+    res = [out]
+    if want_mag:
+        res.append(mag)
+    if want_dk:
+        res.append(dk)
+    return res[0] if len(res) == 1 else tuple(res)
+
+
+def points(x, C_a, w_large, w_dyn, b_dyn, flat_idx, want_mag=False):
+    """Outputs at the given flat indices of out[B,C,H,W], computed one by one."""
+    x, xp = _f32(x)
+    w_large, wp = _f64(w_large)
+    K = int(w_large.shape[-1])
+    B, C, H, W = _dims(x, C_a, K)
+    dk = dynkernel(gap(x, C_a), w_dyn, b_dyn)
+    idx = np.ascontiguousarray(flat_idx, dtype=np.int64)
+    assert idx.ndim == 1 and (idx >= 0).all() and (idx < x.size).all()
+    vals = np.empty(idx.shape, dtype=np.float64)
+    mags = np.empty(idx.shape, dtype=np.float64)
+    _load().convattn_ref_points(
+        xp, B, C, C_a, H, W, K, wp, dk.ctypes.data_as(_f64p), ctypes.c_int64(idx.size),
+        idx.ctypes.data_as(_i64p), vals.ctypes.data_as(_f64p), mags.ctypes.data_as(_f64p),
+    )
+    return (vals, mags) if want_mag else vals

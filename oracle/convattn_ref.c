@@ -1,0 +1,157 @@
+/*
+ * TEST INFRASTRUCTURE -- CPU oracle for the ConvAttn forward pass.
+ *
+ * This file is the slow, obviously-correct definition that the CUDA library is
+ * checked against.  It is used only by the test-suite, by the smoke check and
+ * by the benchmark's CPU-baseline leg; the product never calls it and it shares
+ * no code, header, table or helper with the CUDA path.
+ *
+ * What it computes (ESC paper, Section 3.3 "Convolutional Attention Module",
+ * Eq. 4, in the depth-wise form of Eq. 5 without the point-wise LK^c, and with
+ * the kernel estimator reduced to one linear layer):
+ *
+ *   F_att = x[:, :C_a],  F_idt = x[:, C_a:]                      (Eq. 4, line 1)
+ *   g[b,c]   = mean over (y,x) of F_att[b,c,y,x]                 (GAP, Eq. 4 line 2)
+ *   dk[b,o]  = b_dyn[o] + sum_c W_dyn[o,c] * g[b,c],  o = c*9+i*3+j
+ *   out[b,c] = F_att[b,c] (*) LK[c]  +  F_att[b,c] (*) dk[b,c]   (Eq. 4, line 3)
+ *   out[b, C_a:] = F_idt                                         (Concat, Eq. 4 line 4)
+ *
+ * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
+ * Everything is accumulated in double precision with direct nested loops in
+ * the order written above: no tiling, no merging of the two kernels, no reuse.
+ * Inputs are float arrays holding exactly the values the device sees (bf16
+ * values widen to float without change); weights are passed as double.
+ *
+ * OpenMP only spreads independent (image, channel, row) iterations over
+ * threads for the timing harness; every output value is produced by exactly the
+ * same sequence of operations whatever the thread count.
+ *
+ * Pinned by tests/test_oracle_pins.py (impulse response, constant-input closed
+ * form, zero generator vs a library convolution, scatter-form brute force on
+ * tiny inputs, linearity laws, the Eq. 5 merge identity, permutation / batch
+ * independence, and the GAP->dk stage on non-zero-mean data).
+ */
+#include <stddef.h>
+#include <stdint.h>
+#include <math.h>
+
+#define IDX4(b, c, y, x, C, H, W) ((((size_t)(b) * (C) + (c)) * (H) + (y)) * (size_t)(W) + (x))
+
+/* GAP over the first C_a channels of x[B,C,H,W] (Eq. 4, line 2, inner term). g is [B,C_a]. */
+void convattn_ref_gap(const float *x, int B, int C, int C_a, int H, int W, double *g)
+{
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C_a; ++c) {
+            double s = 0.0;
+            for (int y = 0; y < H; ++y)
+                for (int xx = 0; xx < W; ++xx)
+                    s += (double)x[IDX4(b, c, y, xx, C, H, W)];
+            g[(size_t)b * C_a + c] = s / ((double)H * (double)W);
+        }
+}
+
+/* Kernel estimator: one linear layer C_a -> 9*C_a with bias. dk is [B, C_a*9],
+ * output index o = c*9 + i*3 + j holds tap (i,j) of channel c's 3x3 kernel. */
+void convattn_ref_dynkernel(const double *g, int B, int C_a, const double *w_dyn, const double *b_dyn,
+                            double *dk)
+{
+    for (int b = 0; b < B; ++b)
+        for (int o = 0; o < 9 * C_a; ++o) {
+            double s = b_dyn[o];
+            for (int c = 0; c < C_a; ++c)
+                s += w_dyn[(size_t)o * C_a + c] * g[(size_t)b * C_a + c];
+            dk[(size_t)b * 9 * C_a + o] = s;
+        }
+}
+
+/* One output value of an attention channel (c < C_a): large-kernel taps, then the
+ * dynamic 3x3 taps, both with zero padding.  *mag receives sum |w * x| over the
+ * same taps (the scale that bounds the rounding error of any evaluation order). */
+static double one_output(const float *x, int C, int H, int W, int K, const double *w_large,
+                         const double *dk_b, int b, int c, int y, int xx, double *mag)
+{
+    const int P = (K - 1) / 2;
+    double s = 0.0, m = 0.0;
+    for (int i = 0; i < K; ++i)
+        for (int j = 0; j < K; ++j) {
+            int yy = y + i - P, xc = xx + j - P;
+            if (yy >= 0 && yy < H && xc >= 0 && xc < W) {
+                double t = w_large[((size_t)c * K + i) * K + j] * (double)x[IDX4(b, c, yy, xc, C, H, W)];
+                s += t;
+                m += fabs(t);
+            }
+        }
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) {
+            int yy = y + i - 1, xc = xx + j - 1;
+            if (yy >= 0 && yy < H && xc >= 0 && xc < W) {
+                double t = dk_b[c * 9 + i * 3 + j] * (double)x[IDX4(b, c, yy, xc, C, H, W)];
+                s += t;
+                m += fabs(t);
+            }
+        }
+    if (mag) *mag = m;
+    return s;
+}
+
+/* Stencil stage with an explicit dk[B,C_a*9]: rows y0..y1-1 of every image.
+ * out is [B, C, y1-y0, W] (attention channels convolved, the others copied);
+ * mag (optional, may be NULL) is [B, C_a, y1-y0, W]. */
+void convattn_ref_stencil(const float *x, int B, int C, int C_a, int H, int W, int K,
+                          const double *w_large, const double *dk, int y0, int y1, double *out,
+                          double *mag)
+{
+    const int R = y1 - y0;
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C; ++c)
+            for (int y = y0; y < y1; ++y) {
+                for (int xx = 0; xx < W; ++xx) {
+                    size_t o = IDX4(b, c, y - y0, xx, C, R, W);
+                    if (c < C_a) {
+                        double m;
+                        out[o] = one_output(x, C, H, W, K, w_large, dk + (size_t)b * 9 * C_a, b, c, y, xx, &m);
+                        if (mag) mag[IDX4(b, c, y - y0, xx, C_a, R, W)] = m;
+                    } else {
+                        out[o] = (double)x[IDX4(b, c, y, xx, C, H, W)];
+                    }
+                }
+            }
+}
+
+/* Whole forward pass. g_out [B,C_a] and dk_out [B,C_a*9] are scratch the caller
+ * provides and may inspect; mag may be NULL. */
+void convattn_ref_forward(const float *x, int B, int C, int C_a, int H, int W, int K,
+                          const double *w_large, const double *w_dyn, const double *b_dyn,
+                          double *out, double *g_out, double *dk_out, double *mag)
+{
+    convattn_ref_gap(x, B, C, C_a, H, W, g_out);
+    convattn_ref_dynkernel(g_out, B, C_a, w_dyn, b_dyn, dk_out);
+    convattn_ref_stencil(x, B, C, C_a, H, W, K, w_large, dk_out, 0, H, out, mag);
+}
+
+/* Selected outputs, one by one: idx[n] are flat indices into out[B,C,H,W]; dk is
+ * given (from convattn_ref_gap + convattn_ref_dynkernel). */
+void convattn_ref_points(const float *x, int B, int C, int C_a, int H, int W, int K,
+                         const double *w_large, const double *dk, int64_t n, const int64_t *idx,
+                         double *vals, double *mags)
+{
+    (void)B;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < n; ++t) {
+        int64_t f = idx[t];
+        int xx = (int)(f % W); f /= W;
+        int y = (int)(f % H);  f /= H;
+        int c = (int)(f % C);  f /= C;
+        int b = (int)f;
+        double m = 0.0;
+        if (c < C_a)
+            vals[t] = one_output(x, C, H, W, K, w_large, dk + (size_t)b * 9 * C_a, b, c, y, xx, &m);
+        else {
+            vals[t] = (double)x[IDX4(b, c, y, xx, C, H, W)];
+            m = fabs(vals[t]);
+        }
+        if (mags) mags[t] = m;
+    }
+}
