@@ -1,0 +1,141 @@
+/*
+ * esc_convattn.h -- C ABI of the B200 (sm_100a) ConvAttn forward library.
+ *
+ * The operation is the Convolutional Attention module of the ESC paper
+ * (Section 3.3, Eq. 4), in the depth-wise large-kernel form of Eq. 5 (LK^s, without the
+ * point-wise LK^c) and with the kernel estimator reduced to one linear layer:
+ *
+ *   F_att = x[:, :C_a],  F_idt = x[:, C_a:]                               (Eq. 4, line 1)
+ *   g[b,c]  = mean_{y,x} F_att[b,c,y,x]                                   (GAP, Eq. 4 line 2)
+ *   dk[b,o] = b_dyn[o] + sum_c w_dyn[o,c] * g[b,c],   o = c*9 + i*3 + j   (Eq. 4 line 2)
+ *   out[b,c,y,x] = sum_{i,j<K} w_large[c,i,j] * xp[b,c,y+i-P,x+j-P]
+ *                + sum_{i,j<3} dk[b,c,i,j]    * xp[b,c,y+i-1,x+j-1]       (Eq. 4 line 3)
+ *   out[b, C_a:] = F_idt, bit for bit                                     (Concat, Eq. 4 line 4)
+ *
+ * with P = (K-1)/2, xp = x extended by zeros ('same' padding) and the sums taken as
+ * cross-correlations (no kernel flip).  Internally the two kernels are merged as
+ * ZP(dk) + LK^s (Eq. 5).  g, dk and every accumulation are fp32; each output is rounded
+ * once (round-to-nearest-even) to the storage type.
+ *
+ * General rules
+ *  - Every function returns an esc_status (0 = success).  Nothing throws or aborts.
+ *  - All tensor pointers are DEVICE pointers unless a parameter is named *_host.
+ *    The caller owns every buffer; the library keeps no reference after the work that a
+ *    call enqueued has finished.
+ *  - Logical tensor shape is always [B,C,H,W]; `layout` says how it sits in memory
+ *    (ESC_NCHW: dense [B][C][H][W];  ESC_NHWC: dense [B][H][W][C], PyTorch channels_last).
+ *    Strides are dense.  Weights have the same element type as x.
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *    default stream).  Errors found on the host are returned at once and nothing is
+ *    enqueued.  Device-side conditions (a bounded wait that expired) are recorded in the
+ *    workspace status word and read back with esc_convattn_device_status().
+ *  - Two calls may overlap on the GPU only if they use different workspaces.
+ */
+#ifndef ESC_CONVATTN_H
+#define ESC_CONVATTN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ESC_OK = 0,
+    ESC_ERR_NULL = 1,        /* a required pointer is NULL                                      */
+    ESC_ERR_SHAPE = 2,       /* B,C,H,W <= 0, C_a <= 0, C_a > C, K even or K < 1, size overflow */
+    ESC_ERR_UNSUPPORTED = 3, /* K > ESC_MAX_K, unknown dtype / layout                           */
+    ESC_ERR_ALIGN = 4,       /* a tensor pointer is not aligned to its element size / 16 bytes  */
+    ESC_ERR_ALIAS = 5,       /* out overlaps x (a stencil cannot run in place)                  */
+    ESC_ERR_WORKSPACE = 6,   /* workspace NULL, misaligned or smaller than required             */
+    ESC_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed; text in esc_last_error()   */
+    ESC_DEV_TIMEOUT = 8      /* a bounded device-side wait expired (status word)                */
+} esc_status;
+
+enum { ESC_F32 = 0, ESC_BF16 = 1 };   /* element type of x, out and the three weight tensors */
+enum { ESC_NCHW = 0, ESC_NHWC = 1 };  /* memory layout of x and out                           */
+enum { ESC_MAX_K = 17 };              /* largest supported large-kernel size (odd)            */
+
+/*
+ * ConvAttn forward, Eq. 4 of the paper as restated above.  fp32 tensors in dense NCHW.
+ *   x        [B,C,H,W]   input feature map (device, 16-byte aligned)
+ *   w_large  [C_a,K,K]   shared depth-wise large kernel LK^s (K odd, <= ESC_MAX_K)
+ *   w_dyn    [9*C_a,C_a] kernel-estimator weight, row o = c*9 + i*3 + j
+ *   b_dyn    [9*C_a]     kernel-estimator bias
+ *   out      [B,C,H,W]   result (device, 16-byte aligned, must not overlap x)
+ * Scratch memory is owned by the library (one block per device and stream, created on
+ * first use with cudaMalloc and kept until the process exits).
+ */
+int esc_convattn_forward(const void* x, int B, int C, int C_a, int H, int W, int K,
+                         const void* w_large, const void* w_dyn, const void* b_dyn,
+                         void* out, void* stream);
+
+/*
+ * Same operation with explicit element type, layout and caller-owned scratch.
+ *   dtype      ESC_F32 or ESC_BF16 (bf16 storage, fp32 arithmetic)
+ *   layout     ESC_NCHW or ESC_NHWC
+ *   workspace  device memory of at least esc_convattn_workspace_bytes(...) bytes, 256-byte
+ *              aligned, prepared once with esc_convattn_workspace_init(); it may be reused by
+ *              later calls that do not overlap this one on the GPU.
+ */
+int esc_convattn_forward_ex(const void* x, int B, int C, int C_a, int H, int W, int K,
+                            const void* w_large, const void* w_dyn, const void* b_dyn,
+                            void* out, int dtype, int layout,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch needed by the calls that take a workspace (dk, GAP partial sums,
+ * arrival counters, status word).  Returns 0 for invalid arguments. */
+size_t esc_convattn_workspace_bytes(int B, int C_a, int H, int W, int K);
+
+/* Zero a fresh workspace (enqueued on `stream`).  Needed once per allocation; the kernels
+ * leave the control words ready for the next call. */
+int esc_convattn_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Stage 1 alone (GAP + kernel estimator, Eq. 4 line 2): writes dk_out [B,C_a,3,3] fp32.
+ */
+int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W,
+                           const void* w_dyn, const void* b_dyn, float* dk_out,
+                           int dtype, int layout,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Stage 2 alone (Eq. 4 lines 3-4 with an explicit dk [B,C_a,3,3] fp32 device array):
+ * both depth-wise convolutions, their sum, and the copy of the remaining channels.
+ * `workspace` may be NULL (then device-side time-outs cannot be reported).
+ */
+int esc_convattn_stencil(const void* x, int B, int C, int C_a, int H, int W, int K,
+                         const void* w_large, const float* dk, void* out,
+                         int dtype, int layout,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * End-to-end convenience call on HOST buffers: copies x and the weights to the device,
+ * runs the forward pass, copies out back and synchronises.  Device buffers and a private
+ * stream are kept by the library between calls.  Host buffers should be pinned for full
+ * copy bandwidth but need not be.
+ */
+int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, int W, int K,
+                              const void* w_large_host, const void* w_dyn_host,
+                              const void* b_dyn_host, void* out_host, int dtype, int layout);
+
+/* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
+ * clears it. */
+int esc_convattn_device_status(void* workspace, void* stream);
+
+/* Which stencil implementation the last esc_convattn_forward* / esc_convattn_stencil call on
+ * this thread selected: 0 = none yet, 1 = guarded generic kernel, 2 = TMA-staged register-tiled
+ * kernel.  For tests and benchmarks. */
+int esc_convattn_last_path(void);
+
+/* Number of kernels the last forward / stage call on this thread launched. */
+int esc_convattn_last_launches(void);
+
+const char* esc_status_string(int status);
+const char* esc_last_error(void);   /* thread-local text of the last ESC_ERR_CUDA */
+int esc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ESC_CONVATTN_H */
