@@ -1,0 +1,156 @@
+// Kernel (a): global average pooling of the attention channels fused with the kernel
+// estimator (ESC paper, Section 3.3, Eq. 4 line 2, estimator reduced to one linear layer).
+//
+//   g[b,c]  = (1/HW) sum_{y,x} x[b,c,y,x]            c < C_a
+//   dk[b,o] = b_dyn[o] + sum_c w_dyn[o,c] g[b,c]     o = c*9 + i*3 + j
+//
+// Grid (S, B): every image is cut into S slabs so that a single large image still fills the
+// machine.  A block reduces its slab with 16-byte loads, warp shuffles and one pass through
+// shared memory, and writes C_a partial sums.  The block that arrives last for an image (a
+// wrapping arrival counter, so no counter ever needs re-zeroing) adds the S partial sums in slab
+// order -- the result is bitwise reproducible -- and evaluates the linear layer.
+#pragma once
+#include "common.cuh"
+
+namespace esc {
+
+constexpr int kGapThreads = 256;
+constexpr int kGapWarps = kGapThreads / 32;
+
+template <typename T, int LAYOUT>
+__global__ void __launch_bounds__(kGapThreads)
+gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
+              const T* __restrict__ w_dyn, const T* __restrict__ b_dyn,
+              float* __restrict__ partial,     // [B][S][Ca]
+              unsigned* __restrict__ arrivals, // [B]
+              float* __restrict__ dk)          // [B][9*Ca]
+{
+    constexpr int V = Elem<T>::kVec;
+    extern __shared__ float smem[];            // [kGapWarps][Ca] warp sums, then [Ca] means
+    float* wsum = smem;
+    float* gmean = smem + kGapWarps * Ca;
+    __shared__ bool is_last;
+
+    pdl_launch_dependents();                   // the stencil kernel may start its prologue now
+
+    const int s = blockIdx.x, b = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long HW = (long long)H * W;
+    float* my_partial = partial + ((size_t)b * S + s) * Ca;
+
+    const int cpp = Ca / V;                    // 16-byte chunks per pixel (NHWC)
+    const bool nhwc_vec = LAYOUT == kNHWC && Ca % V == 0 && C % V == 0 && cpp <= 32 && (cpp & (cpp - 1)) == 0;
+
+    if (nhwc_vec) {
+        // Thread t owns chunk (t % cpp) of pixels t/cpp, t/cpp + 256/cpp, ...
+        const long long p0 = HW * s / S, p1 = HW * (s + 1) / S;
+        const int chunk = tid % cpp, ppb = kGapThreads / cpp;
+        float acc[V];
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[v] = 0.f;
+        const T* base = x + ((size_t)b * HW) * C + (size_t)chunk * V;
+        long long p = p0 + tid / cpp;
+        for (; p + 3LL * ppb < p1; p += 4LL * ppb) {      // four independent loads in flight
+            uint4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) q[u] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(p + (long long)u * ppb) * C));
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float f[V];
+                unpack16<T>(q[u], f);
+#pragma unroll
+                for (int v = 0; v < V; ++v) acc[v] += f[v];
+            }
+        }
+        for (; p < p1; p += ppb) {
+            float f[V];
+            unpack16<T>(__ldg(reinterpret_cast<const uint4*>(base + (size_t)p * C)), f);
+#pragma unroll
+            for (int v = 0; v < V; ++v) acc[v] += f[v];
+        }
+        // lanes with equal (lane % cpp) hold the same channels: butterfly over the other lane bits
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+            for (int o = 16; o >= cpp; o >>= 1) acc[v] += __shfl_xor_sync(0xffffffffu, acc[v], o);
+        if (lane < cpp) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) wsum[warp * Ca + lane * V + v] = acc[v];
+        }
+        __syncthreads();
+        for (int c = tid; c < Ca; c += kGapThreads) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < kGapWarps; ++w) t += wsum[w * Ca + c];
+            my_partial[c] = t;
+        }
+    } else {
+        // One warp per channel (channels warp, warp+8, ...); lanes stride over the slab.
+        for (int c = warp; c < Ca; c += kGapWarps) {
+            float acc = 0.f;
+            if (LAYOUT == kNCHW) {
+                const T* plane = x + ((size_t)b * C + c) * HW;
+                if (HW % V == 0) {
+                    const long long nv = HW / V, v0 = nv * s / S, v1 = nv * (s + 1) / S;
+                    const uint4* pv = reinterpret_cast<const uint4*>(plane);
+                    float a4[4] = {0.f, 0.f, 0.f, 0.f};
+                    long long i = v0 + lane;
+                    for (; i + 96 < v1; i += 128) {
+                        uint4 q[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) q[u] = __ldg(pv + i + 32 * u);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            float f[V];
+                            unpack16<T>(q[u], f);
+#pragma unroll
+                            for (int v = 0; v < V; ++v) a4[u] += f[v];
+                        }
+                    }
+                    for (; i < v1; i += 32) {
+                        float f[V];
+                        unpack16<T>(__ldg(pv + i), f);
+#pragma unroll
+                        for (int v = 0; v < V; ++v) a4[0] += f[v];
+                    }
+                    acc = (a4[0] + a4[1]) + (a4[2] + a4[3]);
+                } else {
+                    const long long e0 = HW * s / S, e1 = HW * (s + 1) / S;
+                    for (long long i = e0 + lane; i < e1; i += 32) acc += Elem<T>::to_f32(plane[i]);
+                }
+            } else {
+                const long long p0 = HW * s / S, p1 = HW * (s + 1) / S;
+                const T* base = x + ((size_t)b * HW) * C + c;
+                for (long long p = p0 + lane; p < p1; p += 32) acc += Elem<T>::to_f32(base[(size_t)p * C]);
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) my_partial[c] = acc;
+        }
+    }
+
+    // ---- arrival: the last block of this image finishes the reduction and the linear layer
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned old = atomicInc(arrivals + b, (unsigned)(S - 1));   // wraps back to 0 by itself
+        is_last = (old == (unsigned)(S - 1));
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const float inv_hw = 1.0f / (float)HW;
+    for (int c = tid; c < Ca; c += kGapThreads) {
+        const float* pp = partial + (size_t)b * S * Ca + c;
+        float t = 0.f;
+        for (int k = 0; k < S; ++k) t += __ldcg(pp + (size_t)k * Ca);      // fixed slab order
+        gmean[c] = t * inv_hw;
+    }
+    __syncthreads();
+    for (int o = tid; o < 9 * Ca; o += kGapThreads) {
+        float acc = Elem<T>::to_f32(b_dyn[o]);
+        const T* wr = w_dyn + (size_t)o * Ca;
+        for (int c = 0; c < Ca; ++c) acc = fmaf(Elem<T>::to_f32(wr[c]), gmean[c], acc);
+        dk[(size_t)b * 9 * Ca + o] = acc;
+    }
+}
+
+}  // namespace esc

@@ -1,0 +1,79 @@
+// Guarded generic stencil for any odd K <= 17, any shape, either layout or element type
+// (ESC paper, Section 3.3, Eq. 4 lines 3-4).  One thread per output value: a (TY+K-1) x (TX+K-1)
+// halo tile of one channel is staged in shared memory as fp32 with zeros outside the image, the
+// per-image merged kernel ZP(dk) + LK^s (Eq. 5) sits beside it, and each thread accumulates its
+// K*K taps in fp32.  This is the fall-back when the register-tiled TMA kernel does not apply; it
+// is correct everywhere but makes no attempt to be fast.
+#pragma once
+#include "common.cuh"
+
+namespace esc {
+
+constexpr int kGenTX = 32, kGenTY = 8, kGenMaxK = 17;
+
+template <typename T, int LAYOUT>
+__global__ void __launch_bounds__(kGenTX * kGenTY)
+stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W, int K,
+                const T* __restrict__ w_large, const float* __restrict__ dk,
+                int tiles_x, int tiles_y)
+{
+    __shared__ float tile[(kGenTY + kGenMaxK - 1) * (kGenTX + kGenMaxK - 1)];
+    __shared__ float wm[kGenMaxK * kGenMaxK];
+
+    long long bid = blockIdx.x;
+    const int tx = (int)(bid % tiles_x); bid /= tiles_x;
+    const int ty = (int)(bid % tiles_y); bid /= tiles_y;
+    const int c = (int)(bid % Ca);
+    const int b = (int)(bid / Ca);
+    const int P = (K - 1) / 2;
+    const int tid = threadIdx.y * kGenTX + threadIdx.x;
+    const int TWp = kGenTX + K - 1, THp = kGenTY + K - 1;
+    const int y0 = ty * kGenTY - P, x0 = tx * kGenTX - P;
+
+    pdl_wait_primary();   // dk comes from the preceding kernel when launched as its dependent
+
+    for (int t = tid; t < K * K; t += kGenTX * kGenTY) {
+        const int i = t / K, j = t % K;
+        float w = Elem<T>::to_f32(w_large[(size_t)c * K * K + t]);
+        const int di = i - (P - 1), dj = j - (P - 1);
+        if (di >= 0 && di < 3 && dj >= 0 && dj < 3) w += dk[((size_t)b * Ca + c) * 9 + di * 3 + dj];
+        wm[t] = w;
+    }
+    for (int t = tid; t < TWp * THp; t += kGenTX * kGenTY) {
+        const int r = t / TWp, q = t % TWp;
+        const int y = y0 + r, xx = x0 + q;
+        float v = 0.f;
+        if (y >= 0 && y < H && xx >= 0 && xx < W) v = Elem<T>::to_f32(x[elem_index<LAYOUT>(b, c, y, xx, C, H, W)]);
+        tile[t] = v;
+    }
+    __syncthreads();
+
+    const int oy = ty * kGenTY + threadIdx.y, ox = tx * kGenTX + threadIdx.x;
+    if (oy >= H || ox >= W) return;
+    float acc = 0.f;
+    for (int i = 0; i < K; ++i) {
+        const float* trow = tile + (threadIdx.y + i) * TWp + threadIdx.x;
+        const float* wrow = wm + i * K;
+        for (int j = 0; j < K; ++j) acc = fmaf(wrow[j], trow[j], acc);
+    }
+    out[elem_index<LAYOUT>(b, c, oy, ox, C, H, W)] = Elem<T>::from_f32(acc);
+}
+
+// Copy of the channels that the module leaves untouched (Concat of Eq. 4 line 4), written as a
+// strided 2-D copy: `rows` rows of `row_units` units, `stride_units` apart, starting
+// `offset_units` into both tensors.  U is the widest unit all three quantities divide into.
+template <typename U>
+__global__ void __launch_bounds__(256)
+copy_through(const U* __restrict__ src, U* __restrict__ dst, long long rows, long long row_units,
+             long long stride_units, long long offset_units)
+{
+    const long long total = rows * row_units;
+    const long long step = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += step) {
+        const long long r = i / row_units, q = i - r * row_units;
+        const long long e = r * stride_units + offset_units + q;
+        dst[e] = src[e];
+    }
+}
+
+}  // namespace esc
