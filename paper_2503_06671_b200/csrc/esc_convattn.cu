@@ -1,0 +1,429 @@
+// C ABI of the ConvAttn forward library: argument checks, scratch layout, kernel selection and
+// launches.  The arithmetic lives in the kernels (gap_dynkernel.cuh, stencil_generic.cuh,
+// stencil_tma.cuh); nothing here touches tensor data on the host.
+#include "../../include/esc_convattn.h"
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <utility>
+
+#include "common.cuh"
+#include "gap_dynkernel.cuh"
+#include "stencil_generic.cuh"
+#include "stencil_tma.cuh"
+
+namespace {
+
+thread_local std::string g_last_error;
+thread_local int g_last_path = 0;
+thread_local int g_last_launches = 0;
+
+int cuda_fail(cudaError_t e, const char* what) {
+    char buf[320];
+    snprintf(buf, sizeof buf, "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+    g_last_error = buf;
+    return ESC_ERR_CUDA;
+}
+#define ESC_CUDA(call)                                        \
+    do {                                                      \
+        cudaError_t e__ = (call);                             \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+    } while (0)
+
+size_t elem_size(int dtype) { return dtype == ESC_BF16 ? 2 : 4; }
+
+struct Problem {
+    int B, C, Ca, H, W, K, dtype, layout;
+    size_t es() const { return elem_size(dtype); }
+    size_t elems() const { return (size_t)B * C * H * W; }
+};
+
+int check_shape(const Problem& p) {
+    if (p.B <= 0 || p.C <= 0 || p.H <= 0 || p.W <= 0 || p.Ca <= 0 || p.Ca > p.C) return ESC_ERR_SHAPE;
+    if (p.K < 1 || (p.K & 1) == 0) return ESC_ERR_SHAPE;
+    if (p.K > ESC_MAX_K) return ESC_ERR_UNSUPPORTED;
+    if (p.dtype != ESC_F32 && p.dtype != ESC_BF16) return ESC_ERR_UNSUPPORTED;
+    if (p.layout != ESC_NCHW && p.layout != ESC_NHWC) return ESC_ERR_UNSUPPORTED;
+    // every byte offset the kernels form must fit in 62 bits
+    const long double n = (long double)p.B * p.C * p.H * p.W;
+    if (n > 1.0e18L) return ESC_ERR_SHAPE;
+    return ESC_OK;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_tensors(const Problem& p, const void* x, const void* out) {
+    if (!x || !out) return ESC_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(out, 16)) return ESC_ERR_ALIGN;
+    const uintptr_t xa = reinterpret_cast<uintptr_t>(x), oa = reinterpret_cast<uintptr_t>(out);
+    const size_t bytes = p.elems() * p.es();
+    if (xa < oa + bytes && oa < xa + bytes) return ESC_ERR_ALIAS;
+    return ESC_OK;
+}
+
+// ---- workspace layout -------------------------------------------------------------------
+//   [ctrl words: header + B arrival counters][pad to 256][dk: B*Ca*9 floats][pad][partials: B*S*Ca floats]
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Workspace {
+    unsigned* ctrl;
+    unsigned* arrivals;
+    float* dk;
+    float* partial;
+};
+
+int slabs_for(int B, long long HW) {
+    // about two blocks per SM over the whole batch, at least 512 pixels per slab
+    long long s = (2 * 148 + B - 1) / B;
+    const long long cap = (HW + 511) / 512;
+    if (s > cap) s = cap;
+    if (s > esc::kMaxSlabs) s = esc::kMaxSlabs;
+    if (s < 1) s = 1;
+    return (int)s;
+}
+
+size_t workspace_bytes(int B, int Ca, long long HW) {
+    const int S = slabs_for(B, HW);
+    size_t off = round_up((size_t)(esc::kCtrlHeaderWords + B) * 4, 256);
+    off += round_up((size_t)B * Ca * 9 * 4, 256);
+    off += round_up((size_t)B * S * Ca * 4, 256);
+    return off;
+}
+
+Workspace carve(void* ws, int B, int Ca) {
+    Workspace w;
+    char* p = static_cast<char*>(ws);
+    w.ctrl = reinterpret_cast<unsigned*>(p);
+    w.arrivals = w.ctrl + esc::kCtrlHeaderWords;
+    p += round_up((size_t)(esc::kCtrlHeaderWords + B) * 4, 256);
+    w.dk = reinterpret_cast<float*>(p);
+    p += round_up((size_t)B * Ca * 9 * 4, 256);
+    w.partial = reinterpret_cast<float*>(p);
+    return w;
+}
+
+int check_workspace(const Problem& p, const void* ws, size_t bytes) {
+    if (!ws || !aligned(ws, 256)) return ESC_ERR_WORKSPACE;
+    if (bytes < workspace_bytes(p.B, p.Ca, (long long)p.H * p.W)) return ESC_ERR_WORKSPACE;
+    return ESC_OK;
+}
+
+// ---- stage 1 ------------------------------------------------------------------------------
+template <typename T, int LAYOUT>
+int launch_gap_t(const Problem& p, const void* x, const void* w_dyn, const void* b_dyn,
+                 const Workspace& w, float* dk_out, cudaStream_t st) {
+    const int S = slabs_for(p.B, (long long)p.H * p.W);
+    dim3 grid(S, p.B);
+    const size_t smem = (size_t)(esc::kGapWarps + 1) * p.Ca * sizeof(float);
+    if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
+    esc::gap_dynkernel<T, LAYOUT><<<grid, esc::kGapThreads, smem, st>>>(
+        static_cast<const T*>(x), p.C, p.Ca, p.H, p.W, S, static_cast<const T*>(w_dyn),
+        static_cast<const T*>(b_dyn), w.partial, w.arrivals, dk_out);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
+}
+
+int launch_gap(const Problem& p, const void* x, const void* w_dyn, const void* b_dyn,
+               const Workspace& w, float* dk_out, cudaStream_t st) {
+    if (p.B > 65535) return ESC_ERR_UNSUPPORTED;
+    if (p.dtype == ESC_F32)
+        return p.layout == ESC_NCHW ? launch_gap_t<float, esc::kNCHW>(p, x, w_dyn, b_dyn, w, dk_out, st)
+                                    : launch_gap_t<float, esc::kNHWC>(p, x, w_dyn, b_dyn, w, dk_out, st);
+    return p.layout == ESC_NCHW ? launch_gap_t<__nv_bfloat16, esc::kNCHW>(p, x, w_dyn, b_dyn, w, dk_out, st)
+                                : launch_gap_t<__nv_bfloat16, esc::kNHWC>(p, x, w_dyn, b_dyn, w, dk_out, st);
+}
+
+// ---- stage 2 ------------------------------------------------------------------------------
+template <typename U>
+int launch_copy_u(const void* x, void* out, long long rows, long long row_b, long long stride_b,
+                  long long off_b, cudaStream_t st) {
+    const long long u = sizeof(U);
+    const long long total = rows * (row_b / u);
+    if (total == 0) return ESC_OK;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    esc::copy_through<U><<<(unsigned)blocks, 256, 0, st>>>(static_cast<const U*>(x), static_cast<U*>(out), rows,
+                                                          row_b / u, stride_b / u, off_b / u);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
+}
+
+int launch_copy(const Problem& p, const void* x, void* out, cudaStream_t st) {
+    if (p.Ca == p.C) return ESC_OK;
+    const long long es = (long long)p.es(), HW = (long long)p.H * p.W;
+    long long rows, row_b, stride_b, off_b;
+    if (p.layout == ESC_NCHW) { rows = p.B; row_b = (p.C - p.Ca) * HW * es; stride_b = p.C * HW * es; off_b = p.Ca * HW * es; }
+    else { rows = (long long)p.B * HW; row_b = (p.C - p.Ca) * es; stride_b = p.C * es; off_b = p.Ca * es; }
+    if (row_b % 16 == 0 && stride_b % 16 == 0 && off_b % 16 == 0) return launch_copy_u<uint4>(x, out, rows, row_b, stride_b, off_b, st);
+    if (row_b % 4 == 0 && stride_b % 4 == 0 && off_b % 4 == 0) return launch_copy_u<uint32_t>(x, out, rows, row_b, stride_b, off_b, st);
+    return launch_copy_u<uint16_t>(x, out, rows, row_b, stride_b, off_b, st);
+}
+
+template <typename T, int LAYOUT>
+int launch_generic_t(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
+                     cudaStream_t st, bool dependent) {
+    const int tiles_x = (p.W + esc::kGenTX - 1) / esc::kGenTX, tiles_y = (p.H + esc::kGenTY - 1) / esc::kGenTY;
+    const long long blocks = (long long)p.B * p.Ca * tiles_x * tiles_y;
+    if (blocks > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(esc::kGenTX, esc::kGenTY);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_generic<T, LAYOUT>, static_cast<const T*>(x), static_cast<T*>(out),
+                                p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), dk, tiles_x, tiles_y));
+    ++g_last_launches;
+    return ESC_OK;
+}
+
+int launch_generic(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
+                   cudaStream_t st, bool dependent) {
+    g_last_path = 1;
+    int rc;
+    if (p.dtype == ESC_F32)
+        rc = p.layout == ESC_NCHW ? launch_generic_t<float, esc::kNCHW>(p, x, w_large, dk, out, st, dependent)
+                                  : launch_generic_t<float, esc::kNHWC>(p, x, w_large, dk, out, st, dependent);
+    else
+        rc = p.layout == ESC_NCHW ? launch_generic_t<__nv_bfloat16, esc::kNCHW>(p, x, w_large, dk, out, st, dependent)
+                                  : launch_generic_t<__nv_bfloat16, esc::kNHWC>(p, x, w_large, dk, out, st, dependent);
+    if (rc != ESC_OK) return rc;
+    return launch_copy(p, x, out, st);
+}
+
+int launch_stencil(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
+                   unsigned* ctrl, cudaStream_t st, bool dependent) {
+    int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, out, ctrl, st,
+                                  dependent, &g_last_launches, &g_last_error);
+    if (rc == ESC_OK) { g_last_path = 2; return ESC_OK; }
+    if (rc != esc::tma::kNotApplicable) return rc;
+    return launch_generic(p, x, w_large, dk, out, st, dependent);
+}
+
+// ---- library-owned scratch for the entry point that has no workspace argument --------------
+struct Scratch { void* ptr = nullptr; size_t bytes = 0; };
+std::mutex g_scratch_mu;
+std::map<std::pair<int, void*>, Scratch> g_scratch;
+
+int get_scratch(size_t need, cudaStream_t st, void** out) {
+    int dev = 0;
+    ESC_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(g_scratch_mu);
+    Scratch& s = g_scratch[{dev, (void*)st}];
+    if (s.bytes < need) {
+        if (s.ptr) { ESC_CUDA(cudaFree(s.ptr)); s.ptr = nullptr; s.bytes = 0; }   // cudaFree waits for pending work
+        const size_t cap = round_up(need, 1 << 20);
+        ESC_CUDA(cudaMalloc(&s.ptr, cap));
+        ESC_CUDA(cudaMemset(s.ptr, 0, cap));
+        s.bytes = cap;
+    }
+    *out = s.ptr;
+    return ESC_OK;
+}
+
+int forward_impl(const Problem& p, const void* x, const void* w_large, const void* w_dyn, const void* b_dyn,
+                 void* out, void* ws, cudaStream_t st) {
+    const Workspace w = carve(ws, p.B, p.Ca);
+    int rc = launch_gap(p, x, w_dyn, b_dyn, w, w.dk, st);
+    if (rc != ESC_OK) return rc;
+    return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
+}
+
+// ---- host-buffer path ---------------------------------------------------------------------
+struct HostPath {
+    int dev = -1;
+    cudaStream_t st = nullptr;
+    void *x = nullptr, *out = nullptr, *wts = nullptr, *ws = nullptr;
+    size_t xbytes = 0, wbytes = 0, wsbytes = 0;
+};
+std::mutex g_host_mu;
+HostPath g_host;
+
+}  // namespace
+
+extern "C" {
+
+int esc_version(void) { return 100; }
+
+const char* esc_last_error(void) { return g_last_error.c_str(); }
+
+int esc_convattn_last_path(void) { return g_last_path; }
+int esc_convattn_last_launches(void) { return g_last_launches; }
+
+const char* esc_status_string(int s) {
+    switch (s) {
+        case ESC_OK: return "ok";
+        case ESC_ERR_NULL: return "null pointer";
+        case ESC_ERR_SHAPE: return "invalid shape";
+        case ESC_ERR_UNSUPPORTED: return "unsupported configuration";
+        case ESC_ERR_ALIGN: return "misaligned pointer";
+        case ESC_ERR_ALIAS: return "out overlaps x";
+        case ESC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case ESC_ERR_CUDA: return "CUDA error";
+        case ESC_DEV_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+size_t esc_convattn_workspace_bytes(int B, int C_a, int H, int W, int K) {
+    if (B <= 0 || C_a <= 0 || H <= 0 || W <= 0 || K < 1 || (K & 1) == 0 || K > ESC_MAX_K) return 0;
+    return workspace_bytes(B, C_a, (long long)H * W);
+}
+
+int esc_convattn_workspace_init(void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes_ < 256) return ESC_ERR_WORKSPACE;
+    ESC_CUDA(cudaMemsetAsync(workspace, 0, workspace_bytes_, static_cast<cudaStream_t>(stream)));
+    return ESC_OK;
+}
+
+int esc_convattn_forward_ex(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                            const void* w_dyn, const void* b_dyn, void* out, int dtype, int layout,
+                            void* workspace, size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_large || !w_dyn || !b_dyn) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, p.es()) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    return forward_impl(p, x, w_large, w_dyn, b_dyn, out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_forward(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                         const void* w_dyn, const void* b_dyn, void* out, void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, K, ESC_F32, ESC_NCHW};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_large || !w_dyn || !b_dyn) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, 4) || !aligned(w_dyn, 4) || !aligned(b_dyn, 4)) return ESC_ERR_ALIGN;
+    void* ws = nullptr;
+    rc = get_scratch(workspace_bytes(B, C_a, (long long)H * W), static_cast<cudaStream_t>(stream), &ws);
+    if (rc != ESC_OK) return rc;
+    return forward_impl(p, x, w_large, w_dyn, b_dyn, out, ws, static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W, const void* w_dyn,
+                           const void* b_dyn, float* dk_out, int dtype, int layout, void* workspace,
+                           size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, 1, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!x || !w_dyn || !b_dyn || !dk_out) return ESC_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(dk_out, 4) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    return launch_gap(p, x, w_dyn, b_dyn, carve(workspace, B, C_a), dk_out, static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_stencil(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                         const float* dk, void* out, int dtype, int layout, void* workspace,
+                         size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_large || !dk) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, p.es()) || !aligned(dk, 4)) return ESC_ERR_ALIGN;
+    unsigned* ctrl = nullptr;
+    if (workspace) {
+        rc = check_workspace(p, workspace, workspace_bytes_);
+        if (rc != ESC_OK) return rc;
+        ctrl = carve(workspace, B, C_a).ctrl;
+    }
+    return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
+}
+
+int esc_convattn_device_status(void* workspace, void* stream) {
+    if (!workspace) return ESC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned word[2] = {0, 0};
+    ESC_CUDA(cudaMemcpyAsync(word, workspace, sizeof word, cudaMemcpyDeviceToHost, st));
+    ESC_CUDA(cudaStreamSynchronize(st));
+    if (word[0] != 0) {
+        char buf[96];
+        snprintf(buf, sizeof buf, "device status %u, detail 0x%x", word[0], word[1]);
+        g_last_error = buf;
+        ESC_CUDA(cudaMemsetAsync(workspace, 0, sizeof word, st));
+        ESC_CUDA(cudaStreamSynchronize(st));
+    }
+    return (int)word[0];
+}
+
+int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, int W, int K,
+                              const void* w_large_host, const void* w_dyn_host, const void* b_dyn_host,
+                              void* out_host, int dtype, int layout) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!x_host || !w_large_host || !w_dyn_host || !b_dyn_host || !out_host) return ESC_ERR_NULL;
+    std::lock_guard<std::mutex> lock(g_host_mu);
+    HostPath& h = g_host;
+    int dev = 0;
+    ESC_CUDA(cudaGetDevice(&dev));
+    if (h.dev != dev) {   // first use, or the caller switched device: start over
+        if (h.dev >= 0) {
+            ESC_CUDA(cudaSetDevice(h.dev));
+            cudaFree(h.x); cudaFree(h.out); cudaFree(h.wts); cudaFree(h.ws);
+            if (h.st) cudaStreamDestroy(h.st);
+            ESC_CUDA(cudaSetDevice(dev));
+        }
+        h = HostPath();
+        h.dev = dev;
+        ESC_CUDA(cudaStreamCreateWithFlags(&h.st, cudaStreamNonBlocking));
+    }
+    const size_t es = p.es(), xbytes = p.elems() * es;
+    const size_t n_wl = (size_t)C_a * K * K, n_wd = (size_t)9 * C_a * C_a, n_bd = (size_t)9 * C_a;
+    const size_t off_wd = round_up(n_wl * es, 256), off_bd = off_wd + round_up(n_wd * es, 256);
+    const size_t wbytes = off_bd + round_up(n_bd * es, 256);
+    const size_t wsbytes = workspace_bytes(B, C_a, (long long)H * W);
+    if (h.xbytes < xbytes) {
+        cudaFree(h.x); cudaFree(h.out); h.x = h.out = nullptr; h.xbytes = 0;
+        ESC_CUDA(cudaMalloc(&h.x, xbytes));
+        ESC_CUDA(cudaMalloc(&h.out, xbytes));
+        h.xbytes = xbytes;
+    }
+    if (h.wbytes < wbytes) {
+        cudaFree(h.wts); h.wts = nullptr; h.wbytes = 0;
+        ESC_CUDA(cudaMalloc(&h.wts, wbytes));
+        h.wbytes = wbytes;
+    }
+    if (h.wsbytes < wsbytes) {
+        cudaFree(h.ws); h.ws = nullptr; h.wsbytes = 0;
+        ESC_CUDA(cudaMalloc(&h.ws, wsbytes));
+        ESC_CUDA(cudaMemset(h.ws, 0, wsbytes));
+        h.wsbytes = wsbytes;
+    }
+    char* wts = static_cast<char*>(h.wts);
+    ESC_CUDA(cudaMemcpyAsync(h.x, x_host, xbytes, cudaMemcpyHostToDevice, h.st));
+    ESC_CUDA(cudaMemcpyAsync(wts, w_large_host, n_wl * es, cudaMemcpyHostToDevice, h.st));
+    ESC_CUDA(cudaMemcpyAsync(wts + off_wd, w_dyn_host, n_wd * es, cudaMemcpyHostToDevice, h.st));
+    ESC_CUDA(cudaMemcpyAsync(wts + off_bd, b_dyn_host, n_bd * es, cudaMemcpyHostToDevice, h.st));
+    rc = forward_impl(p, h.x, wts, wts + off_wd, wts + off_bd, h.out, h.ws, h.st);
+    if (rc != ESC_OK) return rc;
+    ESC_CUDA(cudaMemcpyAsync(out_host, h.out, xbytes, cudaMemcpyDeviceToHost, h.st));
+    ESC_CUDA(cudaStreamSynchronize(h.st));
+    return ESC_OK;
+}
+
+}  // extern "C"
