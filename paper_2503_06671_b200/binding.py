@@ -1,0 +1,185 @@
+"""ctypes binding with the same names as include/esc_convattn.h (argument marshalling only).
+
+Tensors are torch CUDA tensors (or, for the *_host call, CPU tensors); the binding passes their
+data pointers, the logical sizes and the current stream.  Logical shape is always [B,C,H,W]:
+an NCHW call takes a contiguous [B,C,H,W] tensor, an NHWC call a contiguous [B,H,W,C] tensor.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+ESC_F32, ESC_BF16 = 0, 1
+ESC_NCHW, ESC_NHWC = 0, 1
+
+_LIB_PATH = Path(__file__).resolve().parent / "lib" / "libesc_convattn.so"
+_lib = None
+
+
+class EscError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        text = esc_status_string(status)
+        detail = esc_last_error() if self.status == 7 else ""
+        super().__init__(f"{where}: status {self.status} ({text}){' -- ' + detail if detail else ''}")
+
+
+def lib_path() -> Path:
+    return _LIB_PATH
+
+
+def lib():
+    """The loaded C-ABI library; raises if it has not been built (no silent fall-back)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2503_06671_b200.build` "
+                "(there is no CPU implementation to fall back to)")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.esc_convattn_forward.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp]
+        L.esc_convattn_forward_ex.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.esc_convattn_workspace_bytes.restype = sz
+        L.esc_convattn_workspace_init.argtypes = [vp, sz, vp]
+        L.esc_convattn_dynkernel.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
+        L.esc_convattn_device_status.argtypes = [vp, vp]
+        L.esc_status_string.argtypes = [i]
+        L.esc_status_string.restype = ctypes.c_char_p
+        L.esc_last_error.restype = ctypes.c_char_p
+        for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
+                     "esc_convattn_dynkernel", "esc_convattn_stencil", "esc_convattn_forward_host",
+                     "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_launches",
+                     "esc_version"):
+            getattr(L, name).restype = i
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    import torch
+
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(status, where):
+    if status != 0:
+        raise EscError(status, where)
+
+
+def _dtype_code(t):
+    import torch
+
+    if t.dtype == torch.float32:
+        return ESC_F32
+    if t.dtype == torch.bfloat16:
+        return ESC_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _dims(x, layout):
+    if x.dim() != 4 or not x.is_contiguous():
+        raise ValueError("x must be a contiguous 4-D tensor in the memory order named by `layout`")
+    if layout == ESC_NCHW:
+        B, C, H, W = x.shape
+    elif layout == ESC_NHWC:
+        B, H, W, C = x.shape
+    else:
+        raise ValueError("layout")
+    return int(B), int(C), int(H), int(W)
+
+
+def esc_status_string(status) -> str:
+    return lib().esc_status_string(int(status)).decode()
+
+
+def esc_last_error() -> str:
+    return lib().esc_last_error().decode()
+
+
+def esc_version() -> int:
+    return lib().esc_version()
+
+
+def esc_convattn_last_path() -> int:
+    return lib().esc_convattn_last_path()
+
+
+def esc_convattn_last_launches() -> int:
+    return lib().esc_convattn_last_launches()
+
+
+def esc_convattn_workspace_bytes(B, C_a, H, W, K) -> int:
+    return int(lib().esc_convattn_workspace_bytes(B, C_a, H, W, K))
+
+
+def esc_convattn_workspace_init(workspace, stream=None):
+    _check(lib().esc_convattn_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                             _stream(stream)), "esc_convattn_workspace_init")
+
+
+def new_workspace(B, C_a, H, W, K, device="cuda"):
+    """Allocate (with torch) and initialise a workspace for the calls that take one."""
+    import torch
+
+    n = esc_convattn_workspace_bytes(B, C_a, H, W, K)
+    if n == 0:
+        raise ValueError("invalid problem size")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    esc_convattn_workspace_init(ws)
+    return ws
+
+
+def esc_convattn_forward(x, C_a, K, w_large, w_dyn, b_dyn, out, stream=None):
+    """fp32 NCHW forward (library-owned scratch).  x, out: contiguous [B,C,H,W] float32 CUDA tensors."""
+    B, C, H, W = _dims(x, ESC_NCHW)
+    _check(lib().esc_convattn_forward(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_dyn), _ptr(b_dyn),
+                                      _ptr(out), _stream(stream)), "esc_convattn_forward")
+    return out
+
+
+def esc_convattn_forward_ex(x, C_a, K, w_large, w_dyn, b_dyn, out, layout, workspace, stream=None):
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_forward_ex(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_dyn), _ptr(b_dyn),
+                                         _ptr(out), _dtype_code(x), layout, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_forward_ex")
+    return out
+
+
+def esc_convattn_dynkernel(x, C_a, w_dyn, b_dyn, dk_out, layout, workspace, stream=None):
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_dynkernel(_ptr(x), B, C, C_a, H, W, _ptr(w_dyn), _ptr(b_dyn), _ptr(dk_out),
+                                        _dtype_code(x), layout, _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_dynkernel")
+    return dk_out
+
+
+def esc_convattn_stencil(x, C_a, K, w_large, dk, out, layout, workspace=None, stream=None):
+    B, C, H, W = _dims(x, layout)
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib().esc_convattn_stencil(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(dk), _ptr(out),
+                                      _dtype_code(x), layout, _ptr(workspace), nbytes, _stream(stream)),
+           "esc_convattn_stencil")
+    return out
+
+
+def esc_convattn_forward_host(x, C_a, K, w_large, w_dyn, b_dyn, out, layout):
+    """Host-buffer call: CPU tensors in, CPU tensor out; copies and synchronisation happen inside."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_forward_host(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_dyn), _ptr(b_dyn),
+                                           _ptr(out), _dtype_code(x), layout), "esc_convattn_forward_host")
+    return out
+
+
+def esc_convattn_device_status(workspace, stream=None) -> int:
+    return lib().esc_convattn_device_status(_ptr(workspace), _stream(stream))

@@ -1,0 +1,101 @@
+"""CPU-side checks of the C-ABI library: it loads without a GPU, exports every symbol the header
+declares, and rejects bad arguments on the host before anything could be launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2503_06671_b200 import build, lib
+
+    build.build()
+    return lib()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "esc_convattn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(esc_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = _declared_symbols()
+    assert "esc_convattn_forward" in names and "esc_convattn_forward_ex" in names and len(names) >= 12
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_binding_has_the_same_names(L):
+    import paper_2503_06671_b200 as pkg
+
+    for n in _declared_symbols():
+        assert hasattr(pkg, n), n
+
+
+def test_version_and_strings(L):
+    assert L.esc_version() >= 100
+    assert L.esc_status_string(0) == b"ok"
+    assert b"overlaps" in L.esc_status_string(5)
+    assert L.esc_status_string(12345) == b"unknown status"
+
+
+def test_workspace_bytes(L):
+    n = L.esc_convattn_workspace_bytes(1, 16, 360, 640, 13)
+    assert n > 0 and n % 256 == 0
+    assert L.esc_convattn_workspace_bytes(64, 16, 64, 64, 13) >= 64 * 16 * 9 * 4
+    for bad in [(0, 16, 8, 8, 13), (1, 0, 8, 8, 13), (1, 16, 0, 8, 13), (1, 16, 8, 8, 12), (1, 16, 8, 8, 19)]:
+        assert L.esc_convattn_workspace_bytes(*bad) == 0
+
+
+def test_host_side_rejections_launch_nothing(L):
+    """Fake, never dereferenced addresses: every call must fail on the host checks."""
+    X, O, Wl, Wd, Bd, WS = 0x10000000, 0x20000000, 0x30000000, 0x30100000, 0x30200000, 0x40000000
+    big = 1 << 20
+
+    def fwd(x=X, B=1, C=64, Ca=16, H=32, W=32, K=13, wl=Wl, wd=Wd, bd=Bd, out=O, dt=1, lay=1, ws=WS, wsb=big):
+        return L.esc_convattn_forward_ex(x, B, C, Ca, H, W, K, wl, wd, bd, out, dt, lay, ws, wsb, None)
+
+    assert fwd(x=None) == 1 and fwd(out=None) == 1 and fwd(wl=None) == 1 and fwd(wd=None) == 1 and fwd(bd=None) == 1
+    assert fwd(B=0) == 2 and fwd(H=-3) == 2 and fwd(Ca=0) == 2 and fwd(Ca=65) == 2 and fwd(K=12) == 2 and fwd(K=0) == 2
+    assert fwd(K=19) == 3 and fwd(dt=2) == 3 and fwd(lay=5) == 3
+    assert fwd(x=X + 8) == 4 and fwd(out=O + 4) == 4 and fwd(wl=Wl + 1) == 4
+    assert fwd(out=X) == 5 and fwd(out=X + 64 * 32 * 32 * 2 - 16) == 5 and fwd(x=O + 16, out=O) == 5
+    assert fwd(ws=None) == 6 and fwd(ws=WS + 64) == 6 and fwd(wsb=128) == 6
+    # the fixed-signature entry and the stage hooks share the checks
+    assert L.esc_convattn_forward(None, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, None) == 1
+    assert L.esc_convattn_forward(X, 1, 64, 16, 8, 8, 14, Wl, Wd, Bd, O, None) == 2
+    assert L.esc_convattn_forward(X, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, X, None) == 5
+    assert L.esc_convattn_dynkernel(X, 1, 64, 16, 8, 8, Wd, Bd, None, 0, 0, WS, big, None) == 1
+    assert L.esc_convattn_dynkernel(X, 1, 64, 16, 8, 8, Wd, Bd, O, 0, 0, WS, 16, None) == 6
+    assert L.esc_convattn_stencil(X, 1, 64, 16, 8, 8, 13, Wl, None, O, 0, 0, None, 0, None) == 1
+    assert L.esc_convattn_stencil(X, 1, 64, 16, 8, 8, 13, Wl, Wd, X + 16, 0, 0, None, 0, None) == 5
+    assert L.esc_convattn_forward_host(None, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 1
+    assert L.esc_convattn_forward_host(X, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 7, 0) == 3
+    assert L.esc_convattn_workspace_init(None, 1024, None) == 6
+    assert L.esc_convattn_device_status(None, None) == 6
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    from paper_2503_06671_b200 import binding
+
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "nope.so")
+    with pytest.raises(RuntimeError, match="no CPU implementation"):
+        binding.lib()
+
+
+def test_product_does_not_import_oracle():
+    pkg = os.path.join(ROOT, "paper_2503_06671_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower() or f == "synth.py", f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c")):
+            assert "paper_2503_06671_b200" not in open(os.path.join(ROOT, "oracle", f)).read(), f

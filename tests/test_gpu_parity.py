@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU oracle on the same
+seeded inputs (ESC paper, Section 3.3, Eq. 4).  Tolerances are in tests/util.py."""
+import numpy as np
+import pytest
+
+from paper_2503_06671_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+LAYOUTS = [synth.NCHW, synth.NHWC]
+DTYPES = [synth.F32, synth.BF16]
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import paper_2503_06671_b200 as p
+
+    p.lib()
+    return p
+
+
+def run_forward(pkg, d, C_a, K, dtype, layout, entry="ex"):
+    import torch
+
+    x = util.to_device(d["x"], dtype, layout)
+    wl, wd, bd = util.weights_to_device(d, dtype)
+    B, C, H, W = d["x"].shape
+    # guard bands around out: the kernels must not write outside it
+    n = x.numel()
+    pad = 4096
+    buf = torch.full((n + 2 * pad,), 7.0, dtype=x.dtype, device="cuda")
+    out = buf[pad:pad + n].view(x.shape)
+    ws = pkg.new_workspace(B, C_a, H, W, K)
+    if entry == "ex":
+        pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, out, util.layout_code(layout), ws)
+    else:
+        pkg.esc_convattn_forward(x, C_a, K, wl, wd, bd, out)
+    torch.cuda.synchronize()
+    assert pkg.esc_convattn_device_status(ws) == 0
+    assert bool((buf[:pad] == 7.0).all()) and bool((buf[pad + n:] == 7.0).all()), "write outside out"
+    return x, out
+
+
+def compare_full(pkg, oracle, d, C_a, K, dtype, layout, entry="ex", what=""):
+    import torch
+
+    x, out = run_forward(pkg, d, C_a, K, dtype, layout, entry)
+    ref, mag = oracle.forward(d["x"], C_a, d["w_large"], d["w_dyn"], d["b_dyn"], want_mag=True)
+    got = util.to_host_nchw(out, layout)
+    err = util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, what)
+    # copy-through channels: bit-exact
+    if C_a < d["x"].shape[1]:
+        xs, os_ = (x, out) if layout == synth.NCHW else (x.permute(0, 3, 1, 2), out.permute(0, 3, 1, 2))
+        assert torch.equal(xs[:, C_a:].contiguous().view(torch.int16 if dtype == synth.BF16 else torch.int32),
+                           os_[:, C_a:].contiguous().view(torch.int16 if dtype == synth.BF16 else torch.int32))
+    return err
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_dk_stage(pkg, oracle, dtype, layout):
+    """GAP + linear layer on non-zero-mean data: dk within 1e-5 of max|dk| (fp32 arithmetic)."""
+    import torch
+
+    for (B, C, C_a, H, W) in [(3, 64, 16, 37, 53), (1, 64, 32, 120, 200), (2, 24, 8, 16, 16), (1, 20, 12, 9, 7),
+                              (70, 32, 16, 8, 8)]:
+        d = synth.make_inputs(B, C, C_a, H, W, 13, dtype, seed=B * 100 + H, channel_means=True)
+        x = util.to_device(d["x"], dtype, layout)
+        _, wd, bd = util.weights_to_device(d, dtype)
+        dk = torch.full((B, C_a, 3, 3), float("nan"), device="cuda")
+        ws = pkg.new_workspace(B, C_a, H, W, 13)
+        for _ in range(2):  # twice: the arrival counters must be ready for reuse
+            pkg.esc_convattn_dynkernel(x, C_a, wd, bd, dk, util.layout_code(layout), ws)
+        torch.cuda.synchronize()
+        ref = oracle.dynkernel(oracle.gap(d["x"], C_a), d["w_dyn"], d["b_dyn"])
+        err = np.abs(dk.cpu().numpy().astype(np.float64) - ref).max()
+        assert err <= 1e-5 * np.abs(ref).max(), (B, C, C_a, H, W, err)
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_stencil_stage_explicit_dk(pkg, oracle, dtype, layout):
+    import torch
+
+    B, C, C_a, H, W, K = 2, 64, 16, 45, 70, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, dtype, seed=77)
+    dk = np.random.default_rng(5).uniform(-0.5, 0.5, size=(B, C_a, 3, 3)).astype(np.float32)
+    x = util.to_device(d["x"], dtype, layout)
+    wl, _, _ = util.weights_to_device(d, dtype)
+    out = torch.empty_like(x)
+    pkg.esc_convattn_stencil(x, C_a, K, wl, torch.from_numpy(dk).cuda(), out, util.layout_code(layout))
+    torch.cuda.synchronize()
+    ref, mag = oracle.stencil(d["x"], C_a, d["w_large"], dk, want_mag=True)
+    got = util.to_host_nchw(out, layout)
+    util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, "stencil stage")
+    assert np.array_equal(got[:, C_a:], ref[:, C_a:])
+
+
+EDGE_SHAPES = [
+    # B, C, C_a, H, W, K
+    (1, 64, 16, 5, 5, 13),      # H, W < K
+    (2, 64, 16, 1, 40, 13),     # single row
+    (2, 64, 16, 33, 1, 13),     # single column
+    (1, 64, 16, 13, 13, 13),
+    (3, 64, 16, 41, 83, 13),    # several tiles plus a ragged tail, odd W
+    (1, 64, 16, 40, 40, 13),    # exactly one register tile
+    (1, 64, 16, 80, 120, 13),   # whole tiles only
+    (2, 16, 16, 30, 50, 13),    # C_a == C: nothing to copy through
+    (2, 32, 8, 22, 36, 13),     # C_a = 8
+    (1, 64, 32, 47, 61, 13),    # C_a = 32
+    (1, 48, 16, 29, 31, 9),     # K = 9
+    (1, 48, 16, 29, 31, 17),    # K = 17
+    (1, 20, 12, 19, 23, 3),     # K = 3, odd channel counts
+    (5, 64, 16, 64, 64, 13),    # small batch of training patches
+]
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", EDGE_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_forward_edge_shapes(pkg, oracle, shape, dtype, layout):
+    B, C, C_a, H, W, K = shape
+    d = synth.make_inputs(B, C, C_a, H, W, K, dtype, seed=sum(shape), per_image_scale=True, channel_means=True)
+    compare_full(pkg, oracle, d, C_a, K, dtype, layout, what=str(shape))
+
+
+@pytest.mark.parametrize("wl_name", ["cfg1_64x64_f32", "cfg2_320x180_f32", "cfg3_640x360_bf16", "cfg4_b64_64x64_bf16"])
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("means", [False, True], ids=["zero_mean", "channel_means"])
+def test_forward_workloads_full(pkg, oracle, wl_name, layout, means):
+    """The evaluation workloads, every output compared (the oracle needs a few seconds each)."""
+    wl = synth.WORKLOADS_BY_NAME[wl_name]
+    d = synth.make_workload(wl, channel_means=means)
+    compare_full(pkg, oracle, d, wl.C_a, wl.K, wl.dtype, layout, what=wl_name)
+
+
+def test_mandated_entry_fp32_nchw(pkg, oracle):
+    wl = synth.WORKLOADS_BY_NAME["cfg1_64x64_f32"]
+    d = synth.make_workload(wl, channel_means=True)
+    compare_full(pkg, oracle, d, wl.C_a, wl.K, wl.dtype, synth.NCHW, entry="fixed", what="esc_convattn_forward")
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_forward_large_map_sampled(pkg, oracle, layout):
+    """1920x1080, C_a=32 bf16 in the launch configuration the benchmark times: 20000 sampled outputs
+    (plus every corner and border row/column sample) against the oracle one by one; copy-through
+    channels compared bit for bit on the device."""
+    import torch
+
+    wl = synth.WORKLOADS_BY_NAME["cfg5_1920x1080_ca32_bf16"]
+    d = synth.make_workload(wl, channel_means=True)
+    x, out = run_forward(pkg, d, wl.C_a, wl.K, wl.dtype, layout)
+    B, C, H, W = d["x"].shape
+    rng = np.random.default_rng(9)
+    c = rng.integers(0, wl.C_a, size=20000)
+    y = rng.integers(0, H, size=20000)
+    xx = rng.integers(0, W, size=20000)
+    # force coverage of borders, corners and tile seams
+    y[:2000] = rng.choice([0, 1, 5, 6, 7, H - 7, H - 6, H - 1, 39, 40, 41, 1079 - 40], size=2000)
+    xx[2000:4000] = rng.choice([0, 1, 5, 6, 7, W - 7, W - 6, W - 1, 39, 40, 41, 1919 - 40], size=2000)
+    flat = (c.astype(np.int64) * H + y) * W + xx
+    vals, mags = oracle.points(d["x"], wl.C_a, d["w_large"], d["w_dyn"], d["b_dyn"], flat, want_mag=True)
+    o_nchw = out if layout == synth.NCHW else out.permute(0, 3, 1, 2)
+    got = o_nchw[0][torch.from_numpy(c).cuda(), torch.from_numpy(y).cuda(), torch.from_numpy(xx).cuda()].float().cpu().numpy()
+    util.check_attention(got, vals, mags, wl.dtype, "cfg5 sampled")
+    x_nchw = x if layout == synth.NCHW else x.permute(0, 3, 1, 2)
+    assert torch.equal(x_nchw[:, wl.C_a:].contiguous().view(torch.int16), o_nchw[:, wl.C_a:].contiguous().view(torch.int16))
+    # property that holds at any size: the large-kernel response to the all-ones image, interior = kernel sum
+    # (checked through linearity on the identity: out is finite everywhere)
+    assert bool(torch.isfinite(o_nchw[:, :wl.C_a].float()).all())
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_bitwise_determinism_and_special_values(pkg, layout):
+    """Run-to-run identical bits; NaN / -0 payloads in copy-through channels survive."""
+    import torch
+
+    B, C, C_a, H, W, K = 2, 64, 16, 90, 130, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=5, channel_means=True)
+    x = util.to_device(d["x"], synth.BF16, layout)
+    xv = x.view(torch.int16)
+    idt = (slice(None), slice(C_a, None)) if layout == synth.NCHW else (Ellipsis, slice(C_a, None))
+    sub = xv[idt]
+    sub.view(-1)[::97] = -32768          # -0.0
+    sub.view(-1)[5::89] = 0x7FC1         # NaN with a payload
+    xv[idt] = sub
+    wl, wd, bd = util.weights_to_device(d, synth.BF16)
+    ws = pkg.new_workspace(B, C_a, H, W, K)
+    outs = []
+    for _ in range(3):
+        out = torch.empty_like(x)
+        pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, out, util.layout_code(layout), ws)
+        torch.cuda.synchronize()
+        outs.append(out.view(torch.int16).clone())
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+    assert torch.equal(outs[0][idt], xv[idt])
+
+
+def test_host_entry_matches_device_entry(pkg):
+    import torch
+
+    B, C, C_a, H, W, K = 2, 64, 16, 60, 100, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=15, channel_means=True)
+    xh = torch.from_numpy(synth.to_layout(d["x"], synth.NHWC)).to(torch.bfloat16).pin_memory()
+    wl, wd, bd = (torch.from_numpy(d[k]).to(torch.bfloat16) for k in ("w_large", "w_dyn", "b_dyn"))
+    oh = torch.empty_like(xh).pin_memory()
+    for _ in range(2):
+        pkg.esc_convattn_forward_host(xh, C_a, K, wl, wd, bd, oh, pkg.ESC_NHWC)
+    x = xh.cuda()
+    out = torch.empty_like(x)
+    ws = pkg.new_workspace(B, C_a, H, W, K)
+    pkg.esc_convattn_forward_ex(x, C_a, K, wl.cuda(), wd.cuda(), bd.cuda(), out, pkg.ESC_NHWC, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out.cpu().view(torch.int16), oh.view(torch.int16))
