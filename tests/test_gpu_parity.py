@@ -46,13 +46,13 @@ def run_forward(pkg, d, C_a, K, dtype, layout, entry="ex"):
     return x, out
 
 
-def compare_full(pkg, oracle, d, C_a, K, dtype, layout, entry="ex", what=""):
+def compare_full(pkg, oracle, d, C_a, K, dtype, layout, entry="ex", what="", unit_variance=False):
     import torch
 
     x, out = run_forward(pkg, d, C_a, K, dtype, layout, entry)
     ref, mag = oracle.forward(d["x"], C_a, d["w_large"], d["w_dyn"], d["b_dyn"], want_mag=True)
     got = util.to_host_nchw(out, layout)
-    err = util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, what)
+    err = util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, what, unit_variance)
     # copy-through channels: bit-exact
     if C_a < d["x"].shape[1]:
         xs, os_ = (x, out) if layout == synth.NCHW else (x.permute(0, 3, 1, 2), out.permute(0, 3, 1, 2))
@@ -97,7 +97,7 @@ def test_stencil_stage_explicit_dk(pkg, oracle, dtype, layout):
     torch.cuda.synchronize()
     ref, mag = oracle.stencil(d["x"], C_a, d["w_large"], dk, want_mag=True)
     got = util.to_host_nchw(out, layout)
-    util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, "stencil stage")
+    util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, "stencil stage", unit_variance=True)
     assert np.array_equal(got[:, C_a:], ref[:, C_a:])
 
 
@@ -136,7 +136,8 @@ def test_forward_workloads_full(pkg, oracle, wl_name, layout, means):
     """The evaluation workloads, every output compared (the oracle needs a few seconds each)."""
     wl = synth.WORKLOADS_BY_NAME[wl_name]
     d = synth.make_workload(wl, channel_means=means)
-    compare_full(pkg, oracle, d, wl.C_a, wl.K, wl.dtype, layout, what=wl_name)
+    compare_full(pkg, oracle, d, wl.C_a, wl.K, wl.dtype, layout, what=wl_name,
+                 unit_variance=not means and not wl.per_image_scale)
 
 
 def test_mandated_entry_fp32_nchw(pkg, oracle):

@@ -43,8 +43,11 @@ def layout_code(layout):
     return ESC_NHWC if layout == synth.NHWC else ESC_NCHW
 
 
-def check_attention(got, ref, mag, dtype, what=""):
-    """got/ref/mag: arrays of attention-channel outputs (any matching shape)."""
+def check_attention(got, ref, mag, dtype, what="", unit_variance=False):
+    """got/ref/mag: arrays of attention-channel outputs (any matching shape).
+
+    The absolute bf16 bar is stated for unit-variance data; inputs with added channel means or
+    per-image scales have larger outputs, so there only the relative and per-element bars apply."""
     got = np.asarray(got, dtype=np.float64)
     err = np.abs(got - ref)
     if dtype == synth.F32:
@@ -53,7 +56,8 @@ def check_attention(got, ref, mag, dtype, what=""):
         fe = (err / np.maximum(mag, 1e-30)).max()
         assert fe <= F32_REL, f"{what}: forward error {fe:.3e} > {F32_REL}"
     else:
-        assert err.max() <= BF16_ABS, f"{what}: max|err|={err.max():.3e} > {BF16_ABS}"
+        if unit_variance:
+            assert err.max() <= BF16_ABS, f"{what}: max|err|={err.max():.3e} > {BF16_ABS}"
         rel = (err / np.maximum(np.abs(ref), 1.0)).max()
         assert rel <= BF16_REL, f"{what}: rel err {rel:.3e} > {BF16_REL}"
         # tighter, scale-aware bar: half a bf16 ulp of the result plus fp32 accumulation noise
