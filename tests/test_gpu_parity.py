@@ -186,7 +186,7 @@ def test_bitwise_determinism_and_special_values(pkg, layout):
     x = util.to_device(d["x"], synth.BF16, layout)
     xv = x.view(torch.int16)
     idt = (slice(None), slice(C_a, None)) if layout == synth.NCHW else (Ellipsis, slice(C_a, None))
-    sub = xv[idt]
+    sub = xv[idt].contiguous().clone()
     sub.view(-1)[::97] = -32768          # -0.0
     sub.view(-1)[5::89] = 0x7FC1         # NaN with a payload
     xv[idt] = sub
