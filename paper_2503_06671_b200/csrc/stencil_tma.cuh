@@ -1,23 +1,28 @@
 // Kernel (b), fast path: TMA-staged, register-tiled fused stencil for K = 13 on NHWC bf16 tensors
 // (ESC paper, Section 3.3, Eq. 4 lines 3-4, evaluated in the merged form ZP(dk) + LK^s of Eq. 5).
 //
-// Work unit: a 40x40 output tile of one image for one group of 16 attention channels.  A CTA
-// (8 compute warps + 1 copy warp, one CTA per SM, persistent over units) does, per unit:
-//   1. one TMA load of the (40+12) x (40+12+1) x 16-channel halo tile; coordinates outside the
-//      image are filled with zeros by the TMA unit, which is the 'same' padding;
-//   2. 169 taps for a 5x10 output patch per lane, two adjacent channels at a time with packed
-//      fp32 FMAs (fma.rn.f32x2): lane = (position q, channel pair p), a warp covers 4 patches x
-//      8 pairs.  Kernel rows are visited in the order 0-4, 8-12, 5-7 so that the per-image dynamic
-//      taps (rows 5-7 of the merged kernel) are needed last and the wait for the kernel that
-//      produces dk costs nothing;
-//   3. one rounding to bf16 and 4-byte stores that fill whole 32-byte sectors across 8 lanes.
-// Meanwhile the copy warp streams the untouched channels of the same tile global -> shared ->
-// global with TMA loads and stores through a small ring, with no register or issue-slot cost.
+// Work unit: a 40x40 output tile of one image for one group of 16 attention channels.  One CTA per
+// SM, persistent over units, three warp groups:
+//   warps 0-7  compute.  lane = (patch position q, channel pair p); a warp covers 4 patches of
+//              5x10 outputs x 8 channel pairs, two channels at a time with packed fp32 FMAs
+//              (fma.rn.f32x2).  The loop runs over the 17 INPUT rows a patch touches: a row is read
+//              from shared memory and widened to fp32 once (22 words), then used by up to five
+//              output rows, each with its own kernel row (7 broadcast-free 16-byte weight loads).
+//              That keeps the non-FMA instructions near 10 % of the issue slots, which matters
+//              because a packed FMA takes two issue slots and nothing is issued in its shadow.
+//   warp 8     tile producer: one TMA load per unit of the (40+12) x (40+12+1) x 16-channel halo
+//              tile into a two-deep ring; coordinates outside the image are zero-filled by the TMA
+//              unit, which is the 'same' padding.
+//   warp 9     copy-through: streams the untouched channels of the same tile global -> shared ->
+//              global with TMA loads and stores through a small ring.
+// The helper warps give their registers to the compute warps (setmaxnreg), which need ~200.
+// Results are rounded once to bf16, staged in the freed input buffer and written with one TMA
+// store per unit (clipped at the image border by the TMA unit).
 //
 // Shared-memory words of the tile hold one pixel's channel pair (bf16x2); a pixel is 8 words
-// (32 bytes), a tile row 53 pixels.  With an odd row pitch and a patch height of 5 the four
-// patches of a warp start at pixel indices that differ mod 4, so the 32 lanes of every LDS.32
-// hit 32 different banks.
+// (32 bytes), a tile row 53 pixels.  The four patches of a warp form a 2x2 block; with an odd row
+// pitch and a patch of 5 rows x 10 columns their first pixels differ mod 4, so the 32 lanes of
+// every LDS.32 hit 32 different banks.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -36,30 +41,35 @@ constexpr int LXP = 4, LYP = 8;           // patches per tile in x and y
 constexpr int TW = OX * LXP, TH = OY * LYP;          // 40 x 40 outputs per tile
 constexpr int THP = TH + K13 - 1;                    // 52 staged rows
 constexpr int PITCH = TW + K13 - 1 + 1;              // 53 staged pixels per row (odd on purpose)
+constexpr int NW = OX + K13 - 1;                     // 22 input pixels per patch row
+constexpr int NR = OY + K13 - 1;                     // 17 input rows per patch
 constexpr int CG = 16;                               // channels per unit
 constexpr int NPAIR = CG / 2;
 constexpr int kComputeWarps = LXP * LYP / 4;         // 8
 constexpr int kComputeThreads = kComputeWarps * 32;  // 256
-constexpr int kThreads = kComputeThreads + 32;       // + copy warp
+constexpr int kThreads = kComputeThreads + 128;      // + helper warp group (producer, copy, 2 idle)
+constexpr int kComputeRegs = 232, kHelperRegs = 24;
 constexpr int TILE_BYTES = THP * PITCH * CG * 2;     // 88,192
+constexpr int OUT_TILE_BYTES = TH * TW * CG * 2;     // 51,200: staged result, reuses the input buffer
 constexpr int WSM_FLOATS = K13 * 7 * NPAIR * 4;      // [i][jj][pair][4]: taps 2jj,2jj+1 of both channels
 constexpr int WSM_BYTES = (WSM_FLOATS * 4 + 127) / 128 * 128;
+constexpr int LKC_BYTES = (CG * 9 * 4 + 127) / 128 * 128;   // pristine centre 3x3 of LK^s
 constexpr int NSLOT = 4, COPY_DEPTH = 3;             // copy ring: slots, loads in flight
 constexpr int kMaxSlotBytes = 8192;
 constexpr unsigned kSpinLimit = 1u << 22;
 
 static_assert(TILE_BYTES % 128 == 0, "tile buffers must keep 128-byte alignment");
-static_assert((OY * PITCH) % 2 == 1, "patch rows must start at distinct pixel indices mod 4");
+static_assert(OUT_TILE_BYTES <= TILE_BYTES, "the result tile is staged in the input buffer");
+static_assert((OY * PITCH) % 2 == 1 && OX % 4 == 2, "2x2 patch block must start at distinct pixel indices mod 4");
 
 struct Params {
     int B, C, Ca, H, W;
-    int tiles_x, tiles_y, groups;     // units = B * tiles_y * tiles_x * groups
+    int tiles_x, tiles_y, groups;     // units = B * groups * tiles_y * tiles_x
     long long units;
     int copy_cc, copy_cw, copy_cr;    // copy box: channels, pixels, rows (copy_cc == 0: nothing to copy)
     int slot_stride;                  // bytes between ring slots (multiple of 128)
     const __nv_bfloat16* w_large;     // [Ca][13][13]
     const float* dk;                  // [B][Ca][9]
-    __nv_bfloat16* out;
     unsigned* ctrl;                   // status words or nullptr
 };
 
@@ -70,6 +80,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity) {
     unsigned ok;
@@ -102,7 +115,10 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void compute_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory"); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 typedef unsigned long long u64;
 __device__ __forceinline__ u64 pack2(float lo, float hi) {
@@ -123,104 +139,137 @@ __device__ __forceinline__ Unit decode_unit(long long u, const Params& p) {
     return r;
 }
 
-// Kernel row visited at step s: rows that never see dk first, the three dk rows last.
-__device__ __forceinline__ int row_order(int s) { return s < 5 ? s : (s < 10 ? s + 3 : s - 5); }
+__device__ __forceinline__ int wsm_index(int c, int i, int j) {
+    return ((i * 7 + (j >> 1)) * NPAIR + (c >> 1)) * 4 + (j & 1) * 2 + (c & 1);
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
-                      const __grid_constant__ CUtensorMap map_cout, const Params p)
+                      const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_res,
+                      const Params p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-    unsigned char* tilebuf = smem;                                   // 2 x TILE_BYTES
-    float* wsm = reinterpret_cast<float*>(smem + 2 * TILE_BYTES);    // merged kernel of the current unit
-    unsigned char* ring = smem + 2 * TILE_BYTES + WSM_BYTES;         // NSLOT x slot_stride
+    unsigned char* tilebuf = smem;                                            // 2 x TILE_BYTES
+    float* wsm = reinterpret_cast<float*>(smem + 2 * TILE_BYTES);             // merged kernel of the current (image, group)
+    float* lkc = reinterpret_cast<float*>(smem + 2 * TILE_BYTES + WSM_BYTES); // centre taps of LK^s alone
+    unsigned char* ring = smem + 2 * TILE_BYTES + WSM_BYTES + LKC_BYTES;      // NSLOT x slot_stride
     u64* bars = reinterpret_cast<u64*>(ring + NSLOT * p.slot_stride);
-    const uint32_t full0 = smem_u32(bars), cfull0 = smem_u32(bars + 2);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 2), cfull0 = smem_u32(bars + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
         mbar_init(full0, 1); mbar_init(full0 + 8, 1);
+        mbar_init(empty0, 1); mbar_init(empty0 + 8, 1);
         for (int s = 0; s < NSLOT; ++s) mbar_init(cfull0 + 8 * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
     const long long first = blockIdx.x, stride = gridDim.x;
+    const long long my_units = first < p.units ? (p.units - first + stride - 1) / stride : 0;
 
-    // ======================= copy warp: untouched channels, TMA in / TMA out ==================
-    if (warp == kComputeWarps) {
-        if (lane != 0 || p.copy_cc == 0) return;
-        const int per_row = TW / p.copy_cw, chunks = per_row * (TH / p.copy_cr);
-        const unsigned bytes = (unsigned)(p.copy_cc * p.copy_cw * p.copy_cr * 2);
-        long long issued = 0, stored = 0;
-        // chunk n of the CTA's stream -> (unit, chunk-in-unit); units with g != 0 copy nothing
-        auto coords = [&](long long n, int& cx, int& cy, int& cb) -> bool {
-            const long long u = first + (n / chunks) * stride;
-            const Unit un = decode_unit(u, p);
-            const int ch = (int)(n % chunks);
-            cx = un.tx * TW + (ch % per_row) * p.copy_cw;
-            cy = un.ty * TH + (ch / per_row) * p.copy_cr;
-            cb = un.b;
-            return un.g == 0 && cx < p.W && cy < p.H;
-        };
-        const long long my_units = first < p.units ? (p.units - first + stride - 1) / stride : 0;
-        const long long total = my_units * chunks;
-        bool alive = true;
-        // Software pipeline: the store of chunk n - COPY_DEPTH goes out first, then the load of
-        // chunk n is issued, so COPY_DEPTH - 1 loads are always in flight behind it.
-        for (long long n = 0; n < total + COPY_DEPTH; ++n) {
-            int cx, cy, cb;
-            const long long m = n - COPY_DEPTH;
-            if (m >= 0 && coords(m, cx, cy, cb)) {
-                const int slot = (int)(stored % NSLOT);
-                if (alive) alive = mbar_wait(cfull0 + 8 * slot, (unsigned)((stored / NSLOT) & 1), p.ctrl, 0xC0000000u | (unsigned)slot);
-                tma_store_4d(&map_cout, smem_u32(ring + slot * p.slot_stride), p.Ca, cx, cy, cb);
-                bulk_commit();
-                ++stored;
+    if (warp >= kComputeWarps) {
+        // ======================= helper warp group ================================================
+        reg_dec<kHelperRegs>();
+        if (lane != 0) return;
+        if (warp == kComputeWarps) {
+            // ---- tile producer: unit k goes to buffer k & 1 once its previous user has released it
+            bool alive = true;
+            for (long long k = 0; k < my_units; ++k) {
+                const int buf = (int)(k & 1);
+                if (k >= 2 && alive) alive = mbar_wait(empty0 + 8 * buf, (unsigned)(((k >> 1) - 1) & 1), p.ctrl, 0xB0000000u | (unsigned)buf);
+                const Unit un = decode_unit(first + k * stride, p);
+                mbar_expect_tx(full0 + 8 * buf, TILE_BYTES);
+                tma_load_4d(smem_u32(tilebuf + (size_t)buf * TILE_BYTES), &map_att, full0 + 8 * buf,
+                            un.g * CG, un.tx * TW - P6, un.ty * TH - P6, un.b);
             }
-            if (n < total && coords(n, cx, cy, cb)) {
-                const int slot = (int)(issued % NSLOT);
-                // the store that last used this slot is at least NSLOT - COPY_DEPTH + 1 groups back
-                bulk_wait_read<NSLOT - COPY_DEPTH>();
-                mbar_expect_tx(cfull0 + 8 * slot, bytes);
-                tma_load_4d(smem_u32(ring + slot * p.slot_stride), &map_cin, cfull0 + 8 * slot, p.Ca, cx, cy, cb);
-                ++issued;
+        } else if (warp == kComputeWarps + 1 && p.copy_cc != 0) {
+            // ---- copy-through of the untouched channels: TMA in, TMA out ---------------------------
+            const int per_row = TW / p.copy_cw, chunks = per_row * (TH / p.copy_cr);
+            const unsigned bytes = (unsigned)(p.copy_cc * p.copy_cw * p.copy_cr * 2);
+            long long issued = 0, stored = 0;
+            // chunk n of the CTA's stream -> (unit, chunk-in-unit); units with g != 0 copy nothing
+            auto coords = [&](long long n, int& cx, int& cy, int& cb) -> bool {
+                const Unit un = decode_unit(first + (n / chunks) * stride, p);
+                const int ch = (int)(n % chunks);
+                cx = un.tx * TW + (ch % per_row) * p.copy_cw;
+                cy = un.ty * TH + (ch / per_row) * p.copy_cr;
+                cb = un.b;
+                return un.g == 0 && cx < p.W && cy < p.H;
+            };
+            const long long total = my_units * chunks;
+            bool alive = true;
+            // Software pipeline: the store of chunk n - COPY_DEPTH goes out first, then the load of
+            // chunk n is issued, so COPY_DEPTH - 1 loads are always in flight behind it.
+            for (long long n = 0; n < total + COPY_DEPTH; ++n) {
+                int cx, cy, cb;
+                const long long m = n - COPY_DEPTH;
+                if (m >= 0 && coords(m, cx, cy, cb)) {
+                    const int slot = (int)(stored % NSLOT);
+                    if (alive) alive = mbar_wait(cfull0 + 8 * slot, (unsigned)((stored / NSLOT) & 1), p.ctrl, 0xC0000000u | (unsigned)slot);
+                    tma_store_4d(&map_cout, smem_u32(ring + slot * p.slot_stride), p.Ca, cx, cy, cb);
+                    bulk_commit();
+                    ++stored;
+                }
+                if (n < total && coords(n, cx, cy, cb)) {
+                    const int slot = (int)(issued % NSLOT);
+                    // the store that last used this slot is at least NSLOT - COPY_DEPTH + 1 groups back
+                    bulk_wait_read<NSLOT - COPY_DEPTH>();
+                    mbar_expect_tx(cfull0 + 8 * slot, bytes);
+                    tma_load_4d(smem_u32(ring + slot * p.slot_stride), &map_cin, cfull0 + 8 * slot, p.Ca, cx, cy, cb);
+                    ++issued;
+                }
             }
+            bulk_wait_all<0>();
         }
-        bulk_wait_all<0>();
         return;
     }
 
-    // ======================= compute warps ====================================================
-    const int q = lane >> 3, pr = lane & 7;                 // patch position in the warp, channel pair
-    const int lx = warp & (LXP - 1), ly = (warp >> 2) * 4 + q;
+    // ======================= compute warps ========================================================
+    reg_inc<kComputeRegs>();
+    const int q = lane >> 3, pr = lane & 7;                 // patch position in the warp's 2x2 block, channel pair
+    const int lx = 2 * (warp & 1) + (q & 1), ly = 2 * (warp >> 1) + (q >> 1);
     const int lane_word = ((ly * OY) * PITCH + lx * OX) * NPAIR + pr;
 
-    if (first < p.units && tid == 0) {
-        const Unit u0 = decode_unit(first, p);
-        mbar_expect_tx(full0, TILE_BYTES);
-        tma_load_4d(smem_u32(tilebuf), &map_att, full0, u0.g * CG, u0.tx * TW - P6, u0.ty * TH - P6, u0.b);
-    }
-
-    int cur_g = -1;
+    int cur_g = -1, cur_b = -1;
     bool alive = true;
-    long long k = 0;
-    for (long long u = first; u < p.units; u += stride, ++k) {
-        const Unit un = decode_unit(u, p);
+    for (long long k = 0; k < my_units; ++k) {
+        const Unit un = decode_unit(first + k * stride, p);
         const int buf = (int)(k & 1);
 
-        // ---- large-kernel taps of this channel group -> shared (fp32, pair-interleaved) -------
-        if (un.g != cur_g) {
+        // ---- merged kernel ZP(dk) + LK^s (Eq. 5) of this (image, channel group) -> shared, fp32 ----
+        if (un.g != cur_g || un.b != cur_b) {
             if (cur_g >= 0) compute_bar();                  // everyone is done with the old table
-            for (int t = tid; t < K13 * 14 * CG; t += kComputeThreads) {
-                const int c = t % CG, j = (t / CG) % 14, i = t / (CG * 14);
-                float w = 0.f;
-                if (j < K13) w = __bfloat162float(p.w_large[((size_t)(un.g * CG + c) * K13 + i) * K13 + j]);
-                wsm[((i * 7 + (j >> 1)) * NPAIR + (c >> 1)) * 4 + (j & 1) * 2 + (c & 1)] = w;
+            if (un.g != cur_g) {
+                const __nv_bfloat16* wg = p.w_large + (size_t)un.g * CG * K13 * K13;
+                constexpr int N = CG * K13 * K13, PER = (N + kComputeThreads - 1) / kComputeThreads;
+                float v[PER];
+#pragma unroll
+                for (int t = 0; t < PER; ++t) {             // coalesced, all loads in flight together
+                    const int idx = tid + t * kComputeThreads;
+                    v[t] = idx < N ? __bfloat162float(wg[idx]) : 0.f;
+                }
+#pragma unroll
+                for (int t = 0; t < PER; ++t) {
+                    const int idx = tid + t * kComputeThreads;
+                    if (idx < N) {
+                        const int c = idx / (K13 * K13), tap = idx % (K13 * K13), i = tap / K13, j = tap % K13;
+                        wsm[wsm_index(c, i, j)] = v[t];
+                        if (i >= 5 && i <= 7 && j >= 5 && j <= 7) lkc[c * 9 + (i - 5) * 3 + (j - 5)] = v[t];
+                    }
+                }
+                if (tid < CG * K13) wsm[wsm_index(tid / K13, tid % K13, K13)] = 0.f;   // pad tap 13
+                compute_bar();
             }
-            cur_g = un.g;
+            if (cur_g < 0) pdl_wait_primary();              // dk is written by the preceding kernel
+            if (tid < CG * 9) {
+                const int c = tid / 9, tap = tid % 9;
+                wsm[wsm_index(c, 5 + tap / 3, 5 + tap % 3)] =
+                    lkc[tid] + p.dk[((size_t)un.b * p.Ca + un.g * CG + c) * 9 + tap];
+            }
+            cur_g = un.g; cur_b = un.b;
             compute_bar();
         }
 
@@ -232,79 +281,75 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
 #pragma unroll
             for (int c = 0; c < OX; ++c) acc[a][c] = 0ull;
 
-        const uint32_t* tw = reinterpret_cast<const uint32_t*>(tilebuf + (size_t)buf * TILE_BYTES) + lane_word;
+        unsigned char* tbuf = tilebuf + (size_t)buf * TILE_BYTES;
+        const uint32_t* tw = reinterpret_cast<const uint32_t*>(tbuf) + lane_word;
+        const float4* wlane = reinterpret_cast<const float4*>(wsm) + pr;
+
+        uint32_t nxt[NW];
+#pragma unroll
+        for (int kk = 0; kk < NW; ++kk) nxt[kk] = tw[kk * NPAIR];
 
 #pragma unroll 1
-        for (int s = 0; s < K13; ++s) {
-            const int i = row_order(s);
-            if (s == 10) {
-                // All warps have finished the previous unit (its buffer and its merged rows are free).
-                compute_bar();
-                if (tid == 0 && u + stride < p.units) {     // prefetch the next unit's tile
-                    const Unit nx = decode_unit(u + stride, p);
-                    mbar_expect_tx(full0 + 8 * (buf ^ 1), TILE_BYTES);
-                    tma_load_4d(smem_u32(tilebuf + (size_t)(buf ^ 1) * TILE_BYTES), &map_att, full0 + 8 * (buf ^ 1),
-                                nx.g * CG, nx.tx * TW - P6, nx.ty * TH - P6, nx.b);
-                }
-                if (k == 0) pdl_wait_primary();             // dk is written by the preceding kernel
-                if (tid < CG * 9) {                          // rows 5-7, columns 5-7: LK^s + dk  (Eq. 5)
-                    const int c = tid / 9, tap = tid % 9, ii = 5 + tap / 3, jj = 5 + tap % 3;
-                    const float w = __bfloat162float(p.w_large[((size_t)(un.g * CG + c) * K13 + ii) * K13 + jj]) +
-                                    p.dk[((size_t)un.b * p.Ca + un.g * CG + c) * 9 + tap];
-                    wsm[((ii * 7 + (jj >> 1)) * NPAIR + (c >> 1)) * 4 + (jj & 1) * 2 + (c & 1)] = w;
-                }
-                compute_bar();
-            }
-            // kernel row i for this lane's channel pair: 13 packed taps
-            u64 w[K13];
-            {
-                const float4* wr = reinterpret_cast<const float4*>(wsm) + (i * 7) * NPAIR + pr;
+        for (int r = 0; r < NR; ++r) {
+            // input row r of the patch window: widen to fp32 pairs once, prefetch the next row
+            u64 in[NW];
 #pragma unroll
-                for (int jj = 0; jj < 7; ++jj) {
-                    const float4 v = wr[jj * NPAIR];
-                    w[2 * jj] = pack2(v.x, v.y);
-                    if (2 * jj + 1 < K13) w[2 * jj + 1] = pack2(v.z, v.w);
-                }
+            for (int kk = 0; kk < NW; ++kk)
+                in[kk] = pack2(__uint_as_float(nxt[kk] << 16), __uint_as_float(nxt[kk] & 0xffff0000u));
+            if (r + 1 < NR) {
+                const uint32_t* rn = tw + (r + 1) * (PITCH * NPAIR);
+#pragma unroll
+                for (int kk = 0; kk < NW; ++kk) nxt[kk] = rn[kk * NPAIR];
             }
-            const uint32_t* trow = tw + i * (PITCH * NPAIR);
 #pragma unroll
             for (int oy = 0; oy < OY; ++oy) {
-                const uint32_t* r = trow + oy * (PITCH * NPAIR);
+                const int i = r - oy;                       // kernel row that maps input row r to output row oy
+                if (i >= 0 && i < K13) {                    // same for the whole warp
+                    u64 w[K13];
+                    const float4* wr = wlane + i * (7 * NPAIR);
 #pragma unroll
-                for (int kk = 0; kk < OX + K13 - 1; ++kk) {
-                    const uint32_t v = r[kk * NPAIR];
-                    const u64 in = pack2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+                    for (int jj = 0; jj < 7; ++jj) {
+                        const float4 v = wr[jj * NPAIR];
+                        w[2 * jj] = pack2(v.x, v.y);
+                        if (2 * jj + 1 < K13) w[2 * jj + 1] = pack2(v.z, v.w);
+                    }
 #pragma unroll
-                    for (int j = 0; j < K13; ++j) {
-                        const int ox = kk - j;
-                        if (ox >= 0 && ox < OX) fma2(acc[oy][ox], w[j], in);
+                    for (int kk = 0; kk < NW; ++kk) {
+#pragma unroll
+                        for (int j = 0; j < K13; ++j) {
+                            const int ox = kk - j;
+                            if (ox >= 0 && ox < OX) fma2(acc[oy][ox], w[j], in[kk]);
+                        }
                     }
                 }
             }
         }
 
-        // ---- epilogue: one rounding to bf16, 4-byte stores (8 lanes = one 32-byte sector) -----
-        const int y0 = un.ty * TH + ly * OY, x0 = un.tx * TW + lx * OX;
-        uint32_t* ow = reinterpret_cast<uint32_t*>(p.out) + un.g * NPAIR + pr;
-        const size_t cw = (size_t)p.C / 2;
+        // ---- epilogue: round once to bf16, stage the 40x40x16 result in the freed input buffer,
+        //      one TMA store (the TMA unit clips at the image border) ---------------------------
+        compute_bar();                                       // every warp has finished reading this buffer
+        {
+            uint32_t* sw = reinterpret_cast<uint32_t*>(tbuf) + ((ly * OY) * TW + lx * OX) * NPAIR + pr;
 #pragma unroll
-        for (int oy = 0; oy < OY; ++oy) {
-            const int y = y0 + oy;
-            if (y < p.H) {
-                const size_t rowbase = ((size_t)un.b * p.H + y) * p.W;
+            for (int oy = 0; oy < OY; ++oy)
 #pragma unroll
                 for (int ox = 0; ox < OX; ++ox) {
-                    const int x = x0 + ox;
-                    if (x < p.W) {
-                        float lo, hi;
-                        unpack2(acc[oy][ox], lo, hi);
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-                        ow[(rowbase + x) * cw] = *reinterpret_cast<const uint32_t*>(&h);
-                    }
+                    float lo, hi;
+                    unpack2(acc[oy][ox], lo, hi);
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+                    sw[(oy * TW + ox) * NPAIR] = *reinterpret_cast<const uint32_t*>(&h);
                 }
-            }
+        }
+        fence_async_smem();
+        compute_bar();
+        if (tid == 0) {
+            tma_store_4d(&map_res, smem_u32(tbuf), un.g * CG, un.tx * TW, un.ty * TH, un.b);
+            bulk_commit();
+            bulk_wait_read<0>();                             // the buffer may be refilled now
+            mbar_arrive(empty0 + 8 * buf);
         }
     }
+    if (tid == 0) bulk_wait_all<0>();
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -374,11 +419,11 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     }
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
     p.dk = dk;
-    p.out = static_cast<__nv_bfloat16*>(out);
     p.ctrl = ctrl;
 
-    CUtensorMap m_att, m_cin, m_cout;
+    CUtensorMap m_att, m_cin, m_cout, m_res;
     if (!make_map(&m_att, x, B, C, H, W, CG, PITCH, THP)) return kNotApplicable;
+    if (!make_map(&m_res, out, B, C, H, W, CG, TW, TH)) return kNotApplicable;
     if (cc > 0) {
         if (!make_map(&m_cin, x, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
         if (!make_map(&m_cout, out, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
@@ -386,7 +431,7 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
         m_cin = m_att; m_cout = m_att;
     }
 
-    const size_t smem = 128 + 2 * (size_t)TILE_BYTES + WSM_BYTES + (size_t)NSLOT * p.slot_stride + 64;
+    const size_t smem = 128 + 2 * (size_t)TILE_BYTES + WSM_BYTES + LKC_BYTES + (size_t)NSLOT * p.slot_stride + 128;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -406,7 +451,7 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16, m_att, m_cin, m_cout, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16, m_att, m_cin, m_cout, m_res, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_tma_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
