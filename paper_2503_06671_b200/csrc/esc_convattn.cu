@@ -120,7 +120,8 @@ int launch_gap_t(const Problem& p, const void* x, const void* w_dyn, const void*
                  const Workspace& w, float* dk_out, cudaStream_t st) {
     const int S = slabs_for(p.B, (long long)p.H * p.W);
     dim3 grid(S, p.B);
-    const size_t smem = (size_t)(esc::kGapWarps + 1) * p.Ca * sizeof(float);
+    const size_t scratch = (size_t)esc::kGapWarps * p.Ca > (size_t)esc::kGapThreads ? (size_t)esc::kGapWarps * p.Ca : (size_t)esc::kGapThreads;
+    const size_t smem = (scratch + p.Ca) * sizeof(float);
     if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
     esc::gap_dynkernel<T, LAYOUT><<<grid, esc::kGapThreads, smem, st>>>(
         static_cast<const T*>(x), p.C, p.Ca, p.H, p.W, S, static_cast<const T*>(w_dyn),

@@ -26,9 +26,9 @@ gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
               float* __restrict__ dk)          // [B][9*Ca]
 {
     constexpr int V = Elem<T>::kVec;
-    extern __shared__ float smem[];            // [kGapWarps][Ca] warp sums, then [Ca] means
+    extern __shared__ float smem[];            // max(kGapWarps*Ca, kGapThreads) floats of scratch, then [Ca] means
     float* wsum = smem;
-    float* gmean = smem + kGapWarps * Ca;
+    float* gmean = smem + (kGapWarps * Ca > kGapThreads ? kGapWarps * Ca : kGapThreads);
     __shared__ bool is_last;
 
     pdl_launch_dependents();                   // the stencil kernel may start its prologue now
@@ -49,24 +49,20 @@ gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
 #pragma unroll
         for (int v = 0; v < V; ++v) acc[v] = 0.f;
         const T* base = x + ((size_t)b * HW) * C + (size_t)chunk * V;
-        long long p = p0 + tid / cpp;
-        for (; p + 3LL * ppb < p1; p += 4LL * ppb) {      // four independent loads in flight
-            uint4 q[4];
+        for (long long p = p0 + tid / cpp; p < p1; p += 8LL * ppb) {   // eight independent loads in flight
+            uint4 q[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) q[u] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(p + (long long)u * ppb) * C));
+            for (int u = 0; u < 8; ++u) {
+                const long long pu = p + (long long)u * ppb;
+                q[u] = pu < p1 ? __ldg(reinterpret_cast<const uint4*>(base + (size_t)pu * C)) : make_uint4(0u, 0u, 0u, 0u);
+            }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 float f[V];
                 unpack16<T>(q[u], f);
 #pragma unroll
                 for (int v = 0; v < V; ++v) acc[v] += f[v];
             }
-        }
-        for (; p < p1; p += ppb) {
-            float f[V];
-            unpack16<T>(__ldg(reinterpret_cast<const uint4*>(base + (size_t)p * C)), f);
-#pragma unroll
-            for (int v = 0; v < V; ++v) acc[v] += f[v];
         }
         // lanes with equal (lane % cpp) hold the same channels: butterfly over the other lane bits
 #pragma unroll
@@ -138,17 +134,50 @@ gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
     if (!is_last) return;
     __threadfence();
     const float inv_hw = 1.0f / (float)HW;
-    for (int c = tid; c < Ca; c += kGapThreads) {
-        const float* pp = partial + (size_t)b * S * Ca + c;
-        float t = 0.f;
-        for (int k = 0; k < S; ++k) t += __ldcg(pp + (size_t)k * Ca);      // fixed slab order
-        gmean[c] = t * inv_hw;
+    // S partial sums per channel, added in a fixed two-level order: group j takes slabs j, j+ng, ...
+    // (all threads busy, loads independent), then the ng group sums are added in order.
+    const int ng = Ca <= kGapThreads / 2 ? kGapThreads / Ca : 1;
+    if (ng > 1) {
+        float* red = wsum;                                   // [ng][Ca] <= 256 floats; the warp sums are dead
+        const int c = tid % Ca, j = tid / Ca;
+        if (j < ng) {
+            const float* pp = partial + (size_t)b * S * Ca + c;
+            float t = 0.f;
+            for (int k = j; k < S; k += 8 * ng) {            // eight independent loads, added in order
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = k + u * ng < S ? __ldcg(pp + (size_t)(k + u * ng) * Ca) : 0.f;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) t += v[u];
+            }
+            red[j * Ca + c] = t;
+        }
+        __syncthreads();
+        if (tid < Ca) {
+            float t = 0.f;
+            for (int j2 = 0; j2 < ng; ++j2) t += red[j2 * Ca + tid];
+            gmean[tid] = t * inv_hw;
+        }
+    } else {
+        for (int c = tid; c < Ca; c += kGapThreads) {
+            const float* pp = partial + (size_t)b * S * Ca + c;
+            float t = 0.f;
+            for (int k = 0; k < S; ++k) t += __ldcg(pp + (size_t)k * Ca);
+            gmean[c] = t * inv_hw;
+        }
     }
     __syncthreads();
     for (int o = tid; o < 9 * Ca; o += kGapThreads) {
         float acc = Elem<T>::to_f32(b_dyn[o]);
         const T* wr = w_dyn + (size_t)o * Ca;
-        for (int c = 0; c < Ca; ++c) acc = fmaf(Elem<T>::to_f32(wr[c]), gmean[c], acc);
+        for (int c0 = 0; c0 < Ca; c0 += 16) {                // sixteen independent loads, FMAs in channel order
+            float wv[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u) wv[u] = c0 + u < Ca ? Elem<T>::to_f32(wr[c0 + u]) : 0.f;
+#pragma unroll
+            for (int u = 0; u < 16; ++u)
+                if (c0 + u < Ca) acc = fmaf(wv[u], gmean[c0 + u], acc);
+        }
         dk[(size_t)b * 9 * Ca + o] = acc;
     }
 }

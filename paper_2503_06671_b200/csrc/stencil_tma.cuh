@@ -48,7 +48,7 @@ constexpr int NPAIR = CG / 2;
 constexpr int kComputeWarps = LXP * LYP / 4;         // 8
 constexpr int kComputeThreads = kComputeWarps * 32;  // 256
 constexpr int kThreads = kComputeThreads + 128;      // + helper warp group (producer, copy, 2 idle)
-constexpr int kComputeRegs = 232, kHelperRegs = 24;
+constexpr int kComputeRegs = 232, kHelperRegs = 40;   // 256*232 + 128*40 = 64,512 <= 65,536
 constexpr int TILE_BYTES = THP * PITCH * CG * 2;     // 88,192
 constexpr int OUT_TILE_BYTES = TH * TW * CG * 2;     // 51,200: staged result, reuses the input buffer
 constexpr int WSM_FLOATS = K13 * 7 * NPAIR * 4;      // [i][jj][pair][4]: taps 2jj,2jj+1 of both channels
@@ -56,7 +56,8 @@ constexpr int WSM_BYTES = (WSM_FLOATS * 4 + 127) / 128 * 128;
 constexpr int LKC_BYTES = (CG * 9 * 4 + 127) / 128 * 128;   // pristine centre 3x3 of LK^s
 constexpr int NSLOT = 4, COPY_DEPTH = 3;             // copy ring: slots, loads in flight
 constexpr int kMaxSlotBytes = 8192;
-constexpr unsigned kSpinLimit = 1u << 22;
+constexpr unsigned kSpinLimit = 1u << 20;    // polls before a wait gives up (each poll may suspend up to the hint)
+constexpr unsigned kSuspendHintNs = 20000;
 
 static_assert(TILE_BYTES % 128 == 0, "tile buffers must keep 128-byte alignment");
 static_assert(OUT_TILE_BYTES <= TILE_BYTES, "the result tile is staged in the input buffer");
@@ -84,21 +85,21 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, unsigned bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// One poll of a phase; the thread is suspended by the hardware until the phase completes or the
+// time hint (ns) runs out, so a waiting thread issues almost no instructions.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity) {
     unsigned ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
     return ok != 0;
 }
 // Bounded wait: gives up after kSpinLimit polls, records where, and lets the caller carry on.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, unsigned parity, unsigned* ctrl, unsigned where) {
-    for (unsigned n = 0; n < kSpinLimit; ++n) {
+    for (unsigned n = 0; n < kSpinLimit; ++n)
         if (mbar_try_wait(bar, parity)) return true;
-        if (n > 64) __nanosleep(64);
-    }
     if (ctrl) { atomicExch(ctrl, kDevTimeout); atomicExch(ctrl + 1, where); }
     return false;
 }
@@ -130,12 +131,13 @@ __device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) { asm("mov.
 __device__ __forceinline__ void fma2(u64& d, u64 a, u64 b) { asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b)); }
 
 struct Unit { int b, g, ty, tx; };
-__device__ __forceinline__ Unit decode_unit(long long u, const Params& p) {
+__device__ __forceinline__ Unit decode_unit(long long u64v, const Params& p) {
+    unsigned u = (unsigned)u64v;                             // the host guarantees units < 2^31
     Unit r;
-    r.tx = (int)(u % p.tiles_x); u /= p.tiles_x;
-    r.ty = (int)(u % p.tiles_y); u /= p.tiles_y;
-    r.g = (int)(u % p.groups);
-    r.b = (int)(u / p.groups);
+    r.tx = (int)(u % (unsigned)p.tiles_x); u /= (unsigned)p.tiles_x;
+    r.ty = (int)(u % (unsigned)p.tiles_y); u /= (unsigned)p.tiles_y;
+    r.g = (int)(u % (unsigned)p.groups);
+    r.b = (int)(u / (unsigned)p.groups);
     return r;
 }
 
@@ -148,8 +150,9 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
                       const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_res,
                       const Params p)
 {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    // The dynamic shared window starts 1024-byte aligned; indexing it directly (no pointer rounding
+    // through integers) lets the compiler keep every access in the shared address space.
+    extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* tilebuf = smem;                                            // 2 x TILE_BYTES
     float* wsm = reinterpret_cast<float*>(smem + 2 * TILE_BYTES);             // merged kernel of the current (image, group)
     float* lkc = reinterpret_cast<float*>(smem + 2 * TILE_BYTES + WSM_BYTES); // centre taps of LK^s alone
@@ -187,39 +190,56 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
             }
         } else if (warp == kComputeWarps + 1 && p.copy_cc != 0) {
             // ---- copy-through of the untouched channels: TMA in, TMA out ---------------------------
+            // Two cursors walk the CTA's chunk stream (units in order, chunks row-major inside a
+            // unit): the load cursor runs COPY_DEPTH chunks ahead of the store cursor.  No division
+            // in the loop: this thread competes with FMA-bound warps for issue slots.
+            struct Cursor {
+                int k, ch, cx0, cy0, cb, col, row; bool live;
+                __device__ void enter_unit(const Params& p, int first, int stride) {
+                    const Unit un = decode_unit(first + k * stride, p);
+                    cx0 = un.tx * TW; cy0 = un.ty * TH; cb = un.b; col = 0; row = 0; ch = 0;
+                    live = un.g == 0;
+                }
+            };
             const int per_row = TW / p.copy_cw, chunks = per_row * (TH / p.copy_cr);
             const unsigned bytes = (unsigned)(p.copy_cc * p.copy_cw * p.copy_cr * 2);
-            long long issued = 0, stored = 0;
-            // chunk n of the CTA's stream -> (unit, chunk-in-unit); units with g != 0 copy nothing
-            auto coords = [&](long long n, int& cx, int& cy, int& cb) -> bool {
-                const Unit un = decode_unit(first + (n / chunks) * stride, p);
-                const int ch = (int)(n % chunks);
-                cx = un.tx * TW + (ch % per_row) * p.copy_cw;
-                cy = un.ty * TH + (ch / per_row) * p.copy_cr;
-                cb = un.b;
-                return un.g == 0 && cx < p.W && cy < p.H;
+            const int nunits = (int)my_units, first_i = (int)first, stride_i = (int)stride;
+            Cursor ld, st;
+            ld.k = st.k = 0;
+            if (nunits > 0) { ld.enter_unit(p, first_i, stride_i); st = ld; }
+            auto advance = [&](Cursor& c) {
+                ++c.ch;
+                if (++c.col == per_row) { c.col = 0; ++c.row; }
+                if (c.ch == chunks) { ++c.k; if (c.k < nunits) c.enter_unit(p, first_i, stride_i); }
             };
-            const long long total = my_units * chunks;
+            int issued = 0, stored = 0, lag = 0;
             bool alive = true;
-            // Software pipeline: the store of chunk n - COPY_DEPTH goes out first, then the load of
-            // chunk n is issued, so COPY_DEPTH - 1 loads are always in flight behind it.
-            for (long long n = 0; n < total + COPY_DEPTH; ++n) {
-                int cx, cy, cb;
-                const long long m = n - COPY_DEPTH;
-                if (m >= 0 && coords(m, cx, cy, cb)) {
-                    const int slot = (int)(stored % NSLOT);
-                    if (alive) alive = mbar_wait(cfull0 + 8 * slot, (unsigned)((stored / NSLOT) & 1), p.ctrl, 0xC0000000u | (unsigned)slot);
-                    tma_store_4d(&map_cout, smem_u32(ring + slot * p.slot_stride), p.Ca, cx, cy, cb);
-                    bulk_commit();
-                    ++stored;
+            while (st.k < nunits) {
+                // store the oldest chunk once COPY_DEPTH loads are in flight (or nothing is left to load)
+                if (lag == COPY_DEPTH || ld.k >= nunits) {
+                    const int cx = st.cx0 + st.col * p.copy_cw, cy = st.cy0 + st.row * p.copy_cr;
+                    if (st.live && cx < p.W && cy < p.H) {
+                        const int slot = stored % NSLOT;
+                        if (alive) alive = mbar_wait(cfull0 + 8 * slot, (unsigned)((stored / NSLOT) & 1), p.ctrl, 0xC0000000u | (unsigned)slot);
+                        tma_store_4d(&map_cout, smem_u32(ring + slot * p.slot_stride), p.Ca, cx, cy, st.cb);
+                        bulk_commit();
+                        ++stored;
+                    }
+                    advance(st);
+                    --lag;
                 }
-                if (n < total && coords(n, cx, cy, cb)) {
-                    const int slot = (int)(issued % NSLOT);
-                    // the store that last used this slot is at least NSLOT - COPY_DEPTH + 1 groups back
-                    bulk_wait_read<NSLOT - COPY_DEPTH>();
-                    mbar_expect_tx(cfull0 + 8 * slot, bytes);
-                    tma_load_4d(smem_u32(ring + slot * p.slot_stride), &map_cin, cfull0 + 8 * slot, p.Ca, cx, cy, cb);
-                    ++issued;
+                if (ld.k < nunits) {
+                    const int cx = ld.cx0 + ld.col * p.copy_cw, cy = ld.cy0 + ld.row * p.copy_cr;
+                    if (ld.live && cx < p.W && cy < p.H) {
+                        const int slot = issued % NSLOT;
+                        // the store that last used this slot is at least NSLOT - COPY_DEPTH + 1 groups back
+                        bulk_wait_read<NSLOT - COPY_DEPTH>();
+                        mbar_expect_tx(cfull0 + 8 * slot, bytes);
+                        tma_load_4d(smem_u32(ring + slot * p.slot_stride), &map_cin, cfull0 + 8 * slot, p.Ca, cx, cy, ld.cb);
+                        ++issued;
+                    }
+                    advance(ld);
+                    ++lag;
                 }
             }
             bulk_wait_all<0>();
@@ -285,21 +305,15 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
         const uint32_t* tw = reinterpret_cast<const uint32_t*>(tbuf) + lane_word;
         const float4* wlane = reinterpret_cast<const float4*>(wsm) + pr;
 
-        uint32_t nxt[NW];
-#pragma unroll
-        for (int kk = 0; kk < NW; ++kk) nxt[kk] = tw[kk * NPAIR];
-
 #pragma unroll 1
         for (int r = 0; r < NR; ++r) {
-            // input row r of the patch window: widen to fp32 pairs once, prefetch the next row
+            // input row r of the patch window: read once, widen to fp32 pairs once
             u64 in[NW];
+            const uint32_t* rn = tw + r * (PITCH * NPAIR);
 #pragma unroll
-            for (int kk = 0; kk < NW; ++kk)
-                in[kk] = pack2(__uint_as_float(nxt[kk] << 16), __uint_as_float(nxt[kk] & 0xffff0000u));
-            if (r + 1 < NR) {
-                const uint32_t* rn = tw + (r + 1) * (PITCH * NPAIR);
-#pragma unroll
-                for (int kk = 0; kk < NW; ++kk) nxt[kk] = rn[kk * NPAIR];
+            for (int kk = 0; kk < NW; ++kk) {
+                const uint32_t v = rn[kk * NPAIR];
+                in[kk] = pack2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
             }
 #pragma unroll
             for (int oy = 0; oy < OY; ++oy) {
@@ -407,6 +421,7 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
     p.tiles_x = (W + TW - 1) / TW; p.tiles_y = (H + TH - 1) / TH; p.groups = Ca / CG;
     p.units = (long long)B * p.groups * p.tiles_x * p.tiles_y;
+    if (p.units > 0x7fffffffLL) return kNotApplicable;
     p.copy_cc = cc; p.copy_cw = TW; p.copy_cr = 2; p.slot_stride = 128;
     if (cc > 0) {
         static const int shapes[5][2] = {{40, 2}, {40, 1}, {20, 1}, {10, 1}, {5, 1}};
@@ -431,7 +446,7 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
         m_cin = m_att; m_cout = m_att;
     }
 
-    const size_t smem = 128 + 2 * (size_t)TILE_BYTES + WSM_BYTES + LKC_BYTES + (size_t)NSLOT * p.slot_stride + 128;
+    const size_t smem = 2 * (size_t)TILE_BYTES + WSM_BYTES + LKC_BYTES + (size_t)NSLOT * p.slot_stride + 128;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
