@@ -79,8 +79,8 @@ struct Workspace {
 };
 
 int slabs_for(int B, long long HW) {
-    // about two blocks per SM over the whole batch, at least 512 pixels per slab
-    long long s = (2 * 148 + B - 1) / B;
+    // about one work item per SM over the whole batch, at least 512 pixels per slab
+    long long s = (148 + B - 1) / B;
     const long long cap = (HW + 511) / 512;
     if (s > cap) s = cap;
     if (s > esc::kMaxSlabs) s = esc::kMaxSlabs;
@@ -119,12 +119,23 @@ template <typename T, int LAYOUT>
 int launch_gap_t(const Problem& p, const void* x, const void* w_dyn, const void* b_dyn,
                  const Workspace& w, float* dk_out, cudaStream_t st) {
     const int S = slabs_for(p.B, (long long)p.H * p.W);
-    dim3 grid(S, p.B);
+    int sms = esc::tma::sm_count();
+    if (sms <= 0) sms = 148;
+    const long long items = (long long)p.B * S;
+    const unsigned grid = (unsigned)(items < sms ? items : sms);   // persistent, at most one block per SM
     const size_t scratch = (size_t)esc::kGapWarps * p.Ca > (size_t)esc::kGapThreads ? (size_t)esc::kGapWarps * p.Ca : (size_t)esc::kGapThreads;
     const size_t smem = (scratch + p.Ca) * sizeof(float);
     if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
+    // Same shared-memory carve-out as the stencil kernel: an SM changes its L1/shared split only
+    // when idle, so with different preferences the two kernels could never share an SM.
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        ESC_CUDA(cudaFuncSetAttribute(esc::gap_dynkernel<T, LAYOUT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      cudaSharedmemCarveoutMaxShared));
+        carveout_set = true;
+    }
     esc::gap_dynkernel<T, LAYOUT><<<grid, esc::kGapThreads, smem, st>>>(
-        static_cast<const T*>(x), p.C, p.Ca, p.H, p.W, S, static_cast<const T*>(w_dyn),
+        static_cast<const T*>(x), p.B, p.C, p.Ca, p.H, p.W, S, static_cast<const T*>(w_dyn),
         static_cast<const T*>(b_dyn), w.partial, w.arrivals, dk_out);
     ESC_CUDA(cudaGetLastError());
     ++g_last_launches;
@@ -133,7 +144,7 @@ int launch_gap_t(const Problem& p, const void* x, const void* w_dyn, const void*
 
 int launch_gap(const Problem& p, const void* x, const void* w_dyn, const void* b_dyn,
                const Workspace& w, float* dk_out, cudaStream_t st) {
-    if (p.B > 65535) return ESC_ERR_UNSUPPORTED;
+    if ((long long)p.B * esc::kMaxSlabs > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
     if (p.dtype == ESC_F32)
         return p.layout == ESC_NCHW ? launch_gap_t<float, esc::kNCHW>(p, x, w_dyn, b_dyn, w, dk_out, st)
                                     : launch_gap_t<float, esc::kNHWC>(p, x, w_dyn, b_dyn, w, dk_out, st);

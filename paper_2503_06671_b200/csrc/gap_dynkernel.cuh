@@ -4,22 +4,27 @@
 //   g[b,c]  = (1/HW) sum_{y,x} x[b,c,y,x]            c < C_a
 //   dk[b,o] = b_dyn[o] + sum_c w_dyn[o,c] g[b,c]     o = c*9 + i*3 + j
 //
-// Grid (S, B): every image is cut into S slabs so that a single large image still fills the
-// machine.  A block reduces its slab with 16-byte loads, warp shuffles and one pass through
-// shared memory, and writes C_a partial sums.  The block that arrives last for an image (a
-// wrapping arrival counter, so no counter ever needs re-zeroing) adds the S partial sums in slab
-// order -- the result is bitwise reproducible -- and evaluates the linear layer.
+// Every image is cut into S slabs so that a single large image still spreads over the machine;
+// the B*S work items are walked by a persistent grid of small blocks (3 warps, at most one block
+// per SM).  The blocks are kept this small on purpose: the stencil kernel is launched as a
+// programmatic dependent of this one and needs nearly a whole SM per block, so the two kernels
+// can only run side by side -- this one bound by DRAM, the other by the FMA pipe -- if this one
+// leaves the registers and shared memory free.  A block reduces a slab with 16-byte loads, warp
+// shuffles and one pass through shared memory, and writes C_a partial sums.  The block that
+// arrives last for an image (a wrapping arrival counter, so no counter ever needs re-zeroing)
+// adds the S partial sums in a fixed order -- the result is bitwise reproducible -- and
+// evaluates the linear layer.
 #pragma once
 #include "common.cuh"
 
 namespace esc {
 
-constexpr int kGapThreads = 256;
+constexpr int kGapThreads = 96;
 constexpr int kGapWarps = kGapThreads / 32;
 
 template <typename T, int LAYOUT>
-__global__ void __launch_bounds__(kGapThreads)
-gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
+__global__ void __maxnreg__(56)
+gap_dynkernel(const T* __restrict__ x, int B, int C, int Ca, int H, int W, int S,
               const T* __restrict__ w_dyn, const T* __restrict__ b_dyn,
               float* __restrict__ partial,     // [B][S][Ca]
               unsigned* __restrict__ arrivals, // [B]
@@ -33,9 +38,10 @@ gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
 
     pdl_launch_dependents();                   // the stencil kernel may start its prologue now
 
-    const int s = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long HW = (long long)H * W;
+    for (int item = blockIdx.x; item < B * S; item += gridDim.x) {
+    const int b = item / S, s = item - b * S;
     float* my_partial = partial + ((size_t)b * S + s) * Ca;
 
     const int cpp = Ca / V;                    // 16-byte chunks per pixel (NHWC)
@@ -131,7 +137,7 @@ gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
         is_last = (old == (unsigned)(S - 1));
     }
     __syncthreads();
-    if (!is_last) return;
+    if (!is_last) continue;
     __threadfence();
     const float inv_hw = 1.0f / (float)HW;
     // S partial sums per channel, added in a fixed two-level order: group j takes slabs j, j+ng, ...
@@ -179,6 +185,8 @@ gap_dynkernel(const T* __restrict__ x, int C, int Ca, int H, int W, int S,
                 if (c0 + u < Ca) acc = fmaf(wv[u], gmean[c0 + u], acc);
         }
         dk[(size_t)b * 9 * Ca + o] = acc;
+    }
+    __syncthreads();                                         // scratch and flag are reused by the next item
     }
 }
 

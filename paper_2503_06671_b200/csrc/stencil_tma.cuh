@@ -48,12 +48,13 @@ constexpr int NPAIR = CG / 2;
 constexpr int kComputeWarps = LXP * LYP / 4;         // 8
 constexpr int kComputeThreads = kComputeWarps * 32;  // 256
 constexpr int kThreads = kComputeThreads + 128;      // + helper warp group (producer, copy, 2 idle)
-constexpr int kComputeRegs = 232, kHelperRegs = 40;   // 256*232 + 128*40 = 64,512 <= 65,536
+constexpr int kLaunchRegs = 152;                      // 384*152 = 58,368: leaves 7,168 registers for one GAP block (96 x 64) per SM
+constexpr int kComputeRegs = 208, kHelperRegs = 40;   // after reallocation: 256*208 + 128*40 = 58,368
 constexpr int TILE_BYTES = THP * PITCH * CG * 2;     // 88,192
 constexpr int OUT_TILE_BYTES = TH * TW * CG * 2;     // 51,200: staged result, reuses the input buffer
 constexpr int WSM_FLOATS = K13 * 7 * NPAIR * 4;      // [i][jj][pair][4]: taps 2jj,2jj+1 of both channels
 constexpr int WSM_BYTES = (WSM_FLOATS * 4 + 127) / 128 * 128;
-constexpr int LKC_BYTES = (CG * 9 * 4 + 127) / 128 * 128;   // pristine centre 3x3 of LK^s
+constexpr int LKC_BYTES = (CG * 9 * 4 + 127) / 128 * 128;
 constexpr int NSLOT = 4, COPY_DEPTH = 3;             // copy ring: slots, loads in flight
 constexpr int kMaxSlotBytes = 8192;
 constexpr unsigned kSpinLimit = 1u << 20;    // polls before a wait gives up (each poll may suspend up to the hint)
@@ -145,7 +146,7 @@ __device__ __forceinline__ int wsm_index(int c, int i, int j) {
     return ((i * 7 + (j >> 1)) * NPAIR + (c >> 1)) * 4 + (j & 1) * 2 + (c & 1);
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __maxnreg__(kLaunchRegs)
 stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
                       const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_res,
                       const Params p)
@@ -154,8 +155,8 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
     // through integers) lets the compiler keep every access in the shared address space.
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* tilebuf = smem;                                            // 2 x TILE_BYTES
-    float* wsm = reinterpret_cast<float*>(smem + 2 * TILE_BYTES);             // merged kernel of the current (image, group)
-    float* lkc = reinterpret_cast<float*>(smem + 2 * TILE_BYTES + WSM_BYTES); // centre taps of LK^s alone
+    float* wsm = reinterpret_cast<float*>(smem + 2 * TILE_BYTES);             // large kernel of the current channel group
+    float* lkc = reinterpret_cast<float*>(smem + 2 * TILE_BYTES + WSM_BYTES); // centre 3x3 of LK^s alone
     unsigned char* ring = smem + 2 * TILE_BYTES + WSM_BYTES + LKC_BYTES;      // NSLOT x slot_stride
     u64* bars = reinterpret_cast<u64*>(ring + NSLOT * p.slot_stride);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 2), cfull0 = smem_u32(bars + 4);
@@ -253,43 +254,35 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
     const int lx = 2 * (warp & 1) + (q & 1), ly = 2 * (warp >> 1) + (q >> 1);
     const int lane_word = ((ly * OY) * PITCH + lx * OX) * NPAIR + pr;
 
-    int cur_g = -1, cur_b = -1;
-    bool alive = true;
+    int cur_g = -1, merged_b = -1;
+    bool alive = true, dk_ready = false;
     for (long long k = 0; k < my_units; ++k) {
         const Unit un = decode_unit(first + k * stride, p);
         const int buf = (int)(k & 1);
 
-        // ---- merged kernel ZP(dk) + LK^s (Eq. 5) of this (image, channel group) -> shared, fp32 ----
-        if (un.g != cur_g || un.b != cur_b) {
+        // ---- large-kernel taps of this channel group -> shared, fp32, pair-interleaved ----------
+        if (un.g != cur_g) {
             if (cur_g >= 0) compute_bar();                  // everyone is done with the old table
-            if (un.g != cur_g) {
-                const __nv_bfloat16* wg = p.w_large + (size_t)un.g * CG * K13 * K13;
-                constexpr int N = CG * K13 * K13, PER = (N + kComputeThreads - 1) / kComputeThreads;
-                float v[PER];
+            const __nv_bfloat16* wg = p.w_large + (size_t)un.g * CG * K13 * K13;
+            constexpr int N = CG * K13 * K13, PER = (N + kComputeThreads - 1) / kComputeThreads;
+            float v[PER];
 #pragma unroll
-                for (int t = 0; t < PER; ++t) {             // coalesced, all loads in flight together
-                    const int idx = tid + t * kComputeThreads;
-                    v[t] = idx < N ? __bfloat162float(wg[idx]) : 0.f;
-                }
+            for (int t = 0; t < PER; ++t) {                 // coalesced, all loads in flight together
+                const int idx = tid + t * kComputeThreads;
+                v[t] = idx < N ? __bfloat162float(wg[idx]) : 0.f;
+            }
 #pragma unroll
-                for (int t = 0; t < PER; ++t) {
-                    const int idx = tid + t * kComputeThreads;
-                    if (idx < N) {
-                        const int c = idx / (K13 * K13), tap = idx % (K13 * K13), i = tap / K13, j = tap % K13;
-                        wsm[wsm_index(c, i, j)] = v[t];
-                        if (i >= 5 && i <= 7 && j >= 5 && j <= 7) lkc[c * 9 + (i - 5) * 3 + (j - 5)] = v[t];
-                    }
+            for (int t = 0; t < PER; ++t) {
+                const int idx = tid + t * kComputeThreads;
+                if (idx < N) {
+                    const int c = idx / (K13 * K13), tap = idx % (K13 * K13);
+                    const int i = tap / K13, j = tap % K13;
+                    wsm[wsm_index(c, i, j)] = v[t];
+                    if (i >= 5 && i <= 7 && j >= 5 && j <= 7) lkc[c * 9 + (i - 5) * 3 + (j - 5)] = v[t];
                 }
-                if (tid < CG * K13) wsm[wsm_index(tid / K13, tid % K13, K13)] = 0.f;   // pad tap 13
-                compute_bar();
             }
-            if (cur_g < 0) pdl_wait_primary();              // dk is written by the preceding kernel
-            if (tid < CG * 9) {
-                const int c = tid / 9, tap = tid % 9;
-                wsm[wsm_index(c, 5 + tap / 3, 5 + tap % 3)] =
-                    lkc[tid] + p.dk[((size_t)un.b * p.Ca + un.g * CG + c) * 9 + tap];
-            }
-            cur_g = un.g; cur_b = un.b;
+            if (tid < CG * K13) wsm[wsm_index(tid / K13, tid % K13, K13)] = 0.f;   // pad tap 13
+            cur_g = un.g; merged_b = -1;
             compute_bar();
         }
 
@@ -306,7 +299,23 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
         const float4* wlane = reinterpret_cast<const float4*>(wsm) + pr;
 
 #pragma unroll 1
-        for (int r = 0; r < NR; ++r) {
+        for (int step = 0; step < NR; ++step) {
+            // Input rows 0-4 and 12-16 only meet kernel rows 0-4 and 8-12; rows 5-11 also meet kernel
+            // rows 5-7, whose centre holds the dynamic taps.  Taking them last means the kernel that
+            // produces dk is needed only when about half of the first unit is done, so the two
+            // kernels run side by side.
+            const int r = step < 5 ? step : (step < 10 ? step + 7 : step - 5);
+            if (step == 10 && merged_b != un.b) {
+                compute_bar();                               // nobody still reads the old centre taps
+                if (!dk_ready) { pdl_wait_primary(); dk_ready = true; }
+                if (tid < CG * 9) {                          // rows 5-7, columns 5-7: LK^s + dk  (Eq. 5)
+                    const int c = tid / 9, tap = tid % 9;
+                    wsm[wsm_index(c, 5 + tap / 3, 5 + tap % 3)] =
+                        lkc[tid] + p.dk[((size_t)un.b * p.Ca + un.g * CG + c) * 9 + tap];
+                }
+                merged_b = un.b;
+                compute_bar();
+            }
             // input row r of the patch window: read once, widen to fp32 pairs once
             u64 in[NW];
             const uint32_t* rn = tw + r * (PITCH * NPAIR);
