@@ -100,6 +100,33 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W,
                            void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Stage 1 for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a packaging variant of esc_convattn_dynkernel, same arithmetic, same result.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a real-time or
+ * safety-certified loop whose memory is fixed at start-up, under an allocator-owning framework
+ * that forbids side allocations, or in a process whose device memory is already fully handed
+ * out.  Such callers cannot create the workspace the other entry points want, so here the
+ * scratch (arrival counters and GAP partial sums) is a fixed 64 KiB array inside the library's
+ * device image.  Every GPU that loads the library holds that array until the process exits.
+ *
+ *  - Limits: B <= 1024 and B * S * C_a <= 15360, where S (slabs per image) is about 148 / B,
+ *    capped at H*W/512.  Larger problems are refused with ESC_ERR_WORKSPACE and a message in
+ *    esc_last_error(); nothing is enqueued.
+ *  - The call itself allocates nothing: no cudaMalloc / cudaFree, no library allocator.  The very
+ *    first call on each device looks up the array's device address (cudaGetSymbolAddress) with
+ *    that device current; make that first call outside any stream capture.
+ *  - All calls in the process share the one array.  The counters are cleared on `stream` at the
+ *    start of every call; partial sums are overwritten before they are read.  Two calls whose GPU
+ *    work overlaps (different streams, or different threads) race on it: serialise them.
+ *  - Other arguments, layout rules, error codes and the result dk_out [B,C_a,3,3] fp32 are exactly
+ *    those of esc_convattn_dynkernel.
+ */
+int esc_convattn_dynkernel_static(const void* x, int B, int C, int C_a, int H, int W,
+                                  const void* w_dyn, const void* b_dyn, float* dk_out,
+                                  int dtype, int layout, void* stream);
+
+/*
  * Stage 2 alone (Eq. 4 lines 3-4 with an explicit dk [B,C_a,3,3] fp32 device array):
  * both depth-wise convolutions, their sum, and the copy of the remaining channels.
  * `workspace` may be NULL (then device-side time-outs cannot be reported).

@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     esc_convattn_forward_ex,
     esc_convattn_forward_host,
     esc_convattn_dynkernel,
+    esc_convattn_dynkernel_static,
     esc_convattn_stencil,
     esc_convattn_workspace_bytes,
     esc_convattn_workspace_init,

@@ -44,6 +44,7 @@ def lib():
         L.esc_convattn_workspace_bytes.restype = sz
         L.esc_convattn_workspace_init.argtypes = [vp, sz, vp]
         L.esc_convattn_dynkernel.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
         L.esc_convattn_device_status.argtypes = [vp, vp]
@@ -51,7 +52,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_stencil", "esc_convattn_forward_host",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_stencil", "esc_convattn_forward_host",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -161,6 +162,19 @@ def esc_convattn_dynkernel(x, C_a, w_dyn, b_dyn, dk_out, layout, workspace, stre
                                         _dtype_code(x), layout, _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), _stream(stream)),
            "esc_convattn_dynkernel")
+    return dk_out
+
+
+def esc_convattn_dynkernel_static(x, C_a, w_dyn, b_dyn, dk_out, layout, stream=None):
+    """Stage 1 without any device allocation: the scratch is a fixed array inside the library.
+
+    For callers that may not call cudaMalloc (fixed-memory real-time loops, frameworks that own
+    the allocator).  Limits and the sharing rule are in include/esc_convattn.h; sizes beyond the
+    fixed scratch raise EscError with status 6."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_dynkernel_static(_ptr(x), B, C, C_a, H, W, _ptr(w_dyn), _ptr(b_dyn), _ptr(dk_out),
+                                               _dtype_code(x), layout, _stream(stream)),
+           "esc_convattn_dynkernel_static")
     return dk_out
 
 

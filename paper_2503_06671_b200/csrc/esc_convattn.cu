@@ -252,6 +252,32 @@ int forward_impl(const Problem& p, const void* x, const void* w_large, const voi
     return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
 }
 
+// ---- fixed scratch for the entry point that must not allocate ------------------------------
+// Layout: [kStaticMaxImages arrival counters][kStaticMaxPartials partial sums].  The array lives in
+// the library's device image: every GPU that loads the library holds these 64 KiB until exit.
+constexpr int kStaticMaxImages = 1024;
+constexpr int kStaticMaxPartials = 15360;
+static __device__ __align__(256) unsigned g_static_scratch[kStaticMaxImages + kStaticMaxPartials];
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+unsigned* g_static_addr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+
+// In host code `g_static_scratch` is only a handle; the address a kernel can use has to be asked
+// for, once per device, with that device current.
+int static_scratch_address(unsigned** out) {
+    int dev = 0;
+    ESC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return ESC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_addr[dev]) {
+        void* ptr = nullptr;
+        ESC_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        g_static_addr[dev] = static_cast<unsigned*>(ptr);
+    }
+    *out = g_static_addr[dev];
+    return ESC_OK;
+}
+
 // ---- host-buffer path ---------------------------------------------------------------------
 struct HostPath {
     int dev = -1;
@@ -343,6 +369,38 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W, c
     rc = check_workspace(p, workspace, workspace_bytes_);
     if (rc != ESC_OK) return rc;
     return launch_gap(p, x, w_dyn, b_dyn, carve(workspace, B, C_a), dk_out, static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_dynkernel_static(const void* x, int B, int C, int C_a, int H, int W, const void* w_dyn,
+                                  const void* b_dyn, float* dk_out, int dtype, int layout, void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, 1, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!x || !w_dyn || !b_dyn || !dk_out) return ESC_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(dk_out, 4) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
+    const int S = slabs_for(B, (long long)H * W);
+    if (B > kStaticMaxImages || (long long)B * S * C_a > kStaticMaxPartials) {
+        char buf[200];
+        snprintf(buf, sizeof buf,
+                 "esc_convattn_dynkernel_static: needs %d counters and %lld partial sums, the fixed scratch holds %d and %d",
+                 B, (long long)B * S * C_a, kStaticMaxImages, kStaticMaxPartials);
+        g_last_error = buf;
+        return ESC_ERR_WORKSPACE;
+    }
+    unsigned* base = nullptr;
+    rc = static_scratch_address(&base);
+    if (rc != ESC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The counters must be zero when the kernel starts; a call that was cut short could have left them
+    // otherwise, and the array is shared by every caller in the process.
+    ESC_CUDA(cudaMemsetAsync(base, 0, (size_t)B * sizeof(unsigned), st));
+    Workspace w;
+    w.ctrl = nullptr;
+    w.arrivals = base;
+    w.dk = dk_out;
+    w.partial = reinterpret_cast<float*>(base + kStaticMaxImages);
+    return launch_gap(p, x, w_dyn, b_dyn, w, dk_out, st);
 }
 
 int esc_convattn_stencil(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
