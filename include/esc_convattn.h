@@ -110,9 +110,9 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W,
  * scratch (arrival counters and GAP partial sums) is a fixed 64 KiB array inside the library's
  * device image.  Every GPU that loads the library holds that array until the process exits.
  *
- *  - Limits: B <= 1024 and B * S * C_a <= 15360, where S (slabs per image) is about 148 / B,
- *    capped at H*W/512.  Larger problems are refused with ESC_ERR_WORKSPACE and a message in
- *    esc_last_error(); nothing is enqueued.
+ *  - Limits: B <= 1024 and B * S * C_a <= 15360, where S (slabs per image) is about 148 / B
+ *    (444 / B once B*H*W reaches 1.5 million pixels), capped at H*W/512.  Larger problems are
+ *    refused with ESC_ERR_WORKSPACE and a message in esc_last_error(); nothing is enqueued.
  *  - The call itself allocates nothing: no cudaMalloc / cudaFree, no library allocator.  The very
  *    first call on each device looks up the array's device address (cudaGetSymbolAddress) with
  *    that device current; make that first call outside any stream capture.

@@ -78,9 +78,14 @@ struct Workspace {
     float* partial;
 };
 
+bool is_large_map(int B, long long HW) { return (long double)B * HW >= 1.5e6L; }
+
 int slabs_for(int B, long long HW) {
-    // about one work item per SM over the whole batch, at least 512 pixels per slab
-    long long s = (148 + B - 1) / B;
+    // About one work item per SM over the whole batch (three for maps so large that the stencil
+    // kernel takes many waves and the GAP kernel runs ahead of it rather than beside it), at least
+    // 512 pixels per slab.
+    const long long target = is_large_map(B, HW) ? 3 * 148 : 148;
+    long long s = (target + B - 1) / B;
     const long long cap = (HW + 511) / 512;
     if (s > cap) s = cap;
     if (s > esc::kMaxSlabs) s = esc::kMaxSlabs;
@@ -122,7 +127,11 @@ int launch_gap_t(const Problem& p, const void* x, const void* w_dyn, const void*
     int sms = esc::tma::sm_count();
     if (sms <= 0) sms = 148;
     const long long items = (long long)p.B * S;
-    const unsigned grid = (unsigned)(items < sms ? items : sms);   // persistent, at most one block per SM
+    // Small maps: at most one block per SM, so that the stencil kernel fits beside this one.
+    // Large maps: the stencil kernel would wait for dk during its first of many units anyway, so
+    // this kernel takes three blocks per SM and finishes sooner.
+    const long long cap = is_large_map(p.B, (long long)p.H * p.W) ? 3LL * sms : sms;
+    const unsigned grid = (unsigned)(items < cap ? items : cap);
     const size_t scratch = (size_t)esc::kGapWarps * p.Ca > (size_t)esc::kGapThreads ? (size_t)esc::kGapWarps * p.Ca : (size_t)esc::kGapThreads;
     const size_t smem = (scratch + p.Ca) * sizeof(float);
     if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
