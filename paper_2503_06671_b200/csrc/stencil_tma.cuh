@@ -215,6 +215,9 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
             };
             int issued = 0, stored = 0, lag = 0;
             bool alive = true;
+            // The copy has the whole kernel to finish, the compute warps cannot start without the
+            // first halo tile: let that tile land before competing with it for DRAM.
+            if (nunits > 0) alive = mbar_wait(full0, 0u, p.ctrl, 0xC1000000u);
             while (st.k < nunits) {
                 // store the oldest chunk once COPY_DEPTH loads are in flight (or nothing is left to load)
                 if (lag == COPY_DEPTH || ld.k >= nunits) {
@@ -393,7 +396,8 @@ inline EncodeTiledFn encode_fn() {
 }
 
 // bf16 NHWC tensor [B][H][W][C] as a 4-D map {C, W, H, B} with the given box.
-inline bool make_map(CUtensorMap* m, const void* base, int B, int C, int H, int W, int bc, int bw, int bh) {
+inline bool make_map(CUtensorMap* m, const void* base, int B, int C, int H, int W, int bc, int bw, int bh,
+                     CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_128B) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
@@ -401,7 +405,7 @@ inline bool make_map(CUtensorMap* m, const void* base, int B, int C, int H, int 
     const cuuint32_t box[4] = {(cuuint32_t)bc, (cuuint32_t)bw, (cuuint32_t)bh, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, promo,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -446,7 +450,9 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     p.ctrl = ctrl;
 
     CUtensorMap m_att, m_cin, m_cout, m_res;
-    if (!make_map(&m_att, x, B, C, H, W, CG, PITCH, THP)) return kNotApplicable;
+    // The halo tile gates the start of the arithmetic: fetch no more than its own 32-byte sectors need
+    // (64-byte promotion measured fastest; 128-byte promotion drags the copy-through channels along).
+    if (!make_map(&m_att, x, B, C, H, W, CG, PITCH, THP, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
     if (!make_map(&m_res, out, B, C, H, W, CG, TW, TH)) return kNotApplicable;
     if (cc > 0) {
         if (!make_map(&m_cin, x, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
