@@ -191,20 +191,27 @@ int launch_copy(const Problem& p, const void* x, void* out, cudaStream_t st) {
 template <typename T, int LAYOUT>
 int launch_generic_t(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                      cudaStream_t st, bool dependent) {
-    const int tiles_x = (p.W + esc::kGenTX - 1) / esc::kGenTX, tiles_y = (p.H + esc::kGenTY - 1) / esc::kGenTY;
+    const bool regtile = p.K == esc::kRtK;             // the paper's kernel size: eight outputs per thread
+    const int TX = regtile ? esc::kRtTX : esc::kGenTX, TY = regtile ? esc::kRtTY : esc::kGenTY;
+    const int tiles_x = (p.W + TX - 1) / TX, tiles_y = (p.H + TY - 1) / TY;
     const long long blocks = (long long)p.B * p.Ca * tiles_x * tiles_y;
     if (blocks > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);
-    cfg.blockDim = dim3(esc::kGenTX, esc::kGenTY);
+    cfg.blockDim = regtile ? dim3(esc::kRtThreads) : dim3(esc::kGenTX, esc::kGenTY);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_generic<T, LAYOUT>, static_cast<const T*>(x), static_cast<T*>(out),
-                                p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), dk, tiles_x, tiles_y));
+    if (regtile)
+        ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT>, static_cast<const T*>(x),
+                                    static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), dk,
+                                    tiles_x, tiles_y));
+    else
+        ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_generic<T, LAYOUT>, static_cast<const T*>(x), static_cast<T*>(out),
+                                    p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), dk, tiles_x, tiles_y));
     ++g_last_launches;
     return ESC_OK;
 }

@@ -59,6 +59,83 @@ stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int
     out[elem_index<LAYOUT>(b, c, oy, ox, C, H, W)] = Elem<T>::from_f32(acc);
 }
 
+// Register-tiled variant for K = 13 (the paper's kernel size) on any layout and element type: the
+// same staging as above, but a 32 x 64 output tile per block and eight adjacent outputs per thread,
+// so that one kernel row costs five 16-byte reads of the input row and four of the weights for
+// 104 FMAs.  It serves the fp32 and NCHW cases that the TMA kernel does not take.
+constexpr int kRtK = 13, kRtTX = 64, kRtTY = 32, kRtOX = 8;
+constexpr int kRtPitch = kRtTX + kRtK - 1;            // 76 floats, a multiple of 4
+constexpr int kRtRows = kRtTY + kRtK - 1;             // 44
+constexpr int kRtThreads = (kRtTX / kRtOX) * kRtTY;   // 256
+
+template <typename T, int LAYOUT>
+__global__ void __launch_bounds__(kRtThreads)
+stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W,
+                    const T* __restrict__ w_large, const float* __restrict__ dk, int tiles_x, int tiles_y)
+{
+    __shared__ __align__(16) float tile[kRtRows * kRtPitch];
+    __shared__ __align__(16) float wm[kRtK * 16];      // merged kernel, rows padded to 16 taps
+
+    long long bid = blockIdx.x;
+    const int tx = (int)(bid % tiles_x); bid /= tiles_x;
+    const int ty = (int)(bid % tiles_y); bid /= tiles_y;
+    const int c = (int)(bid % Ca);
+    const int b = (int)(bid / Ca);
+    constexpr int P = (kRtK - 1) / 2;
+    const int tid = threadIdx.x;
+    const int y0 = ty * kRtTY - P, x0 = tx * kRtTX - P;
+
+    for (int t = tid; t < kRtRows * kRtPitch; t += kRtThreads) {
+        const int r = t / kRtPitch, q = t % kRtPitch;
+        const int y = y0 + r, xx = x0 + q;
+        float v = 0.f;
+        if (y >= 0 && y < H && xx >= 0 && xx < W) v = Elem<T>::to_f32(x[elem_index<LAYOUT>(b, c, y, xx, C, H, W)]);
+        tile[t] = v;
+    }
+    pdl_wait_primary();   // dk comes from the preceding kernel when launched as its dependent
+    for (int t = tid; t < kRtK * 16; t += kRtThreads) {
+        const int i = t / 16, j = t % 16;
+        float w = 0.f;
+        if (j < kRtK) {
+            w = Elem<T>::to_f32(w_large[((size_t)c * kRtK + i) * kRtK + j]);
+            const int di = i - (P - 1), dj = j - (P - 1);
+            if (di >= 0 && di < 3 && dj >= 0 && dj < 3) w += dk[((size_t)b * Ca + c) * 9 + di * 3 + dj];
+        }
+        wm[t] = w;
+    }
+    __syncthreads();
+
+    const int lx = tid % (kRtTX / kRtOX), ly = tid / (kRtTX / kRtOX);
+    float acc[kRtOX];
+#pragma unroll
+    for (int o = 0; o < kRtOX; ++o) acc[o] = 0.f;
+#pragma unroll 1
+    for (int i = 0; i < kRtK; ++i) {
+        float in[kRtOX + kRtK - 1], w[16];
+        const float4* trow = reinterpret_cast<const float4*>(tile + (ly + i) * kRtPitch + lx * kRtOX);
+        const float4* wrow = reinterpret_cast<const float4*>(wm + i * 16);
+#pragma unroll
+        for (int v = 0; v < (kRtOX + kRtK - 1) / 4; ++v) {
+            const float4 q = trow[v];
+            in[4 * v] = q.x; in[4 * v + 1] = q.y; in[4 * v + 2] = q.z; in[4 * v + 3] = q.w;
+        }
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const float4 q = wrow[v];
+            w[4 * v] = q.x; w[4 * v + 1] = q.y; w[4 * v + 2] = q.z; w[4 * v + 3] = q.w;
+        }
+#pragma unroll
+        for (int j = 0; j < kRtK; ++j)
+#pragma unroll
+            for (int o = 0; o < kRtOX; ++o) acc[o] = fmaf(w[j], in[o + j], acc[o]);
+    }
+    const int oy = ty * kRtTY + ly, ox0 = tx * kRtTX + lx * kRtOX;
+    if (oy >= H) return;
+#pragma unroll
+    for (int o = 0; o < kRtOX; ++o)
+        if (ox0 + o < W) out[elem_index<LAYOUT>(b, c, oy, ox0 + o, C, H, W)] = Elem<T>::from_f32(acc[o]);
+}
+
 // Copy of the channels that the module leaves untouched (Concat of Eq. 4 line 4), written as a
 // strided 2-D copy: `rows` rows of `row_units` units, `stride_units` apart, starting
 // `offset_units` into both tensors.  U is the widest unit all three quantities divide into.
