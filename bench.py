@@ -28,6 +28,10 @@ DEFAULT_WORKLOAD = "cfg3_640x360_bf16"       # 640x360x64 bf16: the configuratio
 SM_COUNT_NOMINAL = 148
 FMA_LANES_PER_SM = 128
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one stencil-kernel launch from the ncu capture summarised under
+# profiles/, keyed by (workload, layout, library version the capture was taken with).  Reported only while the
+# library still has that version; otherwise the kernel has changed since and the figure is withheld.
+NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", 101): 29.56e6 + 0.46e6}
 
 
 def peaks():
@@ -345,6 +349,7 @@ def main():
         ach = alg_bytes / (ms_kernel * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
                 "traffic": None, "peak_source": f"{pk['source']} copy bandwidth"}
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name, args.layout, pkg.esc_version()))
     roof.update({"kernel": "stencil (stage 2)", "kernel_ms": ms_kernel, "gap_kernel_ms": ms_gap,
                  "whole_step_frac": max(t_alu, t_hbm) / (ms_step * 1e-3),
                  "hbm_side": {"algorithmic_GBps": alg_bytes / (ms_kernel * 1e-3) / 1e9, "of_peak": alg_bytes / (ms_kernel * 1e-3) / 1e9 / pk["hbm_gbs"]}})
