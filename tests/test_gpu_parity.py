@@ -117,6 +117,10 @@ EDGE_SHAPES = [
     (1, 48, 16, 29, 31, 17),    # K = 17
     (1, 20, 12, 19, 23, 3),     # K = 3, odd channel counts
     (5, 64, 16, 64, 64, 13),    # small batch of training patches
+    (1, 192, 48, 50, 70, 13),   # the paper's large model: C = 192, 48 attention channels (3 channel groups)
+    (2, 48, 16, 45, 45, 13),    # ESC-FP width: C = 48
+    (1, 272, 16, 41, 41, 13),   # 256 copy-through channels: narrowest copy box
+    (1, 288, 16, 20, 20, 13),   # more copy-through channels than a TMA box holds: generic path
 ]
 
 
