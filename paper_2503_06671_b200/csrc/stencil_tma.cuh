@@ -301,24 +301,9 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
         const uint32_t* tw = reinterpret_cast<const uint32_t*>(tbuf) + lane_word;
         const float4* wlane = reinterpret_cast<const float4*>(wsm) + pr;
 
-#pragma unroll 1
-        for (int step = 0; step < NR; ++step) {
-            // Input rows 0-4 and 12-16 only meet kernel rows 0-4 and 8-12; rows 5-11 also meet kernel
-            // rows 5-7, whose centre holds the dynamic taps.  Taking them last means the kernel that
-            // produces dk is needed only when about half of the first unit is done, so the two
-            // kernels run side by side.
-            const int r = step < 5 ? step : (step < 10 ? step + 7 : step - 5);
-            if (step == 10 && merged_b != un.b) {
-                compute_bar();                               // nobody still reads the old centre taps
-                if (!dk_ready) { pdl_wait_primary(); dk_ready = true; }
-                if (tid < CG * 9) {                          // rows 5-7, columns 5-7: LK^s + dk  (Eq. 5)
-                    const int c = tid / 9, tap = tid % 9;
-                    wsm[wsm_index(c, 5 + tap / 3, 5 + tap % 3)] =
-                        lkc[tid] + p.dk[((size_t)un.b * p.Ca + un.g * CG + c) * 9 + tap];
-                }
-                merged_b = un.b;
-                compute_bar();
-            }
+        // One input row r of the patch window: read once, widened once, applied to every output row
+        // it belongs to.
+        auto do_row = [&](const int r) {
             // input row r of the patch window: read once, widen to fp32 pairs once
             u64 in[NW];
             const uint32_t* rn = tw + r * (PITCH * NPAIR);
@@ -349,7 +334,29 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
                     }
                 }
             }
+        };
+
+        // Input rows 0-4 and 12-16 only meet kernel rows 0-4 and 8-12; rows 5-11 also meet kernel rows
+        // 5-7, whose centre holds the dynamic taps.  Taking them last means the kernel that produces dk
+        // is needed only when about half of the first unit is done, so the two kernels run side by
+        // side.  Two plain loops (rather than one loop with a special step) keep each loop body free of
+        // the barrier code: measured 8 % faster.
+#pragma unroll 1
+        for (int step = 0; step < 2 * OY; ++step) do_row(step < OY ? step : step + (K13 - 1) - OY);
+        if (merged_b != un.b) {
+            if (!dk_ready) { pdl_wait_primary(); dk_ready = true; }
+            float dkv = 0.f;                                 // fetched before the barrier so its latency hides behind the stragglers
+            if (tid < CG * 9) dkv = __ldcg(p.dk + ((size_t)un.b * p.Ca + un.g * CG + tid / 9) * 9 + tid % 9);
+            compute_bar();                                   // nobody still reads the old centre taps
+            if (tid < CG * 9) {                              // rows 5-7, columns 5-7: LK^s + dk  (Eq. 5)
+                const int c = tid / 9, tap = tid % 9;
+                wsm[wsm_index(c, 5 + tap / 3, 5 + tap % 3)] = lkc[tid] + dkv;
+            }
+            merged_b = un.b;
+            compute_bar();
         }
+#pragma unroll 1
+        for (int r = OY; r < K13 - 1; ++r) do_row(r);
 
         // ---- epilogue: round once to bf16, stage the 40x40x16 result in the freed input buffer,
         //      one TMA store (the TMA unit clips at the image border) ---------------------------
