@@ -308,7 +308,7 @@ HostPath g_host;
 
 extern "C" {
 
-int esc_version(void) { return 102; }
+int esc_version(void) { return 103; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 

@@ -55,8 +55,10 @@ constexpr int OUT_TILE_BYTES = TH * TW * CG * 2;     // 51,200: staged result, r
 constexpr int WSM_FLOATS = K13 * 7 * NPAIR * 4;      // [i][jj][pair][4]: taps 2jj,2jj+1 of both channels
 constexpr int WSM_BYTES = (WSM_FLOATS * 4 + 127) / 128 * 128;
 constexpr int LKC_BYTES = (CG * 9 * 4 + 127) / 128 * 128;
-constexpr int NSLOT = 4, COPY_DEPTH = 3;             // copy ring: slots, loads in flight
-constexpr int kMaxSlotBytes = 8192;
+constexpr int NSLOT = 2, COPY_DEPTH = 1;             // copy ring: slots, loads in flight (few large chunks: the copy
+                                                     // thread shares a scheduler with two compute warps and every
+                                                     // instruction it issues delays them, then the whole block at the barriers)
+constexpr int kMaxSlotBytes = 16384;
 constexpr unsigned kSpinLimit = 1u << 20;    // polls before a wait gives up (each poll may suspend up to the hint)
 constexpr unsigned kSuspendHintNs = 20000;
 
@@ -444,9 +446,9 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     if (p.units > 0x7fffffffLL) return kNotApplicable;
     p.copy_cc = cc; p.copy_cw = TW; p.copy_cr = 2; p.slot_stride = 128;
     if (cc > 0) {
-        static const int shapes[5][2] = {{40, 2}, {40, 1}, {20, 1}, {10, 1}, {5, 1}};
+        static const int shapes[6][2] = {{40, 4}, {40, 2}, {40, 1}, {20, 1}, {10, 1}, {5, 1}};
         int pick = -1;
-        for (int s = 0; s < 5 && pick < 0; ++s)
+        for (int s = 0; s < 6 && pick < 0; ++s)
             if (cc * 2 * shapes[s][0] * shapes[s][1] <= kMaxSlotBytes) pick = s;
         if (pick < 0) return kNotApplicable;
         p.copy_cw = shapes[pick][0]; p.copy_cr = shapes[pick][1];
