@@ -121,6 +121,9 @@ EDGE_SHAPES = [
     (2, 48, 16, 45, 45, 13),    # ESC-FP width: C = 48
     (1, 272, 16, 41, 41, 13),   # 256 copy-through channels: narrowest copy box
     (1, 288, 16, 20, 20, 13),   # more copy-through channels than a TMA box holds: generic path
+    (130, 32, 16, 40, 40, 13),  # many images of exactly one tile
+    (1, 64, 16, 1200, 20, 13),  # tall and narrow
+    (1, 64, 16, 17, 1500, 13),  # flat and wide
 ]
 
 
@@ -222,3 +225,27 @@ def test_host_entry_matches_device_entry(pkg):
     pkg.esc_convattn_forward_ex(x, C_a, K, wl.cuda(), wd.cuda(), bd.cuda(), out, pkg.ESC_NHWC, ws)
     torch.cuda.synchronize()
     assert torch.equal(out.cpu().view(torch.int16), oh.view(torch.int16))
+
+
+def test_two_streams_two_workspaces(pkg, oracle):
+    """Calls on different streams with different workspaces may overlap on the GPU; each must still be right."""
+    import torch
+
+    B, C, C_a, H, W, K = 2, 64, 16, 120, 200, 13
+    cases = []
+    for seed in (1, 2):
+        d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=9000 + seed, channel_means=True)
+        x = util.to_device(d["x"], synth.BF16, synth.NHWC)
+        wl, wd, bd = util.weights_to_device(d, synth.BF16)
+        cases.append((d, x, wl, wd, bd, torch.empty_like(x), pkg.new_workspace(B, C_a, H, W, K), torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for _ in range(5):
+        for (d, x, wl, wd, bd, out, ws, st) in cases:
+            pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, out, pkg.ESC_NHWC, ws, stream=st)
+    torch.cuda.synchronize()
+    for (d, x, wl, wd, bd, out, ws, st) in cases:
+        assert pkg.esc_convattn_device_status(ws) == 0
+        ref, mag = oracle.forward(d["x"], C_a, d["w_large"], d["w_dyn"], d["b_dyn"], want_mag=True)
+        got = util.to_host_nchw(out, synth.NHWC)
+        util.check_attention(got[:, :C_a], ref[:, :C_a], mag, synth.BF16, "two streams")
+        assert np.array_equal(got[:, C_a:], ref[:, C_a:])
