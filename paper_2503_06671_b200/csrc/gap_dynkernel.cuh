@@ -5,7 +5,7 @@
 //   dk[b,o] = b_dyn[o] + sum_c w_dyn[o,c] g[b,c]     o = c*9 + i*3 + j
 //
 // Every image is cut into S slabs so that a single large image still spreads over the machine;
-// the B*S work items are walked by a persistent grid of small blocks (3 warps, at most one block
+// the B*S work items are walked by a persistent grid of small blocks (4 warps -- one per SM sub-partition --, at most one block
 // per SM).  The blocks are kept this small on purpose: the stencil kernel is launched as a
 // programmatic dependent of this one and needs nearly a whole SM per block, so the two kernels
 // can only run side by side -- this one bound by DRAM, the other by the FMA pipe -- if this one
@@ -19,7 +19,7 @@
 
 namespace esc {
 
-constexpr int kGapThreads = 96;
+constexpr int kGapThreads = 128;
 constexpr int kGapWarps = kGapThreads / 32;
 
 template <typename T, int LAYOUT>

@@ -48,7 +48,7 @@ constexpr int NPAIR = CG / 2;
 constexpr int kComputeWarps = LXP * LYP / 4;         // 8
 constexpr int kComputeThreads = kComputeWarps * 32;  // 256
 constexpr int kThreads = kComputeThreads + 128;      // + helper warp group (producer, copy, 2 idle)
-constexpr int kLaunchRegs = 152;                      // 384*152 = 58,368: leaves 7,168 registers for one GAP block (96 x 64) per SM
+constexpr int kLaunchRegs = 152;                      // 384*152 = 58,368: leaves 7,168 registers (1,792 per sub-partition) for one GAP block (128 x 56) per SM
 constexpr int kComputeRegs = 208, kHelperRegs = 40;   // after reallocation: 256*208 + 128*40 = 58,368
 constexpr int TILE_BYTES = THP * PITCH * CG * 2;     // 88,192
 constexpr int OUT_TILE_BYTES = TH * TW * CG * 2;     // 51,200: staged result, reuses the input buffer
