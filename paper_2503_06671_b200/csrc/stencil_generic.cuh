@@ -60,13 +60,14 @@ stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int
 }
 
 // Register-tiled variant for K = 13 (the paper's kernel size) on any layout and element type: the
-// same staging as above, but a 32 x 64 output tile per block and eight adjacent outputs per thread,
-// so that one kernel row costs five 16-byte reads of the input row and four of the weights for
-// 104 FMAs.  It serves the fp32 and NCHW cases that the TMA kernel does not take.
-constexpr int kRtK = 13, kRtTX = 64, kRtTY = 32, kRtOX = 8;
+// same staging as above, but a 64 x 64 output tile per block and a 4 x 8 patch of outputs per thread.
+// The loop runs over the 16 input rows a patch touches: a row costs five 16-byte reads and is used by
+// up to four output rows, each with its kernel row (four broadcast 16-byte reads), 104 FMAs apiece.
+// It serves the fp32 and NCHW cases that the TMA kernel does not take.
+constexpr int kRtK = 13, kRtTX = 64, kRtTY = 64, kRtOX = 8, kRtOY = 4;
 constexpr int kRtPitch = kRtTX + kRtK - 1;            // 76 floats, a multiple of 4
-constexpr int kRtRows = kRtTY + kRtK - 1;             // 44
-constexpr int kRtThreads = (kRtTX / kRtOX) * kRtTY;   // 256
+constexpr int kRtRows = kRtTY + kRtK - 1;             // 76
+constexpr int kRtThreads = (kRtTX / kRtOX) * (kRtTY / kRtOY);   // 128
 
 template <typename T, int LAYOUT>
 __global__ void __launch_bounds__(kRtThreads)
@@ -106,34 +107,48 @@ stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca,
     __syncthreads();
 
     const int lx = tid % (kRtTX / kRtOX), ly = tid / (kRtTX / kRtOX);
-    float acc[kRtOX];
+    float acc[kRtOY][kRtOX];
 #pragma unroll
-    for (int o = 0; o < kRtOX; ++o) acc[o] = 0.f;
+    for (int a = 0; a < kRtOY; ++a)
+#pragma unroll
+        for (int o = 0; o < kRtOX; ++o) acc[a][o] = 0.f;
 #pragma unroll 1
-    for (int i = 0; i < kRtK; ++i) {
-        float in[kRtOX + kRtK - 1], w[16];
-        const float4* trow = reinterpret_cast<const float4*>(tile + (ly + i) * kRtPitch + lx * kRtOX);
-        const float4* wrow = reinterpret_cast<const float4*>(wm + i * 16);
+    for (int r = 0; r < kRtOY + kRtK - 1; ++r) {          // input row r of the patch window
+        float in[kRtOX + kRtK - 1];
+        const float4* trow = reinterpret_cast<const float4*>(tile + (ly * kRtOY + r) * kRtPitch + lx * kRtOX);
 #pragma unroll
         for (int v = 0; v < (kRtOX + kRtK - 1) / 4; ++v) {
             const float4 q = trow[v];
             in[4 * v] = q.x; in[4 * v + 1] = q.y; in[4 * v + 2] = q.z; in[4 * v + 3] = q.w;
         }
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            const float4 q = wrow[v];
-            w[4 * v] = q.x; w[4 * v + 1] = q.y; w[4 * v + 2] = q.z; w[4 * v + 3] = q.w;
+        for (int a = 0; a < kRtOY; ++a) {
+            const int i = r - a;                           // kernel row that maps input row r to output row a
+            if (i >= 0 && i < kRtK) {
+                float w[16];
+                const float4* wrow = reinterpret_cast<const float4*>(wm + i * 16);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const float4 q = wrow[v];
+                    w[4 * v] = q.x; w[4 * v + 1] = q.y; w[4 * v + 2] = q.z; w[4 * v + 3] = q.w;
+                }
+#pragma unroll
+                for (int j = 0; j < kRtK; ++j)
+#pragma unroll
+                    for (int o = 0; o < kRtOX; ++o) acc[a][o] = fmaf(w[j], in[o + j], acc[a][o]);
+            }
         }
-#pragma unroll
-        for (int j = 0; j < kRtK; ++j)
-#pragma unroll
-            for (int o = 0; o < kRtOX; ++o) acc[o] = fmaf(w[j], in[o + j], acc[o]);
     }
-    const int oy = ty * kRtTY + ly, ox0 = tx * kRtTX + lx * kRtOX;
-    if (oy >= H) return;
+    const int ox0 = tx * kRtTX + lx * kRtOX;
 #pragma unroll
-    for (int o = 0; o < kRtOX; ++o)
-        if (ox0 + o < W) out[elem_index<LAYOUT>(b, c, oy, ox0 + o, C, H, W)] = Elem<T>::from_f32(acc[o]);
+    for (int a = 0; a < kRtOY; ++a) {
+        const int oy = ty * kRtTY + ly * kRtOY + a;
+        if (oy < H) {
+#pragma unroll
+            for (int o = 0; o < kRtOX; ++o)
+                if (ox0 + o < W) out[elem_index<LAYOUT>(b, c, oy, ox0 + o, C, H, W)] = Elem<T>::from_f32(acc[a][o]);
+        }
+    }
 }
 
 // Copy of the channels that the module leaves untouched (Concat of Eq. 4 line 4), written as a
