@@ -110,7 +110,7 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W,
  * scratch (arrival counters and GAP partial sums) is a fixed 64 KiB array inside the library's
  * device image.  Every GPU that loads the library holds that array until the process exits.
  *
- *  - Limits: B <= 1024 and B * S * C_a <= 15360, where S (slabs per image) is about 148 / B
+ *  - Limits: B <= 1024 and B * S * C_a <= 15360, where S (slabs per image) is 148 / B rounded down, at least 1
  *    (444 / B once B*H*W reaches 1.5 million pixels), capped at H*W/512.  Larger problems are
  *    refused with ESC_ERR_WORKSPACE and a message in esc_last_error(); nothing is enqueued.
  *  - The call itself allocates nothing: no cudaMalloc / cudaFree, no library allocator.  The very
@@ -154,6 +154,18 @@ int esc_convattn_device_status(void* workspace, void* stream);
  * this thread selected: 0 = none yet, 1 = guarded generic kernel, 2 = TMA-staged register-tiled
  * kernel.  For tests and benchmarks. */
 int esc_convattn_last_path(void);
+
+/* Width in pixels of the output tile the TMA-staged kernel used in that call (40: 40x40 tiles,
+ * 64: 64x20 tiles, chosen by the tile count's balance over the SMs), 0 when the generic kernel
+ * ran.  For tests and benchmarks. */
+int esc_convattn_last_tile_width(void);
+
+/* Overrides the tile choice of the TMA-staged kernel for later calls on this thread: 0 = choose
+ * by cost (the default), 40 or 64 = always that width.  The geometries add the 169 taps of an
+ * output in different orders, so results differ by fp32 rounding before the final rounding to
+ * bf16 (far inside the module's tolerance); with a fixed width, results are bitwise reproducible.
+ * Returns ESC_ERR_UNSUPPORTED for any other value.  For tests and tuning. */
+int esc_convattn_set_tile_width(int tile_width);
 
 /* Number of kernels the last forward / stage call on this thread launched. */
 int esc_convattn_last_launches(void);

@@ -19,6 +19,8 @@ from .binding import (  # noqa: F401
     esc_convattn_workspace_init,
     esc_convattn_device_status,
     esc_convattn_last_path,
+    esc_convattn_last_tile_width,
+    esc_convattn_set_tile_width,
     esc_convattn_last_launches,
     esc_status_string,
     esc_last_error,

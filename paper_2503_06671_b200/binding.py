@@ -48,12 +48,13 @@ def lib():
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
         L.esc_convattn_device_status.argtypes = [vp, vp]
+        L.esc_convattn_set_tile_width.argtypes = [i]
         L.esc_status_string.argtypes = [i]
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
                      "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_stencil", "esc_convattn_forward_host",
-                     "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_launches",
+                     "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
         _lib = L
@@ -112,6 +113,14 @@ def esc_version() -> int:
 
 def esc_convattn_last_path() -> int:
     return lib().esc_convattn_last_path()
+
+
+def esc_convattn_last_tile_width() -> int:
+    return lib().esc_convattn_last_tile_width()
+
+
+def esc_convattn_set_tile_width(tile_width: int) -> None:
+    _check(lib().esc_convattn_set_tile_width(int(tile_width)), "esc_convattn_set_tile_width")
 
 
 def esc_convattn_last_launches() -> int:

@@ -22,6 +22,8 @@ namespace {
 
 thread_local std::string g_last_error;
 thread_local int g_last_path = 0;
+thread_local int g_last_tile_w = 0;
+thread_local int g_tile_policy = 0;      // 0 = by cost, else the tile width to use
 thread_local int g_last_launches = 0;
 
 int cuda_fail(cudaError_t e, const char* what) {
@@ -81,11 +83,12 @@ struct Workspace {
 bool is_large_map(int B, long long HW) { return (long double)B * HW >= 1.5e6L; }
 
 int slabs_for(int B, long long HW) {
-    // About one work item per SM over the whole batch (three for maps so large that the stencil
-    // kernel takes many waves and the GAP kernel runs ahead of it rather than beside it), at least
-    // 512 pixels per slab.
+    // At most one work item per SM over the whole batch, so that every block walks one item and no
+    // image waits for a second round (three per SM for maps so large that the stencil kernel takes
+    // many waves and the GAP kernel runs ahead of it rather than beside it), at least 512 pixels
+    // per slab.
     const long long target = is_large_map(B, HW) ? 3 * 148 : 148;
-    long long s = (target + B - 1) / B;
+    long long s = target / B;
     const long long cap = (HW + 511) / 512;
     if (s > cap) s = cap;
     if (s > esc::kMaxSlabs) s = esc::kMaxSlabs;
@@ -219,6 +222,7 @@ int launch_generic_t(const Problem& p, const void* x, const void* w_large, const
 int launch_generic(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                    cudaStream_t st, bool dependent) {
     g_last_path = 1;
+    g_last_tile_w = 0;
     int rc;
     if (p.dtype == ESC_F32)
         rc = p.layout == ESC_NCHW ? launch_generic_t<float, esc::kNCHW>(p, x, w_large, dk, out, st, dependent)
@@ -232,9 +236,10 @@ int launch_generic(const Problem& p, const void* x, const void* w_large, const f
 
 int launch_stencil(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                    unsigned* ctrl, cudaStream_t st, bool dependent) {
+    int tile_w = g_tile_policy;
     int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, out, ctrl, st,
-                                  dependent, &g_last_launches, &g_last_error);
-    if (rc == ESC_OK) { g_last_path = 2; return ESC_OK; }
+                                  dependent, &g_last_launches, &g_last_error, &tile_w);
+    if (rc == ESC_OK) { g_last_path = 2; g_last_tile_w = tile_w; return ESC_OK; }
     if (rc != esc::tma::kNotApplicable) return rc;
     return launch_generic(p, x, w_large, dk, out, st, dependent);
 }
@@ -308,11 +313,17 @@ HostPath g_host;
 
 extern "C" {
 
-int esc_version(void) { return 103; }
+int esc_version(void) { return 104; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
 int esc_convattn_last_path(void) { return g_last_path; }
+int esc_convattn_last_tile_width(void) { return g_last_tile_w; }
+int esc_convattn_set_tile_width(int tile_width) {
+    if (tile_width != 0 && tile_width != esc::tma::Geom40::TW && tile_width != esc::tma::Geom64::TW) return ESC_ERR_UNSUPPORTED;
+    g_tile_policy = tile_width;
+    return ESC_OK;
+}
 int esc_convattn_last_launches(void) { return g_last_launches; }
 
 const char* esc_status_string(int s) {

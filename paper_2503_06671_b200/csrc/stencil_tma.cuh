@@ -1,7 +1,10 @@
 // Kernel (b), fast path: TMA-staged, register-tiled fused stencil for K = 13 on NHWC bf16 tensors
 // (ESC paper, Section 3.3, Eq. 4 lines 3-4, evaluated in the merged form ZP(dk) + LK^s of Eq. 5).
 //
-// Work unit: a 40x40 output tile of one image for one group of 16 attention channels.  One CTA per
+// Work unit: an output tile of one image for one group of 16 attention channels.  The kernel is a
+// template over the tile geometry; the description below gives the numbers of the main one (40x40
+// tiles, 5x10 outputs per lane), the second one (64x16 tiles, 4x8 outputs per lane) serves maps
+// that 40x40 tiles cover or balance badly -- the host picks by a cost estimate.  One CTA per
 // SM, persistent over units, three warp groups:
 //   warps 0-7  compute.  lane = (patch position q, channel pair p); a warp covers 4 patches of
 //              5x10 outputs x 8 channel pairs, two channels at a time with packed fp32 FMAs
@@ -36,22 +39,13 @@ namespace esc { namespace tma {
 constexpr int kNotApplicable = -1;
 
 constexpr int K13 = 13, P6 = 6;
-constexpr int OX = 10, OY = 5;            // outputs per lane: OY rows x OX columns
-constexpr int LXP = 4, LYP = 8;           // patches per tile in x and y
-constexpr int TW = OX * LXP, TH = OY * LYP;          // 40 x 40 outputs per tile
-constexpr int THP = TH + K13 - 1;                    // 52 staged rows
-constexpr int PITCH = TW + K13 - 1 + 1;              // 53 staged pixels per row (odd on purpose)
-constexpr int NW = OX + K13 - 1;                     // 22 input pixels per patch row
-constexpr int NR = OY + K13 - 1;                     // 17 input rows per patch
 constexpr int CG = 16;                               // channels per unit
 constexpr int NPAIR = CG / 2;
-constexpr int kComputeWarps = LXP * LYP / 4;         // 8
+constexpr int kComputeWarps = 8;
 constexpr int kComputeThreads = kComputeWarps * 32;  // 256
 constexpr int kThreads = kComputeThreads + 128;      // + helper warp group (producer, copy, 2 idle)
 constexpr int kLaunchRegs = 152;                      // 384*152 = 58,368: leaves 7,168 registers (1,792 per sub-partition) for one GAP block (128 x 56) per SM
 constexpr int kComputeRegs = 208, kHelperRegs = 40;   // after reallocation: 256*208 + 128*40 = 58,368
-constexpr int TILE_BYTES = THP * PITCH * CG * 2;     // 88,192
-constexpr int OUT_TILE_BYTES = TH * TW * CG * 2;     // 51,200: staged result, reuses the input buffer
 constexpr int WSM_FLOATS = K13 * 7 * NPAIR * 4;      // [i][jj][pair][4]: taps 2jj,2jj+1 of both channels
 constexpr int WSM_BYTES = (WSM_FLOATS * 4 + 127) / 128 * 128;
 constexpr int LKC_BYTES = (CG * 9 * 4 + 127) / 128 * 128;
@@ -62,9 +56,46 @@ constexpr int kMaxSlotBytes = 16384;
 constexpr unsigned kSpinLimit = 1u << 20;    // polls before a wait gives up (each poll may suspend up to the hint)
 constexpr unsigned kSuspendHintNs = 20000;
 
-static_assert(TILE_BYTES % 128 == 0, "tile buffers must keep 128-byte alignment");
-static_assert(OUT_TILE_BYTES <= TILE_BYTES, "the result tile is staged in the input buffer");
-static_assert((OY * PITCH) % 2 == 1 && OX % 4 == 2, "2x2 patch block must start at distinct pixel indices mod 4");
+// Tile geometry.  A lane owns a patch of OY rows x OX columns of outputs; a tile is LXP x LYP
+// patches (always 32, i.e. 8 warps of 4 patches x 8 channel pairs).  The 32 lanes of an LDS.32 hit
+// 32 different banks when the four patches of a warp start at pixel indices that differ mod 4:
+//   kBlock2x2   the four patches form a 2x2 block: needs OX = 2 (mod 4) and an odd OY * PITCH;
+//   otherwise   they are stacked vertically: conflict-free only for an odd OY * PITCH.
+template <int OX_, int OY_, int LXP_, int LYP_, bool kBlock2x2_>
+struct Geom {
+    static constexpr int OX = OX_, OY = OY_, LXP = LXP_, LYP = LYP_;
+    static constexpr bool kBlock2x2 = kBlock2x2_;
+    static constexpr int TW = OX * LXP, TH = OY * LYP;            // outputs per tile
+    static constexpr int THP = TH + K13 - 1;                      // staged rows
+    static constexpr int PITCH = (TW + K13 - 1) | 1;              // staged pixels per row, odd on purpose
+    static constexpr int NW = OX + K13 - 1;                       // input pixels per patch row
+    static constexpr int NR = OY + K13 - 1;                       // input rows per patch
+    static constexpr int TILE_BYTES = THP * PITCH * CG * 2;
+    static constexpr int OUT_TILE_BYTES = TH * TW * CG * 2;       // staged result, reuses the input buffer
+    static_assert(LXP * LYP == 4 * kComputeWarps, "one patch per (warp, q)");
+    static_assert(TILE_BYTES % 128 == 0, "tile buffers must keep 128-byte alignment");
+    static_assert(OUT_TILE_BYTES <= TILE_BYTES, "the result tile is staged in the input buffer");
+    static_assert(kBlock2x2 ? ((OY * PITCH) % 2 == 1 && OX % 4 == 2 && LXP % 2 == 0 && LYP % 2 == 0) : (LYP % 4 == 0),
+                  "patch-to-lane mapping does not fit the tile");
+    __device__ static __forceinline__ void patch_of(int warp, int q, int& lx, int& ly) {
+        if (kBlock2x2) {
+            lx = 2 * (warp % (LXP / 2)) + (q & 1);
+            ly = 2 * (warp / (LXP / 2)) + (q >> 1);
+        } else {
+            lx = warp % LXP;
+            ly = 4 * (warp / LXP) + q;
+        }
+    }
+};
+// 40x40 tiles (52 x 53 x 16 staged, 88,192 bytes): the best ratio of arithmetic to halo, loads and
+// per-unit overhead; used whenever the tile count balances over the SMs.
+using Geom40 = Geom<10, 5, 4, 8, true>;
+// 64x16 tiles (28 x 77 x 16 staged, 68,992 bytes) for maps that 40x40 tiles cover badly (a 64x64
+// patch: 64 % useful outputs) or that give too few 40x40 tiles to occupy the SMs.  OY = 4 makes the
+// four stacked patches of a warp share banks (4-way conflict on the 20 input loads per row):
+// measured 15 % more time per FMA than Geom40, 64x20 tiles (OY = 5, conflict-free) 3 % more;
+// on 64x64 patches the exact cover still wins (45.7 us against 50.3 and 58.0).
+using Geom64 = Geom<8, 4, 8, 4, false>;
 
 struct Params {
     int B, C, Ca, H, W;
@@ -148,6 +179,7 @@ __device__ __forceinline__ int wsm_index(int c, int i, int j) {
     return ((i * 7 + (j >> 1)) * NPAIR + (c >> 1)) * 4 + (j & 1) * 2 + (c & 1);
 }
 
+template <class G>
 __global__ void __maxnreg__(kLaunchRegs)
 stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
                       const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_res,
@@ -155,6 +187,8 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
 {
     // The dynamic shared window starts 1024-byte aligned; indexing it directly (no pointer rounding
     // through integers) lets the compiler keep every access in the shared address space.
+    constexpr int OX = G::OX, OY = G::OY, TW = G::TW, TH = G::TH, PITCH = G::PITCH, NW = G::NW;
+    constexpr int TILE_BYTES = G::TILE_BYTES;
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* tilebuf = smem;                                            // 2 x TILE_BYTES
     float* wsm = reinterpret_cast<float*>(smem + 2 * TILE_BYTES);             // large kernel of the current channel group
@@ -200,7 +234,7 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
                 int k, ch, cx0, cy0, cb, col, row; bool live;
                 __device__ void enter_unit(const Params& p, int first, int stride) {
                     const Unit un = decode_unit(first + k * stride, p);
-                    cx0 = un.tx * TW; cy0 = un.ty * TH; cb = un.b; col = 0; row = 0; ch = 0;
+                    cx0 = un.tx * G::TW; cy0 = un.ty * G::TH; cb = un.b; col = 0; row = 0; ch = 0;
                     live = un.g == 0;
                 }
             };
@@ -255,8 +289,9 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
 
     // ======================= compute warps ========================================================
     reg_inc<kComputeRegs>();
-    const int q = lane >> 3, pr = lane & 7;                 // patch position in the warp's 2x2 block, channel pair
-    const int lx = 2 * (warp & 1) + (q & 1), ly = 2 * (warp >> 1) + (q >> 1);
+    const int q = lane >> 3, pr = lane & 7;                 // which of the warp's four patches, channel pair
+    int lx, ly;
+    G::patch_of(warp, q, lx, ly);
     const int lane_word = ((ly * OY) * PITCH + lx * OX) * NPAIR + pr;
 
     int cur_g = -1, merged_b = -1;
@@ -360,7 +395,7 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
 #pragma unroll 1
         for (int r = OY; r < K13 - 1; ++r) do_row(r);
 
-        // ---- epilogue: round once to bf16, stage the 40x40x16 result in the freed input buffer,
+        // ---- epilogue: round once to bf16, stage the TH x TW x 16 result in the freed input buffer,
         //      one TMA store (the TMA unit clips at the image border) ---------------------------
         compute_bar();                                       // every warp has finished reading this buffer
         {
@@ -428,25 +463,35 @@ inline int sm_count() {
     return n;
 }
 
-// Launches the fast kernel if the problem fits it.  Returns 0 on success, kNotApplicable if the
-// generic kernel has to run instead, or an ESC_ERR_* code.
-inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
-                      const void* w_large, const float* dk, void* out, unsigned* ctrl, cudaStream_t st,
-                      bool dependent, int* launches, std::string* err) {
-    if (K != K13 || dtype != 1 /*bf16*/ || layout != kNHWC) return kNotApplicable;
-    if (Ca % CG != 0 || C % 8 != 0) return kNotApplicable;
-    const int cc = C - Ca;
-    if (cc > 256) return kNotApplicable;
-    if (sm_count() <= 0) return kNotApplicable;
+// Units of one launch with geometry G, and the same count as waves over the SMs.
+template <class G>
+inline long long units_of(int B, int Ca, int H, int W) {
+    return (long long)B * (Ca / CG) * ((W + G::TW - 1) / G::TW) * ((H + G::TH - 1) / G::TH);
+}
+// Relative cost of a launch: every CTA walks ceil(units / SMs) units, each costing its tile area
+// plus a fixed per-unit overhead (table merge, barriers, epilogue: about 200 pixels' worth of
+// arithmetic); per_fma is the geometry's cost per FMA relative to the 40x40 tile.
+template <class G>
+inline double cost_of(int B, int Ca, int H, int W, int sms, double per_fma) {
+    const long long u = units_of<G>(B, Ca, H, W);
+    const long long waves = (u + sms - 1) / sms;
+    return (double)waves * ((double)G::TW * G::TH * per_fma + 200.0);
+}
 
+template <class G>
+inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk,
+                       void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err) {
+    const int cc = C - Ca;
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
-    p.tiles_x = (W + TW - 1) / TW; p.tiles_y = (H + TH - 1) / TH; p.groups = Ca / CG;
-    p.units = (long long)B * p.groups * p.tiles_x * p.tiles_y;
+    p.tiles_x = (W + G::TW - 1) / G::TW; p.tiles_y = (H + G::TH - 1) / G::TH; p.groups = Ca / CG;
+    p.units = units_of<G>(B, Ca, H, W);
     if (p.units > 0x7fffffffLL) return kNotApplicable;
-    p.copy_cc = cc; p.copy_cw = TW; p.copy_cr = 2; p.slot_stride = 128;
+    p.copy_cc = cc; p.copy_cw = G::TW; p.copy_cr = 1; p.slot_stride = 128;
     if (cc > 0) {
-        static const int shapes[6][2] = {{40, 4}, {40, 2}, {40, 1}, {20, 1}, {10, 1}, {5, 1}};
+        // chunk = copy_cw pixels x copy_cr rows of the tile; both divide the tile
+        static_assert(G::TH % 4 == 0 && G::TW % 8 == 0, "copy chunk shapes");
+        const int shapes[6][2] = {{G::TW, 4}, {G::TW, 2}, {G::TW, 1}, {G::TW / 2, 1}, {G::TW / 4, 1}, {G::TW / 8, 1}};
         int pick = -1;
         for (int s = 0; s < 6 && pick < 0; ++s)
             if (cc * 2 * shapes[s][0] * shapes[s][1] <= kMaxSlotBytes) pick = s;
@@ -461,8 +506,8 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     CUtensorMap m_att, m_cin, m_cout, m_res;
     // The halo tile gates the start of the arithmetic: fetch no more than its own 32-byte sectors need
     // (64-byte promotion measured fastest; 128-byte promotion drags the copy-through channels along).
-    if (!make_map(&m_att, x, B, C, H, W, CG, PITCH, THP, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
-    if (!make_map(&m_res, out, B, C, H, W, CG, TW, TH)) return kNotApplicable;
+    if (!make_map(&m_att, x, B, C, H, W, CG, G::PITCH, G::THP, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
+    if (!make_map(&m_res, out, B, C, H, W, CG, G::TW, G::TH)) return kNotApplicable;
     if (cc > 0) {
         if (!make_map(&m_cin, x, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
         if (!make_map(&m_cout, out, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
@@ -470,10 +515,10 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
         m_cin = m_att; m_cout = m_att;
     }
 
-    const size_t smem = 2 * (size_t)TILE_BYTES + WSM_BYTES + LKC_BYTES + (size_t)NSLOT * p.slot_stride + 128;
-    static bool attr_set = false;
+    const size_t smem = 2 * (size_t)G::TILE_BYTES + WSM_BYTES + LKC_BYTES + (size_t)NSLOT * p.slot_stride + 128;
+    static bool attr_set = false;                            // one flag per geometry
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
         attr_set = true;
     }
@@ -490,7 +535,7 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16, m_att, m_cin, m_cout, m_res, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16<G>, m_att, m_cin, m_cout, m_res, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_tma_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -499,6 +544,27 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     }
     ++*launches;
     return 0;
+}
+
+// Launches the fast kernel if the problem fits it.  Returns 0 on success, kNotApplicable if the
+// generic kernel has to run instead, or an ESC_ERR_* code.  *tile_w: in, the tile width asked
+// for (0 = choose by cost); out, the one used.
+inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
+                      const void* w_large, const float* dk, void* out, unsigned* ctrl, cudaStream_t st,
+                      bool dependent, int* launches, std::string* err, int* tile_w) {
+    if (K != K13 || dtype != 1 /*bf16*/ || layout != kNHWC) return kNotApplicable;
+    if (Ca % CG != 0 || C % 8 != 0) return kNotApplicable;
+    if (C - Ca > 256) return kNotApplicable;
+    const int sms = sm_count();
+    if (sms <= 0) return kNotApplicable;
+    const bool use64 = *tile_w == Geom64::TW ||
+                       (*tile_w != Geom40::TW && cost_of<Geom64>(B, Ca, H, W, sms, 1.15) < cost_of<Geom40>(B, Ca, H, W, sms, 1.0));
+    if (use64) {
+        *tile_w = Geom64::TW;
+        return launch_geom<Geom64>(B, C, Ca, H, W, x, w_large, dk, out, ctrl, st, dependent, launches, err);
+    }
+    *tile_w = Geom40::TW;
+    return launch_geom<Geom40>(B, C, Ca, H, W, x, w_large, dk, out, ctrl, st, dependent, launches, err);
 }
 
 }}  // namespace esc::tma

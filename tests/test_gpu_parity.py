@@ -1,5 +1,7 @@
 """GPU parity: the CUDA library, called through the C ABI, against the CPU oracle on the same
 seeded inputs (ESC paper, Section 3.3, Eq. 4).  Tolerances are in tests/util.py."""
+import contextlib
+
 import numpy as np
 import pytest
 
@@ -22,6 +24,16 @@ def pkg():
 
     p.lib()
     return p
+
+
+@contextlib.contextmanager
+def tile_width(pkg, width):
+    """Pins the tile geometry of the TMA-staged kernel for the calls inside (0 = chosen by cost)."""
+    pkg.esc_convattn_set_tile_width(width)
+    try:
+        yield
+    finally:
+        pkg.esc_convattn_set_tile_width(0)
 
 
 def run_forward(pkg, d, C_a, K, dtype, layout, entry="ex"):
@@ -136,6 +148,49 @@ def test_forward_edge_shapes(pkg, oracle, shape, dtype, layout):
     compare_full(pkg, oracle, d, C_a, K, dtype, layout, what=str(shape))
 
 
+TILE_SHAPES = [s for s in EDGE_SHAPES if s[5] == 13 and s[2] % 16 == 0 and s[1] - s[2] <= 256] + [
+    (1, 64, 16, 16, 64, 13),    # exactly one 64x16 tile
+    (2, 64, 16, 17, 65, 13),    # one pixel more in both directions
+    (1, 64, 16, 293, 517, 13),  # ragged in both directions, over a hundred tiles of either geometry
+    (3, 48, 32, 100, 129, 13),  # two channel groups, three images
+]
+
+
+@pytest.mark.parametrize("width", [40, 64])
+@pytest.mark.parametrize("shape", TILE_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_forward_both_tile_geometries(pkg, oracle, shape, width):
+    """Every shape the TMA-staged kernel accepts, on each of its two tile geometries."""
+    B, C, C_a, H, W, K = shape
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=sum(shape) + width, per_image_scale=True, channel_means=True)
+    with tile_width(pkg, width):
+        compare_full(pkg, oracle, d, C_a, K, synth.BF16, synth.NHWC, what=f"{shape} tile {width}")
+        assert pkg.esc_convattn_last_path() == 2 and pkg.esc_convattn_last_tile_width() == width
+
+
+def test_tile_choice_and_policy(pkg):
+    """The cost estimate takes 64x16 tiles for a batch of 64x64 patches and for maps with few tiles,
+    40x40 tiles for the large maps; the override rejects widths that do not exist."""
+    import torch
+
+    def used(B, C, C_a, H, W):
+        x = torch.zeros(B, H, W, C, dtype=torch.bfloat16, device="cuda")
+        wl = torch.zeros(C_a, 13, 13, dtype=torch.bfloat16, device="cuda")
+        dk = torch.zeros(B, C_a, 3, 3, device="cuda")
+        ws = pkg.new_workspace(B, C_a, H, W, 13)
+        pkg.esc_convattn_stencil(x, C_a, 13, wl, dk, torch.empty_like(x), pkg.ESC_NHWC, ws)
+        torch.cuda.synchronize()
+        assert pkg.esc_convattn_device_status(ws) == 0
+        return pkg.esc_convattn_last_tile_width()
+
+    assert used(64, 64, 16, 64, 64) == 64
+    assert used(1, 64, 16, 90, 130) == 64
+    assert used(1, 64, 16, 360, 640) == 40
+    assert used(1, 64, 32, 1080, 1920) == 40
+    with pytest.raises(pkg.EscError):
+        pkg.esc_convattn_set_tile_width(48)
+    assert used(1, 64, 16, 360, 640) == 40      # a rejected value leaves the policy alone
+
+
 @pytest.mark.parametrize("wl_name", ["cfg1_64x64_f32", "cfg2_320x180_f32", "cfg3_640x360_bf16", "cfg4_b64_64x64_bf16"])
 @pytest.mark.parametrize("layout", LAYOUTS)
 @pytest.mark.parametrize("means", [False, True], ids=["zero_mean", "channel_means"])
@@ -145,6 +200,16 @@ def test_forward_workloads_full(pkg, oracle, wl_name, layout, means):
     d = synth.make_workload(wl, channel_means=means)
     compare_full(pkg, oracle, d, wl.C_a, wl.K, wl.dtype, layout, what=wl_name,
                  unit_variance=not means and not wl.per_image_scale)
+
+
+@pytest.mark.parametrize("wl_name,width", [("cfg3_640x360_bf16", 64), ("cfg4_b64_64x64_bf16", 40)])
+def test_forward_workloads_other_geometry(pkg, oracle, wl_name, width):
+    """The bf16 workloads on the tile geometry the cost estimate does not pick for them."""
+    wl = synth.WORKLOADS_BY_NAME[wl_name]
+    d = synth.make_workload(wl, channel_means=True)
+    with tile_width(pkg, width):
+        compare_full(pkg, oracle, d, wl.C_a, wl.K, wl.dtype, synth.NHWC, what=f"{wl_name} tile {width}")
+        assert pkg.esc_convattn_last_tile_width() == width
 
 
 def test_mandated_entry_fp32_nchw(pkg, oracle):
