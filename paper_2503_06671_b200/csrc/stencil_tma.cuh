@@ -41,6 +41,7 @@ constexpr int kNotApplicable = -1;
 constexpr int K13 = 13, P6 = 6;
 constexpr int CG = 16;                               // channels per unit
 constexpr int NPAIR = CG / 2;
+static_assert(CG == 16, "index arithmetic below shifts by 4 for the channel group");
 constexpr int kComputeWarps = 8;
 constexpr int kComputeThreads = kComputeWarps * 32;  // 256
 constexpr int kThreads = kComputeThreads + 128;      // + helper warp group (producer, copy, 2 idle)
@@ -304,19 +305,21 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
         if (un.g != cur_g) {
             if (cur_g >= 0) compute_bar();                  // everyone is done with the old table
             const __nv_bfloat16* wg = p.w_large + (size_t)un.g * CG * K13 * K13;
+            // Element e = 16 * tap + channel: the 16 lanes that share a tap write the 16 words of one
+            // (i, jj, j & 1) group -- no bank conflicts in the scatter, one division per element.
             constexpr int N = CG * K13 * K13, PER = (N + kComputeThreads - 1) / kComputeThreads;
             float v[PER];
 #pragma unroll
-            for (int t = 0; t < PER; ++t) {                 // coalesced, all loads in flight together
-                const int idx = tid + t * kComputeThreads;
-                v[t] = idx < N ? __bfloat162float(wg[idx]) : 0.f;
+            for (int t = 0; t < PER; ++t) {                 // all loads in flight together
+                const int e = tid + t * kComputeThreads;
+                v[t] = e < N ? __bfloat162float(wg[(e & (CG - 1)) * (K13 * K13) + (e >> 4)]) : 0.f;
             }
 #pragma unroll
             for (int t = 0; t < PER; ++t) {
-                const int idx = tid + t * kComputeThreads;
-                if (idx < N) {
-                    const int c = idx / (K13 * K13), tap = idx % (K13 * K13);
-                    const int i = tap / K13, j = tap % K13;
+                const int e = tid + t * kComputeThreads;
+                if (e < N) {
+                    const int c = e & (CG - 1), tap = e >> 4;
+                    const int i = tap / K13, j = tap - i * K13;
                     wsm[wsm_index(c, i, j)] = v[t];
                     if (i >= 5 && i <= 7 && j >= 5 && j <= 7) lkc[c * 9 + (i - 5) * 3 + (j - 5)] = v[t];
                 }
