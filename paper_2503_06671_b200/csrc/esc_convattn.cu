@@ -313,7 +313,7 @@ HostPath g_host;
 
 extern "C" {
 
-int esc_version(void) { return 104; }
+int esc_version(void) { return 105; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
