@@ -8,6 +8,8 @@ from .convattn_oracle import (  # noqa: F401
     forward,
     gap,
     dynkernel,
+    dynkernel_mlp,
+    forward_mlp,
     stencil,
     points,
     set_threads,

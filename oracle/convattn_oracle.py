@@ -103,6 +103,35 @@ def dynkernel(g, w_dyn, b_dyn):
     return dk
 
 
+def dynkernel_mlp(g, w_down, b_down, w_up, b_up, want_hidden=False):
+    """dk[B,C_a,3,3] = W_up GELU(W_down g + b_down) + b_up (Eq. 4 line 2 as written, exact-erf GELU)."""
+    g, gp = _f64(g)
+    B, C_a = (int(v) for v in g.shape)
+    w_down, wdp = _f64(w_down)
+    b_down, bdp = _f64(b_down)
+    w_up, wup = _f64(w_up)
+    b_up, bup = _f64(b_up)
+    h = int(w_down.shape[0])
+    assert 1 <= h <= 256
+    assert w_down.shape == (h, C_a) and b_down.shape == (h,)
+    assert w_up.shape == (9 * C_a, h) and b_up.shape == (9 * C_a,)
+    dk = np.empty((B, C_a, 3, 3), dtype=np.float64)
+    hid = np.empty((B, h), dtype=np.float64)
+    _load().convattn_ref_dynkernel_mlp(gp, B, C_a, h, wdp, bdp, wup, bup, hid.ctypes.data_as(_f64p),
+                                       dk.ctypes.data_as(_f64p))
+    return (dk, hid) if want_hidden else dk
+
+
+def forward_mlp(x, C_a, w_large, w_down, b_down, w_up, b_up, want_mag=False, want_dk=False):
+    """Whole forward with the two-layer estimator: GAP, dynkernel_mlp, stencil, in that order."""
+    dk = dynkernel_mlp(gap(x, C_a), w_down, b_down, w_up, b_up)
+    res = stencil(x, C_a, w_large, dk, want_mag=want_mag)
+    res = list(res) if want_mag else [res]
+    if want_dk:
+        res.append(dk)
+    return res[0] if len(res) == 1 else tuple(res)
+
+
 def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
     """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
     x, xp = _f32(x)

@@ -16,6 +16,10 @@
  *   out[b,c] = F_att[b,c] (*) LK[c]  +  F_att[b,c] (*) dk[b,c]   (Eq. 4, line 3)
  *   out[b, C_a:] = F_idt                                         (Concat, Eq. 4 line 4)
  *
+ * convattn_ref_dynkernel_mlp is the estimator exactly as Eq. 4 line 2 writes it,
+ *   dk[b] = W_up . phi(W_down . g[b] + b_down) + b_up,   phi(t) = t * Phi(t)   (GELU, exact erf form)
+ * with hidden width h; the other stages are shared.
+ *
  * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
  * Everything is accumulated in double precision with direct nested loops in
  * the order written above: no tiling, no merging of the two kernels, no reuse.
@@ -29,7 +33,10 @@
  * Pinned by tests/test_oracle_pins.py (impulse response, constant-input closed
  * form, zero generator vs a library convolution, scatter-form brute force on
  * tiny inputs, linearity laws, the Eq. 5 merge identity, permutation / batch
- * independence, and the GAP->dk stage on non-zero-mean data).
+ * independence, and the GAP->dk stage on non-zero-mean data); the two-layer
+ * estimator by tabulated values of the normal distribution function, the
+ * reflection law of phi, its two linear limits (which reduce it to the one-layer
+ * estimator with composed weights) and a math.erf brute force.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -63,6 +70,39 @@ void convattn_ref_dynkernel(const double *g, int B, int C_a, const double *w_dyn
                 s += w_dyn[(size_t)o * C_a + c] * g[(size_t)b * C_a + c];
             dk[(size_t)b * 9 * C_a + o] = s;
         }
+}
+
+/* Gaussian error linear unit: phi(t) = t * Phi(t), Phi the standard normal distribution function,
+ * Phi(t) = (1 + erf(t / sqrt 2)) / 2 = erfc(-t / sqrt 2) / 2; the erfc form keeps full relative
+ * accuracy in the left tail, where 1 + erf cancels. */
+static double gelu(double t)
+{
+    return t * 0.5 * erfc(-t / sqrt(2.0));
+}
+
+/* Kernel estimator of Eq. 4 line 2: Conv_up(phi(Conv_down(g))), both 1x1 convolutions on a 1x1 map, i.e.
+ * two dense layers with bias.  w_down [h, C_a], b_down [h], w_up [9*C_a, h], b_up [9*C_a]; hidden (may be
+ * NULL) receives phi(...) [B, h]; dk is [B, C_a*9] with the same output order as the one-layer estimator. */
+void convattn_ref_dynkernel_mlp(const double *g, int B, int C_a, int h, const double *w_down,
+                                const double *b_down, const double *w_up, const double *b_up,
+                                double *hidden, double *dk)
+{
+    for (int b = 0; b < B; ++b) {
+        double a[256];                       /* h <= 256, checked by the caller */
+        for (int j = 0; j < h; ++j) {
+            double t = b_down[j];
+            for (int c = 0; c < C_a; ++c)
+                t += w_down[(size_t)j * C_a + c] * g[(size_t)b * C_a + c];
+            a[j] = gelu(t);
+            if (hidden) hidden[(size_t)b * h + j] = a[j];
+        }
+        for (int o = 0; o < 9 * C_a; ++o) {
+            double s = b_up[o];
+            for (int j = 0; j < h; ++j)
+                s += w_up[(size_t)o * h + j] * a[j];
+            dk[(size_t)b * 9 * C_a + o] = s;
+        }
+    }
 }
 
 /* One output value of an attention channel (c < C_a): large-kernel taps, then the

@@ -126,6 +126,24 @@ def make_inputs(B, C, C_a, H, W, K=13, dtype=F32, seed=0, per_image_scale=False,
     }
 
 
+def make_estimator_mlp(C_a, h, dtype=F32, seed=0):
+    """Weights of the two-layer kernel estimator (hidden width h), float32 arrays rounded to `dtype`:
+    w_down [h,C_a], b_down [h] ~ U(-1,1)/sqrt(C_a) * 4 (so that the pre-activations of pooled
+    features of order one fall across the curved part of the activation, not only its linear tails),
+    w_up [9*C_a,h], b_up [9*C_a] kaiming-uniform with fan_in h."""
+    rng = np.random.default_rng(1000003 * (seed + 1) + h)
+    w_down = 4.0 * _kaiming_uniform(rng, (h, C_a), C_a)
+    b_down = 4.0 * _kaiming_uniform(rng, (h,), C_a)
+    w_up = _kaiming_uniform(rng, (9 * C_a, h), h)
+    b_up = _kaiming_uniform(rng, (9 * C_a,), h)
+    return {
+        "w_down": round_to(w_down, dtype),
+        "b_down": round_to(b_down, dtype),
+        "w_up": round_to(w_up, dtype),
+        "b_up": round_to(b_up, dtype),
+    }
+
+
 def make_workload(wl: Workload, channel_means=False):
     return make_inputs(wl.B, wl.C, wl.C_a, wl.H, wl.W, wl.K, wl.dtype, wl.seed, wl.per_image_scale,
                        channel_means)
