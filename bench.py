@@ -31,7 +31,8 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one stencil-kernel launch from the ncu capture summarised under
 # profiles/, keyed by (workload, layout, library version the capture was taken with).  Reported only while the
 # library still has that version; otherwise the kernel has changed since and the figure is withheld.
-NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", 105): 29.56e6 + 0.30e6}
+# (Version 106 added the two-layer estimator to stage 1; the stencil kernel is the one captured at 105.)
+NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", v): 29.56e6 + 0.30e6 for v in (105, 106)}
 
 
 def peaks():
@@ -332,6 +333,9 @@ def main():
 
     ms_kernel = timed(lambda i: pkg.esc_convattn_stencil(xs[i % n_rot], wl.C_a, wl.K, wl_d, dk, outs[i % n_rot], lay_code, ws))
     ms_gap = timed(lambda i: pkg.esc_convattn_dynkernel(xs[i % n_rot], wl.C_a, wd_d, bd_d, dk, lay_code, ws))
+    # the whole step once more with the paper's two-layer estimator (hidden width 8, exact GELU), for comparison
+    mlp_d = [torch.from_numpy(v).to(tdt).cuda() for v in synth.make_estimator_mlp(wl.C_a, 8, wl.dtype, wl.seed).values()]
+    ms_step_mlp = timed(lambda i: pkg.esc_convattn_forward_mlp(xs[i % n_rot], wl.C_a, wl.K, wl_d, *mlp_d, outs[i % n_rot], lay_code, ws))
 
     pk = peaks()
     flops = 2.0 * wl.K * wl.K * wl.C_a * wl.pixels                    # merged 169-tap form, Eq. 5
@@ -382,11 +386,12 @@ def main():
                        "storage": wl.dtype, "layout": args.layout, "sharding": "replicas: one image batch per GPU, no collective",
                        "l2": f"inputs larger than L2: {n_rot} rotating (x,out) pairs, {n_rot * 2 * tensor_bytes / 1e6:.0f} MB",
                        "stencil_path": {1: "generic", 2: "tma"}.get(path, str(path)),
-                       "launch": launch_mode},
+                       "launch": launch_mode, "estimator": "one linear layer"},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
             "gpu_launches": launches_per_step * args.steps,
             "launches_per_step": launches_per_step, "stencil_stage_launches": stencil_launches,
             "GB_per_s_whole_step": alg_bytes / (ms_step * 1e-3) / 1e9,
+            "ms_per_step_two_layer_estimator_h8": ms_step_mlp,
         }))
     if world > 1:
         dist.destroy_process_group()

@@ -100,6 +100,30 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W,
                            void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The forward pass with the kernel estimator exactly as Eq. 4 line 2 of the paper writes it:
+ *   DK = Conv_up(phi(Conv_down(GAP(F_att)))),  phi(t) = t * Phi(t)  (Gaussian error linear unit,
+ * exact form through erfc, not the tanh approximation); both 1x1 convolutions carry a bias
+ * (pass zeros for a bias-free estimator).  Section 3.3 sets the hidden width h to 4 or 8, the
+ * larger model of the appendix to 24.
+ *   w_down  [hidden,C_a]    b_down [hidden]
+ *   w_up    [9*C_a,hidden]  b_up   [9*C_a]      row o = c*9 + i*3 + j, 1 <= hidden <= 128
+ * All four in the tensor's dtype on the device; everything else as for esc_convattn_forward_ex,
+ * including the workspace size.  ESC_ERR_SHAPE for hidden outside 1..128.
+ */
+int esc_convattn_forward_mlp(const void* x, int B, int C, int C_a, int H, int W, int K,
+                             const void* w_large, const void* w_down, const void* b_down,
+                             const void* w_up, const void* b_up, int hidden,
+                             void* out, int dtype, int layout,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Stage 1 alone with that two-layer estimator: writes dk_out [B,C_a,3,3] fp32. */
+int esc_convattn_dynkernel_mlp(const void* x, int B, int C, int C_a, int H, int W,
+                               const void* w_down, const void* b_down,
+                               const void* w_up, const void* b_up, int hidden, float* dk_out,
+                               int dtype, int layout,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Stage 1 for callers that must not allocate device memory.  (The paper has no counterpart:
  * this is a packaging variant of esc_convattn_dynkernel, same arithmetic, same result.)
  *

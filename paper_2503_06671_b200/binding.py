@@ -44,6 +44,8 @@ def lib():
         L.esc_convattn_workspace_bytes.restype = sz
         L.esc_convattn_workspace_init.argtypes = [vp, sz, vp]
         L.esc_convattn_dynkernel.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_forward_mlp.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, i, vp, i, i, vp, sz, vp]
+        L.esc_convattn_dynkernel_mlp.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, i, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -53,7 +55,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_stencil", "esc_convattn_forward_host",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_stencil", "esc_convattn_forward_host",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -171,6 +173,27 @@ def esc_convattn_dynkernel(x, C_a, w_dyn, b_dyn, dk_out, layout, workspace, stre
                                         _dtype_code(x), layout, _ptr(workspace),
                                         workspace.numel() * workspace.element_size(), _stream(stream)),
            "esc_convattn_dynkernel")
+    return dk_out
+
+
+def esc_convattn_forward_mlp(x, C_a, K, w_large, w_down, b_down, w_up, b_up, out, layout, workspace, stream=None):
+    """Forward pass with the two-layer kernel estimator (hidden width = w_down.shape[0])."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_forward_mlp(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_down), _ptr(b_down),
+                                          _ptr(w_up), _ptr(b_up), int(w_down.shape[0]), _ptr(out), _dtype_code(x),
+                                          layout, _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                          _stream(stream)),
+           "esc_convattn_forward_mlp")
+    return out
+
+
+def esc_convattn_dynkernel_mlp(x, C_a, w_down, b_down, w_up, b_up, dk_out, layout, workspace, stream=None):
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_dynkernel_mlp(_ptr(x), B, C, C_a, H, W, _ptr(w_down), _ptr(b_down), _ptr(w_up),
+                                            _ptr(b_up), int(w_down.shape[0]), _ptr(dk_out), _dtype_code(x), layout,
+                                            _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                            _stream(stream)),
+           "esc_convattn_dynkernel_mlp")
     return dk_out
 
 

@@ -123,8 +123,15 @@ int check_workspace(const Problem& p, const void* ws, size_t bytes) {
 }
 
 // ---- stage 1 ------------------------------------------------------------------------------
+// The estimator's weights: one linear layer (hidden == 0: w_last [9*Ca][Ca]) or two layers with the
+// GELU between them (w_down [hidden][Ca], b_down [hidden], w_last = w_up [9*Ca][hidden]).
+struct Estimator {
+    const void *w_last, *b_last, *w_down, *b_down;
+    int hidden;
+};
+
 template <typename T, int LAYOUT>
-int launch_gap_t(const Problem& p, const void* x, const void* w_dyn, const void* b_dyn,
+int launch_gap_t(const Problem& p, const void* x, const Estimator& est,
                  const Workspace& w, float* dk_out, cudaStream_t st) {
     const int S = slabs_for(p.B, (long long)p.H * p.W);
     int sms = esc::tma::sm_count();
@@ -147,21 +154,32 @@ int launch_gap_t(const Problem& p, const void* x, const void* w_dyn, const void*
         carveout_set = true;
     }
     esc::gap_dynkernel<T, LAYOUT><<<grid, esc::kGapThreads, smem, st>>>(
-        static_cast<const T*>(x), p.B, p.C, p.Ca, p.H, p.W, S, static_cast<const T*>(w_dyn),
-        static_cast<const T*>(b_dyn), w.partial, w.arrivals, dk_out);
+        static_cast<const T*>(x), p.B, p.C, p.Ca, p.H, p.W, S, static_cast<const T*>(est.w_last),
+        static_cast<const T*>(est.b_last), static_cast<const T*>(est.w_down), static_cast<const T*>(est.b_down),
+        est.hidden, w.partial, w.arrivals, dk_out);
     ESC_CUDA(cudaGetLastError());
     ++g_last_launches;
     return ESC_OK;
 }
 
-int launch_gap(const Problem& p, const void* x, const void* w_dyn, const void* b_dyn,
+int launch_gap(const Problem& p, const void* x, const Estimator& est,
                const Workspace& w, float* dk_out, cudaStream_t st) {
     if ((long long)p.B * esc::kMaxSlabs > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
     if (p.dtype == ESC_F32)
-        return p.layout == ESC_NCHW ? launch_gap_t<float, esc::kNCHW>(p, x, w_dyn, b_dyn, w, dk_out, st)
-                                    : launch_gap_t<float, esc::kNHWC>(p, x, w_dyn, b_dyn, w, dk_out, st);
-    return p.layout == ESC_NCHW ? launch_gap_t<__nv_bfloat16, esc::kNCHW>(p, x, w_dyn, b_dyn, w, dk_out, st)
-                                : launch_gap_t<__nv_bfloat16, esc::kNHWC>(p, x, w_dyn, b_dyn, w, dk_out, st);
+        return p.layout == ESC_NCHW ? launch_gap_t<float, esc::kNCHW>(p, x, est, w, dk_out, st)
+                                    : launch_gap_t<float, esc::kNHWC>(p, x, est, w, dk_out, st);
+    return p.layout == ESC_NCHW ? launch_gap_t<__nv_bfloat16, esc::kNCHW>(p, x, est, w, dk_out, st)
+                                : launch_gap_t<__nv_bfloat16, esc::kNHWC>(p, x, est, w, dk_out, st);
+}
+
+int check_estimator(const Problem& p, const Estimator& e) {
+    if (!e.w_last || !e.b_last) return ESC_ERR_NULL;
+    if (!aligned(e.w_last, p.es()) || !aligned(e.b_last, p.es())) return ESC_ERR_ALIGN;
+    if (e.hidden == 0) return ESC_OK;
+    if (e.hidden < 0 || e.hidden > esc::kMaxHidden) return ESC_ERR_SHAPE;
+    if (!e.w_down || !e.b_down) return ESC_ERR_NULL;
+    if (!aligned(e.w_down, p.es()) || !aligned(e.b_down, p.es())) return ESC_ERR_ALIGN;
+    return ESC_OK;
 }
 
 // ---- stage 2 ------------------------------------------------------------------------------
@@ -265,10 +283,10 @@ int get_scratch(size_t need, cudaStream_t st, void** out) {
     return ESC_OK;
 }
 
-int forward_impl(const Problem& p, const void* x, const void* w_large, const void* w_dyn, const void* b_dyn,
+int forward_impl(const Problem& p, const void* x, const void* w_large, const Estimator& est,
                  void* out, void* ws, cudaStream_t st) {
     const Workspace w = carve(ws, p.B, p.Ca);
-    int rc = launch_gap(p, x, w_dyn, b_dyn, w, w.dk, st);
+    int rc = launch_gap(p, x, est, w, w.dk, st);
     if (rc != ESC_OK) return rc;
     return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
 }
@@ -313,7 +331,7 @@ HostPath g_host;
 
 extern "C" {
 
-int esc_version(void) { return 105; }
+int esc_version(void) { return 106; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
@@ -365,7 +383,8 @@ int esc_convattn_forward_ex(const void* x, int B, int C, int C_a, int H, int W, 
     if (!aligned(w_large, p.es()) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
     rc = check_workspace(p, workspace, workspace_bytes_);
     if (rc != ESC_OK) return rc;
-    return forward_impl(p, x, w_large, w_dyn, b_dyn, out, workspace, static_cast<cudaStream_t>(stream));
+    return forward_impl(p, x, w_large, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, out, workspace,
+                        static_cast<cudaStream_t>(stream));
 }
 
 int esc_convattn_forward(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
@@ -381,7 +400,7 @@ int esc_convattn_forward(const void* x, int B, int C, int C_a, int H, int W, int
     void* ws = nullptr;
     rc = get_scratch(workspace_bytes(B, C_a, (long long)H * W), static_cast<cudaStream_t>(stream), &ws);
     if (rc != ESC_OK) return rc;
-    return forward_impl(p, x, w_large, w_dyn, b_dyn, out, ws, static_cast<cudaStream_t>(stream));
+    return forward_impl(p, x, w_large, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, out, ws, static_cast<cudaStream_t>(stream));
 }
 
 int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W, const void* w_dyn,
@@ -395,7 +414,47 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W, c
     if (!aligned(x, 16) || !aligned(dk_out, 4) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
     rc = check_workspace(p, workspace, workspace_bytes_);
     if (rc != ESC_OK) return rc;
-    return launch_gap(p, x, w_dyn, b_dyn, carve(workspace, B, C_a), dk_out, static_cast<cudaStream_t>(stream));
+    return launch_gap(p, x, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, carve(workspace, B, C_a), dk_out,
+                      static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_forward_mlp(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                             const void* w_down, const void* b_down, const void* w_up, const void* b_up, int hidden,
+                             void* out, int dtype, int layout, void* workspace, size_t workspace_bytes_,
+                             void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (hidden < 1) return ESC_ERR_SHAPE;
+    if (!w_large) return ESC_ERR_NULL;
+    const Estimator est{w_up, b_up, w_down, b_down, hidden};
+    rc = check_estimator(p, est);
+    if (rc != ESC_OK) return rc;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, p.es())) return ESC_ERR_ALIGN;
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    return forward_impl(p, x, w_large, est, out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_dynkernel_mlp(const void* x, int B, int C, int C_a, int H, int W, const void* w_down,
+                               const void* b_down, const void* w_up, const void* b_up, int hidden, float* dk_out,
+                               int dtype, int layout, void* workspace, size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C_a, H, W, 1, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (hidden < 1) return ESC_ERR_SHAPE;
+    if (!x || !dk_out) return ESC_ERR_NULL;
+    const Estimator est{w_up, b_up, w_down, b_down, hidden};
+    rc = check_estimator(p, est);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(x, 16) || !aligned(dk_out, 4)) return ESC_ERR_ALIGN;
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    return launch_gap(p, x, est, carve(workspace, B, C_a), dk_out, static_cast<cudaStream_t>(stream));
 }
 
 int esc_convattn_dynkernel_static(const void* x, int B, int C, int C_a, int H, int W, const void* w_dyn,
@@ -427,7 +486,7 @@ int esc_convattn_dynkernel_static(const void* x, int B, int C, int C_a, int H, i
     w.arrivals = base;
     w.dk = dk_out;
     w.partial = reinterpret_cast<float*>(base + kStaticMaxImages);
-    return launch_gap(p, x, w_dyn, b_dyn, w, dk_out, st);
+    return launch_gap(p, x, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, w, dk_out, st);
 }
 
 int esc_convattn_stencil(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
@@ -516,7 +575,7 @@ int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, 
     ESC_CUDA(cudaMemcpyAsync(wts, w_large_host, n_wl * es, cudaMemcpyHostToDevice, h.st));
     ESC_CUDA(cudaMemcpyAsync(wts + off_wd, w_dyn_host, n_wd * es, cudaMemcpyHostToDevice, h.st));
     ESC_CUDA(cudaMemcpyAsync(wts + off_bd, b_dyn_host, n_bd * es, cudaMemcpyHostToDevice, h.st));
-    rc = forward_impl(p, h.x, wts, wts + off_wd, wts + off_bd, h.out, h.ws, h.st);
+    rc = forward_impl(p, h.x, wts, Estimator{wts + off_wd, wts + off_bd, nullptr, nullptr, 0}, h.out, h.ws, h.st);
     if (rc != ESC_OK) return rc;
     ESC_CUDA(cudaMemcpyAsync(out_host, h.out, xbytes, cudaMemcpyDeviceToHost, h.st));
     ESC_CUDA(cudaStreamSynchronize(h.st));

@@ -1,8 +1,12 @@
 // Kernel (a): global average pooling of the attention channels fused with the kernel
-// estimator (ESC paper, Section 3.3, Eq. 4 line 2, estimator reduced to one linear layer).
+// estimator (ESC paper, Section 3.3, Eq. 4 line 2), either reduced to one linear layer
 //
 //   g[b,c]  = (1/HW) sum_{y,x} x[b,c,y,x]            c < C_a
 //   dk[b,o] = b_dyn[o] + sum_c w_dyn[o,c] g[b,c]     o = c*9 + i*3 + j
+// or, with hidden > 0, the estimator as Eq. 4 line 2 writes it -- two 1x1 convolutions on the pooled
+// vector with the Gaussian error linear unit phi(t) = t * Phi(t) between them:
+//   a[b,j]  = phi(b_down[j] + sum_c w_down[j,c] g[b,c])      j < hidden
+//   dk[b,o] = b_up[o] + sum_j w_up[o,j] a[b,j]
 //
 // Every image is cut into S slabs so that a single large image still spreads over the machine;
 // the B*S work items are walked by a persistent grid of small blocks (4 warps -- one per SM sub-partition --, at most one block
@@ -13,7 +17,7 @@
 // shuffles and one pass through shared memory, and writes C_a partial sums.  The block that
 // arrives last for an image (a wrapping arrival counter, so no counter ever needs re-zeroing)
 // adds the S partial sums in a fixed order -- the result is bitwise reproducible -- and
-// evaluates the linear layer.
+// evaluates the estimator.
 #pragma once
 #include "common.cuh"
 
@@ -21,11 +25,17 @@ namespace esc {
 
 constexpr int kGapThreads = 128;
 constexpr int kGapWarps = kGapThreads / 32;
+constexpr int kMaxHidden = kGapThreads;        // hidden activations live in the block's scratch
+
+// phi(t) = t * Phi(t) with Phi(t) = erfc(-t / sqrt 2) / 2 (no cancellation in the left tail).
+__device__ __forceinline__ float gelu_exact(float t) { return 0.5f * t * erfcf(-0.70710678118654752f * t); }
 
 template <typename T, int LAYOUT>
 __global__ void __maxnreg__(56)
 gap_dynkernel(const T* __restrict__ x, int B, int C, int Ca, int H, int W, int S,
-              const T* __restrict__ w_dyn, const T* __restrict__ b_dyn,
+              const T* __restrict__ w_dyn, const T* __restrict__ b_dyn,   // last layer: [9*Ca][n_in], [9*Ca]
+              const T* __restrict__ w_down, const T* __restrict__ b_down, // hidden layer [hidden][Ca], [hidden] (hidden > 0)
+              int hidden,                      // 0: one linear layer, n_in = Ca; else n_in = hidden
               float* __restrict__ partial,     // [B][S][Ca]
               unsigned* __restrict__ arrivals, // [B]
               float* __restrict__ dk)          // [B][9*Ca]
@@ -144,7 +154,7 @@ gap_dynkernel(const T* __restrict__ x, int B, int C, int Ca, int H, int W, int S
     // (all threads busy, loads independent), then the ng group sums are added in order.
     const int ng = Ca <= kGapThreads / 2 ? kGapThreads / Ca : 1;
     if (ng > 1) {
-        float* red = wsum;                                   // [ng][Ca] <= 256 floats; the warp sums are dead
+        float* red = wsum;                                   // [ng][Ca] <= kGapThreads floats; the warp sums are dead
         const int c = tid % Ca, j = tid / Ca;
         if (j < ng) {
             const float* pp = partial + (size_t)b * S * Ca + c;
@@ -173,16 +183,29 @@ gap_dynkernel(const T* __restrict__ x, int B, int C, int Ca, int H, int W, int S
         }
     }
     __syncthreads();
+    const float* vin = gmean;                                // input of the last layer
+    int n_in = Ca;
+    if (hidden > 0) {
+        float* act = wsum;                                   // the warp and group sums are dead
+        for (int j = tid; j < hidden; j += kGapThreads) {
+            float t = Elem<T>::to_f32(b_down[j]);
+            const T* wr = w_down + (size_t)j * Ca;
+            for (int c = 0; c < Ca; ++c) t = fmaf(Elem<T>::to_f32(wr[c]), gmean[c], t);
+            act[j] = gelu_exact(t);
+        }
+        __syncthreads();
+        vin = act; n_in = hidden;
+    }
     for (int o = tid; o < 9 * Ca; o += kGapThreads) {
         float acc = Elem<T>::to_f32(b_dyn[o]);
-        const T* wr = w_dyn + (size_t)o * Ca;
-        for (int c0 = 0; c0 < Ca; c0 += 16) {                // sixteen independent loads, FMAs in channel order
+        const T* wr = w_dyn + (size_t)o * n_in;
+        for (int c0 = 0; c0 < n_in; c0 += 16) {              // sixteen independent loads, FMAs in input order
             float wv[16];
 #pragma unroll
-            for (int u = 0; u < 16; ++u) wv[u] = c0 + u < Ca ? Elem<T>::to_f32(wr[c0 + u]) : 0.f;
+            for (int u = 0; u < 16; ++u) wv[u] = c0 + u < n_in ? Elem<T>::to_f32(wr[c0 + u]) : 0.f;
 #pragma unroll
             for (int u = 0; u < 16; ++u)
-                if (c0 + u < Ca) acc = fmaf(wv[u], gmean[c0 + u], acc);
+                if (c0 + u < n_in) acc = fmaf(wv[u], vin[c0 + u], acc);
         }
         dk[(size_t)b * 9 * Ca + o] = acc;
     }
