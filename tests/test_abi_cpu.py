@@ -76,6 +76,18 @@ def test_host_side_rejections_launch_nothing(L):
     assert L.esc_convattn_stencil(X, 1, 64, 16, 8, 8, 13, Wl, Wd, X + 16, 0, 0, None, 0, None) == 5
     assert L.esc_convattn_forward_host(None, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 1
     assert L.esc_convattn_forward_host(X, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 7, 0) == 3
+    # two-layer estimator: the same checks plus the hidden width
+    Wu, Bu = 0x30300000, 0x30400000
+
+    def mlp(x=X, wd=Wd, bd=Bd, wu=Wu, bu=Bu, h=8, out=O, ws=WS, wsb=big, K=13):
+        return L.esc_convattn_forward_mlp(x, 1, 64, 16, 32, 32, K, Wl, wd, bd, wu, bu, h, out, 1, 1, ws, wsb, None)
+
+    assert mlp(h=0) == 2 and mlp(h=-4) == 2 and mlp(h=129) == 2 and mlp(K=12) == 2
+    assert mlp(wd=None) == 1 and mlp(bd=None) == 1 and mlp(wu=None) == 1 and mlp(bu=None) == 1 and mlp(x=None) == 1
+    assert mlp(wu=Wu + 1) == 4 and mlp(out=X) == 5 and mlp(wsb=64) == 6
+    assert L.esc_convattn_dynkernel_mlp(X, 1, 64, 16, 8, 8, Wd, Bd, Wu, Bu, 0, O, 0, 0, WS, big, None) == 2
+    assert L.esc_convattn_dynkernel_mlp(X, 1, 64, 16, 8, 8, Wd, Bd, Wu, Bu, 8, None, 0, 0, WS, big, None) == 1
+    assert L.esc_convattn_set_tile_width(48) == 3 and L.esc_convattn_set_tile_width(0) == 0
     assert L.esc_convattn_workspace_init(None, 1024, None) == 6
     assert L.esc_convattn_device_status(None, None) == 6
 
