@@ -11,6 +11,9 @@ from .convattn_oracle import (  # noqa: F401
     dynkernel_mlp,
     forward_mlp,
     stencil,
+    pointwise,
+    stencil_pw,
+    forward_pw,
     points,
     set_threads,
     max_threads,

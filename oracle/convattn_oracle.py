@@ -132,6 +132,48 @@ def forward_mlp(x, C_a, w_large, w_down, b_down, w_up, b_up, want_mag=False, wan
     return res[0] if len(res) == 1 else tuple(res)
 
 
+def pointwise(x, C_a, w_point, want_abs=False):
+    """xm[B,C_a,H,W] = 1x1 convolution of the attention channels with w_point[C_a,C_a] (Eq. 5, LK^c), no bias."""
+    x, xp = _f32(x)
+    B, C, H, W = (int(v) for v in x.shape)
+    w_point, wp = _f64(w_point)
+    assert w_point.shape == (C_a, C_a) and C_a <= C
+    xm = np.empty((B, C_a, H, W), dtype=np.float64)
+    xabs = np.empty((B, C_a, H, W), dtype=np.float64) if want_abs else None
+    _load().convattn_ref_pointwise(xp, B, C, C_a, H, W, wp, xm.ctypes.data_as(_f64p),
+                                   xabs.ctypes.data_as(_f64p) if want_abs else None)
+    return (xm, xabs) if want_abs else xm
+
+
+def stencil_pw(x, C_a, w_large, w_point, dk, want_mag=False):
+    """Decomposed form of Eq. 5 with an explicit dk: (F_att * LK^c) * (ZP(dk) + LK^s); other channels copied."""
+    x, xp = _f32(x)
+    w_large, wp = _f64(w_large)
+    K = int(w_large.shape[-1])
+    B, C, H, W = _dims(x, C_a, K)
+    assert w_large.shape == (C_a, K, K)
+    dk, dp = _f64(dk)
+    assert dk.size == B * C_a * 9
+    xm, xabs = pointwise(x, C_a, w_point, want_abs=True)
+    out = np.empty((B, C, H, W), dtype=np.float64)
+    mag = np.empty((B, C_a, H, W), dtype=np.float64) if want_mag else None
+    _load().convattn_ref_stencil_mixed(
+        xp, xm.ctypes.data_as(_f64p), xabs.ctypes.data_as(_f64p), B, C, C_a, H, W, K, wp, dp,
+        out.ctypes.data_as(_f64p), mag.ctypes.data_as(_f64p) if want_mag else None,
+    )
+    return (out, mag) if want_mag else out
+
+
+def forward_pw(x, C_a, w_large, w_point, w_dyn, b_dyn, want_mag=False, want_dk=False):
+    """Whole forward in the decomposed form: dk from GAP(F_att) (one-layer estimator), then stencil_pw."""
+    dk = dynkernel(gap(x, C_a), w_dyn, b_dyn)
+    res = stencil_pw(x, C_a, w_large, w_point, dk, want_mag=want_mag)
+    res = list(res) if want_mag else [res]
+    if want_dk:
+        res.append(dk)
+    return res[0] if len(res) == 1 else tuple(res)
+
+
 def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
     """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
     x, xp = _f32(x)

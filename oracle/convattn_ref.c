@@ -20,6 +20,11 @@
  *   dk[b] = W_up . phi(W_down . g[b] + b_down) + b_up,   phi(t) = t * Phi(t)   (GELU, exact erf form)
  * with hidden width h; the other stages are shared.
  *
+ * convattn_ref_pointwise + convattn_ref_stencil_mixed are the decomposed form of Eq. 5,
+ *   out[b,:C_a] = (F_att (*) LK^c) (*) (ZP(dk) + LK^s),  LK^c a 1x1 convolution over the C_a channels,
+ * taken in that order: mix first, then the depth-wise stage on the mixed features; dk still
+ * comes from GAP(F_att) as in Eq. 4 line 2.
+ *
  * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
  * Everything is accumulated in double precision with direct nested loops in
  * the order written above: no tiling, no merging of the two kernels, no reuse.
@@ -36,7 +41,9 @@
  * independence, and the GAP->dk stage on non-zero-mean data); the two-layer
  * estimator by tabulated values of the normal distribution function, the
  * reflection law of phi, its two linear limits (which reduce it to the one-layer
- * estimator with composed weights) and a math.erf brute force.
+ * estimator with composed weights) and a math.erf brute force; the decomposed form
+ * by the identity mix, library 1x1 + depth-wise convolutions, the commutation with a
+ * channel-independent spatial kernel, permutation mixes and a brute force.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -169,6 +176,73 @@ void convattn_ref_forward(const float *x, int B, int C, int C_a, int H, int W, i
     convattn_ref_gap(x, B, C, C_a, H, W, g_out);
     convattn_ref_dynkernel(g_out, B, C_a, w_dyn, b_dyn, dk_out);
     convattn_ref_stencil(x, B, C, C_a, H, W, K, w_large, dk_out, 0, H, out, mag);
+}
+
+/* Point-wise large-kernel filter LK^c of the decomposed form (Eq. 5, first factor F_att (*) LK^c):
+ * a 1x1 convolution over the attention channels, no bias.
+ *   xm[b,n,y,x] = sum_k w_point[n,k] * x[b,k,y,x]        n, k < C_a
+ * xm is [B, C_a, H, W]; xabs (optional) receives sum_k |w_point[n,k] * x[b,k,y,x]|. */
+void convattn_ref_pointwise(const float *x, int B, int C, int C_a, int H, int W, const double *w_point,
+                            double *xm, double *xabs)
+{
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < C_a; ++n)
+            for (int y = 0; y < H; ++y)
+                for (int xx = 0; xx < W; ++xx) {
+                    double s = 0.0, m = 0.0;
+                    for (int k = 0; k < C_a; ++k) {
+                        double t = w_point[(size_t)n * C_a + k] * (double)x[IDX4(b, k, y, xx, C, H, W)];
+                        s += t;
+                        m += fabs(t);
+                    }
+                    xm[IDX4(b, n, y, xx, C_a, H, W)] = s;
+                    if (xabs) xabs[IDX4(b, n, y, xx, C_a, H, W)] = m;
+                }
+}
+
+/* Eq. 5, second factor: the mixed features xm [B,C_a,H,W] convolved depth-wise with LK^s and with
+ * the dynamic 3x3 kernel (the two convolutions of Eq. 4 line 3, summed; same taps as ZP(DK) + LK^s),
+ * zero padding; identity channels copied from x.  out is [B,C,H,W]; mag (optional) [B,C_a,H,W]
+ * receives sum |w| * xabs over the same taps when xabs is given, else sum |w * xm|. */
+void convattn_ref_stencil_mixed(const float *x, const double *xm, const double *xabs, int B, int C, int C_a,
+                                int H, int W, int K, const double *w_large, const double *dk, double *out,
+                                double *mag)
+{
+    const int P = (K - 1) / 2;
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C; ++c)
+            for (int y = 0; y < H; ++y)
+                for (int xx = 0; xx < W; ++xx) {
+                    if (c >= C_a) {
+                        out[IDX4(b, c, y, xx, C, H, W)] = (double)x[IDX4(b, c, y, xx, C, H, W)];
+                        continue;
+                    }
+                    double s = 0.0, m = 0.0;
+                    for (int i = 0; i < K; ++i)
+                        for (int j = 0; j < K; ++j) {
+                            int yy = y + i - P, xc = xx + j - P;
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W) {
+                                size_t q = IDX4(b, c, yy, xc, C_a, H, W);
+                                double w = w_large[((size_t)c * K + i) * K + j];
+                                s += w * xm[q];
+                                m += fabs(w) * (xabs ? xabs[q] : fabs(xm[q]));
+                            }
+                        }
+                    for (int i = 0; i < 3; ++i)
+                        for (int j = 0; j < 3; ++j) {
+                            int yy = y + i - 1, xc = xx + j - 1;
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W) {
+                                size_t q = IDX4(b, c, yy, xc, C_a, H, W);
+                                double w = dk[(size_t)b * 9 * C_a + c * 9 + i * 3 + j];
+                                s += w * xm[q];
+                                m += fabs(w) * (xabs ? xabs[q] : fabs(xm[q]));
+                            }
+                        }
+                    out[IDX4(b, c, y, xx, C, H, W)] = s;
+                    if (mag) mag[IDX4(b, c, y, xx, C_a, H, W)] = m;
+                }
 }
 
 /* Selected outputs, one by one: idx[n] are flat indices into out[B,C,H,W]; dk is

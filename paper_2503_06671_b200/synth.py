@@ -144,6 +144,14 @@ def make_estimator_mlp(C_a, h, dtype=F32, seed=0):
     }
 
 
+def make_pointwise(C_a, dtype=F32, seed=0):
+    """w_point [C_a,C_a] (row = output channel): the 1x1 large-kernel filter of the decomposed form,
+    kaiming-uniform with fan_in C_a plus the identity, float32 rounded to `dtype`."""
+    rng = np.random.default_rng(7000003 * (seed + 1) + C_a)
+    w = _kaiming_uniform(rng, (C_a, C_a), C_a) + np.eye(C_a, dtype=np.float32)
+    return round_to(w, dtype)
+
+
 def make_workload(wl: Workload, channel_means=False):
     return make_inputs(wl.B, wl.C, wl.C_a, wl.H, wl.W, wl.K, wl.dtype, wl.seed, wl.per_image_scale,
                        channel_means)
