@@ -170,6 +170,27 @@ int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, 
                               const void* w_large_host, const void* w_dyn_host,
                               const void* b_dyn_host, void* out_host, int dtype, int layout);
 
+/*
+ * The decomposed large kernel of Eq. 5, F_res = (F_att (*) LK^c) (*) (ZP(DK) + LK^s): the attention
+ * channels first go through the point-wise filter LK^c (a 1x1 convolution, no bias),
+ *   w_point [C_a,C_a]   row n = output channel: mixed[n] = sum_k w_point[n,k] * F_att[k]
+ * (device, the tensor's dtype), then through the same depth-wise stage as above; DK still comes from
+ * GAP(F_att), the unmixed features (Eq. 4 line 2).  With bf16 storage the mixed features are rounded
+ * to bf16 once where the fast kernel runs (NHWC, K = 13, C_a = 16: tensor-core mix inside the staged
+ * tile) and kept in fp32 on the generic path.  Other arguments as for esc_convattn_forward_ex and
+ * esc_convattn_stencil.
+ */
+int esc_convattn_forward_pw(const void* x, int B, int C, int C_a, int H, int W, int K,
+                            const void* w_large, const void* w_point,
+                            const void* w_dyn, const void* b_dyn,
+                            void* out, int dtype, int layout,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+int esc_convattn_stencil_pw(const void* x, int B, int C, int C_a, int H, int W, int K,
+                            const void* w_large, const void* w_point, const float* dk,
+                            void* out, int dtype, int layout,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

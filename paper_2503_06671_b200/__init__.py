@@ -19,6 +19,8 @@ from .binding import (  # noqa: F401
     esc_convattn_workspace_init,
     esc_convattn_device_status,
     esc_convattn_forward_mlp,
+    esc_convattn_forward_pw,
+    esc_convattn_stencil_pw,
     esc_convattn_dynkernel_mlp,
     esc_convattn_last_path,
     esc_convattn_last_tile_width,

@@ -46,6 +46,8 @@ def lib():
         L.esc_convattn_dynkernel.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_mlp.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, i, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_mlp.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, i, vp, i, i, vp, sz, vp]
+        L.esc_convattn_forward_pw.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_stencil_pw.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -55,7 +57,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_stencil", "esc_convattn_forward_host",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_stencil", "esc_convattn_forward_host",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -195,6 +197,26 @@ def esc_convattn_dynkernel_mlp(x, C_a, w_down, b_down, w_up, b_up, dk_out, layou
                                             _stream(stream)),
            "esc_convattn_dynkernel_mlp")
     return dk_out
+
+
+def esc_convattn_forward_pw(x, C_a, K, w_large, w_point, w_dyn, b_dyn, out, layout, workspace, stream=None):
+    """Forward pass in the decomposed form of Eq. 5: point-wise filter w_point [C_a,C_a], then the depth-wise stage."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_forward_pw(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_point), _ptr(w_dyn),
+                                         _ptr(b_dyn), _ptr(out), _dtype_code(x), layout, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_forward_pw")
+    return out
+
+
+def esc_convattn_stencil_pw(x, C_a, K, w_large, w_point, dk, out, layout, workspace=None, stream=None):
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_stencil_pw(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_point), _ptr(dk),
+                                         _ptr(out), _dtype_code(x), layout, _ptr(workspace),
+                                         0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                         _stream(stream)),
+           "esc_convattn_stencil_pw")
+    return out
 
 
 def esc_convattn_dynkernel_static(x, C_a, w_dyn, b_dyn, dk_out, layout, stream=None):

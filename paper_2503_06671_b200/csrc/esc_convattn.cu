@@ -42,6 +42,7 @@ size_t elem_size(int dtype) { return dtype == ESC_BF16 ? 2 : 4; }
 
 struct Problem {
     int B, C, Ca, H, W, K, dtype, layout;
+    const void* w_point = nullptr;   // [Ca][Ca] point-wise filter LK^c of the decomposed form (Eq. 5), or none
     size_t es() const { return elem_size(dtype); }
     size_t elems() const { return (size_t)B * C * H * W; }
 };
@@ -228,11 +229,11 @@ int launch_generic_t(const Problem& p, const void* x, const void* w_large, const
     cfg.numAttrs = dependent ? 1 : 0;
     if (regtile)
         ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT>, static_cast<const T*>(x),
-                                    static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), dk,
+                                    static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk,
                                     tiles_x, tiles_y));
     else
         ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_generic<T, LAYOUT>, static_cast<const T*>(x), static_cast<T*>(out),
-                                    p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), dk, tiles_x, tiles_y));
+                                    p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk, tiles_x, tiles_y));
     ++g_last_launches;
     return ESC_OK;
 }
@@ -255,8 +256,8 @@ int launch_generic(const Problem& p, const void* x, const void* w_large, const f
 int launch_stencil(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                    unsigned* ctrl, cudaStream_t st, bool dependent) {
     int tile_w = g_tile_policy;
-    int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, out, ctrl, st,
-                                  dependent, &g_last_launches, &g_last_error, &tile_w);
+    int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, p.w_point, dk, out, ctrl,
+                                  st, dependent, &g_last_launches, &g_last_error, &tile_w);
     if (rc == ESC_OK) { g_last_path = 2; g_last_tile_w = tile_w; return ESC_OK; }
     if (rc != esc::tma::kNotApplicable) return rc;
     return launch_generic(p, x, w_large, dk, out, st, dependent);
@@ -331,7 +332,7 @@ HostPath g_host;
 
 extern "C" {
 
-int esc_version(void) { return 106; }
+int esc_version(void) { return 107; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
@@ -507,6 +508,46 @@ int esc_convattn_stencil(const void* x, int B, int C, int C_a, int H, int W, int
         ctrl = carve(workspace, B, C_a).ctrl;
     }
     return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
+}
+
+int esc_convattn_stencil_pw(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                            const void* w_point, const float* dk, void* out, int dtype, int layout, void* workspace,
+                            size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_large || !w_point || !dk) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, p.es()) || !aligned(w_point, p.es()) || !aligned(dk, 4)) return ESC_ERR_ALIGN;
+    p.w_point = w_point;
+    unsigned* ctrl = nullptr;
+    if (workspace) {
+        rc = check_workspace(p, workspace, workspace_bytes_);
+        if (rc != ESC_OK) return rc;
+        ctrl = carve(workspace, B, C_a).ctrl;
+    }
+    return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
+}
+
+int esc_convattn_forward_pw(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                            const void* w_point, const void* w_dyn, const void* b_dyn, void* out, int dtype,
+                            int layout, void* workspace, size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_large || !w_point || !w_dyn || !b_dyn) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, p.es()) || !aligned(w_point, p.es()) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es()))
+        return ESC_ERR_ALIGN;
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    p.w_point = w_point;
+    return forward_impl(p, x, w_large, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, out, workspace,
+                        static_cast<cudaStream_t>(stream));
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {

@@ -11,10 +11,24 @@ namespace esc {
 
 constexpr int kGenTX = 32, kGenTY = 8, kGenMaxK = 17;
 
+// One staged input value of attention channel c: the feature itself, or -- in the decomposed form of
+// Eq. 5, (F_att * LK^c) * (ZP(DK) + LK^s) -- the point-wise mix sum_k w_point[c][k] * x[k] of the
+// pixel's C_a attention channels (fp32, channel order).  Outside the image both are zero.
+template <typename T, int LAYOUT>
+__device__ __forceinline__ float staged_value(const T* __restrict__ x, const T* __restrict__ w_point, int b, int c,
+                                              int y, int xx, int C, int Ca, int H, int W) {
+    if (y < 0 || y >= H || xx < 0 || xx >= W) return 0.f;
+    if (w_point == nullptr) return Elem<T>::to_f32(x[elem_index<LAYOUT>(b, c, y, xx, C, H, W)]);
+    float v = 0.f;
+    for (int k = 0; k < Ca; ++k)
+        v = fmaf(Elem<T>::to_f32(w_point[(size_t)c * Ca + k]), Elem<T>::to_f32(x[elem_index<LAYOUT>(b, k, y, xx, C, H, W)]), v);
+    return v;
+}
+
 template <typename T, int LAYOUT>
 __global__ void __launch_bounds__(kGenTX * kGenTY)
 stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W, int K,
-                const T* __restrict__ w_large, const float* __restrict__ dk,
+                const T* __restrict__ w_large, const T* __restrict__ w_point, const float* __restrict__ dk,
                 int tiles_x, int tiles_y)
 {
     __shared__ float tile[(kGenTY + kGenMaxK - 1) * (kGenTX + kGenMaxK - 1)];
@@ -41,10 +55,7 @@ stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int
     }
     for (int t = tid; t < TWp * THp; t += kGenTX * kGenTY) {
         const int r = t / TWp, q = t % TWp;
-        const int y = y0 + r, xx = x0 + q;
-        float v = 0.f;
-        if (y >= 0 && y < H && xx >= 0 && xx < W) v = Elem<T>::to_f32(x[elem_index<LAYOUT>(b, c, y, xx, C, H, W)]);
-        tile[t] = v;
+        tile[t] = staged_value<T, LAYOUT>(x, w_point, b, c, y0 + r, x0 + q, C, Ca, H, W);
     }
     __syncthreads();
 
@@ -72,7 +83,8 @@ constexpr int kRtThreads = (kRtTX / kRtOX) * (kRtTY / kRtOY);   // 128
 template <typename T, int LAYOUT>
 __global__ void __launch_bounds__(kRtThreads)
 stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W,
-                    const T* __restrict__ w_large, const float* __restrict__ dk, int tiles_x, int tiles_y)
+                    const T* __restrict__ w_large, const T* __restrict__ w_point, const float* __restrict__ dk,
+                    int tiles_x, int tiles_y)
 {
     __shared__ __align__(16) float tile[kRtRows * kRtPitch];
     __shared__ __align__(16) float wm[kRtK * 16];      // merged kernel, rows padded to 16 taps
@@ -88,10 +100,7 @@ stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca,
 
     for (int t = tid; t < kRtRows * kRtPitch; t += kRtThreads) {
         const int r = t / kRtPitch, q = t % kRtPitch;
-        const int y = y0 + r, xx = x0 + q;
-        float v = 0.f;
-        if (y >= 0 && y < H && xx >= 0 && xx < W) v = Elem<T>::to_f32(x[elem_index<LAYOUT>(b, c, y, xx, C, H, W)]);
-        tile[t] = v;
+        tile[t] = staged_value<T, LAYOUT>(x, w_point, b, c, y0 + r, x0 + q, C, Ca, H, W);
     }
     pdl_wait_primary();   // dk comes from the preceding kernel when launched as its dependent
     for (int t = tid; t < kRtK * 16; t += kRtThreads) {

@@ -31,6 +31,7 @@
 #include <cuda_runtime.h>
 #include <string>
 #include <cstdio>
+#include <cstdint>
 
 #include "common.cuh"
 
@@ -105,6 +106,7 @@ struct Params {
     int copy_cc, copy_cw, copy_cr;    // copy box: channels, pixels, rows (copy_cc == 0: nothing to copy)
     int slot_stride;                  // bytes between ring slots (multiple of 128)
     const __nv_bfloat16* w_large;     // [Ca][13][13]
+    const __nv_bfloat16* w_point;     // [16][16] point-wise filter LK^c of the decomposed form, or nullptr
     const float* dk;                  // [B][Ca][9]
     unsigned* ctrl;                   // status words or nullptr
 };
@@ -180,7 +182,78 @@ __device__ __forceinline__ int wsm_index(int c, int i, int j) {
     return ((i * 7 + (j >> 1)) * NPAIR + (c >> 1)) * 4 + (j & 1) * 2 + (c & 1);
 }
 
-template <class G>
+// D (16x8, fp32) = A (16x16, bf16, row-major) x B (16x8, bf16, column-major): the warp-level tensor-core
+// instruction, used only for the small point-wise mix below.
+__device__ __forceinline__ void mma_16x8x16_bf16(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// Decomposed form of Eq. 5, first factor: every staged pixel's 16 channels are replaced in place by
+// LK^c applied to them, F <- F * LK^c (1x1 convolution, out[n] = sum_k w_point[n][k] in[k]), with fp32
+// accumulation on the tensor cores and one rounding back to bf16.  Zero-filled halo pixels stay zero,
+// which is the zero padding of the mixed feature map.  A warp takes 16 pixels at a time: pixel rows are
+// the A matrix, LK^c the B matrix in two halves of 8 output channels; a lane reads and writes only its
+// own eight bytes of two pixels, so the update needs no staging.
+// The tensor-core instruction sums over k and fills column n in a fixed lane layout, but which channel
+// a k or an n stands for is free as long as A, B and D agree.  Both are permuted here so that lane
+// (g, t) -- g = lane / 4, t = lane % 4 -- deals with channels 4t..4t+3 only, on the input and on the
+// output side: its A fragment is one 8-byte read per pixel, its D fragments one 8-byte write, and a
+// warp's reads and writes cover whole 256-byte runs of the tile (no bank conflicts; with the natural
+// order every access touches half of each 32-byte pixel and the mix is twice as slow, bound by
+// shared-memory bandwidth either way).
+//   k = 2t + e      <-> input channel 4t + e          k = 8 + 2t + e      <-> input channel 4t + 2 + e
+//   n = 2j + e, first half <-> output channel 4j + e  second half         <-> output channel 4j + 2 + e
+__device__ __forceinline__ void load_mix_fragments(const __nv_bfloat16* __restrict__ w_point, int lane, uint32_t (&bf)[4]) {
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t* wp = reinterpret_cast<const uint32_t*>(w_point);        // word n*8 + c/2 = (w[n][c], w[n][c+1])
+    const int n0 = 4 * (g >> 1) + (g & 1), n1 = n0 + 2;                      // output channels of column g in either half
+    bf[0] = __ldg(wp + n0 * 8 + 2 * t); bf[1] = __ldg(wp + n0 * 8 + 2 * t + 1);
+    bf[2] = __ldg(wp + n1 * 8 + 2 * t); bf[3] = __ldg(wp + n1 * 8 + 2 * t + 1);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+template <int NPIX>
+__device__ __forceinline__ void pointwise_mix_tile(uint32_t* tile, const uint32_t (&bf)[4], int warp, int lane) {
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t b0[2] = {bf[0], bf[1]}, b1[2] = {bf[2], bf[3]};
+    uint2* t2 = reinterpret_cast<uint2*>(tile) + t;          // pixel p, channels 4t..4t+3: t2[p * 4]
+    constexpr int U = 4, STEP = kComputeWarps * 16;          // groups of 16 pixels in flight per warp
+#pragma unroll 1
+    for (int base = warp * 16; base < NPIX; base += U * STEP) {
+        // all loads, then all products, then all stores: a warp issues in order and the loads of one
+        // group may not move above the stores of another (same array)
+        uint32_t a[U][4];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int pa = base + u * STEP + g, pb = pa + 8;
+            const uint2 va = pa < NPIX ? t2[pa * 4] : make_uint2(0u, 0u);
+            const uint2 vb = pb < NPIX ? t2[pb * 4] : make_uint2(0u, 0u);
+            a[u][0] = va.x; a[u][2] = va.y; a[u][1] = vb.x; a[u][3] = vb.y;
+        }
+        float d0[U][4], d1[U][4];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) d0[u][e] = d1[u][e] = 0.f;
+            mma_16x8x16_bf16(d0[u], a[u], b0);
+            mma_16x8x16_bf16(d1[u], a[u], b1);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int pa = base + u * STEP + g, pb = pa + 8;
+            if (pa < NPIX) t2[pa * 4] = make_uint2(pack_bf16x2(d0[u][0], d0[u][1]), pack_bf16x2(d1[u][0], d1[u][1]));
+            if (pb < NPIX) t2[pb * 4] = make_uint2(pack_bf16x2(d0[u][2], d0[u][3]), pack_bf16x2(d1[u][2], d1[u][3]));
+        }
+    }
+}
+
+template <class G, bool kMix>
 __global__ void __maxnreg__(kLaunchRegs)
 stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
                       const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_res,
@@ -329,6 +402,9 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
             compute_bar();
         }
 
+        uint32_t mixb[4];
+        if (kMix) load_mix_fragments(p.w_point, lane, mixb);   // issued before the wait: a cold miss hides behind the tile
+
         if (alive) alive = mbar_wait(full0 + 8 * buf, (unsigned)((k >> 1) & 1), p.ctrl, 0xA0000000u | (unsigned)buf);
 
         u64 acc[OY][OX];
@@ -338,6 +414,10 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
             for (int c = 0; c < OX; ++c) acc[a][c] = 0ull;
 
         unsigned char* tbuf = tilebuf + (size_t)buf * TILE_BYTES;
+        if (kMix) {                                          // Eq. 5: the depth-wise stage sees F_att * LK^c
+            pointwise_mix_tile<G::THP * G::PITCH>(reinterpret_cast<uint32_t*>(tbuf), mixb, warp, lane);
+            compute_bar();
+        }
         const uint32_t* tw = reinterpret_cast<const uint32_t*>(tbuf) + lane_word;
         const float4* wlane = reinterpret_cast<const float4*>(wsm) + pr;
 
@@ -481,9 +561,10 @@ inline double cost_of(int B, int Ca, int H, int W, int sms, double per_fma) {
     return (double)waves * ((double)G::TW * G::TH * per_fma + 200.0);
 }
 
-template <class G>
-inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk,
-                       void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err) {
+template <class G, bool kMix>
+inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const void* w_point,
+                       const float* dk, void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches,
+                       std::string* err) {
     const int cc = C - Ca;
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -503,6 +584,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
         p.slot_stride = (cc * 2 * p.copy_cw * p.copy_cr + 127) / 128 * 128;
     }
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
+    p.w_point = static_cast<const __nv_bfloat16*>(w_point);
     p.dk = dk;
     p.ctrl = ctrl;
 
@@ -521,7 +603,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     const size_t smem = 2 * (size_t)G::TILE_BYTES + WSM_BYTES + LKC_BYTES + (size_t)NSLOT * p.slot_stride + 128;
     static bool attr_set = false;                            // one flag per geometry
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16<G, kMix>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
         attr_set = true;
     }
@@ -538,7 +620,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16<G>, m_att, m_cin, m_cout, m_res, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16<G, kMix>, m_att, m_cin, m_cout, m_res, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_tma_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -553,21 +635,25 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
 // generic kernel has to run instead, or an ESC_ERR_* code.  *tile_w: in, the tile width asked
 // for (0 = choose by cost); out, the one used.
 inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
-                      const void* w_large, const float* dk, void* out, unsigned* ctrl, cudaStream_t st,
-                      bool dependent, int* launches, std::string* err, int* tile_w) {
+                      const void* w_large, const void* w_point, const float* dk, void* out, unsigned* ctrl,
+                      cudaStream_t st, bool dependent, int* launches, std::string* err, int* tile_w) {
     if (K != K13 || dtype != 1 /*bf16*/ || layout != kNHWC) return kNotApplicable;
     if (Ca % CG != 0 || C % 8 != 0) return kNotApplicable;
     if (C - Ca > 256) return kNotApplicable;
+    if (w_point && Ca != CG) return kNotApplicable;         // the mix needs all C_a channels of a pixel in one tile
+    if (w_point && (reinterpret_cast<uintptr_t>(w_point) & 3) != 0) return kNotApplicable;   // read as 32-bit words
     const int sms = sm_count();
     if (sms <= 0) return kNotApplicable;
     const bool use64 = *tile_w == Geom64::TW ||
                        (*tile_w != Geom40::TW && cost_of<Geom64>(B, Ca, H, W, sms, 1.15) < cost_of<Geom40>(B, Ca, H, W, sms, 1.0));
     if (use64) {
         *tile_w = Geom64::TW;
-        return launch_geom<Geom64>(B, C, Ca, H, W, x, w_large, dk, out, ctrl, st, dependent, launches, err);
+        return w_point ? launch_geom<Geom64, true>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err)
+                       : launch_geom<Geom64, false>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err);
     }
     *tile_w = Geom40::TW;
-    return launch_geom<Geom40>(B, C, Ca, H, W, x, w_large, dk, out, ctrl, st, dependent, launches, err);
+    return w_point ? launch_geom<Geom40, true>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err)
+                   : launch_geom<Geom40, false>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err);
 }
 
 }}  // namespace esc::tma

@@ -88,6 +88,15 @@ def test_host_side_rejections_launch_nothing(L):
     assert L.esc_convattn_dynkernel_mlp(X, 1, 64, 16, 8, 8, Wd, Bd, Wu, Bu, 0, O, 0, 0, WS, big, None) == 2
     assert L.esc_convattn_dynkernel_mlp(X, 1, 64, 16, 8, 8, Wd, Bd, Wu, Bu, 8, None, 0, 0, WS, big, None) == 1
     assert L.esc_convattn_set_tile_width(48) == 3 and L.esc_convattn_set_tile_width(0) == 0
+    # decomposed large kernel: the point-wise filter is one more checked pointer
+    Wp = 0x30500000
+
+    def pw(x=X, wp=Wp, out=O, K=13, ws=WS, wsb=big):
+        return L.esc_convattn_forward_pw(x, 1, 64, 16, 32, 32, K, Wl, wp, Wd, Bd, out, 1, 1, ws, wsb, None)
+
+    assert pw(wp=None) == 1 and pw(x=None) == 1 and pw(K=14) == 2 and pw(wp=Wp + 1) == 4 and pw(out=X) == 5 and pw(wsb=8) == 6
+    assert L.esc_convattn_stencil_pw(X, 1, 64, 16, 8, 8, 13, Wl, None, Wd, O, 0, 0, None, 0, None) == 1
+    assert L.esc_convattn_stencil_pw(X, 1, 64, 16, 8, 8, 13, Wl, Wp, Wd, X + 16, 0, 0, None, 0, None) == 5
     assert L.esc_convattn_workspace_init(None, 1024, None) == 6
     assert L.esc_convattn_device_status(None, None) == 6
 

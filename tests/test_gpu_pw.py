@@ -1,0 +1,123 @@
+"""GPU parity for the decomposed large kernel (ESC paper, Section 3.3, Eq. 5:
+F_res = (F_att * LK^c) * (ZP(DK) + LK^s)), through the C ABI against the CPU oracle."""
+import numpy as np
+import pytest
+
+from paper_2503_06671_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+LAYOUTS = [synth.NCHW, synth.NHWC]
+DTYPES = [synth.F32, synth.BF16]
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import paper_2503_06671_b200 as p
+
+    p.lib()
+    return p
+
+
+SHAPES = [
+    # B, C, C_a, H, W, K
+    (2, 48, 16, 64, 64, 13),     # ESC-FP width, training patches
+    (1, 48, 16, 90, 130, 13),    # several tiles, ragged
+    (1, 64, 16, 5, 7, 13),       # smaller than the kernel
+    (3, 16, 16, 41, 83, 13),     # nothing to copy through
+    (1, 64, 32, 47, 61, 13),     # C_a = 32: generic path (the tile holds 16 channels)
+    (1, 20, 12, 19, 23, 3),      # K = 3, odd channel counts
+    (1, 48, 16, 29, 31, 9),      # K = 9
+]
+
+
+def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True):
+    import torch
+
+    B, C, C_a, H, W, K = shape
+    d = synth.make_inputs(B, C, C_a, H, W, K, dtype, seed=sum(shape), per_image_scale=True, channel_means=True)
+    wp = synth.make_pointwise(C_a, dtype, seed=sum(shape))
+    x = util.to_device(d["x"], dtype, layout)
+    wl, wd, bd = util.weights_to_device(d, dtype)
+    wp_d = torch.from_numpy(wp).to("cuda", util.torch_dtype(dtype))
+    out = torch.full_like(x, 7.0)
+    ws = pkg.new_workspace(B, C_a, H, W, K)
+    pkg.esc_convattn_set_tile_width(width)
+    try:
+        if forward:
+            pkg.esc_convattn_forward_pw(x, C_a, K, wl, wp_d, wd, bd, out, util.layout_code(layout), ws)
+            ref, mag = oracle.forward_pw(d["x"], C_a, d["w_large"], wp, d["w_dyn"], d["b_dyn"], want_mag=True)
+        else:
+            dk = np.random.default_rng(5).uniform(-0.5, 0.5, size=(B, C_a, 3, 3)).astype(np.float32)
+            pkg.esc_convattn_stencil_pw(x, C_a, K, wl, wp_d, torch.from_numpy(dk).cuda(), out, util.layout_code(layout), ws)
+            ref, mag = oracle.stencil_pw(d["x"], C_a, d["w_large"], wp, dk, want_mag=True)
+        torch.cuda.synchronize()
+    finally:
+        pkg.esc_convattn_set_tile_width(0)
+    assert pkg.esc_convattn_device_status(ws) == 0
+    got = util.to_host_nchw(out, layout)
+    path = pkg.esc_convattn_last_path()
+    if dtype == synth.BF16 and path == 2:
+        # The fast kernel keeps the mixed features in its bf16 tile: one rounding of F_att * LK^c, as a
+        # bf16 network stores that tensor.  (a) Against the exact oracle the error is bounded by the two
+        # roundings: 2^-9 * sum|w||mixed| for the intermediate plus 2^-9 * |out| for the result, both
+        # <= 2^-9 * mag.  (b) Against the oracle fed with the same rounded intermediate the usual bf16
+        # bar holds.
+        err = np.abs(got[:, :C_a] - ref[:, :C_a])
+        assert (err <= 2.0 ** -8 * mag + 1e-6).all(), f"pw {shape}: {(err / np.maximum(mag, 1e-30)).max():.3e} of mag"
+        x2 = d["x"].copy()
+        x2[:, :C_a] = synth.round_to(oracle.pointwise(d["x"], C_a, wp).astype(np.float32), synth.BF16)
+        dk_used = dk if not forward else oracle.dynkernel(oracle.gap(d["x"], C_a), d["w_dyn"], d["b_dyn"])
+        ref2, mag2 = oracle.stencil(x2, C_a, d["w_large"], dk_used, want_mag=True)
+        err2 = np.abs(got[:, :C_a] - ref2[:, :C_a])
+        assert (err2 / np.maximum(np.abs(ref2[:, :C_a]), 1.0)).max() <= util.BF16_REL
+        # one bf16 rounding of the result plus fp32 noise -- except where the fp32-accumulated mix and the
+        # oracle's fp64 mix round a value to different bf16 neighbours, which moves an output by one
+        # tap's worth; that may happen to a few outputs in a hundred thousand, not more
+        tight = 2.0 ** -8 * np.abs(ref2[:, :C_a]) + 1e-5 * mag2 + 1e-30
+        assert (err2 > tight).mean() <= 1e-4, f"pw {shape}: {(err2 > tight).mean():.2e} of outputs beyond one rounding"
+    else:
+        util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, f"pw {shape}")
+    assert np.array_equal(got[:, C_a:], ref[:, C_a:])
+    return path, pkg.esc_convattn_last_tile_width()
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_forward_pw(pkg, oracle, shape, dtype, layout):
+    path, _ = _run(pkg, oracle, shape, dtype, layout)
+    fast = dtype == synth.BF16 and layout == synth.NHWC and shape[5] == 13 and shape[2] == 16
+    assert path == (2 if fast else 1)
+
+
+@pytest.mark.parametrize("width", [40, 64])
+@pytest.mark.parametrize("shape", [s for s in SHAPES if s[2] == 16 and s[5] == 13] + [(1, 64, 16, 293, 517, 13)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_stencil_pw_both_tile_geometries(pkg, oracle, shape, width):
+    path, used = _run(pkg, oracle, shape, synth.BF16, synth.NHWC, width=width, forward=False)
+    assert path == 2 and used == width
+
+
+def test_identity_mix_reproduces_the_plain_forward_bit_for_bit(pkg):
+    """With LK^c = I the tensor-core mix returns every bf16 value unchanged, so the result equals the
+    depth-wise forward exactly."""
+    import torch
+
+    B, C, C_a, H, W, K = 2, 64, 16, 70, 100, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=21, channel_means=True)
+    x = util.to_device(d["x"], synth.BF16, synth.NHWC)
+    wl, wd, bd = util.weights_to_device(d, synth.BF16)
+    eye = torch.eye(C_a, dtype=torch.bfloat16, device="cuda")
+    ws = pkg.new_workspace(B, C_a, H, W, K)
+    a, b = torch.empty_like(x), torch.empty_like(x)
+    pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, a, pkg.ESC_NHWC, ws)
+    pkg.esc_convattn_forward_pw(x, C_a, K, wl, eye, wd, bd, b, pkg.ESC_NHWC, ws)
+    torch.cuda.synchronize()
+    assert pkg.esc_convattn_last_path() == 2
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
