@@ -109,6 +109,7 @@ struct Params {
     const __nv_bfloat16* w_point;     // [16][16] point-wise filter LK^c of the decomposed form, or nullptr
     const float* dk;                  // [B][Ca][9]
     unsigned* ctrl;                   // status words or nullptr
+    int wait_first;                   // 1: nothing may be read before the previous kernel of the stream has finished
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -281,6 +282,15 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
     }
     __syncthreads();
 
+    // Programmatic stream serialization.  As the dependent of the GAP kernel (wait_first == 0) this
+    // kernel starts beside it: x is complete (the GAP kernel lets its dependent go only after its own
+    // predecessor has finished), dk is waited for where it is needed.  Launched on its own
+    // (wait_first == 1) it may be resident before its predecessor has finished and waits here.  Either
+    // way the next kernel of the stream may be scheduled from now on; it has to wait for this grid
+    // itself before it touches anything, as the two kernels of this library do.
+    if (p.wait_first) pdl_wait_primary();
+    pdl_launch_dependents();
+
     const long long first = blockIdx.x, stride = gridDim.x;
     const long long my_units = first < p.units ? (p.units - first + stride - 1) / stride : 0;
 
@@ -369,7 +379,7 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
     const int lane_word = ((ly * OY) * PITCH + lx * OX) * NPAIR + pr;
 
     int cur_g = -1, merged_b = -1;
-    bool alive = true, dk_ready = false;
+    bool alive = true, dk_ready = p.wait_first != 0;
     for (long long k = 0; k < my_units; ++k) {
         const Unit un = decode_unit(first + k * stride, p);
         const int buf = (int)(k & 1);
@@ -587,6 +597,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     p.w_point = static_cast<const __nv_bfloat16*>(w_point);
     p.dk = dk;
     p.ctrl = ctrl;
+    p.wait_first = dependent ? 0 : 1;
 
     CUtensorMap m_att, m_cin, m_cout, m_res;
     // The halo tile gates the start of the arithmetic: fetch no more than its own 32-byte sectors need
@@ -619,7 +630,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = dependent ? 1 : 0;
+    cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16<G, kMix>, m_att, m_cin, m_cout, m_res, p);
     if (e != cudaSuccess) {
         char buf[256];
