@@ -148,11 +148,13 @@ int launch_gap_t(const Problem& p, const void* x, const Estimator& est,
     if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
     // Same shared-memory carve-out as the stencil kernel: an SM changes its L1/shared split only
     // when idle, so with different preferences the two kernels could never share an SM.
-    static bool carveout_set = false;
-    if (!carveout_set) {
+    static bool carveout_set[esc::tma::kMaxDevices] = {};   // per device and per instantiation
+    const int dev = esc::tma::current_device();
+    if (dev < 0) return ESC_ERR_UNSUPPORTED;
+    if (!carveout_set[dev]) {
         ESC_CUDA(cudaFuncSetAttribute(esc::gap_dynkernel<T, LAYOUT>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                       cudaSharedmemCarveoutMaxShared));
-        carveout_set = true;
+        carveout_set[dev] = true;
     }
     esc::gap_dynkernel<T, LAYOUT><<<grid, esc::kGapThreads, smem, st>>>(
         static_cast<const T*>(x), p.B, p.C, p.Ca, p.H, p.W, S, static_cast<const T*>(est.w_last),

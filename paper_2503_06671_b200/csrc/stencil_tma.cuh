@@ -546,14 +546,26 @@ inline bool make_map(CUtensorMap* m, const void* base, int B, int C, int H, int 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+constexpr int kMaxDevices = 64;
+
+// Index of the current device, or -1.
+inline int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
+// SM count of the current device (asked once per device).
 inline int sm_count() {
-    static int n = []() {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    static int cached[kMaxDevices] = {};
+    const int dev = current_device();
+    if (dev < 0) return 0;
+    if (cached[dev] == 0) {
+        int v = 0;
         if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        return v;
-    }();
-    return n;
+        cached[dev] = v;
+    }
+    return cached[dev];
 }
 
 // Units of one launch with geometry G, and the same count as waves over the SMs.
@@ -612,11 +624,13 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     }
 
     const size_t smem = 2 * (size_t)G::TILE_BYTES + WSM_BYTES + LKC_BYTES + (size_t)NSLOT * p.slot_stride + 128;
-    static bool attr_set = false;                            // one flag per geometry
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {};                  // function attributes are per device; one array per instantiation
+    const int dev = current_device();
+    if (dev < 0) return kNotApplicable;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16<G, kMix>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
-        attr_set = true;
+        attr_set[dev] = true;
     }
     if (smem > 227 * 1024) return kNotApplicable;
 
