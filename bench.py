@@ -31,9 +31,7 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one stencil-kernel launch from the ncu capture summarised under
 # profiles/, keyed by (workload, layout, library version the capture was taken with).  Reported only while the
 # library still has that version; otherwise the kernel has changed since and the figure is withheld.
-# (Versions 106 and 107 added the two-layer estimator to stage 1 and a separate instantiation of the stencil kernel
-# for the decomposed large kernel; the instantiation timed here is the one captured at 105.)
-NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", v): 29.56e6 + 0.30e6 for v in (105, 106, 107)}
+NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", 108): 29.56e6 + 0.47e6}
 
 
 def peaks():

@@ -334,7 +334,7 @@ HostPath g_host;
 
 extern "C" {
 
-int esc_version(void) { return 107; }
+int esc_version(void) { return 108; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
