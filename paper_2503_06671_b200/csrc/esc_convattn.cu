@@ -143,7 +143,7 @@ int launch_gap_t(const Problem& p, const void* x, const Estimator& est,
     // this kernel takes three blocks per SM and finishes sooner.
     const long long cap = is_large_map(p.B, (long long)p.H * p.W) ? 3LL * sms : sms;
     const unsigned grid = (unsigned)(items < cap ? items : cap);
-    const size_t scratch = (size_t)esc::kGapWarps * p.Ca > (size_t)esc::kGapThreads ? (size_t)esc::kGapWarps * p.Ca : (size_t)esc::kGapThreads;
+    const size_t scratch = (size_t)esc::gap_scratch_floats(LAYOUT, p.C, p.Ca, esc::Elem<T>::kVec);
     const size_t smem = (scratch + p.Ca) * sizeof(float);
     if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
     // Same shared-memory carve-out as the stencil kernel: an SM changes its L1/shared split only

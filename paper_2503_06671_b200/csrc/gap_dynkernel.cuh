@@ -27,6 +27,24 @@ constexpr int kGapThreads = 128;
 constexpr int kGapWarps = kGapThreads / 32;
 constexpr int kMaxHidden = kGapThreads;        // hidden activations live in the block's scratch
 
+// How the block reads an NHWC slab: 16-byte chunks of the attention channels, cpp = C_a / V chunks per
+// pixel.  kVecPow2: cpp is a power of two <= 32, lanes with equal lane % cpp hold the same channels and
+// a shuffle butterfly adds them.  kVecAny: any other cpp (C_a = 48: six chunks), one row of cpp threads
+// per pixel and a reduction through shared memory.  kScalar: channel counts that do not fill chunks.
+enum GapRead { kScalar = 0, kVecPow2 = 1, kVecAny = 2 };
+__host__ __device__ inline int gap_read_mode(int layout, int C, int Ca, int V) {
+    if (layout != kNHWC || Ca % V != 0 || C % V != 0) return kScalar;
+    const int cpp = Ca / V;
+    if (cpp <= 32 && (cpp & (cpp - 1)) == 0) return kVecPow2;
+    return cpp <= kGapThreads ? kVecAny : kScalar;
+}
+// Floats of block scratch in front of the C_a means.
+__host__ __device__ inline int gap_scratch_floats(int layout, int C, int Ca, int V) {
+    int n = kGapWarps * Ca > kGapThreads ? kGapWarps * Ca : kGapThreads;
+    if (gap_read_mode(layout, C, Ca, V) == kVecAny && kGapThreads * V > n) n = kGapThreads * V;
+    return n;
+}
+
 // phi(t) = t * Phi(t) with Phi(t) = erfc(-t / sqrt 2) / 2 (no cancellation in the left tail).
 __device__ __forceinline__ float gelu_exact(float t) { return 0.5f * t * erfcf(-0.70710678118654752f * t); }
 
@@ -41,9 +59,9 @@ gap_dynkernel(const T* __restrict__ x, int B, int C, int Ca, int H, int W, int S
               float* __restrict__ dk)          // [B][9*Ca]
 {
     constexpr int V = Elem<T>::kVec;
-    extern __shared__ float smem[];            // max(kGapWarps*Ca, kGapThreads) floats of scratch, then [Ca] means
+    extern __shared__ float smem[];            // gap_scratch_floats() floats of scratch, then [Ca] means
     float* wsum = smem;
-    float* gmean = smem + (kGapWarps * Ca > kGapThreads ? kGapWarps * Ca : kGapThreads);
+    float* gmean = smem + gap_scratch_floats(LAYOUT, C, Ca, V);
     __shared__ bool is_last;
 
     pdl_launch_dependents();                   // the stencil kernel may start its prologue now
@@ -55,9 +73,43 @@ gap_dynkernel(const T* __restrict__ x, int B, int C, int Ca, int H, int W, int S
     float* my_partial = partial + ((size_t)b * S + s) * Ca;
 
     const int cpp = Ca / V;                    // 16-byte chunks per pixel (NHWC)
-    const bool nhwc_vec = LAYOUT == kNHWC && Ca % V == 0 && C % V == 0 && cpp <= 32 && (cpp & (cpp - 1)) == 0;
+    const int mode = gap_read_mode(LAYOUT, C, Ca, V);
 
-    if (nhwc_vec) {
+    if (mode == kVecAny) {
+        // Thread t owns chunk t % cpp of pixels t / cpp, t / cpp + ppb, ...; the last 128 % cpp threads idle.
+        const long long p0 = HW * s / S, p1 = HW * (s + 1) / S;
+        const int chunk = tid % cpp, prow = tid / cpp, ppb = kGapThreads / cpp;
+        float acc[V];
+#pragma unroll
+        for (int v = 0; v < V; ++v) acc[v] = 0.f;
+        if (prow < ppb) {
+            const T* base = x + ((size_t)b * HW) * C + (size_t)chunk * V;
+            for (long long p = p0 + prow; p < p1; p += 8LL * ppb) {        // eight independent loads in flight
+                uint4 q[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const long long pu = p + (long long)u * ppb;
+                    q[u] = pu < p1 ? __ldg(reinterpret_cast<const uint4*>(base + (size_t)pu * C)) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float f[V];
+                    unpack16<T>(q[u], f);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) acc[v] += f[v];
+                }
+            }
+        }
+#pragma unroll
+        for (int v = 0; v < V; ++v) wsum[tid * V + v] = acc[v];
+        __syncthreads();
+        for (int c = tid; c < Ca; c += kGapThreads) {                      // rows added in order: reproducible
+            const float* col = wsum + (c / V) * V + (c % V);
+            float t = 0.f;
+            for (int r = 0; r < ppb; ++r) t += col[r * cpp * V];
+            my_partial[c] = t;
+        }
+    } else if (mode == kVecPow2) {
         // Thread t owns chunk (t % cpp) of pixels t/cpp, t/cpp + 256/cpp, ...
         const long long p0 = HW * s / S, p1 = HW * (s + 1) / S;
         const int chunk = tid % cpp, ppb = kGapThreads / cpp;

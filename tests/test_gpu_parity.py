@@ -80,7 +80,8 @@ def test_dk_stage(pkg, oracle, dtype, layout):
     import torch
 
     for (B, C, C_a, H, W) in [(3, 64, 16, 37, 53), (1, 64, 32, 120, 200), (2, 24, 8, 16, 16), (1, 20, 12, 9, 7),
-                              (70, 32, 16, 8, 8)]:
+                              (70, 32, 16, 8, 8),
+                              (2, 192, 48, 33, 47), (1, 48, 24, 20, 30), (1, 144, 144, 12, 12)]:   # 6, 3 and 18 (or 12, 6, 36) chunks per pixel
         d = synth.make_inputs(B, C, C_a, H, W, 13, dtype, seed=B * 100 + H, channel_means=True)
         x = util.to_device(d["x"], dtype, layout)
         _, wd, bd = util.weights_to_device(d, dtype)
