@@ -171,6 +171,22 @@ int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, 
                               const void* b_dyn_host, void* out_host, int dtype, int layout);
 
 /*
+ * The same end-to-end call split in two, so that a caller can keep the PCIe link busy in both
+ * directions: submit enqueues the copies and the kernels on one of two private slots (slot 0 or 1,
+ * each with its own device buffers and stream) and returns without waiting; wait blocks until that
+ * slot's last submit has finished and out_host is complete.  With two slots in turn --
+ * submit(i % 2) for step i, then wait((i - 1) % 2) -- the upload of one step overlaps the download
+ * of the step before.  The host buffers must be pinned (page-locked) for the copies to be
+ * asynchronous and must stay valid and untouched until the matching wait returns; two steps in
+ * flight need two out_host buffers.  esc_convattn_forward_host is submit(0) followed by wait(0).
+ * ESC_ERR_UNSUPPORTED for a slot other than 0 or 1.
+ */
+int esc_convattn_forward_host_submit(int slot, const void* x_host, int B, int C, int C_a, int H, int W, int K,
+                                     const void* w_large_host, const void* w_dyn_host,
+                                     const void* b_dyn_host, void* out_host, int dtype, int layout);
+int esc_convattn_forward_host_wait(int slot);
+
+/*
  * The decomposed large kernel of Eq. 5, F_res = (F_att (*) LK^c) (*) (ZP(DK) + LK^s): the attention
  * channels first go through the point-wise filter LK^c (a 1x1 convolution, no bias),
  *   w_point [C_a,C_a]   row n = output channel: mixed[n] = sum_k w_point[n,k] * F_att[k]

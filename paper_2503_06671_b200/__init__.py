@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     esc_convattn_workspace_bytes,
     esc_convattn_workspace_init,
     esc_convattn_device_status,
+    esc_convattn_forward_host_submit,
+    esc_convattn_forward_host_wait,
     esc_convattn_forward_mlp,
     esc_convattn_forward_pw,
     esc_convattn_stencil_pw,

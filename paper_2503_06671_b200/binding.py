@@ -52,12 +52,14 @@ def lib():
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
         L.esc_convattn_device_status.argtypes = [vp, vp]
+        L.esc_convattn_forward_host_submit.argtypes = [i, vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
+        L.esc_convattn_forward_host_wait.argtypes = [i]
         L.esc_convattn_set_tile_width.argtypes = [i]
         L.esc_status_string.argtypes = [i]
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_stencil", "esc_convattn_forward_host",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -247,6 +249,19 @@ def esc_convattn_forward_host(x, C_a, K, w_large, w_dyn, b_dyn, out, layout):
     _check(lib().esc_convattn_forward_host(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_dyn), _ptr(b_dyn),
                                            _ptr(out), _dtype_code(x), layout), "esc_convattn_forward_host")
     return out
+
+
+def esc_convattn_forward_host_submit(slot, x, C_a, K, w_large, w_dyn, b_dyn, out, layout):
+    """Asynchronous half of the host-buffer call: enqueue on slot 0 or 1 and return.  The CPU tensors must be
+    pinned and stay untouched until esc_convattn_forward_host_wait(slot) returns."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_forward_host_submit(int(slot), _ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_dyn),
+                                                  _ptr(b_dyn), _ptr(out), _dtype_code(x), layout),
+           "esc_convattn_forward_host_submit")
+
+
+def esc_convattn_forward_host_wait(slot) -> None:
+    _check(lib().esc_convattn_forward_host_wait(int(slot)), "esc_convattn_forward_host_wait")
 
 
 def esc_convattn_device_status(workspace, stream=None) -> int:

@@ -327,8 +327,9 @@ struct HostPath {
     void *x = nullptr, *out = nullptr, *wts = nullptr, *ws = nullptr;
     size_t xbytes = 0, wbytes = 0, wsbytes = 0;
 };
+constexpr int kHostSlots = 2;
 std::mutex g_host_mu;
-HostPath g_host;
+HostPath g_host[kHostSlots];
 
 }  // namespace
 
@@ -568,21 +569,23 @@ int esc_convattn_device_status(void* workspace, void* stream) {
     return (int)word[0];
 }
 
-int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, int W, int K,
-                              const void* w_large_host, const void* w_dyn_host, const void* b_dyn_host,
-                              void* out_host, int dtype, int layout) {
+int esc_convattn_forward_host_submit(int slot, const void* x_host, int B, int C, int C_a, int H, int W, int K,
+                                     const void* w_large_host, const void* w_dyn_host, const void* b_dyn_host,
+                                     void* out_host, int dtype, int layout) {
     g_last_launches = 0;
+    if (slot < 0 || slot >= kHostSlots) return ESC_ERR_UNSUPPORTED;
     const Problem p{B, C, C_a, H, W, K, dtype, layout};
     int rc = check_shape(p);
     if (rc != ESC_OK) return rc;
     if (!x_host || !w_large_host || !w_dyn_host || !b_dyn_host || !out_host) return ESC_ERR_NULL;
     std::lock_guard<std::mutex> lock(g_host_mu);
-    HostPath& h = g_host;
+    HostPath& h = g_host[slot];
     int dev = 0;
     ESC_CUDA(cudaGetDevice(&dev));
     if (h.dev != dev) {   // first use, or the caller switched device: start over
         if (h.dev >= 0) {
             ESC_CUDA(cudaSetDevice(h.dev));
+            if (h.st) cudaStreamSynchronize(h.st);
             cudaFree(h.x); cudaFree(h.out); cudaFree(h.wts); cudaFree(h.ws);
             if (h.st) cudaStreamDestroy(h.st);
             ESC_CUDA(cudaSetDevice(dev));
@@ -596,6 +599,8 @@ int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, 
     const size_t off_wd = round_up(n_wl * es, 256), off_bd = off_wd + round_up(n_wd * es, 256);
     const size_t wbytes = off_bd + round_up(n_bd * es, 256);
     const size_t wsbytes = workspace_bytes(B, C_a, (long long)H * W);
+    if (h.xbytes < xbytes || h.wbytes < wbytes || h.wsbytes < wsbytes)
+        ESC_CUDA(cudaStreamSynchronize(h.st));               // nothing of this slot may still use the old buffers
     if (h.xbytes < xbytes) {
         cudaFree(h.x); cudaFree(h.out); h.x = h.out = nullptr; h.xbytes = 0;
         ESC_CUDA(cudaMalloc(&h.x, xbytes));
@@ -621,8 +626,28 @@ int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, 
     rc = forward_impl(p, h.x, wts, Estimator{wts + off_wd, wts + off_bd, nullptr, nullptr, 0}, h.out, h.ws, h.st);
     if (rc != ESC_OK) return rc;
     ESC_CUDA(cudaMemcpyAsync(out_host, h.out, xbytes, cudaMemcpyDeviceToHost, h.st));
-    ESC_CUDA(cudaStreamSynchronize(h.st));
     return ESC_OK;
+}
+
+int esc_convattn_forward_host_wait(int slot) {
+    if (slot < 0 || slot >= kHostSlots) return ESC_ERR_UNSUPPORTED;
+    cudaStream_t st = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_host_mu);
+        if (g_host[slot].dev < 0) return ESC_OK;             // nothing was ever submitted here
+        st = g_host[slot].st;
+    }
+    ESC_CUDA(cudaStreamSynchronize(st));
+    return ESC_OK;
+}
+
+int esc_convattn_forward_host(const void* x_host, int B, int C, int C_a, int H, int W, int K,
+                              const void* w_large_host, const void* w_dyn_host, const void* b_dyn_host,
+                              void* out_host, int dtype, int layout) {
+    int rc = esc_convattn_forward_host_submit(0, x_host, B, C, C_a, H, W, K, w_large_host, w_dyn_host, b_dyn_host,
+                                              out_host, dtype, layout);
+    if (rc != ESC_OK) return rc;
+    return esc_convattn_forward_host_wait(0);
 }
 
 }  // extern "C"

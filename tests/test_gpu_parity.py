@@ -293,6 +293,31 @@ def test_host_entry_matches_device_entry(pkg):
     assert torch.equal(out.cpu().view(torch.int16), oh.view(torch.int16))
 
 
+def test_host_submit_wait_two_slots_in_turn(pkg):
+    """The asynchronous host-buffer pair: steps alternate between the two slots, every result equals the
+    blocking call's bit for bit, and a second shape on the same slots works (buffers regrow)."""
+    import torch
+
+    with pytest.raises(pkg.EscError):
+        pkg.esc_convattn_forward_host_wait(2)
+    for (B, C, C_a, H, W, K) in [(1, 64, 16, 60, 100, 13), (2, 64, 16, 90, 130, 13)]:
+        steps = []
+        for seed in range(4):
+            d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=300 + seed, channel_means=True)
+            xh = torch.from_numpy(synth.to_layout(d["x"], synth.NHWC)).to(torch.bfloat16).pin_memory()
+            w = [torch.from_numpy(d[k]).to(torch.bfloat16).pin_memory() for k in ("w_large", "w_dyn", "b_dyn")]
+            ref = torch.empty_like(xh).pin_memory()
+            pkg.esc_convattn_forward_host(xh, C_a, K, *w, ref, pkg.ESC_NHWC)
+            steps.append((xh, w, ref, torch.zeros_like(xh).pin_memory()))
+        for i, (xh, w, ref, out) in enumerate(steps):
+            pkg.esc_convattn_forward_host_submit(i % 2, xh, C_a, K, *w, out, pkg.ESC_NHWC)
+            if i > 0:
+                pkg.esc_convattn_forward_host_wait((i - 1) % 2)
+                assert torch.equal(steps[i - 1][3].view(torch.int16), steps[i - 1][2].view(torch.int16))
+        pkg.esc_convattn_forward_host_wait((len(steps) - 1) % 2)
+        assert torch.equal(steps[-1][3].view(torch.int16), steps[-1][2].view(torch.int16))
+
+
 def test_two_streams_two_workspaces(pkg, oracle):
     """Calls on different streams with different workspaces may overlap on the GPU; each must still be right."""
     import torch
