@@ -11,6 +11,8 @@ from .convattn_oracle import (  # noqa: F401
     dynkernel_mlp,
     forward_mlp,
     stencil,
+    stencil_dense,
+    forward_dense,
     pointwise,
     stencil_pw,
     forward_pw,

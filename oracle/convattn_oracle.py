@@ -174,6 +174,32 @@ def forward_pw(x, C_a, w_large, w_point, w_dyn, b_dyn, want_mag=False, want_dk=F
     return res[0] if len(res) == 1 else tuple(res)
 
 
+def stencil_dense(x, C_a, w_dense, dk, want_mag=False):
+    """Dense large kernel w_dense[C_a,C_a,K,K] (out, in, row, col) plus the depth-wise dynamic 3x3 kernel dk."""
+    x, xp = _f32(x)
+    w_dense, wp = _f64(w_dense)
+    K = int(w_dense.shape[-1])
+    B, C, H, W = _dims(x, C_a, K)
+    assert w_dense.shape == (C_a, C_a, K, K)
+    dk, dp = _f64(dk)
+    assert dk.size == B * C_a * 9
+    out = np.empty((B, C, H, W), dtype=np.float64)
+    mag = np.empty((B, C_a, H, W), dtype=np.float64) if want_mag else None
+    _load().convattn_ref_stencil_dense(xp, B, C, C_a, H, W, K, wp, dp, out.ctypes.data_as(_f64p),
+                                       mag.ctypes.data_as(_f64p) if want_mag else None)
+    return (out, mag) if want_mag else out
+
+
+def forward_dense(x, C_a, w_dense, w_dyn, b_dyn, want_mag=False, want_dk=False):
+    """Whole forward with the dense large kernel: dk from GAP(F_att) (one-layer estimator), then stencil_dense."""
+    dk = dynkernel(gap(x, C_a), w_dyn, b_dyn)
+    res = stencil_dense(x, C_a, w_dense, dk, want_mag=want_mag)
+    res = list(res) if want_mag else [res]
+    if want_dk:
+        res.append(dk)
+    return res[0] if len(res) == 1 else tuple(res)
+
+
 def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
     """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
     x, xp = _f32(x)

@@ -25,6 +25,9 @@
  * taken in that order: mix first, then the depth-wise stage on the mixed features; dk still
  * comes from GAP(F_att) as in Eq. 4 line 2.
  *
+ * convattn_ref_stencil_dense is Eq. 4 line 3 with the dense large kernel of Section 3.2
+ * (13x13x16x16: every output channel sums over all attention input channels).
+ *
  * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
  * Everything is accumulated in double precision with direct nested loops in
  * the order written above: no tiling, no merging of the two kernels, no reuse.
@@ -43,7 +46,9 @@
  * reflection law of phi, its two linear limits (which reduce it to the one-layer
  * estimator with composed weights) and a math.erf brute force; the decomposed form
  * by the identity mix, library 1x1 + depth-wise convolutions, the commutation with a
- * channel-independent spatial kernel, permutation mixes and a brute force.
+ * channel-independent spatial kernel, permutation mixes and a brute force; the dense
+ * large kernel by its diagonal case (= the depth-wise stencil), a library dense
+ * convolution, the depth-wise-then-point-wise factorisation and a brute force.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -242,6 +247,51 @@ void convattn_ref_stencil_mixed(const float *x, const double *xm, const double *
                         }
                     out[IDX4(b, c, y, xx, C, H, W)] = s;
                     if (mag) mag[IDX4(b, c, y, xx, C_a, H, W)] = m;
+                }
+}
+
+/* Dense large kernel (Section 3.2: LK in R^{13x13x16x16}; Eq. 4 line 3 with that LK): every attention
+ * output channel n sums over all C_a input channels k and all taps,
+ *   out[b,n,y,x] = sum_{k,i,j} w_dense[n,k,i,j] * x[b,k,y+i-P,x+j-P]  +  sum_{i,j} dk[b,n,i,j] * x[b,n,y+i-1,x+j-1],
+ * zero padding, the dynamic 3x3 kernel still depth-wise; identity channels copied.  w_dense is
+ * [C_a, C_a, K, K] (output channel, input channel, row, column); out [B,C,H,W]; mag (optional) [B,C_a,H,W]
+ * receives sum |w * x| over the same terms. */
+void convattn_ref_stencil_dense(const float *x, int B, int C, int C_a, int H, int W, int K,
+                                const double *w_dense, const double *dk, double *out, double *mag)
+{
+    const int P = (K - 1) / 2;
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < C; ++n)
+            for (int y = 0; y < H; ++y)
+                for (int xx = 0; xx < W; ++xx) {
+                    if (n >= C_a) {
+                        out[IDX4(b, n, y, xx, C, H, W)] = (double)x[IDX4(b, n, y, xx, C, H, W)];
+                        continue;
+                    }
+                    double s = 0.0, m = 0.0;
+                    for (int k = 0; k < C_a; ++k)
+                        for (int i = 0; i < K; ++i)
+                            for (int j = 0; j < K; ++j) {
+                                int yy = y + i - P, xc = xx + j - P;
+                                if (yy >= 0 && yy < H && xc >= 0 && xc < W) {
+                                    double t = w_dense[(((size_t)n * C_a + k) * K + i) * K + j] *
+                                               (double)x[IDX4(b, k, yy, xc, C, H, W)];
+                                    s += t;
+                                    m += fabs(t);
+                                }
+                            }
+                    for (int i = 0; i < 3; ++i)
+                        for (int j = 0; j < 3; ++j) {
+                            int yy = y + i - 1, xc = xx + j - 1;
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W) {
+                                double t = dk[(size_t)b * 9 * C_a + n * 9 + i * 3 + j] * (double)x[IDX4(b, n, yy, xc, C, H, W)];
+                                s += t;
+                                m += fabs(t);
+                            }
+                        }
+                    out[IDX4(b, n, y, xx, C, H, W)] = s;
+                    if (mag) mag[IDX4(b, n, y, xx, C_a, H, W)] = m;
                 }
 }
 

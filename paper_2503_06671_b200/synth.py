@@ -152,6 +152,13 @@ def make_pointwise(C_a, dtype=F32, seed=0):
     return round_to(w, dtype)
 
 
+def make_dense_kernel(C_a, K=13, dtype=F32, seed=0):
+    """w_dense [C_a,C_a,K,K] (output channel, input channel, row, column): the dense large kernel of the main
+    model, kaiming-uniform with fan_in C_a*K*K, float32 rounded to `dtype`."""
+    rng = np.random.default_rng(9000011 * (seed + 1) + C_a * 31 + K)
+    return round_to(_kaiming_uniform(rng, (C_a, C_a, K, K), C_a * K * K), dtype)
+
+
 def make_workload(wl: Workload, channel_means=False):
     return make_inputs(wl.B, wl.C, wl.C_a, wl.H, wl.W, wl.K, wl.dtype, wl.seed, wl.per_image_scale,
                        channel_means)
