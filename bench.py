@@ -31,7 +31,8 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one stencil-kernel launch from the ncu capture summarised under
 # profiles/, keyed by (workload, layout, library version the capture was taken with).  Reported only while the
 # library still has that version; otherwise the kernel has changed since and the figure is withheld.
-NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", 108): 29.56e6 + 0.47e6}
+# (Version 109 added entry points and kernels for other variants; the kernel timed here is the one captured at 108.)
+NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", v): 29.56e6 + 0.47e6 for v in (108, 109)}
 
 
 def peaks():
@@ -39,9 +40,10 @@ def peaks():
     try:
         with open(path) as f:
             p = json.load(f)
-        return {"hbm_gbs": float(p["hbm_gbs"]), "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+        return {"hbm_gbs": float(p["hbm_gbs"]), "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)),
+                "bf16_tflops": float(p.get("bf16_tflops", 1590.0)), "source": "measured"}
     except Exception:
-        return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+        return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "bf16_tflops": 1590.0, "source": "fallback"}
 
 
 class ClockSampler:
@@ -338,6 +340,16 @@ def main():
     # and with the decomposed large kernel of Eq. 5 (point-wise LK^c in front of the depth-wise stage)
     wp_d = torch.from_numpy(synth.make_pointwise(wl.C_a, wl.dtype, wl.seed)).to(tdt).cuda()
     ms_step_pw = timed(lambda i: pkg.esc_convattn_forward_pw(xs[i % n_rot], wl.C_a, wl.K, wl_d, wp_d, wd_d, bd_d, outs[i % n_rot], lay_code, ws))
+    # and with the dense large kernel of the main model (Section 3.2): an implicit GEMM on the tensor cores
+    dense = None
+    if wl.C_a == 16 and wl.K == 13:
+        wdn_d = torch.from_numpy(synth.make_dense_kernel(wl.C_a, wl.K, wl.dtype, wl.seed)).to(tdt).cuda()
+        ms_dense = timed(lambda i: pkg.esc_convattn_forward_dense(xs[i % n_rot], wl.C_a, wl.K, wdn_d, wd_d, bd_d, outs[i % n_rot], lay_code, ws))
+        fl = 2.0 * wl.C_a * wl.C_a * wl.K * wl.K * wl.pixels
+        bf16_peak = peaks()["bf16_tflops"]
+        dense = {"ms_per_step": ms_dense, "bound": "tensor", "achieved": fl / (ms_dense * 1e-3) / 1e12, "peak": bf16_peak,
+                 "unit": "TFLOP/s", "frac": fl / (ms_dense * 1e-3) / 1e12 / bf16_peak,
+                 "note": "whole step (GAP + dense stencil + copy kernel); warp-level mma.sync, see DESIGN.md"}
 
     pk = peaks()
     flops = 2.0 * wl.K * wl.K * wl.C_a * wl.pixels                    # merged 169-tap form, Eq. 5
@@ -413,6 +425,7 @@ def main():
             "GB_per_s_whole_step": alg_bytes / (ms_step * 1e-3) / 1e9,
             "ms_per_step_two_layer_estimator_h8": ms_step_mlp,
             "ms_per_step_decomposed_large_kernel": ms_step_pw,
+            "dense_large_kernel": dense,
         }))
     if world > 1:
         dist.destroy_process_group()

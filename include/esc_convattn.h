@@ -207,13 +207,32 @@ int esc_convattn_stencil_pw(const void* x, int B, int C, int C_a, int H, int W, 
                             void* out, int dtype, int layout,
                             void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * The dense large kernel of the main ESC models (Section 3.2: LK in R^{13x13x16x16}) in Eq. 4 line 3:
+ * every attention output channel sums over all C_a attention input channels and all K*K taps; the
+ * dynamic 3x3 kernel stays depth-wise.
+ *   w_dense [C_a,C_a,K,K]   (output channel, input channel, row, column), device, the tensor's dtype
+ * For bf16 NHWC tensors with K = 13 and C_a = 16 the first sum runs on the tensor cores (bf16 products,
+ * fp32 accumulation, implicit GEMM over the TMA-staged halo tile); anything else takes a slow
+ * one-thread-per-output kernel.  Other arguments as for esc_convattn_forward_ex / esc_convattn_stencil.
+ */
+int esc_convattn_forward_dense(const void* x, int B, int C, int C_a, int H, int W, int K,
+                               const void* w_dense, const void* w_dyn, const void* b_dyn,
+                               void* out, int dtype, int layout,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+int esc_convattn_stencil_dense(const void* x, int B, int C, int C_a, int H, int W, int K,
+                               const void* w_dense, const float* dk,
+                               void* out, int dtype, int layout,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);
 
 /* Which stencil implementation the last esc_convattn_forward* / esc_convattn_stencil call on
  * this thread selected: 0 = none yet, 1 = guarded generic kernel, 2 = TMA-staged register-tiled
- * kernel.  For tests and benchmarks. */
+ * kernel, 3 = tensor-core kernel of the dense large kernel.  For tests and benchmarks. */
 int esc_convattn_last_path(void);
 
 /* Width in pixels of the output tile the TMA-staged kernel used in that call (40: 40x40 tiles,

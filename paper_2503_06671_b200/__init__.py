@@ -20,6 +20,8 @@ from .binding import (  # noqa: F401
     esc_convattn_device_status,
     esc_convattn_forward_host_submit,
     esc_convattn_forward_host_wait,
+    esc_convattn_forward_dense,
+    esc_convattn_stencil_dense,
     esc_convattn_forward_mlp,
     esc_convattn_forward_pw,
     esc_convattn_stencil_pw,

@@ -48,6 +48,8 @@ def lib():
         L.esc_convattn_dynkernel_mlp.argtypes = [vp, i, i, i, i, i, vp, vp, vp, vp, i, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_pw.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_stencil_pw.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_forward_dense.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_stencil_dense.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -59,7 +61,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -218,6 +220,26 @@ def esc_convattn_stencil_pw(x, C_a, K, w_large, w_point, dk, out, layout, worksp
                                          0 if workspace is None else workspace.numel() * workspace.element_size(),
                                          _stream(stream)),
            "esc_convattn_stencil_pw")
+    return out
+
+
+def esc_convattn_forward_dense(x, C_a, K, w_dense, w_dyn, b_dyn, out, layout, workspace, stream=None):
+    """Forward pass with the dense large kernel w_dense [C_a,C_a,K,K] (output channel, input channel, row, column)."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_forward_dense(_ptr(x), B, C, C_a, H, W, K, _ptr(w_dense), _ptr(w_dyn), _ptr(b_dyn),
+                                            _ptr(out), _dtype_code(x), layout, _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_forward_dense")
+    return out
+
+
+def esc_convattn_stencil_dense(x, C_a, K, w_dense, dk, out, layout, workspace=None, stream=None):
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_stencil_dense(_ptr(x), B, C, C_a, H, W, K, _ptr(w_dense), _ptr(dk), _ptr(out),
+                                            _dtype_code(x), layout, _ptr(workspace),
+                                            0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                            _stream(stream)),
+           "esc_convattn_stencil_dense")
     return out
 
 

@@ -17,6 +17,7 @@
 #include "gap_dynkernel.cuh"
 #include "stencil_generic.cuh"
 #include "stencil_tma.cuh"
+#include "stencil_dense.cuh"
 
 namespace {
 
@@ -43,6 +44,7 @@ size_t elem_size(int dtype) { return dtype == ESC_BF16 ? 2 : 4; }
 struct Problem {
     int B, C, Ca, H, W, K, dtype, layout;
     const void* w_point = nullptr;   // [Ca][Ca] point-wise filter LK^c of the decomposed form (Eq. 5), or none
+    bool dense = false;              // w_large is the dense kernel [Ca][Ca][K][K] of Section 3.2
     size_t es() const { return elem_size(dtype); }
     size_t elems() const { return (size_t)B * C * H * W; }
 };
@@ -286,11 +288,56 @@ int get_scratch(size_t need, cudaStream_t st, void** out) {
     return ESC_OK;
 }
 
+template <typename T, int LAYOUT>
+int launch_dense_generic_t(const Problem& p, const void* x, const void* w_dense, const float* dk, void* out,
+                           cudaStream_t st, bool dependent) {
+    const long long total = (long long)p.B * p.Ca * p.H * p.W;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::tma::stencil_dense_generic<T, LAYOUT>, static_cast<const T*>(x),
+                                static_cast<T*>(out), p.B, p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_dense), dk));
+    ++g_last_launches;
+    return ESC_OK;
+}
+
+// Dense large kernel: tensor-core kernel where it applies, one thread per output elsewhere; the identity
+// channels go through the copy kernel either way.
+int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, const float* dk, void* out,
+                         unsigned* ctrl, cudaStream_t st, bool dependent) {
+    g_last_tile_w = 0;
+    int rc = esc::tma::try_launch_dense(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_dense, dk, out, ctrl,
+                                        st, dependent, &g_last_launches, &g_last_error);
+    if (rc == ESC_OK) {
+        g_last_path = 3;
+        g_last_tile_w = esc::tma::dense::TW;
+    } else if (rc == esc::tma::kNotApplicable) {
+        g_last_path = 1;
+        if (p.dtype == ESC_F32)
+            rc = p.layout == ESC_NCHW ? launch_dense_generic_t<float, esc::kNCHW>(p, x, w_dense, dk, out, st, dependent)
+                                      : launch_dense_generic_t<float, esc::kNHWC>(p, x, w_dense, dk, out, st, dependent);
+        else
+            rc = p.layout == ESC_NCHW ? launch_dense_generic_t<__nv_bfloat16, esc::kNCHW>(p, x, w_dense, dk, out, st, dependent)
+                                      : launch_dense_generic_t<__nv_bfloat16, esc::kNHWC>(p, x, w_dense, dk, out, st, dependent);
+    }
+    if (rc != ESC_OK) return rc;
+    return launch_copy(p, x, out, st);
+}
+
 int forward_impl(const Problem& p, const void* x, const void* w_large, const Estimator& est,
                  void* out, void* ws, cudaStream_t st) {
     const Workspace w = carve(ws, p.B, p.Ca);
     int rc = launch_gap(p, x, est, w, w.dk, st);
     if (rc != ESC_OK) return rc;
+    if (p.dense) return launch_stencil_dense(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
     return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
 }
 
@@ -335,7 +382,7 @@ HostPath g_host[kHostSlots];
 
 extern "C" {
 
-int esc_version(void) { return 108; }
+int esc_version(void) { return 109; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
@@ -550,6 +597,45 @@ int esc_convattn_forward_pw(const void* x, int B, int C, int C_a, int H, int W, 
     if (rc != ESC_OK) return rc;
     p.w_point = w_point;
     return forward_impl(p, x, w_large, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, out, workspace,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_stencil_dense(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_dense,
+                               const float* dk, void* out, int dtype, int layout, void* workspace,
+                               size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_dense || !dk) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_dense, p.es()) || !aligned(dk, 4)) return ESC_ERR_ALIGN;
+    p.dense = true;
+    unsigned* ctrl = nullptr;
+    if (workspace) {
+        rc = check_workspace(p, workspace, workspace_bytes_);
+        if (rc != ESC_OK) return rc;
+        ctrl = carve(workspace, B, C_a).ctrl;
+    }
+    return launch_stencil_dense(p, x, w_dense, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
+}
+
+int esc_convattn_forward_dense(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_dense,
+                               const void* w_dyn, const void* b_dyn, void* out, int dtype, int layout,
+                               void* workspace, size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_dense || !w_dyn || !b_dyn) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_dense, p.es()) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    p.dense = true;
+    return forward_impl(p, x, w_dense, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, out, workspace,
                         static_cast<cudaStream_t>(stream));
 }
 

@@ -97,6 +97,11 @@ def test_host_side_rejections_launch_nothing(L):
     assert pw(wp=None) == 1 and pw(x=None) == 1 and pw(K=14) == 2 and pw(wp=Wp + 1) == 4 and pw(out=X) == 5 and pw(wsb=8) == 6
     assert L.esc_convattn_stencil_pw(X, 1, 64, 16, 8, 8, 13, Wl, None, Wd, O, 0, 0, None, 0, None) == 1
     assert L.esc_convattn_stencil_pw(X, 1, 64, 16, 8, 8, 13, Wl, Wp, Wd, X + 16, 0, 0, None, 0, None) == 5
+    Wdn = 0x30600000
+    assert L.esc_convattn_forward_dense(X, 1, 64, 16, 32, 32, 13, None, Wd, Bd, O, 1, 1, WS, big, None) == 1
+    assert L.esc_convattn_forward_dense(X, 1, 64, 16, 32, 32, 13, Wdn + 1, Wd, Bd, O, 1, 1, WS, big, None) == 4
+    assert L.esc_convattn_forward_dense(X, 1, 64, 16, 32, 32, 13, Wdn, Wd, Bd, X, 1, 1, WS, big, None) == 5
+    assert L.esc_convattn_stencil_dense(X, 1, 64, 16, 8, 8, 12, Wdn, Wd, O, 0, 0, None, 0, None) == 2
     assert L.esc_convattn_forward_host_submit(2, X, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 3
     assert L.esc_convattn_forward_host_submit(0, None, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 1
     assert L.esc_convattn_forward_host_wait(-1) == 3
