@@ -6,8 +6,8 @@
 // The first sum is an implicit GEMM, M = pixels, N = 16 output channels, K = 16 input channels x 169 taps.
 // For one tap the A operand of a 16-pixel run is simply the 16 x 16-channel block of the staged halo tile
 // shifted by that tap (a pixel's 16 channels are its 32 contiguous bytes), so the tile is never unfolded:
-// one CTA per SM walks 64x16-pixel output tiles; each of its 8 warps owns two tile rows = 8 runs of 16
-// pixels x 16 output channels (64 fp32 accumulators per lane) and, per tap, reads its B fragments (one
+// one CTA per SM walks 64x16-pixel output tiles; each of its 16 warps owns one tile row = 4 runs of 16
+// pixels x 16 output channels (32 fp32 accumulators per lane) and, per tap, reads its B fragments (one
 // 16-byte load from a fragment-ordered weight table in shared memory), then per run its A fragment (two
 // 8-byte loads, conflict-free thanks to a permutation of k) and issues two mma.sync.m16n8k16 (bf16 in,
 // fp32 accumulate).  The dynamic 3x3 kernel stays depth-wise and in fp32: nine FMAs per output on the
@@ -30,11 +30,12 @@ constexpr int PITCH = TW + K13 - 1;                // 76 staged pixels per row
 constexpr int TILE_BYTES = THP * PITCH * CG * 2;   // 68,096
 constexpr int WFRAG_BYTES = K13 * K13 * 32 * 16;   // 86,528: [tap][lane] x 4 words
 constexpr int DK_BYTES = ((CG * 9 * 4) + 127) / 128 * 128;
-constexpr int kThreads = 256, kWarps = 8;
-constexpr int RUNS = (TW / 16) * (TH / kWarps);    // 8 runs of 16 pixels per warp
+constexpr int kThreads = 512, kWarps = 16;
+constexpr int RPW = TH / kWarps;                   // tile rows per warp
+constexpr int RUNS = (TW / 16) * RPW;              // runs of 16 pixels per warp
 static_assert(TILE_BYTES % 128 == 0, "tile buffers keep 128-byte alignment");
 static_assert(TH * TW * CG * 2 <= TILE_BYTES, "the result tile is staged in the consumed input buffer");
-static_assert(TH % kWarps == 0 && TW % 16 == 0, "tile splits into whole runs per warp");
+static_assert(TH % kWarps == 0 && TW == 64, "tile splits into whole runs per warp; u >> 2 and u & 3 assume four runs per row");
 constexpr size_t kSmemBytes = 2 * (size_t)TILE_BYTES + WFRAG_BYTES + DK_BYTES + 128;
 
 struct Params {
@@ -119,8 +120,8 @@ stencil_dense_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __gri
 #pragma unroll
                 for (int e = 0; e < 4; ++e) d[u][h][e] = 0.f;
 
-        // lane's first pixel of run u for tap (0,0): staged row 2*warp + (u >> 2), staged column 16*(u & 3) + g
-        const uint2* a2 = reinterpret_cast<const uint2*>(tbuf) + ((2 * warp) * PITCH + g) * 4 + t;
+        // lane's first pixel of run u for tap (0,0): staged row RPW*warp + (u >> 2), staged column 16*(u & 3) + g
+        const uint2* a2 = reinterpret_cast<const uint2*>(tbuf) + ((RPW * warp) * PITCH + g) * 4 + t;
 #pragma unroll 1
         for (int i = 0; i < K13; ++i) {
             if (i == 1 && tid == 0 && k + 1 < my_units) {
@@ -162,7 +163,7 @@ stencil_dense_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __gri
                 const int off = ((P6 - 1 + tap / 3) * PITCH + (P6 - 1 + tap % 3)) * NPAIR;
 #pragma unroll
                 for (int u = 0; u < RUNS; ++u) {
-                    const int px = ((2 * warp + (u >> 2)) * PITCH + (u & 3) * 16 + g) * NPAIR + off;
+                    const int px = ((RPW * warp + (u >> 2)) * PITCH + (u & 3) * 16 + g) * NPAIR + off;
 #pragma unroll
                     for (int r = 0; r < 2; ++r) {            // pixel g, pixel g + 8
                         const uint32_t v0 = x32[px + r * 8 * NPAIR + t], v1 = x32[px + r * 8 * NPAIR + 4 + t];
@@ -181,7 +182,7 @@ stencil_dense_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __gri
             uint32_t* s32 = reinterpret_cast<uint32_t*>(tbuf);
 #pragma unroll
             for (int u = 0; u < RUNS; ++u) {
-                const int px = ((2 * warp + (u >> 2)) * TW + (u & 3) * 16 + g) * NPAIR;
+                const int px = ((RPW * warp + (u >> 2)) * TW + (u & 3) * 16 + g) * NPAIR;
 #pragma unroll
                 for (int r = 0; r < 2; ++r) {
                     s32[px + r * 8 * NPAIR + t] = pack_bf16x2(d[u][0][2 * r], d[u][0][2 * r + 1]);
