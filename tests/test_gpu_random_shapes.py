@@ -34,13 +34,16 @@ def _cases(n, seed):
         K = int(rng.choice([13, 13, 13, 13, 5, 17]))
         dtype = synth.BF16 if rng.random() < 0.6 else synth.F32
         layout = synth.NHWC if rng.random() < 0.6 else synth.NCHW
-        variant = ["plain", "mlp", "pw"][i % 3]
+        variant = ["plain", "mlp", "pw", "dense"][i % 4]
+        if variant == "dense":                              # the oracle does 16 x K x K terms per output: keep it small
+            H, W, C_a = min(H, 48), min(W, 80), 16 if rng.random() < 0.7 else C_a
+            C = max(C, C_a)
         width = int(rng.choice([0, 0, 40, 64]))
         out.append((B, C, C_a, H, W, K, dtype, layout, variant, width))
     return out
 
 
-CASES = _cases(45, seed=20250306)
+CASES = _cases(60, seed=20250306)
 
 
 @pytest.mark.parametrize("case", CASES, ids=lambda c: "-".join(map(str, c)))
@@ -69,6 +72,10 @@ def test_random_case(pkg, oracle, case):
             keys = ("w_down", "b_down", "w_up", "b_up")
             pkg.esc_convattn_forward_mlp(x, C_a, K, wl, *(torch.from_numpy(m[k]).to("cuda", tdt) for k in keys), out, lay, ws)
             ref, mag = oracle.forward_mlp(d["x"], C_a, d["w_large"], *(m[k] for k in keys), want_mag=True)
+        elif variant == "dense":
+            wdn = synth.make_dense_kernel(C_a, K, dtype, seed=seed)
+            pkg.esc_convattn_forward_dense(x, C_a, K, torch.from_numpy(wdn).to("cuda", tdt), wd, bd, out, lay, ws)
+            ref, mag = oracle.forward_dense(d["x"], C_a, wdn, d["w_dyn"], d["b_dyn"], want_mag=True)
         else:
             wp = synth.make_pointwise(C_a, dtype, seed=seed)
             pkg.esc_convattn_forward_pw(x, C_a, K, wl, torch.from_numpy(wp).to("cuda", tdt), wd, bd, out, lay, ws)
@@ -87,6 +94,7 @@ def test_random_case(pkg, oracle, case):
         # accumulation noise; where the fast kernel also keeps the mixed features in bf16, one more rounding
         # of every input of the depth-wise stage, bounded by 2^-8 of sum |w| |mixed| <= 2^-8 * mag
         extra = 2.0 ** -8 * mag if variant == "pw" and pkg.esc_convattn_last_path() == 2 else 0.0
-        bar = 2.0 ** -8 * np.abs(ref[:, :C_a]) * 1.001 + extra + 1e-5 * mag + 1e-30
+        noise = 5e-5 if variant == "dense" else 1e-5       # 16 x K x K terms through the tensor cores' fp32 adders
+        bar = 2.0 ** -8 * np.abs(ref[:, :C_a]) * 1.001 + extra + noise * mag + 1e-30
         assert (err <= bar).all(), f"{case}: {int((err > bar).sum())} outputs beyond the rounding bound"
     assert np.array_equal(got[:, C_a:], ref[:, C_a:])
