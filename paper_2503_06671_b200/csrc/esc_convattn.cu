@@ -214,6 +214,28 @@ int launch_copy(const Problem& p, const void* x, void* out, cudaStream_t st) {
     return launch_copy_u<uint16_t>(x, out, rows, row_b, stride_b, off_b, st);
 }
 
+// The identity channels as a copy job for extra blocks of a stencil launch (blocks == 0: nothing to copy).
+esc::CopyJob make_copy_job(const Problem& p, const void* x, void* out, long long first_block, int threads) {
+    esc::CopyJob j = {};
+    if (p.Ca == p.C) return j;
+    const long long es = (long long)p.es(), HW = (long long)p.H * p.W;
+    long long rows, row_b, stride_b, off_b;
+    if (p.layout == ESC_NCHW) { rows = p.B; row_b = (p.C - p.Ca) * HW * es; stride_b = p.C * HW * es; off_b = p.Ca * HW * es; }
+    else { rows = (long long)p.B * HW; row_b = (p.C - p.Ca) * es; stride_b = p.C * es; off_b = p.Ca * es; }
+    const int u = (row_b % 16 == 0 && stride_b % 16 == 0 && off_b % 16 == 0) ? 16
+                : (row_b % 4 == 0 && stride_b % 4 == 0 && off_b % 4 == 0) ? 4 : 2;
+    j.src = x; j.dst = out;
+    j.rows = rows; j.row_units = row_b / u; j.stride_units = stride_b / u; j.offset_units = off_b / u;
+    j.unit_bytes = u;
+    const long long total = rows * j.row_units;
+    long long blocks = (total + (long long)threads * 4 - 1) / ((long long)threads * 4);   // about four units per thread
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks < 1) blocks = 1;
+    j.first_block = (unsigned)first_block;
+    j.blocks = (unsigned)blocks;
+    return j;
+}
+
 template <typename T, int LAYOUT>
 int launch_generic_t(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                      cudaStream_t st, bool dependent) {
@@ -221,9 +243,10 @@ int launch_generic_t(const Problem& p, const void* x, const void* w_large, const
     const int TX = regtile ? esc::kRtTX : esc::kGenTX, TY = regtile ? esc::kRtTY : esc::kGenTY;
     const int tiles_x = (p.W + TX - 1) / TX, tiles_y = (p.H + TY - 1) / TY;
     const long long blocks = (long long)p.B * p.Ca * tiles_x * tiles_y;
-    if (blocks > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
+    const esc::CopyJob job = make_copy_job(p, x, out, blocks, regtile ? esc::kRtThreads : esc::kGenTX * esc::kGenTY);
+    if (blocks + job.blocks > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.gridDim = dim3((unsigned)(blocks + job.blocks));   // the copy blocks come last
     cfg.blockDim = regtile ? dim3(esc::kRtThreads) : dim3(esc::kGenTX, esc::kGenTY);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -234,10 +257,10 @@ int launch_generic_t(const Problem& p, const void* x, const void* w_large, const
     if (regtile)
         ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT>, static_cast<const T*>(x),
                                     static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk,
-                                    tiles_x, tiles_y));
+                                    tiles_x, tiles_y, job));
     else
         ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_generic<T, LAYOUT>, static_cast<const T*>(x), static_cast<T*>(out),
-                                    p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk, tiles_x, tiles_y));
+                                    p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk, tiles_x, tiles_y, job));
     ++g_last_launches;
     return ESC_OK;
 }
@@ -253,8 +276,7 @@ int launch_generic(const Problem& p, const void* x, const void* w_large, const f
     else
         rc = p.layout == ESC_NCHW ? launch_generic_t<__nv_bfloat16, esc::kNCHW>(p, x, w_large, dk, out, st, dependent)
                                   : launch_generic_t<__nv_bfloat16, esc::kNHWC>(p, x, w_large, dk, out, st, dependent);
-    if (rc != ESC_OK) return rc;
-    return launch_copy(p, x, out, st);
+    return rc;                                             // the identity channels went along as copy blocks
 }
 
 int launch_stencil(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,

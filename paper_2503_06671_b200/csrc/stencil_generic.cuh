@@ -25,14 +25,48 @@ __device__ __forceinline__ float staged_value(const T* __restrict__ x, const T* 
     return v;
 }
 
+// The identity channels (Concat of Eq. 4 line 4) as a strided 2-D copy -- `rows` rows of `row_units` units of
+// `unit_bytes` bytes, `stride_units` apart, starting `offset_units` into both tensors -- done by the last
+// `blocks` blocks (from `first_block` on) of the same launch that computes the attention channels, so that
+// the copy, bound by HBM, runs beside the tail of the arithmetic instead of in a launch of its own after it
+// (measured: better than putting the copy blocks first).  blocks == 0: nothing to copy.
+struct CopyJob {
+    const void* src;
+    void* dst;
+    long long rows, row_units, stride_units, offset_units;
+    int unit_bytes;
+    unsigned first_block, blocks;
+};
+
+template <typename U>
+__device__ __forceinline__ void copy_job_units(const CopyJob& j, unsigned rank, unsigned tid, unsigned nthreads) {
+    const U* __restrict__ src = static_cast<const U*>(j.src);
+    U* __restrict__ dst = static_cast<U*>(j.dst);
+    const long long total = j.rows * j.row_units, step = (long long)j.blocks * nthreads;
+    for (long long i = (long long)rank * nthreads + tid; i < total; i += step) {
+        const long long r = i / j.row_units, q = i - r * j.row_units;
+        const long long e = r * j.stride_units + j.offset_units + q;
+        dst[e] = src[e];
+    }
+}
+__device__ __forceinline__ void run_copy_job(const CopyJob& j, unsigned rank, unsigned tid, unsigned nthreads) {
+    if (j.unit_bytes == 16) copy_job_units<uint4>(j, rank, tid, nthreads);
+    else if (j.unit_bytes == 4) copy_job_units<uint32_t>(j, rank, tid, nthreads);
+    else copy_job_units<uint16_t>(j, rank, tid, nthreads);
+}
+
 template <typename T, int LAYOUT>
 __global__ void __launch_bounds__(kGenTX * kGenTY)
 stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W, int K,
                 const T* __restrict__ w_large, const T* __restrict__ w_point, const float* __restrict__ dk,
-                int tiles_x, int tiles_y)
+                int tiles_x, int tiles_y, const CopyJob job)
 {
     __shared__ float tile[(kGenTY + kGenMaxK - 1) * (kGenTX + kGenMaxK - 1)];
     __shared__ float wm[kGenMaxK * kGenMaxK];
+    if (job.blocks != 0 && blockIdx.x >= job.first_block) {
+        run_copy_job(job, blockIdx.x - job.first_block, threadIdx.y * kGenTX + threadIdx.x, kGenTX * kGenTY);
+        return;
+    }
 
     long long bid = blockIdx.x;
     const int tx = (int)(bid % tiles_x); bid /= tiles_x;
@@ -84,10 +118,14 @@ template <typename T, int LAYOUT>
 __global__ void __launch_bounds__(kRtThreads)
 stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W,
                     const T* __restrict__ w_large, const T* __restrict__ w_point, const float* __restrict__ dk,
-                    int tiles_x, int tiles_y)
+                    int tiles_x, int tiles_y, const CopyJob job)
 {
     __shared__ __align__(16) float tile[kRtRows * kRtPitch];
     __shared__ __align__(16) float wm[kRtK * 16];      // merged kernel, rows padded to 16 taps
+    if (job.blocks != 0 && blockIdx.x >= job.first_block) {
+        run_copy_job(job, blockIdx.x - job.first_block, threadIdx.x, kRtThreads);
+        return;
+    }
 
     long long bid = blockIdx.x;
     const int tx = (int)(bid % tiles_x); bid /= tiles_x;
