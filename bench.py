@@ -349,7 +349,7 @@ def main():
         bf16_peak = peaks()["bf16_tflops"]
         dense = {"ms_per_step": ms_dense, "bound": "tensor", "achieved": fl / (ms_dense * 1e-3) / 1e12, "peak": bf16_peak,
                  "unit": "TFLOP/s", "frac": fl / (ms_dense * 1e-3) / 1e12 / bf16_peak,
-                 "note": "whole step (GAP + dense stencil + copy kernel); warp-level mma.sync"}
+                 "note": "whole step (GAP kernel + dense stencil kernel with copy blocks); warp-level mma.sync"}
 
     pk = peaks()
     flops = 2.0 * wl.K * wl.K * wl.C_a * wl.pixels                    # merged 169-tap form, Eq. 5

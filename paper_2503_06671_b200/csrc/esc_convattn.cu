@@ -336,11 +336,14 @@ int launch_dense_generic_t(const Problem& p, const void* x, const void* w_dense,
 int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, const float* dk, void* out,
                          unsigned* ctrl, cudaStream_t st, bool dependent) {
     g_last_tile_w = 0;
+    esc::CopyJob job = make_copy_job(p, x, out, 0, esc::tma::dense::kThreads);
+    if (job.blocks > 148) job.blocks = 148;                // every block of that launch takes a whole SM
     int rc = esc::tma::try_launch_dense(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_dense, dk, out, ctrl,
-                                        st, dependent, &g_last_launches, &g_last_error);
+                                        st, dependent, job, &g_last_launches, &g_last_error);
     if (rc == ESC_OK) {
         g_last_path = 3;
         g_last_tile_w = esc::tma::dense::TW;
+        return ESC_OK;                                     // the identity channels went along as copy blocks
     } else if (rc == esc::tma::kNotApplicable) {
         g_last_path = 1;
         if (p.dtype == ESC_F32)

@@ -19,6 +19,7 @@
 // kernel needs 1/8 byte of shared-memory bandwidth per multiply-add: at 128 bytes per clock and SM that
 // caps it at 1024 MAC/clk/SM whichever tensor-core instruction consumes the fragments.
 #pragma once
+#include "stencil_generic.cuh"
 #include "stencil_tma.cuh"
 
 namespace esc { namespace tma {
@@ -51,9 +52,17 @@ struct Params {
 
 __global__ void __launch_bounds__(dense::kThreads, 1)
 stencil_dense_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_res,
-                        const dense::Params p)
+                        const dense::Params p, const CopyJob job)
 {
     using namespace dense;
+    // The last blocks of the grid copy the identity channels.  They need a whole SM like every block of this
+    // launch, so they run where a tile-walking CTA has already finished (the tile count is rarely a multiple
+    // of the SM count) or after them, without a launch of their own.
+    if (job.blocks != 0 && blockIdx.x >= job.first_block) {
+        if (p.wait_first) pdl_wait_primary();              // launched on its own: x may still be in the making
+        run_copy_job(job, blockIdx.x - job.first_block, threadIdx.x, dense::kThreads);
+        return;
+    }
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* tilebuf = smem;                                               // 2 x TILE_BYTES
     uint4* wfrag = reinterpret_cast<uint4*>(smem + 2 * TILE_BYTES);              // [tap][lane]
@@ -70,7 +79,7 @@ stencil_dense_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __gri
     if (p.wait_first) pdl_wait_primary();
     pdl_launch_dependents();
 
-    const long long first = blockIdx.x, stride = gridDim.x;
+    const long long first = blockIdx.x, stride = job.blocks != 0 ? job.first_block : gridDim.x;
     const long long my_units = first < p.units ? (p.units - first + stride - 1) / stride : 0;
     auto coords = [&](long long k, int& b, int& ty, int& tx) {
         unsigned u = (unsigned)(first + k * stride);                             // the host guarantees units < 2^31
@@ -240,7 +249,7 @@ stencil_dense_generic(const T* __restrict__ x, T* __restrict__ out, int B, int C
 // Returns 0, kNotApplicable, or an ESC_ERR_* code.
 inline int try_launch_dense(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
                             const void* w_dense, const float* dk, void* out, unsigned* ctrl, cudaStream_t st,
-                            bool dependent, int* launches, std::string* err) {
+                            bool dependent, CopyJob job, int* launches, std::string* err) {
     using namespace dense;
     if (K != K13 || dtype != 1 /*bf16*/ || layout != kNHWC || Ca != CG || C % 8 != 0) return kNotApplicable;
     if ((reinterpret_cast<uintptr_t>(w_dense) & 1) != 0) return kNotApplicable;
@@ -267,7 +276,9 @@ inline int try_launch_dense(int B, int C, int Ca, int H, int W, int K, int dtype
         attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(p.units < sms ? p.units : sms));
+    const unsigned walkers = (unsigned)(p.units < sms ? p.units : sms);
+    if (job.blocks != 0) job.first_block = walkers;
+    cfg.gridDim = dim3(walkers + job.blocks);
     cfg.blockDim = dim3(dense::kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = st;
@@ -276,7 +287,7 @@ inline int try_launch_dense(int B, int C, int Ca, int H, int W, int K, int dtype
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_dense_nhwc_bf16, m_att, m_res, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_dense_nhwc_bf16, m_att, m_res, p, job);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_dense_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
