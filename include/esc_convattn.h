@@ -226,6 +226,25 @@ int esc_convattn_stencil_dense(const void* x, int B, int C, int C_a, int H, int 
                                void* out, int dtype, int layout,
                                void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Any combination of large-kernel form and estimator, i.e. the module as the paper's model variants use
+ * it: ESC and ESC-light -- dense LK (Section 3.2) with the two-layer estimator, h = 8; ESC-FP -- the
+ * decomposed LK of Eq. 5 with the two-layer estimator (Section 3.3 gives h = 4 or 8).
+ *   large_kernel  ESC_LK_DEPTHWISE: w_large [C_a,K,K], w_point ignored
+ *                 ESC_LK_DECOMPOSED: w_large [C_a,K,K] and w_point [C_a,C_a]
+ *                 ESC_LK_DENSE: w_large [C_a,C_a,K,K], w_point ignored
+ *   hidden        0: one linear layer, w_up [9*C_a,C_a] and b_up [9*C_a] play w_dyn and b_dyn, w_down and
+ *                 b_down are ignored; 1..128: the two-layer estimator with the exact GELU
+ * Everything else as for esc_convattn_forward_ex.  ESC_ERR_UNSUPPORTED for an unknown large_kernel.
+ */
+enum { ESC_LK_DEPTHWISE = 0, ESC_LK_DECOMPOSED = 1, ESC_LK_DENSE = 2 };
+int esc_convattn_forward_variant(const void* x, int B, int C, int C_a, int H, int W, int K, int large_kernel,
+                                 const void* w_large, const void* w_point,
+                                 const void* w_down, const void* b_down,
+                                 const void* w_up, const void* b_up, int hidden,
+                                 void* out, int dtype, int layout,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

@@ -22,6 +22,8 @@ from .binding import (  # noqa: F401
     esc_convattn_forward_host_wait,
     esc_convattn_forward_dense,
     esc_convattn_stencil_dense,
+    esc_convattn_forward_variant,
+    ESC_LK_DEPTHWISE, ESC_LK_DECOMPOSED, ESC_LK_DENSE,
     esc_convattn_forward_mlp,
     esc_convattn_forward_pw,
     esc_convattn_stencil_pw,

@@ -50,6 +50,7 @@ def lib():
         L.esc_convattn_stencil_pw.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_dense.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_stencil_dense.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_forward_variant.argtypes = [vp, i, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -61,7 +62,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -240,6 +241,22 @@ def esc_convattn_stencil_dense(x, C_a, K, w_dense, dk, out, layout, workspace=No
                                             0 if workspace is None else workspace.numel() * workspace.element_size(),
                                             _stream(stream)),
            "esc_convattn_stencil_dense")
+    return out
+
+
+ESC_LK_DEPTHWISE, ESC_LK_DECOMPOSED, ESC_LK_DENSE = 0, 1, 2
+
+
+def esc_convattn_forward_variant(x, C_a, K, large_kernel, w_large, w_point, w_down, b_down, w_up, b_up, out, layout,
+                                 workspace, stream=None):
+    """Any large-kernel form (ESC_LK_*) with either estimator: w_down None means one linear layer (w_up, b_up)."""
+    B, C, H, W = _dims(x, layout)
+    hidden = 0 if w_down is None else int(w_down.shape[0])
+    _check(lib().esc_convattn_forward_variant(_ptr(x), B, C, C_a, H, W, K, int(large_kernel), _ptr(w_large), _ptr(w_point),
+                                              _ptr(w_down), _ptr(b_down), _ptr(w_up), _ptr(b_up), hidden, _ptr(out),
+                                              _dtype_code(x), layout, _ptr(workspace),
+                                              workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_forward_variant")
     return out
 
 

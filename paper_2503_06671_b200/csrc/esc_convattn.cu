@@ -407,7 +407,7 @@ HostPath g_host[kHostSlots];
 
 extern "C" {
 
-int esc_version(void) { return 109; }
+int esc_version(void) { return 110; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
@@ -662,6 +662,31 @@ int esc_convattn_forward_dense(const void* x, int B, int C, int C_a, int H, int 
     p.dense = true;
     return forward_impl(p, x, w_dense, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, out, workspace,
                         static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_forward_variant(const void* x, int B, int C, int C_a, int H, int W, int K, int large_kernel,
+                                 const void* w_large, const void* w_point, const void* w_down, const void* b_down,
+                                 const void* w_up, const void* b_up, int hidden, void* out, int dtype, int layout,
+                                 void* workspace, size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (large_kernel != ESC_LK_DEPTHWISE && large_kernel != ESC_LK_DECOMPOSED && large_kernel != ESC_LK_DENSE)
+        return ESC_ERR_UNSUPPORTED;
+    if (hidden < 0) return ESC_ERR_SHAPE;
+    if (!w_large || (large_kernel == ESC_LK_DECOMPOSED && !w_point)) return ESC_ERR_NULL;
+    const Estimator est{w_up, b_up, hidden > 0 ? w_down : nullptr, hidden > 0 ? b_down : nullptr, hidden};
+    rc = check_estimator(p, est);
+    if (rc != ESC_OK) return rc;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, p.es()) || (large_kernel == ESC_LK_DECOMPOSED && !aligned(w_point, p.es()))) return ESC_ERR_ALIGN;
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    if (large_kernel == ESC_LK_DECOMPOSED) p.w_point = w_point;
+    p.dense = large_kernel == ESC_LK_DENSE;
+    return forward_impl(p, x, w_large, est, out, workspace, static_cast<cudaStream_t>(stream));
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {

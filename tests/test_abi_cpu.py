@@ -102,6 +102,10 @@ def test_host_side_rejections_launch_nothing(L):
     assert L.esc_convattn_forward_dense(X, 1, 64, 16, 32, 32, 13, Wdn + 1, Wd, Bd, O, 1, 1, WS, big, None) == 4
     assert L.esc_convattn_forward_dense(X, 1, 64, 16, 32, 32, 13, Wdn, Wd, Bd, X, 1, 1, WS, big, None) == 5
     assert L.esc_convattn_stencil_dense(X, 1, 64, 16, 8, 8, 12, Wdn, Wd, O, 0, 0, None, 0, None) == 2
+    assert L.esc_convattn_forward_variant(X, 1, 64, 16, 32, 32, 13, 9, Wl, None, None, None, Wd, Bd, 0, O, 1, 1, WS, big, None) == 3
+    assert L.esc_convattn_forward_variant(X, 1, 64, 16, 32, 32, 13, 1, Wl, None, None, None, Wd, Bd, 0, O, 1, 1, WS, big, None) == 1
+    assert L.esc_convattn_forward_variant(X, 1, 64, 16, 32, 32, 13, 0, Wl, None, None, None, Wd, Bd, 8, O, 1, 1, WS, big, None) == 1
+    assert L.esc_convattn_forward_variant(X, 1, 64, 16, 32, 32, 13, 0, Wl, None, None, None, Wd, Bd, -1, O, 1, 1, WS, big, None) == 2
     assert L.esc_convattn_forward_host_submit(2, X, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 3
     assert L.esc_convattn_forward_host_submit(0, None, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 1
     assert L.esc_convattn_forward_host_wait(-1) == 3
