@@ -11,6 +11,7 @@ from .convattn_oracle import (  # noqa: F401
     dynkernel_mlp,
     forward_mlp,
     stencil,
+    backward,
     stencil_dense,
     forward_dense,
     pointwise,

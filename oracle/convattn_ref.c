@@ -28,6 +28,9 @@
  * convattn_ref_stencil_dense is Eq. 4 line 3 with the dense large kernel of Section 3.2
  * (13x13x16x16: every output channel sums over all attention input channels).
  *
+ * convattn_ref_backward is the gradient of the first form above with respect to x, LK, W_dyn and
+ * b_dyn, by the chain rule written out.
+ *
  * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
  * Everything is accumulated in double precision with direct nested loops in
  * the order written above: no tiling, no merging of the two kernels, no reuse.
@@ -48,11 +51,15 @@
  * by the identity mix, library 1x1 + depth-wise convolutions, the commutation with a
  * channel-independent spatial kernel, permutation mixes and a brute force; the dense
  * large kernel by its diagonal case (= the depth-wise stencil), a library dense
- * convolution, the depth-wise-then-point-wise factorisation and a brute force.
+ * convolution, the depth-wise-then-point-wise factorisation and a brute force; the
+ * backward pass by central differences of the pinned forward (exact for this
+ * function, which is quadratic in x and bilinear in weights and x) and the
+ * adjoint identity.
  */
 #include <stddef.h>
 #include <stdint.h>
 #include <math.h>
+#include <stdlib.h>
 
 #define IDX4(b, c, y, x, C, H, W) ((((size_t)(b) * (C) + (c)) * (H) + (y)) * (size_t)(W) + (x))
 
@@ -293,6 +300,120 @@ void convattn_ref_stencil_dense(const float *x, int B, int C, int C_a, int H, in
                     out[IDX4(b, n, y, xx, C, H, W)] = s;
                     if (mag) mag[IDX4(b, n, y, xx, C_a, H, W)] = m;
                 }
+}
+
+/* Backward pass of the forward above (one-layer estimator, depth-wise LK; Eq. 4), by the chain rule written
+ * out.  With go = dL/dout [B,C,H,W], Wm[b,c] = LK[c] + ZP(dk[b,c]) and x~ the zero-padded input:
+ *   g_tap[b,c,i,j] = sum_{y,x} go[b,c,y,x] * x~[b,c,y+i-P,x+j-P]              (per-image tap gradient)
+ *   g_lk[c,i,j]    = sum_b g_tap[b,c,i,j]                                      (dL/dLK)
+ *   g_dk[b,c,i,j]  = g_tap[b,c,i+P-1,j+P-1]                                    (its central 3x3: dL/ddk)
+ *   g_b[o]         = sum_b g_dk[b,o]            g_W[o,k] = sum_b g_dk[b,o] * g[b,k]
+ *   g_g[b,k]       = sum_o W[o,k] * g_dk[b,o]
+ *   g_x[b,c,y,x]   = sum_{i,j} Wm[b,c,i,j] * go~[b,c,y-(i-P),x-(j-P)] + g_g[b,c] / (H*W)      c < C_a
+ *   g_x[b,c]       = go[b,c]                                                                   c >= C_a
+ * Outputs: gx [B,C,H,W], glk [C_a,K,K], gw [9*C_a,C_a], gb [9*C_a]; any of them may be NULL. */
+void convattn_ref_backward(const float *x, const float *go, int B, int C, int C_a, int H, int W, int K,
+                           const double *w_large, const double *w_dyn, const double *b_dyn,
+                           double *gx, double *glk, double *gw, double *gb)
+{
+    const int P = (K - 1) / 2;
+    const size_t nt = (size_t)B * C_a * K * K;
+    double *g = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    double *dk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    double *gtap = (double *)malloc(sizeof(double) * nt);
+    double *gg = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    convattn_ref_gap(x, B, C, C_a, H, W, g);
+    convattn_ref_dynkernel(g, B, C_a, w_dyn, b_dyn, dk);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C_a; ++c)
+            for (int i = 0; i < K; ++i)
+                for (int j = 0; j < K; ++j) {
+                    double s = 0.0;
+                    for (int y = 0; y < H; ++y)
+                        for (int xx = 0; xx < W; ++xx) {
+                            int yy = y + i - P, xc = xx + j - P;
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                s += (double)go[IDX4(b, c, y, xx, C, H, W)] * (double)x[IDX4(b, c, yy, xc, C, H, W)];
+                        }
+                    gtap[(((size_t)b * C_a + c) * K + i) * K + j] = s;
+                }
+    if (glk)
+        for (int c = 0; c < C_a; ++c)
+            for (int t = 0; t < K * K; ++t) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gtap[((size_t)b * C_a + c) * K * K + t];
+                glk[(size_t)c * K * K + t] = s;
+            }
+    /* dL/ddk[b,o], o = c*9 + i*3 + j: the central 3x3 of the tap gradient (zero where K < 3 leaves no such tap) */
+#define GDK(b, c, i, j) (((i) + P - 1 >= 0 && (i) + P - 1 < K && (j) + P - 1 >= 0 && (j) + P - 1 < K) \
+                             ? gtap[(((size_t)(b) * C_a + (c)) * K + (i) + P - 1) * K + (j) + P - 1] : 0.0)
+    /* for K = 1 the dynamic taps other than the centre have no LK counterpart: take them directly */
+    double *gdk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C_a; ++c)
+            for (int i = 0; i < 3; ++i)
+                for (int j = 0; j < 3; ++j) {
+                    double s;
+                    if (K >= 3) s = GDK(b, c, i, j);
+                    else {
+                        s = 0.0;
+                        for (int y = 0; y < H; ++y)
+                            for (int xx = 0; xx < W; ++xx) {
+                                int yy = y + i - 1, xc = xx + j - 1;
+                                if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                    s += (double)go[IDX4(b, c, y, xx, C, H, W)] * (double)x[IDX4(b, c, yy, xc, C, H, W)];
+                            }
+                    }
+                    gdk[((size_t)b * C_a + c) * 9 + i * 3 + j] = s;
+                }
+#undef GDK
+    if (gb)
+        for (int o = 0; o < 9 * C_a; ++o) {
+            double s = 0.0;
+            for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o];
+            gb[o] = s;
+        }
+    if (gw)
+        for (int o = 0; o < 9 * C_a; ++o)
+            for (int k = 0; k < C_a; ++k) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o] * g[(size_t)b * C_a + k];
+                gw[(size_t)o * C_a + k] = s;
+            }
+    for (int b = 0; b < B; ++b)
+        for (int k = 0; k < C_a; ++k) {
+            double s = 0.0;
+            for (int o = 0; o < 9 * C_a; ++o) s += w_dyn[(size_t)o * C_a + k] * gdk[(size_t)b * 9 * C_a + o];
+            gg[(size_t)b * C_a + k] = s;
+        }
+    if (gx) {
+#pragma omp parallel for collapse(3) schedule(static)
+        for (int b = 0; b < B; ++b)
+            for (int c = 0; c < C; ++c)
+                for (int y = 0; y < H; ++y)
+                    for (int xx = 0; xx < W; ++xx) {
+                        if (c >= C_a) {
+                            gx[IDX4(b, c, y, xx, C, H, W)] = (double)go[IDX4(b, c, y, xx, C, H, W)];
+                            continue;
+                        }
+                        double s = 0.0;
+                        for (int i = 0; i < K; ++i)
+                            for (int j = 0; j < K; ++j) {
+                                int yy = y - (i - P), xc = xx - (j - P);
+                                if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                    s += w_large[((size_t)c * K + i) * K + j] * (double)go[IDX4(b, c, yy, xc, C, H, W)];
+                            }
+                        for (int i = 0; i < 3; ++i)
+                            for (int j = 0; j < 3; ++j) {
+                                int yy = y - (i - 1), xc = xx - (j - 1);
+                                if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                    s += dk[((size_t)b * C_a + c) * 9 + i * 3 + j] * (double)go[IDX4(b, c, yy, xc, C, H, W)];
+                            }
+                        gx[IDX4(b, c, y, xx, C, H, W)] = s + gg[(size_t)b * C_a + c] / ((double)H * (double)W);
+                    }
+    }
+    free(g); free(dk); free(gtap); free(gg); free(gdk);
 }
 
 /* Selected outputs, one by one: idx[n] are flat indices into out[B,C,H,W]; dk is
