@@ -31,8 +31,8 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one stencil-kernel launch from the ncu capture summarised under
 # profiles/, keyed by (workload, layout, library version the capture was taken with).  Reported only while the
 # library still has that version; otherwise the kernel has changed since and the figure is withheld.
-# (Versions 109 and 110 added entry points and kernels for other variants; the kernel timed here is the one captured at 108.)
-NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", v): 29.56e6 + 0.47e6 for v in (108, 109, 110)}
+# (Versions 109 to 111 added entry points and kernels for other variants; the kernel timed here is the one captured at 108.)
+NCU_TRAFFIC_BYTES = {("cfg3_640x360_bf16", "nhwc", v): 29.56e6 + 0.47e6 for v in (108, 109, 110, 111)}
 
 
 def peaks():

@@ -245,6 +245,26 @@ int esc_convattn_forward_variant(const void* x, int B, int C, int C_a, int H, in
                                  void* out, int dtype, int layout,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Backward pass of esc_convattn_forward_ex (one-layer estimator, depth-wise LK; the chain rule applied to
+ * Eq. 4): given grad_out = dL/dout, writes
+ *   grad_x        [B,C,H,W]    dL/dx, element type and layout of x (identity channels: grad_out itself; attention
+ *                              channels: grad_out correlated with the 180-degree-rotated merged kernels, plus the
+ *                              path through the GAP and the estimator)
+ *   grad_w_large  [C_a,K,K]    fp32   dL/dLK        (may be NULL)
+ *   grad_w_dyn    [9*C_a,C_a]  fp32   dL/dW_dyn     (may be NULL)
+ *   grad_b_dyn    [9*C_a]      fp32   dL/db_dyn     (may be NULL)
+ * K must be 13 (ESC_ERR_UNSUPPORTED otherwise).  grad_x must not overlap x or grad_out.  The workspace is one of
+ * esc_convattn_backward_workspace_bytes(...) bytes, 256-byte aligned, zeroed once with
+ * esc_convattn_workspace_init(); it is not the forward workspace.  All sums are added in a fixed order.
+ */
+size_t esc_convattn_backward_workspace_bytes(int B, int C_a, int H, int W, int K);
+int esc_convattn_backward(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                          const void* w_large, const void* w_dyn, const void* b_dyn,
+                          void* grad_x, float* grad_w_large, float* grad_w_dyn, float* grad_b_dyn,
+                          int dtype, int layout,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

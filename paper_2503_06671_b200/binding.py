@@ -51,6 +51,9 @@ def lib():
         L.esc_convattn_forward_dense.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_stencil_dense.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_variant.argtypes = [vp, i, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, vp, i, i, vp, sz, vp]
+        L.esc_convattn_backward_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.esc_convattn_backward_workspace_bytes.restype = sz
+        L.esc_convattn_backward.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -62,7 +65,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -245,6 +248,34 @@ def esc_convattn_stencil_dense(x, C_a, K, w_dense, dk, out, layout, workspace=No
 
 
 ESC_LK_DEPTHWISE, ESC_LK_DECOMPOSED, ESC_LK_DENSE = 0, 1, 2
+
+
+def esc_convattn_backward_workspace_bytes(B, C_a, H, W, K) -> int:
+    return int(lib().esc_convattn_backward_workspace_bytes(B, C_a, H, W, K))
+
+
+def new_backward_workspace(B, C_a, H, W, K, device="cuda"):
+    """Allocate (with torch) and zero a workspace for esc_convattn_backward."""
+    import torch
+
+    n = esc_convattn_backward_workspace_bytes(B, C_a, H, W, K)
+    if n == 0:
+        raise ValueError("invalid problem size, or K is not 13")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    esc_convattn_workspace_init(ws)
+    return ws
+
+
+def esc_convattn_backward(x, grad_out, C_a, K, w_large, w_dyn, b_dyn, grad_x, grad_w_large, grad_w_dyn, grad_b_dyn,
+                          layout, workspace, stream=None):
+    """Gradients of esc_convattn_forward_ex: grad_x like x; the three weight gradients are fp32 tensors or None."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_backward(_ptr(x), _ptr(grad_out), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_dyn), _ptr(b_dyn),
+                                       _ptr(grad_x), _ptr(grad_w_large), _ptr(grad_w_dyn), _ptr(grad_b_dyn),
+                                       _dtype_code(x), layout, _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_backward")
+    return grad_x
 
 
 def esc_convattn_forward_variant(x, C_a, K, large_kernel, w_large, w_point, w_down, b_down, w_up, b_up, out, layout,

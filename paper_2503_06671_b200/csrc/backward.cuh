@@ -1,0 +1,194 @@
+// Backward pass of the ConvAttn forward (ESC paper, Section 3.3, Eq. 4, one-layer estimator, depth-wise LK),
+// the chain rule written out.  With go = dL/dout and Wm[b,c] = LK[c] + ZP(dk[b,c]):
+//
+//   g_tap[b,c,i,j] = sum_{y,x} go[b,c,y,x] * x~[b,c,y+i-6,x+j-6]      per-image tap gradient  (kernel tap_grad)
+//   g_lk = sum_b g_tap;   g_dk = central 3x3 of g_tap;   g_b = sum_b g_dk;   g_W[o,k] = sum_b g_dk[b,o] g[b,k]
+//   g_g[b,k] = sum_o W[o,k] g_dk[b,o]                                                        (kernel finish)
+//   g_x[b,c] = go[b,c] (*) flip(Wm[b,c]) + g_g[b,c] / (H W)   (c < C_a),   g_x[b,c] = go[b,c]  (c >= C_a)
+//
+// The last line is the forward stencil applied to go with both kernels rotated by 180 degrees and a
+// per-(image, channel) constant added, so it runs on the forward kernels; `finish` prepares the rotated
+// kernels and the constants for it.  Every reduction is done in a fixed order: results are reproducible.
+#pragma once
+#include "common.cuh"
+#include "stencil_generic.cuh"
+
+namespace esc { namespace bwd {
+
+constexpr int K = 13, P = 6, TAPS = K * K;
+constexpr int TX = 64, TY = 64, OX = 8, OY = 4;           // tile of go per block, patch of go per thread
+constexpr int XP = TX + K - 1;                            // 76 floats per staged x row (a multiple of 4)
+constexpr int XR = TY + K - 1;                            // 76 staged x rows
+constexpr int kThreads = (TX / OX) * (TY / OY);           // 128
+constexpr int kSlot = 176;                                // floats per (image, channel, tile): 169 taps, sum of x, padding
+static_assert(XP % 4 == 0 && TAPS + 1 <= kSlot, "layout");
+
+// ---- kernel 1: per-tile partial tap gradients and partial sums of x ---------------------------------------
+// Block = (image b, attention channel c, 64x64 tile).  The x halo tile (zeros outside the image) and the go
+// tile (zeros outside) are staged in shared memory as fp32; a thread keeps its 4x8 patch of go in registers
+// and, for every kernel row i, reads the four x rows its patch meets (five 16-byte reads each) and forms the
+// 13 partial sums of that row: 416 FMAs per 20 reads.  The 13 sums are then added over the block in a fixed
+// order (shuffle butterfly inside a warp, warps in order).
+template <typename T, int LAYOUT>
+__global__ void __launch_bounds__(kThreads)
+tap_grad(const T* __restrict__ x, const T* __restrict__ go, int C, int Ca, int H, int W, int tiles_x, int tiles_y,
+         float* __restrict__ part)      // [B][Ca][tiles][kSlot]
+{
+    __shared__ __align__(16) float xt[XR * XP];
+    __shared__ __align__(16) float gt[TY * TX];
+    __shared__ float red[kThreads / 32][16];
+
+    long long bid = blockIdx.x;
+    const int tiles = tiles_x * tiles_y;
+    const int tile = (int)(bid % tiles); bid /= tiles;
+    const int c = (int)(bid % Ca);
+    const int b = (int)(bid / Ca);
+    const int tx = tile % tiles_x, ty = tile / tiles_x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int y0 = ty * TY, x0 = tx * TX;
+
+    for (int t = tid; t < XR * XP; t += kThreads) {
+        const int r = t / XP, q = t % XP;
+        const int y = y0 - P + r, xx = x0 - P + q;
+        xt[t] = (y >= 0 && y < H && xx >= 0 && xx < W) ? Elem<T>::to_f32(x[elem_index<LAYOUT>(b, c, y, xx, C, H, W)]) : 0.f;
+    }
+    for (int t = tid; t < TY * TX; t += kThreads) {
+        const int r = t / TX, q = t % TX;
+        const int y = y0 + r, xx = x0 + q;
+        gt[t] = (y < H && xx < W) ? Elem<T>::to_f32(go[elem_index<LAYOUT>(b, c, y, xx, C, H, W)]) : 0.f;
+    }
+    __syncthreads();
+
+    const int lx = tid % (TX / OX), ly = tid / (TX / OX);
+    float g[OY][OX];
+    float sx = 0.f;                                       // sum of x over the patch (for the GAP of this image)
+#pragma unroll
+    for (int a = 0; a < OY; ++a) {
+        const float4* gr = reinterpret_cast<const float4*>(gt + (ly * OY + a) * TX + lx * OX);
+        const float4 q0 = gr[0], q1 = gr[1];
+        g[a][0] = q0.x; g[a][1] = q0.y; g[a][2] = q0.z; g[a][3] = q0.w;
+        g[a][4] = q1.x; g[a][5] = q1.y; g[a][6] = q1.z; g[a][7] = q1.w;
+        const float4* xr = reinterpret_cast<const float4*>(xt + (ly * OY + a + P) * XP + lx * OX + P - 2);   // 16-byte aligned: P - 2 = 4
+        // the patch's own pixels sit at columns lx*OX + P .. +7: floats 2..9 of the three reads from column lx*OX + 4
+        const float4 u0 = xr[0], u1 = xr[1], u2 = xr[2];
+        sx += (u0.z + u0.w) + (u1.x + u1.y + u1.z + u1.w) + (u2.x + u2.y);
+    }
+    float* slot = part + (((size_t)b * Ca + c) * tiles + tile) * kSlot;
+
+#pragma unroll 1
+    for (int i = 0; i < K; ++i) {
+        float s[K];
+#pragma unroll
+        for (int j = 0; j < K; ++j) s[j] = 0.f;
+#pragma unroll
+        for (int a = 0; a < OY; ++a) {
+            float in[OX + K - 1];                         // x row (ly*OY + a + i), columns lx*OX .. lx*OX + 19
+            const float4* xr = reinterpret_cast<const float4*>(xt + (ly * OY + a + i) * XP + lx * OX);
+#pragma unroll
+            for (int v = 0; v < (OX + K - 1) / 4; ++v) {
+                const float4 q = xr[v];
+                in[4 * v] = q.x; in[4 * v + 1] = q.y; in[4 * v + 2] = q.z; in[4 * v + 3] = q.w;
+            }
+#pragma unroll
+            for (int j = 0; j < K; ++j)
+#pragma unroll
+                for (int o = 0; o < OX; ++o) s[j] = fmaf(g[a][o], in[o + j], s[j]);
+        }
+        // block sum of the 13 values, fixed order
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) s[j] += __shfl_xor_sync(0xffffffffu, s[j], o);
+        if (lane == 0) {
+#pragma unroll
+            for (int j = 0; j < K; ++j) red[warp][j] = s[j];
+        }
+        __syncthreads();
+        if (tid < K) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) t += red[w][tid];
+            slot[i * K + tid] = t;
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, o);
+    if (lane == 0) red[warp][0] = sx;
+    __syncthreads();
+    if (tid == 0) {
+        float t = 0.f;
+        for (int w = 0; w < kThreads / 32; ++w) t += red[w][0];
+        slot[TAPS] = t;
+    }
+}
+
+// ---- kernel 2a: add the tiles of one (image, channel) in order ---------------------------------------------
+__global__ void __launch_bounds__(192)
+sum_tiles(const float* __restrict__ part, int tiles, float* __restrict__ gtap)   // gtap [B*Ca][kSlot]
+{
+    const size_t bc = blockIdx.x;
+    const int t = threadIdx.x;
+    if (t > TAPS) return;
+    const float* p = part + bc * tiles * kSlot + t;
+    float s = 0.f;
+    for (int k = 0; k < tiles; ++k) s += p[(size_t)k * kSlot];
+    gtap[bc * kSlot + t] = s;
+}
+
+// ---- kernel 2b: everything small; every output element is independent, a few blocks share them ------------
+// From g_tap [B][Ca][169 + sum x]: g_lk, g_b, g_W (fp32 outputs), and for the stencil pass that follows the
+// kernels rotated by 180 degrees -- w_flip (element type T), dk_flip [B][Ca][9] -- and the constants
+// bias[b][c] = g_g[b,c] / (H W).  g[b,k] = sum x / (H W) and dk = b_dyn + W g are recomputed here.
+template <typename T>
+__global__ void __launch_bounds__(256)
+finish(const float* __restrict__ gtap, int B, int Ca, int H, int W, const T* __restrict__ w_large,
+       const T* __restrict__ w_dyn, const T* __restrict__ b_dyn, float* __restrict__ g_lk, float* __restrict__ g_w,
+       float* __restrict__ g_b, T* __restrict__ w_flip, float* __restrict__ dk_flip, float* __restrict__ bias)
+{
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    const float inv_hw = 1.0f / ((float)H * (float)W);
+    auto gdk = [&](int b, int o) {                        // o = c*9 + i*3 + j -> central 3x3 of the tap gradient
+        const int c = o / 9, i = (o % 9) / 3, j = o % 3;
+        return gtap[((size_t)b * Ca + c) * kSlot + (i + P - 1) * K + (j + P - 1)];
+    };
+    auto gmean = [&](int b, int k) { return gtap[((size_t)b * Ca + k) * kSlot + TAPS] * inv_hw; };
+    if (g_lk)
+        for (int e = tid; e < Ca * TAPS; e += nth) {
+            const int c = e / TAPS, t = e % TAPS;
+            float s = 0.f;
+            for (int b = 0; b < B; ++b) s += gtap[((size_t)b * Ca + c) * kSlot + t];
+            g_lk[e] = s;
+        }
+    if (g_b)
+        for (int o = tid; o < 9 * Ca; o += nth) {
+            float s = 0.f;
+            for (int b = 0; b < B; ++b) s += gdk(b, o);
+            g_b[o] = s;
+        }
+    if (g_w)
+        for (int e = tid; e < 9 * Ca * Ca; e += nth) {
+            const int o = e / Ca, k = e % Ca;
+            float s = 0.f;
+            for (int b = 0; b < B; ++b) s = fmaf(gdk(b, o), gmean(b, k), s);
+            g_w[e] = s;
+        }
+    for (int e = tid; e < Ca * TAPS; e += nth) {
+        const int c = e / TAPS, t = e % TAPS;
+        w_flip[(size_t)c * TAPS + (TAPS - 1 - t)] = w_large[e];
+    }
+    for (int e = tid; e < B * Ca * 9; e += nth) {
+        const int b = e / (9 * Ca), o = e % (9 * Ca), c = o / 9, t = o % 9;
+        float s = Elem<T>::to_f32(b_dyn[o]);
+        for (int k = 0; k < Ca; ++k) s = fmaf(Elem<T>::to_f32(w_dyn[(size_t)o * Ca + k]), gmean(b, k), s);
+        dk_flip[((size_t)b * Ca + c) * 9 + (8 - t)] = s;
+    }
+    for (int e = tid; e < B * Ca; e += nth) {
+        const int b = e / Ca, k = e % Ca;
+        float s = 0.f;
+        for (int o = 0; o < 9 * Ca; ++o) s = fmaf(Elem<T>::to_f32(w_dyn[(size_t)o * Ca + k]), gdk(b, o), s);
+        bias[e] = s * inv_hw;
+    }
+}
+
+}}  // namespace esc::bwd

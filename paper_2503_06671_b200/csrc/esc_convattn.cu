@@ -18,6 +18,7 @@
 #include "stencil_generic.cuh"
 #include "stencil_tma.cuh"
 #include "stencil_dense.cuh"
+#include "backward.cuh"
 
 namespace {
 
@@ -45,6 +46,7 @@ struct Problem {
     int B, C, Ca, H, W, K, dtype, layout;
     const void* w_point = nullptr;   // [Ca][Ca] point-wise filter LK^c of the decomposed form (Eq. 5), or none
     bool dense = false;              // w_large is the dense kernel [Ca][Ca][K][K] of Section 3.2
+    const float* bias = nullptr;     // [B][Ca] constant per (image, channel) added to the attention outputs (backward pass)
     size_t es() const { return elem_size(dtype); }
     size_t elems() const { return (size_t)B * C * H * W; }
 };
@@ -257,10 +259,10 @@ int launch_generic_t(const Problem& p, const void* x, const void* w_large, const
     if (regtile)
         ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT>, static_cast<const T*>(x),
                                     static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk,
-                                    tiles_x, tiles_y, job));
+                                    tiles_x, tiles_y, job, p.bias));
     else
         ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_generic<T, LAYOUT>, static_cast<const T*>(x), static_cast<T*>(out),
-                                    p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk, tiles_x, tiles_y, job));
+                                    p.C, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk, tiles_x, tiles_y, job, p.bias));
     ++g_last_launches;
     return ESC_OK;
 }
@@ -282,8 +284,8 @@ int launch_generic(const Problem& p, const void* x, const void* w_large, const f
 int launch_stencil(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                    unsigned* ctrl, cudaStream_t st, bool dependent) {
     int tile_w = g_tile_policy;
-    int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, p.w_point, dk, out, ctrl,
-                                  st, dependent, &g_last_launches, &g_last_error, &tile_w);
+    int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, p.w_point, dk, p.bias, out,
+                                  ctrl, st, dependent, &g_last_launches, &g_last_error, &tile_w);
     if (rc == ESC_OK) { g_last_path = 2; g_last_tile_w = tile_w; return ESC_OK; }
     if (rc != esc::tma::kNotApplicable) return rc;
     return launch_generic(p, x, w_large, dk, out, st, dependent);
@@ -366,6 +368,49 @@ int forward_impl(const Problem& p, const void* x, const void* w_large, const Est
     return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
 }
 
+// ---- backward pass -------------------------------------------------------------------------
+// Workspace: [ctrl 256 B | per-tile partial tap gradients B*Ca*tiles*kSlot | tap gradients B*Ca*kSlot |
+//             rotated LK Ca*169 elements | rotated dk B*Ca*9 | constants B*Ca], each part 256-byte aligned.
+struct BackwardWs {
+    unsigned* ctrl;
+    float *part, *gtap, *dk_flip, *bias;
+    void* w_flip;
+    size_t bytes;
+};
+BackwardWs carve_backward(void* ws, const Problem& p) {
+    const int tiles = ((p.W + esc::bwd::TX - 1) / esc::bwd::TX) * ((p.H + esc::bwd::TY - 1) / esc::bwd::TY);
+    BackwardWs w;
+    char* base = static_cast<char*>(ws);
+    size_t off = 256;
+    w.ctrl = reinterpret_cast<unsigned*>(base);
+    w.part = reinterpret_cast<float*>(base + off); off += round_up((size_t)p.B * p.Ca * tiles * esc::bwd::kSlot * 4, 256);
+    w.gtap = reinterpret_cast<float*>(base + off); off += round_up((size_t)p.B * p.Ca * esc::bwd::kSlot * 4, 256);
+    w.w_flip = base + off;                          off += round_up((size_t)p.Ca * esc::bwd::TAPS * 4, 256);
+    w.dk_flip = reinterpret_cast<float*>(base + off); off += round_up((size_t)p.B * p.Ca * 9 * 4, 256);
+    w.bias = reinterpret_cast<float*>(base + off);  off += round_up((size_t)p.B * p.Ca * 4, 256);
+    w.bytes = off;
+    return w;
+}
+
+template <typename T, int LAYOUT>
+int backward_t(const Problem& p, const void* x, const void* go, const void* w_large, const void* w_dyn,
+               const void* b_dyn, const BackwardWs& w, float* g_lk, float* g_w, float* g_b, cudaStream_t st) {
+    const int tiles_x = (p.W + esc::bwd::TX - 1) / esc::bwd::TX, tiles_y = (p.H + esc::bwd::TY - 1) / esc::bwd::TY;
+    const long long blocks = (long long)p.B * p.Ca * tiles_x * tiles_y;
+    if (blocks > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
+    esc::bwd::tap_grad<T, LAYOUT><<<(unsigned)blocks, esc::bwd::kThreads, 0, st>>>(
+        static_cast<const T*>(x), static_cast<const T*>(go), p.C, p.Ca, p.H, p.W, tiles_x, tiles_y, w.part);
+    ESC_CUDA(cudaGetLastError());
+    esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), 192, 0, st>>>(w.part, tiles_x * tiles_y, w.gtap);
+    ESC_CUDA(cudaGetLastError());
+    esc::bwd::finish<T><<<64, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, static_cast<const T*>(w_large),
+                                            static_cast<const T*>(w_dyn), static_cast<const T*>(b_dyn), g_lk, g_w, g_b,
+                                            static_cast<T*>(w.w_flip), w.dk_flip, w.bias);
+    ESC_CUDA(cudaGetLastError());
+    g_last_launches += 3;
+    return ESC_OK;
+}
+
 // ---- fixed scratch for the entry point that must not allocate ------------------------------
 // Layout: [kStaticMaxImages arrival counters][kStaticMaxPartials partial sums].  The array lives in
 // the library's device image: every GPU that loads the library holds these 64 KiB until exit.
@@ -407,7 +452,7 @@ HostPath g_host[kHostSlots];
 
 extern "C" {
 
-int esc_version(void) { return 110; }
+int esc_version(void) { return 111; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
@@ -687,6 +732,51 @@ int esc_convattn_forward_variant(const void* x, int B, int C, int C_a, int H, in
     if (large_kernel == ESC_LK_DECOMPOSED) p.w_point = w_point;
     p.dense = large_kernel == ESC_LK_DENSE;
     return forward_impl(p, x, w_large, est, out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+size_t esc_convattn_backward_workspace_bytes(int B, int C_a, int H, int W, int K) {
+    if (B <= 0 || C_a <= 0 || H <= 0 || W <= 0 || K != esc::bwd::K) return 0;
+    const Problem p{B, C_a, C_a, H, W, K, ESC_F32, ESC_NCHW};
+    return carve_backward(nullptr, p).bytes;
+}
+
+int esc_convattn_backward(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                          const void* w_large, const void* w_dyn, const void* b_dyn, void* grad_x,
+                          float* grad_w_large, float* grad_w_dyn, float* grad_b_dyn, int dtype, int layout,
+                          void* workspace, size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (K != esc::bwd::K) return ESC_ERR_UNSUPPORTED;
+    if ((long long)B * C_a > 0x7fffffffLL / esc::bwd::kSlot) return ESC_ERR_UNSUPPORTED;
+    if (!x || !grad_out || !grad_x || !w_large || !w_dyn || !b_dyn) return ESC_ERR_NULL;
+    rc = check_tensors(p, grad_out, grad_x);                 // the stencil pass reads grad_out and writes grad_x
+    if (rc != ESC_OK) return rc;
+    if (!aligned(x, 16)) return ESC_ERR_ALIGN;
+    {
+        const uintptr_t xa = reinterpret_cast<uintptr_t>(x), oa = reinterpret_cast<uintptr_t>(grad_x);
+        const size_t bytes = p.elems() * p.es();
+        if (xa < oa + bytes && oa < xa + bytes) return ESC_ERR_ALIAS;
+    }
+    if (!aligned(w_large, p.es()) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
+    if ((grad_w_large && !aligned(grad_w_large, 4)) || (grad_w_dyn && !aligned(grad_w_dyn, 4)) ||
+        (grad_b_dyn && !aligned(grad_b_dyn, 4)))
+        return ESC_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256)) return ESC_ERR_WORKSPACE;
+    const BackwardWs w = carve_backward(workspace, p);
+    if (workspace_bytes_ < w.bytes) return ESC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == ESC_F32)
+        rc = layout == ESC_NCHW ? backward_t<float, esc::kNCHW>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st)
+                                : backward_t<float, esc::kNHWC>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st);
+    else
+        rc = layout == ESC_NCHW ? backward_t<__nv_bfloat16, esc::kNCHW>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st)
+                                : backward_t<__nv_bfloat16, esc::kNHWC>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st);
+    if (rc != ESC_OK) return rc;
+    // grad_x: the forward stencil on grad_out with both kernels rotated by 180 degrees, plus the constants
+    p.bias = w.bias;
+    return launch_stencil(p, grad_out, w.w_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false);
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {

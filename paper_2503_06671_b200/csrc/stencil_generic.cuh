@@ -59,7 +59,7 @@ template <typename T, int LAYOUT>
 __global__ void __launch_bounds__(kGenTX * kGenTY)
 stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W, int K,
                 const T* __restrict__ w_large, const T* __restrict__ w_point, const float* __restrict__ dk,
-                int tiles_x, int tiles_y, const CopyJob job)
+                int tiles_x, int tiles_y, const CopyJob job, const float* __restrict__ bias)
 {
     __shared__ float tile[(kGenTY + kGenMaxK - 1) * (kGenTX + kGenMaxK - 1)];
     __shared__ float wm[kGenMaxK * kGenMaxK];
@@ -95,7 +95,7 @@ stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int
 
     const int oy = ty * kGenTY + threadIdx.y, ox = tx * kGenTX + threadIdx.x;
     if (oy >= H || ox >= W) return;
-    float acc = 0.f;
+    float acc = bias ? bias[(size_t)b * Ca + c] : 0.f;   // the backward pass adds a constant per (image, channel)
     for (int i = 0; i < K; ++i) {
         const float* trow = tile + (threadIdx.y + i) * TWp + threadIdx.x;
         const float* wrow = wm + i * K;
@@ -118,7 +118,7 @@ template <typename T, int LAYOUT>
 __global__ void __launch_bounds__(kRtThreads)
 stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W,
                     const T* __restrict__ w_large, const T* __restrict__ w_point, const float* __restrict__ dk,
-                    int tiles_x, int tiles_y, const CopyJob job)
+                    int tiles_x, int tiles_y, const CopyJob job, const float* __restrict__ bias)
 {
     __shared__ __align__(16) float tile[kRtRows * kRtPitch];
     __shared__ __align__(16) float wm[kRtK * 16];      // merged kernel, rows padded to 16 taps
@@ -155,10 +155,11 @@ stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca,
 
     const int lx = tid % (kRtTX / kRtOX), ly = tid / (kRtTX / kRtOX);
     float acc[kRtOY][kRtOX];
+    const float acc0 = bias ? bias[(size_t)b * Ca + c] : 0.f;   // the backward pass adds a constant per (image, channel)
 #pragma unroll
     for (int a = 0; a < kRtOY; ++a)
 #pragma unroll
-        for (int o = 0; o < kRtOX; ++o) acc[a][o] = 0.f;
+        for (int o = 0; o < kRtOX; ++o) acc[a][o] = acc0;
 #pragma unroll 1
     for (int r = 0; r < kRtOY + kRtK - 1; ++r) {          // input row r of the patch window
         float in[kRtOX + kRtK - 1];

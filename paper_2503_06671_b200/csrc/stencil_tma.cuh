@@ -108,6 +108,7 @@ struct Params {
     const __nv_bfloat16* w_large;     // [Ca][13][13]
     const __nv_bfloat16* w_point;     // [16][16] point-wise filter LK^c of the decomposed form, or nullptr
     const float* dk;                  // [B][Ca][9]
+    const float* bias;                // [B][Ca] constant added to every output of (image, channel), or nullptr
     unsigned* ctrl;                   // status words or nullptr
     int wait_first;                   // 1: nothing may be read before the previous kernel of the stream has finished
 };
@@ -254,7 +255,7 @@ __device__ __forceinline__ void pointwise_mix_tile(uint32_t* tile, const uint32_
     }
 }
 
-template <class G, bool kMix>
+template <class G, bool kMix, bool kBias>
 __global__ void __maxnreg__(kLaunchRegs)
 stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
                       const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_res,
@@ -418,10 +419,19 @@ stencil_tma_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_
         if (alive) alive = mbar_wait(full0 + 8 * buf, (unsigned)((k >> 1) & 1), p.ctrl, 0xA0000000u | (unsigned)buf);
 
         u64 acc[OY][OX];
+        if (kBias) {                                         // the backward pass adds a constant per (image, channel)
+            const u64 z = pack2(__ldg(p.bias + (size_t)un.b * p.Ca + un.g * CG + 2 * pr),
+                                __ldg(p.bias + (size_t)un.b * p.Ca + un.g * CG + 2 * pr + 1));
 #pragma unroll
-        for (int a = 0; a < OY; ++a)
+            for (int a = 0; a < OY; ++a)
 #pragma unroll
-            for (int c = 0; c < OX; ++c) acc[a][c] = 0ull;
+                for (int c = 0; c < OX; ++c) acc[a][c] = z;
+        } else {
+#pragma unroll
+            for (int a = 0; a < OY; ++a)
+#pragma unroll
+                for (int c = 0; c < OX; ++c) acc[a][c] = 0ull;
+        }
 
         unsigned char* tbuf = tilebuf + (size_t)buf * TILE_BYTES;
         if (kMix) {                                          // Eq. 5: the depth-wise stage sees F_att * LK^c
@@ -583,10 +593,10 @@ inline double cost_of(int B, int Ca, int H, int W, int sms, double per_fma) {
     return (double)waves * ((double)G::TW * G::TH * per_fma + 200.0);
 }
 
-template <class G, bool kMix>
+template <class G, bool kMix, bool kBias>
 inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const void* w_point,
-                       const float* dk, void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches,
-                       std::string* err) {
+                       const float* dk, const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent,
+                       int* launches, std::string* err) {
     const int cc = C - Ca;
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -608,6 +618,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
     p.w_point = static_cast<const __nv_bfloat16*>(w_point);
     p.dk = dk;
+    p.bias = bias;
     p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
 
@@ -628,7 +639,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     const int dev = current_device();
     if (dev < 0) return kNotApplicable;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16<G, kMix>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stencil_tma_nhwc_bf16<G, kMix, kBias>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
         attr_set[dev] = true;
     }
@@ -645,7 +656,7 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16<G, kMix>, m_att, m_cin, m_cout, m_res, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_tma_nhwc_bf16<G, kMix, kBias>, m_att, m_cin, m_cout, m_res, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_tma_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -660,8 +671,8 @@ inline int launch_geom(int B, int C, int Ca, int H, int W, const void* x, const 
 // generic kernel has to run instead, or an ESC_ERR_* code.  *tile_w: in, the tile width asked
 // for (0 = choose by cost); out, the one used.
 inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
-                      const void* w_large, const void* w_point, const float* dk, void* out, unsigned* ctrl,
-                      cudaStream_t st, bool dependent, int* launches, std::string* err, int* tile_w) {
+                      const void* w_large, const void* w_point, const float* dk, const float* bias, void* out,
+                      unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err, int* tile_w) {
     if (K != K13 || dtype != 1 /*bf16*/ || layout != kNHWC) return kNotApplicable;
     if (Ca % CG != 0 || C % 8 != 0) return kNotApplicable;
     if (C - Ca > 256) return kNotApplicable;
@@ -671,14 +682,20 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
     if (sms <= 0) return kNotApplicable;
     const bool use64 = *tile_w == Geom64::TW ||
                        (*tile_w != Geom40::TW && cost_of<Geom64>(B, Ca, H, W, sms, 1.15) < cost_of<Geom40>(B, Ca, H, W, sms, 1.0));
+    // the combinations in use: plain, with the point-wise mix, with the backward pass's constants
+#define ESC_TMA_ARGS B, C, Ca, H, W, x, w_large, w_point, dk, bias, out, ctrl, st, dependent, launches, err
+    if (w_point && bias) return kNotApplicable;
     if (use64) {
         *tile_w = Geom64::TW;
-        return w_point ? launch_geom<Geom64, true>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err)
-                       : launch_geom<Geom64, false>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err);
+        return w_point ? launch_geom<Geom64, true, false>(ESC_TMA_ARGS)
+             : bias    ? launch_geom<Geom64, false, true>(ESC_TMA_ARGS)
+                       : launch_geom<Geom64, false, false>(ESC_TMA_ARGS);
     }
     *tile_w = Geom40::TW;
-    return w_point ? launch_geom<Geom40, true>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err)
-                   : launch_geom<Geom40, false>(B, C, Ca, H, W, x, w_large, w_point, dk, out, ctrl, st, dependent, launches, err);
+    return w_point ? launch_geom<Geom40, true, false>(ESC_TMA_ARGS)
+         : bias    ? launch_geom<Geom40, false, true>(ESC_TMA_ARGS)
+                   : launch_geom<Geom40, false, false>(ESC_TMA_ARGS);
+#undef ESC_TMA_ARGS
 }
 
 }}  // namespace esc::tma

@@ -106,6 +106,12 @@ def test_host_side_rejections_launch_nothing(L):
     assert L.esc_convattn_forward_variant(X, 1, 64, 16, 32, 32, 13, 1, Wl, None, None, None, Wd, Bd, 0, O, 1, 1, WS, big, None) == 1
     assert L.esc_convattn_forward_variant(X, 1, 64, 16, 32, 32, 13, 0, Wl, None, None, None, Wd, Bd, 8, O, 1, 1, WS, big, None) == 1
     assert L.esc_convattn_forward_variant(X, 1, 64, 16, 32, 32, 13, 0, Wl, None, None, None, Wd, Bd, -1, O, 1, 1, WS, big, None) == 2
+    GO, GX = 0x50000000, 0x60000000
+    assert L.esc_convattn_backward(X, GO, 1, 64, 16, 32, 32, 13, Wl, Wd, Bd, None, None, None, None, 1, 1, WS, big, None) == 1
+    assert L.esc_convattn_backward(X, GO, 1, 64, 16, 32, 32, 9, Wl, Wd, Bd, GX, None, None, None, 1, 1, WS, big, None) == 3
+    assert L.esc_convattn_backward(X, GO, 1, 64, 16, 32, 32, 13, Wl, Wd, Bd, X, None, None, None, 1, 1, WS, big, None) == 5
+    assert L.esc_convattn_backward(X, GO, 1, 64, 16, 32, 32, 13, Wl, Wd, Bd, GO + 32, None, None, None, 1, 1, WS, big, None) == 5
+    assert L.esc_convattn_backward(X, GO, 1, 64, 16, 32, 32, 13, Wl, Wd, Bd, GX, None, None, None, 1, 1, WS, 64, None) == 6
     assert L.esc_convattn_forward_host_submit(2, X, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 3
     assert L.esc_convattn_forward_host_submit(0, None, 1, 64, 16, 8, 8, 13, Wl, Wd, Bd, O, 0, 0) == 1
     assert L.esc_convattn_forward_host_wait(-1) == 3

@@ -1,0 +1,91 @@
+"""GPU parity for the backward pass (gradients of the ConvAttn forward of ESC Section 3.3, Eq. 4, one-layer
+estimator, depth-wise LK) through the C ABI against the CPU oracle, which is pinned by exact finite differences."""
+import numpy as np
+import pytest
+
+from paper_2503_06671_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+LAYOUTS = [synth.NCHW, synth.NHWC]
+DTYPES = [synth.F32, synth.BF16]
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import paper_2503_06671_b200 as p
+
+    p.lib()
+    return p
+
+
+SHAPES = [
+    # B, C, C_a, H, W
+    (2, 64, 16, 64, 64),      # one tile per image
+    (1, 64, 16, 70, 131),     # several tiles, ragged in both directions
+    (3, 24, 8, 9, 11),        # smaller than the kernel, C_a = 8
+    (1, 48, 32, 37, 90),      # two channel groups
+    (2, 16, 16, 20, 65),      # nothing but attention channels
+]
+
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_backward(pkg, oracle, shape, dtype, layout):
+    import torch
+
+    B, C, C_a, H, W = shape
+    K = 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, dtype, seed=sum(shape), per_image_scale=True, channel_means=True)
+    go = synth.round_to(np.random.default_rng(sum(shape) + 1).standard_normal(size=d["x"].shape).astype(np.float32), dtype)
+    x = util.to_device(d["x"], dtype, layout)
+    go_d = util.to_device(go, dtype, layout)
+    wl, wd, bd = util.weights_to_device(d, dtype)
+    gx = torch.full_like(x, 7.0)
+    g_lk = torch.full((C_a, K, K), float("nan"), device="cuda")
+    g_w = torch.full((9 * C_a, C_a), float("nan"), device="cuda")
+    g_b = torch.full((9 * C_a,), float("nan"), device="cuda")
+    ws = pkg.new_backward_workspace(B, C_a, H, W, K)
+    for _ in range(2):                                   # twice: nothing in the workspace may need re-zeroing
+        pkg.esc_convattn_backward(x, go_d, C_a, K, wl, wd, bd, gx, g_lk, g_w, g_b, util.layout_code(layout), ws)
+    torch.cuda.synchronize()
+    assert pkg.esc_convattn_device_status(ws) == 0
+
+    rx, rlk, rw, rb = oracle.backward(d["x"], go, C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    # scales of the sums: the same gradients of |x|, |go| (every term replaced by its magnitude)
+    _, alk, aw, ab = oracle.backward(np.abs(d["x"]), np.abs(go), C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    for name, got, ref, scale in (("w_large", g_lk, rlk, alk), ("w_dyn", g_w, rw, aw), ("b_dyn", g_b, rb, ab)):
+        err = np.abs(got.cpu().numpy().astype(np.float64) - ref)
+        assert (err <= 1e-5 * scale + 1e-30).all(), f"grad {name}: worst {(err / np.maximum(scale, 1e-30)).max():.3e} of its scale"
+
+    got = util.to_host_nchw(gx, layout)
+    assert np.array_equal(got[:, C_a:], go[:, C_a:].astype(np.float64)), "identity channels: grad_x must be grad_out"
+    # magnitude of the stencil part: |go| through |rotated kernels| = the pinned stencil on magnitudes
+    dk = oracle.dynkernel(oracle.gap(d["x"], C_a), d["w_dyn"], d["b_dyn"])
+    mag = oracle.stencil(np.abs(go), C_a, np.abs(d["w_large"][:, ::-1, ::-1]).copy(), np.abs(dk[:, :, ::-1, ::-1]).copy())[:, :C_a]
+    err = np.abs(got[:, :C_a] - rx[:, :C_a])
+    # the constant from the GAP path comes from the fp32 tap gradients: allow their 1e-5 relative noise on its scale
+    gg_scale = np.abs(np.einsum("ok,bo->bk", np.abs(d["w_dyn"].astype(np.float64)), np.abs(ab.reshape(1, -1)).repeat(B, 0))) / (H * W)
+    bar = 1e-5 * mag + 1e-5 * gg_scale[:, :, None, None] + 1e-30
+    if dtype == synth.BF16:
+        bar = bar + 2.0 ** -8 * np.abs(rx[:, :C_a]) * 1.001
+    assert (err <= bar).all(), f"grad x: {int((err > bar).sum())} values beyond the bound"
+
+
+def test_backward_rejections(pkg):
+    import torch
+
+    x = torch.zeros(1, 8, 8, 16, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(16, 9, 9, dtype=torch.bfloat16, device="cuda")
+    assert pkg.esc_convattn_backward_workspace_bytes(1, 16, 8, 8, 9) == 0          # K = 13 only
+    L = pkg.lib()
+    ws = pkg.new_backward_workspace(1, 16, 8, 8, 13)
+    rc = L.esc_convattn_backward(x.data_ptr(), x.data_ptr(), 1, 16, 16, 8, 8, 9, w.data_ptr(), w.data_ptr(), w.data_ptr(),
+                                 x.data_ptr(), None, None, None, 1, 1, ws.data_ptr(), ws.numel(), None)
+    assert rc == 3
