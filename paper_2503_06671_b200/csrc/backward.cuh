@@ -123,6 +123,121 @@ tap_grad(const T* __restrict__ x, const T* __restrict__ go, int C, int Ca, int H
     }
 }
 
+// ---- kernel 1, NHWC form: eight channels per block -----------------------------------------------------------
+// In NHWC a block per channel would fetch every pixel's line once per channel with 2-byte loads.  Here a block
+// takes eight neighbouring channels (16 bytes of a bf16 pixel, 32 of an fp32 one) of a 32x32 tile: pixels are
+// read with 16-byte loads and spread over eight planar fp32 tiles in shared memory; warp w then works on channel
+// w exactly as above (4x8 patch of go per lane), so the block sum of the 13 values is one shuffle butterfly.
+namespace n8 {
+constexpr int TX = 32, TY = 32, CH = 8;
+constexpr int XP = TX + K - 1, XR = TY + K - 1;          // 44 x 44 staged x per channel (44 is a multiple of 4)
+constexpr int kThreads = CH * 32;                        // 256
+constexpr size_t kSmemBytes = (size_t)CH * (XR * XP + TY * TX) * sizeof(float);   // 94,720
+static_assert(XP % 4 == 0 && (TX / OX) * (TY / OY) == 32, "one warp covers a channel's tile");
+}  // namespace n8
+
+template <typename T>
+__global__ void __launch_bounds__(n8::kThreads)
+tap_grad_nhwc8(const T* __restrict__ x, const T* __restrict__ go, int C, int Ca, int H, int W, int tiles_x, int tiles_y,
+               float* __restrict__ part)      // [B][Ca][tiles][kSlot]
+{
+    constexpr int TX = n8::TX, TY = n8::TY, CH = n8::CH, XP = n8::XP, XR = n8::XR, kThreads = n8::kThreads;
+    constexpr int V = Elem<T>::kVec;                      // elements per 16-byte load: 8 (bf16) or 4 (fp32)
+    extern __shared__ __align__(16) float sm[];
+    float* xt = sm;                                       // [CH][XR*XP]
+    float* gt = sm + CH * XR * XP;                        // [CH][TY*TX]
+
+    long long bid = blockIdx.x;
+    const int tiles = tiles_x * tiles_y, octets = Ca / CH;
+    const int tile = (int)(bid % tiles); bid /= tiles;
+    const int oct = (int)(bid % octets);
+    const int b = (int)(bid / octets);
+    const int tx = tile % tiles_x, ty = tile / tiles_x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int y0 = ty * TY, x0 = tx * TX;
+    const T* xb = x + (size_t)b * H * W * C + oct * CH;
+    const T* gb = go + (size_t)b * H * W * C + oct * CH;
+
+    for (int t = tid; t < XR * XP * (CH / V); t += kThreads) {
+        const int h = t % (CH / V), pix = t / (CH / V);   // which 16-byte piece of the pixel's eight channels
+        const int r = pix / XP, q = pix % XP;
+        const int y = y0 - P + r, xx = x0 - P + q;
+        float f[V];
+        if (y >= 0 && y < H && xx >= 0 && xx < W)
+            unpack16<T>(__ldg(reinterpret_cast<const uint4*>(xb + ((size_t)y * W + xx) * C + h * V)), f);
+        else {
+#pragma unroll
+            for (int v = 0; v < V; ++v) f[v] = 0.f;
+        }
+#pragma unroll
+        for (int v = 0; v < V; ++v) xt[(h * V + v) * (XR * XP) + pix] = f[v];
+    }
+    for (int t = tid; t < TY * TX * (CH / V); t += kThreads) {
+        const int h = t % (CH / V), pix = t / (CH / V);
+        const int r = pix / TX, q = pix % TX;
+        const int y = y0 + r, xx = x0 + q;
+        float f[V];
+        if (y < H && xx < W)
+            unpack16<T>(__ldg(reinterpret_cast<const uint4*>(gb + ((size_t)y * W + xx) * C + h * V)), f);
+        else {
+#pragma unroll
+            for (int v = 0; v < V; ++v) f[v] = 0.f;
+        }
+#pragma unroll
+        for (int v = 0; v < V; ++v) gt[(h * V + v) * (TY * TX) + pix] = f[v];
+    }
+    __syncthreads();
+
+    const float* xc = xt + warp * (XR * XP);              // this warp's channel
+    const float* gc = gt + warp * (TY * TX);
+    const int lx = lane % (TX / OX), ly = lane / (TX / OX);
+    float g[OY][OX];
+    float sx = 0.f;
+#pragma unroll
+    for (int a = 0; a < OY; ++a) {
+        const float4* gr = reinterpret_cast<const float4*>(gc + (ly * OY + a) * TX + lx * OX);
+        const float4 q0 = gr[0], q1 = gr[1];
+        g[a][0] = q0.x; g[a][1] = q0.y; g[a][2] = q0.z; g[a][3] = q0.w;
+        g[a][4] = q1.x; g[a][5] = q1.y; g[a][6] = q1.z; g[a][7] = q1.w;
+        const float4* xr = reinterpret_cast<const float4*>(xc + (ly * OY + a + P) * XP + lx * OX + P - 2);
+        const float4 u0 = xr[0], u1 = xr[1], u2 = xr[2];  // the patch's own pixels are floats 2..9 of these
+        sx += (u0.z + u0.w) + (u1.x + u1.y + u1.z + u1.w) + (u2.x + u2.y);
+    }
+    float* slot = part + (((size_t)b * Ca + oct * CH + warp) * tiles + tile) * kSlot;
+
+#pragma unroll 1
+    for (int i = 0; i < K; ++i) {
+        float s[K];
+#pragma unroll
+        for (int j = 0; j < K; ++j) s[j] = 0.f;
+#pragma unroll
+        for (int a = 0; a < OY; ++a) {
+            float in[OX + K - 1];
+            const float4* xr = reinterpret_cast<const float4*>(xc + (ly * OY + a + i) * XP + lx * OX);
+#pragma unroll
+            for (int v = 0; v < (OX + K - 1) / 4; ++v) {
+                const float4 q = xr[v];
+                in[4 * v] = q.x; in[4 * v + 1] = q.y; in[4 * v + 2] = q.z; in[4 * v + 3] = q.w;
+            }
+#pragma unroll
+            for (int j = 0; j < K; ++j)
+#pragma unroll
+                for (int o = 0; o < OX; ++o) s[j] = fmaf(g[a][o], in[o + j], s[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) s[j] += __shfl_xor_sync(0xffffffffu, s[j], o);
+        // after the butterfly every lane holds all 13 sums: lane j writes the j-th
+#pragma unroll
+        for (int j = 0; j < K; ++j)
+            if (lane == j) slot[i * K + j] = s[j];
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, o);
+    if (lane == 0) slot[TAPS] = sx;
+}
+
 // ---- kernel 2a: add the tiles of one (image, channel) in order ---------------------------------------------
 __global__ void __launch_bounds__(192)
 sum_tiles(const float* __restrict__ part, int tiles, float* __restrict__ gtap)   // gtap [B*Ca][kSlot]

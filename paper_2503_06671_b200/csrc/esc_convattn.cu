@@ -378,7 +378,8 @@ struct BackwardWs {
     size_t bytes;
 };
 BackwardWs carve_backward(void* ws, const Problem& p) {
-    const int tiles = ((p.W + esc::bwd::TX - 1) / esc::bwd::TX) * ((p.H + esc::bwd::TY - 1) / esc::bwd::TY);
+    // sized for the finer of the two tilings the tap-gradient kernels use (32x32)
+    const int tiles = ((p.W + esc::bwd::n8::TX - 1) / esc::bwd::n8::TX) * ((p.H + esc::bwd::n8::TY - 1) / esc::bwd::n8::TY);
     BackwardWs w;
     char* base = static_cast<char*>(ws);
     size_t off = 256;
@@ -395,11 +396,27 @@ BackwardWs carve_backward(void* ws, const Problem& p) {
 template <typename T, int LAYOUT>
 int backward_t(const Problem& p, const void* x, const void* go, const void* w_large, const void* w_dyn,
                const void* b_dyn, const BackwardWs& w, float* g_lk, float* g_w, float* g_b, cudaStream_t st) {
-    const int tiles_x = (p.W + esc::bwd::TX - 1) / esc::bwd::TX, tiles_y = (p.H + esc::bwd::TY - 1) / esc::bwd::TY;
-    const long long blocks = (long long)p.B * p.Ca * tiles_x * tiles_y;
+    // NHWC with whole octets of channels: eight channels per block, 16-byte loads; else a block per channel
+    const bool oct = LAYOUT == esc::kNHWC && p.Ca % 8 == 0 && p.C % 8 == 0;
+    const int TXs = oct ? esc::bwd::n8::TX : esc::bwd::TX, TYs = oct ? esc::bwd::n8::TY : esc::bwd::TY;
+    const int tiles_x = (p.W + TXs - 1) / TXs, tiles_y = (p.H + TYs - 1) / TYs;
+    const long long blocks = (long long)p.B * (oct ? p.Ca / 8 : p.Ca) * tiles_x * tiles_y;
     if (blocks > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
-    esc::bwd::tap_grad<T, LAYOUT><<<(unsigned)blocks, esc::bwd::kThreads, 0, st>>>(
-        static_cast<const T*>(x), static_cast<const T*>(go), p.C, p.Ca, p.H, p.W, tiles_x, tiles_y, w.part);
+    if (oct) {
+        static bool attr_set[esc::tma::kMaxDevices] = {};
+        const int dev = esc::tma::current_device();
+        if (dev < 0) return ESC_ERR_UNSUPPORTED;
+        if (!attr_set[dev]) {
+            ESC_CUDA(cudaFuncSetAttribute(esc::bwd::tap_grad_nhwc8<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)esc::bwd::n8::kSmemBytes));
+            attr_set[dev] = true;
+        }
+        esc::bwd::tap_grad_nhwc8<T><<<(unsigned)blocks, esc::bwd::n8::kThreads, esc::bwd::n8::kSmemBytes, st>>>(
+            static_cast<const T*>(x), static_cast<const T*>(go), p.C, p.Ca, p.H, p.W, tiles_x, tiles_y, w.part);
+    } else {
+        esc::bwd::tap_grad<T, LAYOUT><<<(unsigned)blocks, esc::bwd::kThreads, 0, st>>>(
+            static_cast<const T*>(x), static_cast<const T*>(go), p.C, p.Ca, p.H, p.W, tiles_x, tiles_y, w.part);
+    }
     ESC_CUDA(cudaGetLastError());
     esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), 192, 0, st>>>(w.part, tiles_x * tiles_y, w.gtap);
     ESC_CUDA(cudaGetLastError());
