@@ -127,13 +127,13 @@ tap_grad(const T* __restrict__ x, const T* __restrict__ go, int C, int Ca, int H
 // In NHWC a block per channel would fetch every pixel's line once per channel with 2-byte loads.  Here a block
 // takes eight neighbouring channels (16 bytes of a bf16 pixel, 32 of an fp32 one) of a 32x32 tile: pixels are
 // read with 16-byte loads and spread over eight planar fp32 tiles in shared memory; warp w then works on channel
-// w exactly as above (4x8 patch of go per lane), so the block sum of the 13 values is one shuffle butterfly.
+// w on its own (8x4 patch of go per lane), so the block sum of the 13 values is one shuffle butterfly.
 namespace n8 {
 constexpr int TX = 32, TY = 32, CH = 8;
 constexpr int XP = TX + K - 1, XR = TY + K - 1;          // 44 x 44 staged x per channel (44 is a multiple of 4)
 constexpr int kThreads = CH * 32;                        // 256
 constexpr size_t kSmemBytes = (size_t)CH * (XR * XP + TY * TX) * sizeof(float);   // 94,720
-static_assert(XP % 4 == 0 && (TX / OX) * (TY / OY) == 32, "one warp covers a channel's tile");
+static_assert(XP % 4 == 0, "16-byte reads of staged rows");
 }  // namespace n8
 
 template <typename T>
@@ -190,18 +190,20 @@ tap_grad_nhwc8(const T* __restrict__ x, const T* __restrict__ go, int C, int Ca,
 
     const float* xc = xt + warp * (XR * XP);              // this warp's channel
     const float* gc = gt + warp * (TY * TX);
-    const int lx = lane % (TX / OX), ly = lane / (TX / OX);
-    float g[OY][OX];
+    // A lane's patch is 8 rows x 4 columns here: the eight lanes that share a 16-byte read phase then sit
+    // side by side (16 bytes apart, 128 contiguous bytes) and the reads are free of bank conflicts.
+    constexpr int PY = 8, PX = 4;
+    static_assert((TX / PX) * (TY / PY) == 32, "one warp covers a channel's tile");
+    const int lx = lane % (TX / PX), ly = lane / (TX / PX);
+    float g[PY][PX];
     float sx = 0.f;
 #pragma unroll
-    for (int a = 0; a < OY; ++a) {
-        const float4* gr = reinterpret_cast<const float4*>(gc + (ly * OY + a) * TX + lx * OX);
-        const float4 q0 = gr[0], q1 = gr[1];
+    for (int a = 0; a < PY; ++a) {
+        const float4 q0 = *reinterpret_cast<const float4*>(gc + (ly * PY + a) * TX + lx * PX);
         g[a][0] = q0.x; g[a][1] = q0.y; g[a][2] = q0.z; g[a][3] = q0.w;
-        g[a][4] = q1.x; g[a][5] = q1.y; g[a][6] = q1.z; g[a][7] = q1.w;
-        const float4* xr = reinterpret_cast<const float4*>(xc + (ly * OY + a + P) * XP + lx * OX + P - 2);
-        const float4 u0 = xr[0], u1 = xr[1], u2 = xr[2];  // the patch's own pixels are floats 2..9 of these
-        sx += (u0.z + u0.w) + (u1.x + u1.y + u1.z + u1.w) + (u2.x + u2.y);
+        const float4* xr = reinterpret_cast<const float4*>(xc + (ly * PY + a + P) * XP + lx * PX + P - 2);
+        const float4 u0 = xr[0], u1 = xr[1];              // the patch's own pixels are floats 2..5 of these
+        sx += (u0.z + u0.w) + (u1.x + u1.y);
     }
     float* slot = part + (((size_t)b * Ca + oct * CH + warp) * tiles + tile) * kSlot;
 
@@ -211,18 +213,18 @@ tap_grad_nhwc8(const T* __restrict__ x, const T* __restrict__ go, int C, int Ca,
 #pragma unroll
         for (int j = 0; j < K; ++j) s[j] = 0.f;
 #pragma unroll
-        for (int a = 0; a < OY; ++a) {
-            float in[OX + K - 1];
-            const float4* xr = reinterpret_cast<const float4*>(xc + (ly * OY + a + i) * XP + lx * OX);
+        for (int a = 0; a < PY; ++a) {
+            float in[PX + K - 1];                         // 16 floats: four 16-byte reads
+            const float4* xr = reinterpret_cast<const float4*>(xc + (ly * PY + a + i) * XP + lx * PX);
 #pragma unroll
-            for (int v = 0; v < (OX + K - 1) / 4; ++v) {
+            for (int v = 0; v < (PX + K - 1) / 4; ++v) {
                 const float4 q = xr[v];
                 in[4 * v] = q.x; in[4 * v + 1] = q.y; in[4 * v + 2] = q.z; in[4 * v + 3] = q.w;
             }
 #pragma unroll
             for (int j = 0; j < K; ++j)
 #pragma unroll
-                for (int o = 0; o < OX; ++o) s[j] = fmaf(g[a][o], in[o + j], s[j]);
+                for (int o = 0; o < PX; ++o) s[j] = fmaf(g[a][o], in[o + j], s[j]);
         }
 #pragma unroll
         for (int j = 0; j < K; ++j)
