@@ -43,7 +43,7 @@ extern "C" {
 typedef enum {
     ESC_OK = 0,
     ESC_ERR_NULL = 1,        /* a required pointer is NULL                                      */
-    ESC_ERR_SHAPE = 2,       /* B,C,H,W <= 0, C_a <= 0, C_a > C, K even or K < 1, size overflow */
+    ESC_ERR_SHAPE = 2,       /* B,C,H,W <= 0, C_a <= 0, C_a > C, K even or K < 3, size overflow */
     ESC_ERR_UNSUPPORTED = 3, /* K > ESC_MAX_K, unknown dtype / layout                           */
     ESC_ERR_ALIGN = 4,       /* a tensor pointer is not aligned to its element size / 16 bytes  */
     ESC_ERR_ALIAS = 5,       /* out overlaps x (a stencil cannot run in place)                  */
@@ -275,7 +275,7 @@ int esc_convattn_device_status(void* workspace, void* stream);
 int esc_convattn_last_path(void);
 
 /* Width in pixels of the output tile the TMA-staged kernel used in that call (40: 40x40 tiles,
- * 64: 64x20 tiles, chosen by the tile count's balance over the SMs), 0 when the generic kernel
+ * 64: 64x16 tiles, chosen by the tile count's balance over the SMs), 0 when the generic kernel
  * ran.  For tests and benchmarks. */
 int esc_convattn_last_tile_width(void);
 

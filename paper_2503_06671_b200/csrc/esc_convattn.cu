@@ -53,7 +53,7 @@ struct Problem {
 
 int check_shape(const Problem& p) {
     if (p.B <= 0 || p.C <= 0 || p.H <= 0 || p.W <= 0 || p.Ca <= 0 || p.Ca > p.C) return ESC_ERR_SHAPE;
-    if (p.K < 1 || (p.K & 1) == 0) return ESC_ERR_SHAPE;
+    if (p.K < 3 || (p.K & 1) == 0) return ESC_ERR_SHAPE;   // the 3x3 dynamic kernel is folded into the K x K one
     if (p.K > ESC_MAX_K) return ESC_ERR_UNSUPPORTED;
     if (p.dtype != ESC_F32 && p.dtype != ESC_BF16) return ESC_ERR_UNSUPPORTED;
     if (p.layout != ESC_NCHW && p.layout != ESC_NHWC) return ESC_ERR_UNSUPPORTED;
@@ -87,12 +87,20 @@ struct Workspace {
 
 bool is_large_map(int B, long long HW) { return (long double)B * HW >= 1.5e6L; }
 
+// SM count of the current device; a B200's 148 where no device can be asked (size queries on a
+// machine without a GPU).
+int sms_or_nominal() {
+    const int v = esc::tma::sm_count();
+    return v > 0 ? v : 148;
+}
+
 int slabs_for(int B, long long HW) {
     // At most one work item per SM over the whole batch, so that every block walks one item and no
     // image waits for a second round (three per SM for maps so large that the stencil kernel takes
     // many waves and the GAP kernel runs ahead of it rather than beside it), at least 512 pixels
     // per slab.
-    const long long target = is_large_map(B, HW) ? 3 * 148 : 148;
+    const long long sms = sms_or_nominal();
+    const long long target = is_large_map(B, HW) ? 3 * sms : sms;
     long long s = target / B;
     const long long cap = (HW + 511) / 512;
     if (s > cap) s = cap;
@@ -139,8 +147,7 @@ template <typename T, int LAYOUT>
 int launch_gap_t(const Problem& p, const void* x, const Estimator& est,
                  const Workspace& w, float* dk_out, cudaStream_t st) {
     const int S = slabs_for(p.B, (long long)p.H * p.W);
-    int sms = esc::tma::sm_count();
-    if (sms <= 0) sms = 148;
+    const int sms = sms_or_nominal();
     const long long items = (long long)p.B * S;
     // Small maps: at most one block per SM, so that the stencil kernel fits beside this one.
     // Large maps: the stencil kernel would wait for dk during its first of many units anyway, so
@@ -197,7 +204,7 @@ int launch_copy_u(const void* x, void* out, long long rows, long long row_b, lon
     const long long total = rows * (row_b / u);
     if (total == 0) return ESC_OK;
     long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > 16LL * sms_or_nominal()) blocks = 16LL * sms_or_nominal();
     esc::copy_through<U><<<(unsigned)blocks, 256, 0, st>>>(static_cast<const U*>(x), static_cast<U*>(out), rows,
                                                           row_b / u, stride_b / u, off_b / u);
     ESC_CUDA(cudaGetLastError());
@@ -231,7 +238,7 @@ esc::CopyJob make_copy_job(const Problem& p, const void* x, void* out, long long
     j.unit_bytes = u;
     const long long total = rows * j.row_units;
     long long blocks = (total + (long long)threads * 4 - 1) / ((long long)threads * 4);   // about four units per thread
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > 8LL * sms_or_nominal()) blocks = 8LL * sms_or_nominal();
     if (blocks < 1) blocks = 1;
     j.first_block = (unsigned)first_block;
     j.blocks = (unsigned)blocks;
@@ -317,7 +324,7 @@ int launch_dense_generic_t(const Problem& p, const void* x, const void* w_dense,
                            cudaStream_t st, bool dependent) {
     const long long total = (long long)p.B * p.Ca * p.H * p.W;
     long long blocks = (total + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > 8LL * sms_or_nominal()) blocks = 8LL * sms_or_nominal();
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)blocks);
     cfg.blockDim = dim3(256);
@@ -339,7 +346,7 @@ int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, c
                          unsigned* ctrl, cudaStream_t st, bool dependent) {
     g_last_tile_w = 0;
     esc::CopyJob job = make_copy_job(p, x, out, 0, esc::tma::dense::kThreads);
-    if (job.blocks > 148) job.blocks = 148;                // every block of that launch takes a whole SM
+    if (job.blocks > (unsigned)sms_or_nominal()) job.blocks = (unsigned)sms_or_nominal();   // every block of that launch takes a whole SM
     int rc = esc::tma::try_launch_dense(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_dense, dk, out, ctrl,
                                         st, dependent, job, &g_last_launches, &g_last_error);
     if (rc == ESC_OK) {
@@ -498,7 +505,7 @@ const char* esc_status_string(int s) {
 }
 
 size_t esc_convattn_workspace_bytes(int B, int C_a, int H, int W, int K) {
-    if (B <= 0 || C_a <= 0 || H <= 0 || W <= 0 || K < 1 || (K & 1) == 0 || K > ESC_MAX_K) return 0;
+    if (B <= 0 || C_a <= 0 || H <= 0 || W <= 0 || K < 3 || (K & 1) == 0 || K > ESC_MAX_K) return 0;
     return workspace_bytes(B, C_a, (long long)H * W);
 }
 
@@ -545,7 +552,7 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W, c
                            const void* b_dyn, float* dk_out, int dtype, int layout, void* workspace,
                            size_t workspace_bytes_, void* stream) {
     g_last_launches = 0;
-    const Problem p{B, C, C_a, H, W, 1, dtype, layout};
+    const Problem p{B, C, C_a, H, W, 3, dtype, layout};   // stage 1 has no large kernel: any valid K
     int rc = check_shape(p);
     if (rc != ESC_OK) return rc;
     if (!x || !w_dyn || !b_dyn || !dk_out) return ESC_ERR_NULL;
@@ -581,7 +588,7 @@ int esc_convattn_dynkernel_mlp(const void* x, int B, int C, int C_a, int H, int 
                                const void* b_down, const void* w_up, const void* b_up, int hidden, float* dk_out,
                                int dtype, int layout, void* workspace, size_t workspace_bytes_, void* stream) {
     g_last_launches = 0;
-    const Problem p{B, C, C_a, H, W, 1, dtype, layout};
+    const Problem p{B, C, C_a, H, W, 3, dtype, layout};   // stage 1 has no large kernel: any valid K
     int rc = check_shape(p);
     if (rc != ESC_OK) return rc;
     if (hidden < 1) return ESC_ERR_SHAPE;
@@ -598,7 +605,7 @@ int esc_convattn_dynkernel_mlp(const void* x, int B, int C, int C_a, int H, int 
 int esc_convattn_dynkernel_static(const void* x, int B, int C, int C_a, int H, int W, const void* w_dyn,
                                   const void* b_dyn, float* dk_out, int dtype, int layout, void* stream) {
     g_last_launches = 0;
-    const Problem p{B, C, C_a, H, W, 1, dtype, layout};
+    const Problem p{B, C, C_a, H, W, 3, dtype, layout};   // stage 1 has no large kernel: any valid K
     int rc = check_shape(p);
     if (rc != ESC_OK) return rc;
     if (!x || !w_dyn || !b_dyn || !dk_out) return ESC_ERR_NULL;

@@ -48,7 +48,7 @@ def test_workspace_bytes(L):
     n = L.esc_convattn_workspace_bytes(1, 16, 360, 640, 13)
     assert n > 0 and n % 256 == 0
     assert L.esc_convattn_workspace_bytes(64, 16, 64, 64, 13) >= 64 * 16 * 9 * 4
-    for bad in [(0, 16, 8, 8, 13), (1, 0, 8, 8, 13), (1, 16, 0, 8, 13), (1, 16, 8, 8, 12), (1, 16, 8, 8, 19)]:
+    for bad in [(0, 16, 8, 8, 13), (1, 0, 8, 8, 13), (1, 16, 0, 8, 13), (1, 16, 8, 8, 12), (1, 16, 8, 8, 19), (1, 16, 8, 8, 1), (1, 16, 8, 8, -3)]:
         assert L.esc_convattn_workspace_bytes(*bad) == 0
 
 
@@ -62,6 +62,7 @@ def test_host_side_rejections_launch_nothing(L):
 
     assert fwd(x=None) == 1 and fwd(out=None) == 1 and fwd(wl=None) == 1 and fwd(wd=None) == 1 and fwd(bd=None) == 1
     assert fwd(B=0) == 2 and fwd(H=-3) == 2 and fwd(Ca=0) == 2 and fwd(Ca=65) == 2 and fwd(K=12) == 2 and fwd(K=0) == 2
+    assert fwd(K=1) == 2 and fwd(K=-1) == 2   # a 1x1 large kernel cannot hold the 3x3 dynamic kernel it is merged with
     assert fwd(K=19) == 3 and fwd(dt=2) == 3 and fwd(lay=5) == 3
     assert fwd(x=X + 8) == 4 and fwd(out=O + 4) == 4 and fwd(wl=Wl + 1) == 4
     assert fwd(out=X) == 5 and fwd(out=X + 64 * 32 * 32 * 2 - 16) == 5 and fwd(x=O + 16, out=O) == 5

@@ -46,7 +46,10 @@ TENSOR_SHAPES = [
     (1, 48, 16, 90, 200),     # several tiles per CTA in both directions
     (1, 64, 16, 1, 300),      # single row
     (1, 64, 16, 150, 1),      # single column
-    (40, 32, 16, 40, 40),     # more tiles than SMs: every CTA walks several, the ring wraps
+    (40, 32, 16, 40, 40),     # 120 tiles: one per CTA, many images
+    (1, 64, 16, 360, 640),    # 230 tiles of 64x16: two per CTA on 148 SMs (the benchmark's launch)
+    (50, 32, 16, 96, 128),    # 600 tiles: four or five per CTA -- both buffers re-used, the barrier phase wraps,
+                              # the image (and its dk) changes inside a CTA's walk
 ]
 
 
