@@ -271,16 +271,31 @@ int esc_convattn_device_status(void* workspace, void* stream);
 
 /* Which stencil implementation the last esc_convattn_forward* / esc_convattn_stencil call on
  * this thread selected: 0 = none yet, 1 = guarded generic kernel, 2 = TMA-staged register-tiled
- * kernel, 3 = tensor-core kernel of the dense large kernel.  For tests and benchmarks. */
+ * FP32 kernel, 3 = tensor-core kernel of the dense large kernel, 4 = tensor-core (banded Toeplitz)
+ * kernel of the depth-wise large kernel.  For tests and benchmarks. */
 int esc_convattn_last_path(void);
 
-/* Width in pixels of the output tile the TMA-staged kernel used in that call (40: 40x40 tiles,
- * 64: 64x16 tiles, chosen by the tile count's balance over the SMs), 0 when the generic kernel
- * ran.  For tests and benchmarks. */
+/* Which arithmetic units evaluate the depth-wise 13x13 stage of Eq. 4 line 3 on NHWC bf16 tensors, for
+ * later calls on this thread.  ESC_ENGINE_AUTO (default): the tensor-core kernel where it applies
+ * (K = 13, C_a a multiple of 16, C a multiple of 8, no point-wise LK^c), else the FP32 kernels.
+ * ESC_ENGINE_FP32: never the tensor-core kernel.  ESC_ENGINE_TENSOR: the tensor-core kernel or, where
+ * it does not apply, the guarded generic kernel.  Both engines multiply exactly (bf16 x bf16 in fp32) and
+ * accumulate in fp32; they differ in the order of the 169 additions, i.e. by fp32 rounding before
+ * the single rounding of the result to bf16.  In the tensor-core kernel one instruction sums 16
+ * horizontally adjacent inputs, three of which may lie outside an output's 13-tap window with weight
+ * zero: a non-finite attention input therefore turns outputs up to 15 pixels beyond its window into
+ * NaN (finite data are unaffected).  Returns ESC_ERR_UNSUPPORTED for any other value. */
+enum { ESC_ENGINE_AUTO = 0, ESC_ENGINE_FP32 = 1, ESC_ENGINE_TENSOR = 2 };
+int esc_convattn_set_stencil_engine(int engine);
+
+/* Width in pixels of the output tile the TMA-staged kernel used in that call (FP32 kernel: 40 = 40x40
+ * tiles, 64 = 64x16 tiles, chosen by the tile count's balance over the SMs; tensor-core kernel: 64 =
+ * 64x16 tiles), 0 when the generic kernel ran.  For tests and benchmarks. */
 int esc_convattn_last_tile_width(void);
 
-/* Overrides the tile choice of the TMA-staged kernel for later calls on this thread: 0 = choose
- * by cost (the default), 40 or 64 = always that width.  The geometries add the 169 taps of an
+/* Overrides the tile choice of the TMA-staged FP32 kernel for later calls on this thread (and, when
+ * not 0, selects that kernel as ESC_ENGINE_FP32 does): 0 = choose by cost (the default), 40 or 64 =
+ * always that width.  The geometries add the 169 taps of an
  * output in different orders, so results differ by fp32 rounding before the final rounding to
  * bf16 (far inside the module's tolerance); with a fixed width, results are bitwise reproducible.
  * Returns ESC_ERR_UNSUPPORTED for any other value.  For tests and tuning. */

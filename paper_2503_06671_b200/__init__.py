@@ -34,6 +34,8 @@ from .binding import (  # noqa: F401
     esc_convattn_last_path,
     esc_convattn_last_tile_width,
     esc_convattn_set_tile_width,
+    esc_convattn_set_stencil_engine,
+    ESC_ENGINE_AUTO, ESC_ENGINE_FP32, ESC_ENGINE_TENSOR,
     esc_convattn_last_launches,
     esc_status_string,
     esc_last_error,

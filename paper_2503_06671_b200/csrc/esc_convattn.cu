@@ -17,6 +17,7 @@
 #include "gap_dynkernel.cuh"
 #include "stencil_generic.cuh"
 #include "stencil_tma.cuh"
+#include "stencil_toeplitz.cuh"
 #include "stencil_dense.cuh"
 #include "backward.cuh"
 
@@ -26,6 +27,7 @@ thread_local std::string g_last_error;
 thread_local int g_last_path = 0;
 thread_local int g_last_tile_w = 0;
 thread_local int g_tile_policy = 0;      // 0 = by cost, else the tile width to use
+thread_local int g_engine_policy = 0;    // ESC_ENGINE_AUTO / _FP32 / _TENSOR for the depth-wise stencil
 thread_local int g_last_launches = 0;
 
 int cuda_fail(cudaError_t e, const char* what) {
@@ -94,13 +96,21 @@ int sms_or_nominal() {
     return v > 0 ? v : 148;
 }
 
-int slabs_for(int B, long long HW) {
-    // At most one work item per SM over the whole batch, so that every block walks one item and no
-    // image waits for a second round (three per SM for maps so large that the stencil kernel takes
-    // many waves and the GAP kernel runs ahead of it rather than beside it), at least 512 pixels
-    // per slab.
+// Grid policy of the GAP kernel.  Narrow: at most one block per SM, which is what fits beside a CTA of the
+// FP32 stencil kernel (58 k registers).  Wide: three blocks per SM -- for maps so large that the stencil
+// kernel takes many waves and the GAP kernel runs ahead of it rather than beside it, and for batches in
+// front of the tensor-core stencil kernel, whose CTAs need every image's dk early (measured on 64 patches
+// of 64x64: 35.5 us per forward against 37.8; a single 640x360 map: 37.4 against 36.2, so single images
+// keep the narrow grid).
+bool wide_gap(int B, long long HW, bool tensor_stencil) {
+    return (tensor_stencil && B > 1) || is_large_map(B, HW);
+}
+
+int slabs_for(int B, long long HW, bool wide) {
+    // At most one work item per block over the whole batch, so that every block walks one item and no
+    // image waits for a second round; at least 512 pixels per slab.
     const long long sms = sms_or_nominal();
-    const long long target = is_large_map(B, HW) ? 3 * sms : sms;
+    const long long target = wide ? 3 * sms : sms;
     long long s = target / B;
     const long long cap = (HW + 511) / 512;
     if (s > cap) s = cap;
@@ -110,7 +120,7 @@ int slabs_for(int B, long long HW) {
 }
 
 size_t workspace_bytes(int B, int Ca, long long HW) {
-    const int S = slabs_for(B, HW);
+    const int S = slabs_for(B, HW, true);                   // room for either grid policy
     size_t off = round_up((size_t)(esc::kCtrlHeaderWords + B) * 4, 256);
     off += round_up((size_t)B * Ca * 9 * 4, 256);
     off += round_up((size_t)B * S * Ca * 4, 256);
@@ -145,14 +155,11 @@ struct Estimator {
 
 template <typename T, int LAYOUT>
 int launch_gap_t(const Problem& p, const void* x, const Estimator& est,
-                 const Workspace& w, float* dk_out, cudaStream_t st) {
-    const int S = slabs_for(p.B, (long long)p.H * p.W);
+                 const Workspace& w, float* dk_out, cudaStream_t st, bool wide) {
+    const int S = slabs_for(p.B, (long long)p.H * p.W, wide);
     const int sms = sms_or_nominal();
     const long long items = (long long)p.B * S;
-    // Small maps: at most one block per SM, so that the stencil kernel fits beside this one.
-    // Large maps: the stencil kernel would wait for dk during its first of many units anyway, so
-    // this kernel takes three blocks per SM and finishes sooner.
-    const long long cap = is_large_map(p.B, (long long)p.H * p.W) ? 3LL * sms : sms;
+    const long long cap = wide ? 3LL * sms : sms;
     const unsigned grid = (unsigned)(items < cap ? items : cap);
     const size_t scratch = (size_t)esc::gap_scratch_floats(LAYOUT, p.C, p.Ca, esc::Elem<T>::kVec);
     const size_t smem = (scratch + p.Ca) * sizeof(float);
@@ -177,13 +184,14 @@ int launch_gap_t(const Problem& p, const void* x, const Estimator& est,
 }
 
 int launch_gap(const Problem& p, const void* x, const Estimator& est,
-               const Workspace& w, float* dk_out, cudaStream_t st) {
+               const Workspace& w, float* dk_out, cudaStream_t st, bool tensor_stencil = false) {
     if ((long long)p.B * esc::kMaxSlabs > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
+    const bool wide = wide_gap(p.B, (long long)p.H * p.W, tensor_stencil);
     if (p.dtype == ESC_F32)
-        return p.layout == ESC_NCHW ? launch_gap_t<float, esc::kNCHW>(p, x, est, w, dk_out, st)
-                                    : launch_gap_t<float, esc::kNHWC>(p, x, est, w, dk_out, st);
-    return p.layout == ESC_NCHW ? launch_gap_t<__nv_bfloat16, esc::kNCHW>(p, x, est, w, dk_out, st)
-                                : launch_gap_t<__nv_bfloat16, esc::kNHWC>(p, x, est, w, dk_out, st);
+        return p.layout == ESC_NCHW ? launch_gap_t<float, esc::kNCHW>(p, x, est, w, dk_out, st, wide)
+                                    : launch_gap_t<float, esc::kNHWC>(p, x, est, w, dk_out, st, wide);
+    return p.layout == ESC_NCHW ? launch_gap_t<__nv_bfloat16, esc::kNCHW>(p, x, est, w, dk_out, st, wide)
+                                : launch_gap_t<__nv_bfloat16, esc::kNHWC>(p, x, est, w, dk_out, st, wide);
 }
 
 int check_estimator(const Problem& p, const Estimator& e) {
@@ -290,12 +298,29 @@ int launch_generic(const Problem& p, const void* x, const void* w_large, const f
 
 int launch_stencil(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                    unsigned* ctrl, cudaStream_t st, bool dependent) {
+    // Depth-wise K = 13 on NHWC bf16: the tensor-core (Toeplitz) kernel unless the caller pinned the FP32
+    // kernel (by engine or by one of its tile widths) or asked for the point-wise mix, which only the
+    // FP32 kernel carries.
+    if (!p.w_point && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0) {
+        int tw = 0;
+        const int rc = esc::tma::toep::try_launch_toeplitz(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, p.bias,
+                                                           out, ctrl, st, dependent, &g_last_launches, &g_last_error, &tw);
+        if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
+        if (rc != esc::tma::kNotApplicable) return rc;
+    }
+    if (g_engine_policy == ESC_ENGINE_TENSOR) return launch_generic(p, x, w_large, dk, out, st, dependent);
     int tile_w = g_tile_policy;
     int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, p.w_point, dk, p.bias, out,
                                   ctrl, st, dependent, &g_last_launches, &g_last_error, &tile_w);
     if (rc == ESC_OK) { g_last_path = 2; g_last_tile_w = tile_w; return ESC_OK; }
     if (rc != esc::tma::kNotApplicable) return rc;
     return launch_generic(p, x, w_large, dk, out, st, dependent);
+}
+
+// Whether launch_stencil will take the tensor-core kernel for this problem (same conditions).
+bool tensor_stencil_follows(const Problem& p) {
+    return !p.dense && !p.w_point && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
+           esc::tma::toep::applies(p.C, p.Ca, p.K, p.dtype, p.layout);
 }
 
 // ---- library-owned scratch for the entry point that has no workspace argument --------------
@@ -369,7 +394,7 @@ int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, c
 int forward_impl(const Problem& p, const void* x, const void* w_large, const Estimator& est,
                  void* out, void* ws, cudaStream_t st) {
     const Workspace w = carve(ws, p.B, p.Ca);
-    int rc = launch_gap(p, x, est, w, w.dk, st);
+    int rc = launch_gap(p, x, est, w, w.dk, st, tensor_stencil_follows(p));
     if (rc != ESC_OK) return rc;
     if (p.dense) return launch_stencil_dense(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
     return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
@@ -485,6 +510,11 @@ int esc_convattn_last_tile_width(void) { return g_last_tile_w; }
 int esc_convattn_set_tile_width(int tile_width) {
     if (tile_width != 0 && tile_width != esc::tma::Geom40::TW && tile_width != esc::tma::Geom64::TW) return ESC_ERR_UNSUPPORTED;
     g_tile_policy = tile_width;
+    return ESC_OK;
+}
+int esc_convattn_set_stencil_engine(int engine) {
+    if (engine != ESC_ENGINE_AUTO && engine != ESC_ENGINE_FP32 && engine != ESC_ENGINE_TENSOR) return ESC_ERR_UNSUPPORTED;
+    g_engine_policy = engine;
     return ESC_OK;
 }
 int esc_convattn_last_launches(void) { return g_last_launches; }
@@ -610,7 +640,7 @@ int esc_convattn_dynkernel_static(const void* x, int B, int C, int C_a, int H, i
     if (rc != ESC_OK) return rc;
     if (!x || !w_dyn || !b_dyn || !dk_out) return ESC_ERR_NULL;
     if (!aligned(x, 16) || !aligned(dk_out, 4) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
-    const int S = slabs_for(B, (long long)H * W);
+    const int S = slabs_for(B, (long long)H * W, wide_gap(B, (long long)H * W, false));
     if (B > kStaticMaxImages || (long long)B * S * C_a > kStaticMaxPartials) {
         char buf[200];
         snprintf(buf, sizeof buf,

@@ -90,7 +90,7 @@ def test_forward_mlp(pkg, oracle, shape, dtype, layout):
     util.check_attention(got[:, :C_a], ref[:, :C_a], mag, dtype, f"mlp {shape}")
     assert np.array_equal(got[:, C_a:], ref[:, C_a:])
     if dtype == synth.BF16 and layout == synth.NHWC and K == 13:
-        assert pkg.esc_convattn_last_path() == 2
+        assert pkg.esc_convattn_last_path() in (2, 4)
 
 
 def test_mlp_differs_from_linear_and_rejects_bad_width(pkg, oracle):

@@ -169,7 +169,7 @@ def test_forward_both_tile_geometries(pkg, oracle, shape, width):
 
 
 def test_tile_choice_and_policy(pkg):
-    """The cost estimate takes 64x16 tiles for a batch of 64x64 patches and for maps with few tiles,
+    """FP32 engine: the cost estimate takes 64x16 tiles for a batch of 64x64 patches and for maps with few tiles,
     40x40 tiles for the large maps; the override rejects widths that do not exist."""
     import torch
 
@@ -183,13 +183,17 @@ def test_tile_choice_and_policy(pkg):
         assert pkg.esc_convattn_device_status(ws) == 0
         return pkg.esc_convattn_last_tile_width()
 
-    assert used(64, 64, 16, 64, 64) == 64
-    assert used(1, 64, 16, 90, 130) == 64
-    assert used(1, 64, 16, 360, 640) == 40
-    assert used(1, 64, 32, 1080, 1920) == 40
-    with pytest.raises(pkg.EscError):
-        pkg.esc_convattn_set_tile_width(48)
-    assert used(1, 64, 16, 360, 640) == 40      # a rejected value leaves the policy alone
+    pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32)
+    try:
+        assert used(64, 64, 16, 64, 64) == 64
+        assert used(1, 64, 16, 90, 130) == 64
+        assert used(1, 64, 16, 360, 640) == 40
+        assert used(1, 64, 32, 1080, 1920) == 40
+        with pytest.raises(pkg.EscError):
+            pkg.esc_convattn_set_tile_width(48)
+        assert used(1, 64, 16, 360, 640) == 40      # a rejected value leaves the policy alone
+    finally:
+        pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
 
 
 @pytest.mark.parametrize("wl_name", ["cfg1_64x64_f32", "cfg2_320x180_f32", "cfg3_640x360_bf16", "cfg4_b64_64x64_bf16"])

@@ -106,7 +106,7 @@ def test_stencil_pw_both_tile_geometries(pkg, oracle, shape, width):
 
 def test_identity_mix_reproduces_the_plain_forward_bit_for_bit(pkg):
     """With LK^c = I the tensor-core mix returns every bf16 value unchanged, so the result equals the
-    depth-wise forward exactly."""
+    depth-wise forward of the same (FP32) stencil kernel exactly."""
     import torch
 
     B, C, C_a, H, W, K = 2, 64, 16, 70, 100, 13
@@ -116,7 +116,11 @@ def test_identity_mix_reproduces_the_plain_forward_bit_for_bit(pkg):
     eye = torch.eye(C_a, dtype=torch.bfloat16, device="cuda")
     ws = pkg.new_workspace(B, C_a, H, W, K)
     a, b = torch.empty_like(x), torch.empty_like(x)
-    pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, a, pkg.ESC_NHWC, ws)
+    pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32)      # the mix lives in the FP32 kernel: compare like with like
+    try:
+        pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, a, pkg.ESC_NHWC, ws)
+    finally:
+        pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
     pkg.esc_convattn_forward_pw(x, C_a, K, wl, eye, wd, bd, b, pkg.ESC_NHWC, ws)
     torch.cuda.synchronize()
     assert pkg.esc_convattn_last_path() == 2

@@ -1,0 +1,98 @@
+"""GPU parity of the tensor-core (banded Toeplitz) form of the depth-wise stage (ESC paper, Section 3.3,
+Eq. 4 line 3 with the large kernel of Eq. 5's depth-wise form) against the CPU oracle, every output
+compared.  Bar: one bf16 rounding of the result plus fp32 accumulation noise (tests/util.py)."""
+import contextlib
+
+import numpy as np
+import pytest
+
+from paper_2503_06671_b200 import synth
+from tests import util
+from tests.test_gpu_parity import TILE_SHAPES, compare_full
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import paper_2503_06671_b200 as p
+
+    p.lib()
+    return p
+
+
+@contextlib.contextmanager
+def engine(pkg, which):
+    pkg.esc_convattn_set_stencil_engine(which)
+    try:
+        yield
+    finally:
+        pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
+
+
+@pytest.mark.parametrize("shape", TILE_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_forward_tensor_engine(pkg, oracle, shape):
+    """Every shape the kernel accepts: maps smaller than the kernel, single rows and columns, ragged tails,
+    one to three channel groups, no and many copy-through channels."""
+    B, C, C_a, H, W, K = shape
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=sum(shape) + 4, per_image_scale=True, channel_means=True)
+    with engine(pkg, pkg.ESC_ENGINE_TENSOR):
+        compare_full(pkg, oracle, d, C_a, K, synth.BF16, synth.NHWC, what=f"{shape} tensor engine")
+        assert pkg.esc_convattn_last_path() == 4
+
+
+def test_engines_agree_and_switch(pkg, oracle):
+    """The same call on either engine: both within the bar of the oracle, the switch selects the kernel, an
+    unknown engine is refused and leaves the choice alone."""
+    B, C, C_a, H, W, K = 2, 64, 16, 77, 150, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=31, per_image_scale=True, channel_means=True)
+    for which, path in ((pkg.ESC_ENGINE_FP32, 2), (pkg.ESC_ENGINE_TENSOR, 4), (pkg.ESC_ENGINE_AUTO, 4)):
+        with engine(pkg, which):
+            compare_full(pkg, oracle, d, C_a, K, synth.BF16, synth.NHWC, what=f"engine {which}")
+            assert pkg.esc_convattn_last_path() == path
+    with pytest.raises(pkg.EscError):
+        pkg.esc_convattn_set_stencil_engine(7)
+    # shapes the tensor-core kernel does not take fall to the guarded generic kernel when it is demanded
+    d = synth.make_inputs(1, 20, 12, 19, 23, 13, synth.BF16, seed=32, channel_means=True)
+    with engine(pkg, pkg.ESC_ENGINE_TENSOR):
+        compare_full(pkg, oracle, d, 12, 13, synth.BF16, synth.NHWC, what="C_a = 12")
+        assert pkg.esc_convattn_last_path() == 1
+
+
+def test_many_units_per_cta(pkg, oracle):
+    """Eight images, two channel groups, 280x400: 2,016 units of 64x16, thirteen or fourteen per CTA on 148
+    SMs, with image and channel-group changes inside every CTA's walk; all outputs compared."""
+    B, C, C_a, H, W, K = 8, 64, 32, 280, 400, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=2031, per_image_scale=True, channel_means=True)
+    with engine(pkg, pkg.ESC_ENGINE_TENSOR):
+        compare_full(pkg, oracle, d, C_a, K, synth.BF16, synth.NHWC, what="many units, tensor engine")
+        assert pkg.esc_convattn_last_path() == 4
+
+
+def test_stencil_stage_explicit_dk_and_determinism(pkg, oracle):
+    """The stage alone with a given dk (so that a wrong 3x3 tap order cannot hide behind small dynamic taps),
+    and bitwise identical results run to run."""
+    import torch
+
+    B, C, C_a, H, W, K = 2, 64, 16, 45, 70, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=78)
+    dk = np.random.default_rng(6).uniform(-0.5, 0.5, size=(B, C_a, 3, 3)).astype(np.float32)
+    x = util.to_device(d["x"], synth.BF16, synth.NHWC)
+    wl, _, _ = util.weights_to_device(d, synth.BF16)
+    outs = []
+    with engine(pkg, pkg.ESC_ENGINE_TENSOR):
+        for _ in range(3):
+            out = torch.empty_like(x)
+            pkg.esc_convattn_stencil(x, C_a, K, wl, torch.from_numpy(dk).cuda(), out, pkg.ESC_NHWC)
+            torch.cuda.synchronize()
+            assert pkg.esc_convattn_last_path() == 4
+            outs.append(out)
+    ref, mag = oracle.stencil(d["x"], C_a, d["w_large"], dk, want_mag=True)
+    got = util.to_host_nchw(outs[0], synth.NHWC)
+    util.check_attention(got[:, :C_a], ref[:, :C_a], mag, synth.BF16, "stencil stage, tensor engine", unit_variance=True)
+    assert np.array_equal(got[:, C_a:], ref[:, C_a:])
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16)) and torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
