@@ -288,6 +288,17 @@ int esc_convattn_last_path(void);
 enum { ESC_ENGINE_AUTO = 0, ESC_ENGINE_FP32 = 1, ESC_ENGINE_TENSOR = 2 };
 int esc_convattn_set_stencil_engine(int engine);
 
+/* Whether a forward call on this thread may run as ONE launch of the tensor-core kernel with stage 1 (Eq. 4
+ * line 2: pooled means and the kernel estimator) inside it (default: on).  It does so where that kernel applies,
+ * C_a <= 128, and no CTA gets more than two 64x16 tiles (about 300,000 pixels per 16 attention channels on a
+ * B200): every CTA adds up the interiors of its own staged tiles, the CTAs exchange the sums through the
+ * workspace and each evaluates the estimator for the channels it works on.  The launch is cooperative (CTAs
+ * wait on one another, all waits bounded: ESC_DEV_TIMEOUT through esc_convattn_device_status); if the device
+ * refuses it, or with 0 here, the forward is the usual two launches.  The pooled means are then sums over tiles
+ * instead of slabs: dk differs by fp32 rounding (about 1e-7 relative).  A workspace whose launch was cut short
+ * must be zeroed again with esc_convattn_workspace_init before its next use.  For tests and tuning. */
+int esc_convattn_set_fused_stage1(int on);
+
 /* Width in pixels of the output tile the TMA-staged kernel used in that call (FP32 kernel: 40 = 40x40
  * tiles, 64 = 64x16 tiles, chosen by the tile count's balance over the SMs; tensor-core kernel: 64 =
  * 64x16 tiles), 0 when the generic kernel ran.  For tests and benchmarks. */

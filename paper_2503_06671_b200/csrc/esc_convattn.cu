@@ -29,6 +29,7 @@ thread_local int g_last_tile_w = 0;
 thread_local int g_tile_policy = 0;      // 0 = by cost, else the tile width to use
 thread_local int g_engine_policy = 0;    // ESC_ENGINE_AUTO / _FP32 / _TENSOR for the depth-wise stencil
 thread_local int g_last_launches = 0;
+thread_local bool g_fuse_stage1 = true;  // tensor-core kernel: stage 1 inside it where every CTA has at most two units
 
 int cuda_fail(cudaError_t e, const char* what) {
     char buf[320];
@@ -77,14 +78,17 @@ int check_tensors(const Problem& p, const void* x, const void* out) {
 }
 
 // ---- workspace layout -------------------------------------------------------------------
-//   [ctrl words: header + B arrival counters][pad to 256][dk: B*Ca*9 floats][pad][partials: B*S*Ca floats]
+//   [ctrl words: header + B arrival counters + B launch flags][pad to 256][dk: B*Ca*9 floats][pad]
+//   [partials: B*S*Ca floats][pad][per-unit sums of the fused stage 1: 2 * SMs * 16 floats]
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Workspace {
     unsigned* ctrl;
     unsigned* arrivals;
+    unsigned* flags;
     float* dk;
     float* partial;
+    float* unit_sums;
 };
 
 bool is_large_map(int B, long long HW) { return (long double)B * HW >= 1.5e6L; }
@@ -121,21 +125,25 @@ int slabs_for(int B, long long HW, bool wide) {
 
 size_t workspace_bytes(int B, int Ca, long long HW) {
     const int S = slabs_for(B, HW, true);                   // room for either grid policy
-    size_t off = round_up((size_t)(esc::kCtrlHeaderWords + B) * 4, 256);
+    size_t off = round_up((size_t)(esc::kCtrlHeaderWords + 2 * (size_t)B) * 4, 256);
     off += round_up((size_t)B * Ca * 9 * 4, 256);
     off += round_up((size_t)B * S * Ca * 4, 256);
+    off += round_up((size_t)2 * sms_or_nominal() * 16 * 4, 256);
     return off;
 }
 
-Workspace carve(void* ws, int B, int Ca) {
+Workspace carve(void* ws, int B, int Ca, long long HW) {
     Workspace w;
     char* p = static_cast<char*>(ws);
     w.ctrl = reinterpret_cast<unsigned*>(p);
     w.arrivals = w.ctrl + esc::kCtrlHeaderWords;
-    p += round_up((size_t)(esc::kCtrlHeaderWords + B) * 4, 256);
+    w.flags = w.arrivals + B;
+    p += round_up((size_t)(esc::kCtrlHeaderWords + 2 * (size_t)B) * 4, 256);
     w.dk = reinterpret_cast<float*>(p);
     p += round_up((size_t)B * Ca * 9 * 4, 256);
     w.partial = reinterpret_cast<float*>(p);
+    p += round_up((size_t)B * slabs_for(B, HW, true) * Ca * 4, 256);
+    w.unit_sums = reinterpret_cast<float*>(p);
     return w;
 }
 
@@ -393,7 +401,20 @@ int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, c
 
 int forward_impl(const Problem& p, const void* x, const void* w_large, const Estimator& est,
                  void* out, void* ws, cudaStream_t st) {
-    const Workspace w = carve(ws, p.B, p.Ca);
+    const Workspace w = carve(ws, p.B, p.Ca, (long long)p.H * p.W);
+    // Small problems on the tensor-core kernel: one launch, stage 1 inside the stencil kernel.
+    if (g_fuse_stage1 && tensor_stencil_follows(p)) {
+        const esc::tma::toep::Fused fu{est.w_last, est.b_last, est.w_down, est.b_down, est.hidden, w.unit_sums, w.arrivals, w.flags};
+        int tw = 0;
+        const int rc = esc::tma::toep::try_launch_fused(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, fu, out,
+                                                        w.ctrl, st, &g_last_launches, &g_last_error, &tw);
+        if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
+        if (rc != esc::tma::kNotApplicable) {
+            // a cooperative launch can be refused (SMs held by another context): fall back to two kernels
+            (void)cudaGetLastError();
+            g_last_error.clear();
+        }
+    }
     int rc = launch_gap(p, x, est, w, w.dk, st, tensor_stencil_follows(p));
     if (rc != ESC_OK) return rc;
     if (p.dense) return launch_stencil_dense(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
@@ -517,6 +538,10 @@ int esc_convattn_set_stencil_engine(int engine) {
     g_engine_policy = engine;
     return ESC_OK;
 }
+int esc_convattn_set_fused_stage1(int on) {
+    g_fuse_stage1 = on != 0;
+    return ESC_OK;
+}
 int esc_convattn_last_launches(void) { return g_last_launches; }
 
 const char* esc_status_string(int s) {
@@ -589,7 +614,7 @@ int esc_convattn_dynkernel(const void* x, int B, int C, int C_a, int H, int W, c
     if (!aligned(x, 16) || !aligned(dk_out, 4) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
     rc = check_workspace(p, workspace, workspace_bytes_);
     if (rc != ESC_OK) return rc;
-    return launch_gap(p, x, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, carve(workspace, B, C_a), dk_out,
+    return launch_gap(p, x, Estimator{w_dyn, b_dyn, nullptr, nullptr, 0}, carve(workspace, B, C_a, (long long)H * W), dk_out,
                       static_cast<cudaStream_t>(stream));
 }
 
@@ -629,7 +654,7 @@ int esc_convattn_dynkernel_mlp(const void* x, int B, int C, int C_a, int H, int 
     if (!aligned(x, 16) || !aligned(dk_out, 4)) return ESC_ERR_ALIGN;
     rc = check_workspace(p, workspace, workspace_bytes_);
     if (rc != ESC_OK) return rc;
-    return launch_gap(p, x, est, carve(workspace, B, C_a), dk_out, static_cast<cudaStream_t>(stream));
+    return launch_gap(p, x, est, carve(workspace, B, C_a, (long long)H * W), dk_out, static_cast<cudaStream_t>(stream));
 }
 
 int esc_convattn_dynkernel_static(const void* x, int B, int C, int C_a, int H, int W, const void* w_dyn,
@@ -679,7 +704,7 @@ int esc_convattn_stencil(const void* x, int B, int C, int C_a, int H, int W, int
     if (workspace) {
         rc = check_workspace(p, workspace, workspace_bytes_);
         if (rc != ESC_OK) return rc;
-        ctrl = carve(workspace, B, C_a).ctrl;
+        ctrl = carve(workspace, B, C_a, (long long)H * W).ctrl;
     }
     return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
 }
@@ -700,7 +725,7 @@ int esc_convattn_stencil_pw(const void* x, int B, int C, int C_a, int H, int W, 
     if (workspace) {
         rc = check_workspace(p, workspace, workspace_bytes_);
         if (rc != ESC_OK) return rc;
-        ctrl = carve(workspace, B, C_a).ctrl;
+        ctrl = carve(workspace, B, C_a, (long long)H * W).ctrl;
     }
     return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
 }
@@ -740,7 +765,7 @@ int esc_convattn_stencil_dense(const void* x, int B, int C, int C_a, int H, int 
     if (workspace) {
         rc = check_workspace(p, workspace, workspace_bytes_);
         if (rc != ESC_OK) return rc;
-        ctrl = carve(workspace, B, C_a).ctrl;
+        ctrl = carve(workspace, B, C_a, (long long)H * W).ctrl;
     }
     return launch_stencil_dense(p, x, w_dense, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
 }

@@ -28,6 +28,7 @@
 //   warp 8      tile producer (TMA), warp 9 copy-through of the untouched channels (TMA in / out).
 #pragma once
 #include "stencil_tma.cuh"
+#include "gap_dynkernel.cuh"
 
 namespace esc { namespace tma { namespace toep {
 
@@ -66,7 +67,18 @@ struct Params {
     __nv_bfloat16* out;
     unsigned* ctrl;
     int wait_first;
+    // Fused stage 1 (kFused): the estimator's weights (bf16; one layer when hidden == 0, see gap_dynkernel.cuh),
+    // one slot of 16 partial sums per unit, and per image an arrival counter and a flag that counts launches.
+    const __nv_bfloat16 *w_last, *b_last, *w_down, *b_down;
+    int hidden;
+    float* gpart;
+    unsigned *garr, *gflag;
+    int upi;                          // units per image = groups * tiles_y * tiles_x
 };
+constexpr int kFusedMaxCa = 128;      // channels the fused estimator keeps in shared memory
+// scratch of the fused stage 1, a multiple of 128 bytes (the copy ring behind it is a TMA destination)
+constexpr int FUSED_SMEM_FLOATS = (kMmaThreads + kFusedMaxCa + kMaxHidden + CG * 9 + kWarps * CG + 31) / 32 * 32;
+constexpr unsigned kFlagPolls = 1u << 22;   // polls of another CTA's flag before a wait gives up (about half a second)
 
 __device__ __forceinline__ Unit decode(long long u64v, const Params& p) {
     unsigned u = (unsigned)u64v;
@@ -97,7 +109,25 @@ __device__ __forceinline__ float bf16_at(const unsigned char* plane, int row, in
     return __uint_as_float((unsigned)v << 16);
 }
 
-template <class S, bool kBias>
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// kFused: stage 1 of the module (Eq. 4 line 2) inside this kernel, for launches in which no CTA has more
+// than two units.  The pooled means come from the staged tiles themselves: every CTA adds up the interiors
+// of its own tiles, which partition the image, writes 16 sums per unit and arrives on the image's counter
+// (the atomic is issued by the otherwise idle producer lane, so its round trip stays off the working warps'
+// path); the CTA that arrives last advances the image's flag; every CTA then adds the partial sums of the
+// image in a fixed order and evaluates the estimator for the 16 channels it is working on.  No second
+// kernel, no second pass over the attention channels, and dk is there when the tensor-core work of a CTA's
+// first unit is done.  CTAs wait on one another: the launch is cooperative (all CTAs resident, one per SM)
+// and every wait is bounded.
+template <class S, bool kBias, bool kFused>
 __global__ void __launch_bounds__(kThreads, 1)
 stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
                            const __grid_constant__ CUtensorMap map_cout, const Params p)
@@ -108,15 +138,17 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
     unsigned char* stage = smem;                                   // NHWC halo tile as it lands: [ROWS][SW][16] bf16
     unsigned char* planes = smem + S::STAGE_BYTES;                 // 16 x [ROWS][PP] bf16
     uint32_t* ptab = reinterpret_cast<uint32_t*>(planes + CG * PLANE);   // [16][13][PT] packed tap pairs
-    unsigned char* ring = reinterpret_cast<unsigned char*>(ptab) + PTAB_BYTES;
+    float* fsm = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(ptab) + PTAB_BYTES);   // fused stage 1 scratch
+    unsigned char* ring = reinterpret_cast<unsigned char*>(fsm) + (kFused ? FUSED_SMEM_FLOATS * 4 : 0);
     u64* bars = reinterpret_cast<u64*>(ring + NSLOT * p.slot_stride);
-    const uint32_t full = smem_u32(bars), empty = full + 8, cfull0 = full + 16;
+    const uint32_t full = smem_u32(bars), empty = full + 8, cfull0 = full + 16, sumdone = cfull0 + 8 * NSLOT;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         mbar_init(full, 1);
         mbar_init(empty, kWarps);
         for (int s = 0; s < NSLOT; ++s) mbar_init(cfull0 + 8 * s, 1);
+        mbar_init(sumdone, CG);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -129,13 +161,24 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
     if (warp >= kWarps) {
         if (lane != 0) return;
         if (warp == kWarps) {
-            // ---- tile producer: the staging buffer is free again once every warp has transposed its share
+            // ---- tile producer: the staging buffer is free again once every warp has transposed its share.
+            //      With stage 1 fused this lane also performs the arrivals on the images' counters, once the
+            //      working warps have written a unit's 16 sums.
             bool alive = true;
             for (long long k = 0; k < my_units; ++k) {
-                if (k >= 1 && alive) alive = mbar_wait(empty, (unsigned)((k - 1) & 1), p.ctrl, 0xB8000000u);
                 const Unit un = decode(first + k * stride, p);
+                unsigned seen = 0u;
+                if (kFused) seen = ld_acquire(p.gflag + un.b);       // before this CTA's arrival: the flag cannot have advanced yet
+                if (k >= 1 && alive) alive = mbar_wait(empty, (unsigned)((k - 1) & 1), p.ctrl, 0xB8000000u);
                 mbar_expect_tx(full, S::STAGE_BYTES);
                 tma_load_4d(smem_u32(stage), &map_att, full, un.g * CG, un.tx * TW - P6, un.ty * TH - P6, un.b);
+                if (kFused) {
+                    if (alive) alive = mbar_wait(sumdone, (unsigned)(k & 1), p.ctrl, 0xB9000000u);
+                    // release: the 16 sums (seen through the barrier) are visible to whoever reads the counter or the flag
+                    unsigned old;
+                    asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.garr + un.b), "r"((unsigned)(p.upi - 1)) : "memory");
+                    if (old == (unsigned)(p.upi - 1)) st_release(p.gflag + un.b, seen + 1u);   // the counter has wrapped back to 0
+                }
             }
         } else if (p.copy_cc != 0) {
             // ---- copy-through of the untouched channels (same scheme as the FP32 kernel's copy warp)
@@ -203,6 +246,113 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
 
     int cur_g = -1;
     bool alive = true, dk_ready = p.wait_first != 0;
+
+    // ---- fused stage 1 ------------------------------------------------------------------------------
+    float* f_sub = fsm;                                      // [256] sub-sums of the partial sums
+    float* f_mean = fsm + kMmaThreads;                       // [Ca] pooled means of the current image
+    float* f_act = f_mean + kFusedMaxCa;                     // [hidden] activations of the two-layer estimator
+    float* f_dk = f_act + kMaxHidden;                        // [16][9] dynamic taps of the current (image, group)
+    float* f_red = f_dk + CG * 9;                            // [8 warps][16] tile sums
+    unsigned flag0[2] = {0u, 0u};                            // the images' flags as they stood before this launch
+    int dk_b = -1, dk_g = -1;
+    if (kFused) {
+        // read before this CTA arrives anywhere: the flag cannot have advanced yet
+        for (int k = 0; k < (int)my_units && k < 2; ++k) flag0[k] = ld_acquire(p.gflag + decode(first + k * stride, p).b);
+    }
+    // Sum of the staged tile's interior per channel (the tiles' interiors partition the image; pixels outside
+    // it are zero-filled), in a fixed order; 16 sums to the unit's slot, then the producer lane is told.
+    auto tile_sum = [&](const long long unit_index) {
+        const int gsub = lane >> 3, pr = lane & 7;           // pixel 4i + gsub of a row, channel pair pr: conflict-free
+        const uint32_t* st32 = reinterpret_cast<const uint32_t*>(stage);
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int rr = 0; rr < NA; ++rr)
+#pragma unroll
+            for (int i = 0; i < TW / 4; ++i) {
+                const uint32_t v = st32[((P6 + warp * NA + rr) * SW + P6 + 4 * i + gsub) * NPAIR + pr];
+                s0 += __uint_as_float(v << 16);
+                s1 += __uint_as_float(v & 0xffff0000u);
+            }
+        s0 += __shfl_xor_sync(0xffffffffu, s0, 8);  s1 += __shfl_xor_sync(0xffffffffu, s1, 8);
+        s0 += __shfl_xor_sync(0xffffffffu, s0, 16); s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+        if (lane < 8) { f_red[warp * CG + 2 * lane] = s0; f_red[warp * CG + 2 * lane + 1] = s1; }
+        mma_bar();
+        if (tid < CG) {
+            float tsum = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) tsum += f_red[w * CG + tid];
+            p.gpart[unit_index * CG + tid] = tsum;
+            mbar_arrive(sumdone);
+        }
+    };
+    // dk of (image, group) of `un` into f_dk: wait for the image's flag, add the image's partial sums in a fixed
+    // order, evaluate the estimator (Eq. 4 line 2) for the 16 channels of the group.
+    auto obtain_dk = [&](const Unit& un, const unsigned seen) {
+        if (un.b == dk_b && un.g == dk_g) return;
+        if (un.b != dk_b) {
+            if (tid == 0 && alive) {
+                unsigned n = 0;
+                while (ld_acquire(p.gflag + un.b) == seen) {
+                    __nanosleep(100);
+                    if (++n > kFlagPolls) { if (p.ctrl) { atomicExch(p.ctrl, kDevTimeout); atomicExch(p.ctrl + 1, 0xF0000000u | (unsigned)un.b); } break; }
+                }
+            }
+            mma_bar();
+            // means: thread (sub, c) adds tiles sub, sub + nsub, ... of channel c's group; then the sub-sums in order
+            const int Ca = p.Ca, nsub = kMmaThreads / Ca, tpi = p.upi / p.groups;
+            const int c = tid % Ca, sub = tid / Ca;
+            if (sub < nsub) {
+                const float* src = p.gpart + ((size_t)un.b * p.upi + (size_t)(c / CG) * tpi) * CG + (c % CG);
+                float tsum = 0.f;
+                for (int tl = sub; tl < tpi; tl += 8 * nsub) {
+                    float v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = tl + u * nsub < tpi ? __ldcg(src + (size_t)(tl + u * nsub) * CG) : 0.f;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) tsum += v[u];
+                }
+                f_sub[tid] = tsum;
+            }
+            mma_bar();
+            if (tid < Ca) {
+                float tsum = 0.f;
+                for (int j = 0; j < nsub; ++j) tsum += f_sub[j * Ca + tid];
+                f_mean[tid] = tsum * (1.0f / (float)((long long)p.H * p.W));
+            }
+            mma_bar();
+            if (p.hidden > 0) {
+                for (int j = tid; j < p.hidden; j += kMmaThreads) {
+                    float tsum = __bfloat162float(p.b_down[j]);
+                    const __nv_bfloat16* wr = p.w_down + (size_t)j * Ca;
+                    for (int cc = 0; cc < Ca; ++cc) tsum = fmaf(__bfloat162float(wr[cc]), f_mean[cc], tsum);
+                    f_act[j] = gelu_exact(tsum);
+                }
+                mma_bar();
+            }
+            dk_b = un.b;
+        }
+        {
+            const float* vin = p.hidden > 0 ? f_act : f_mean;
+            const int n_in = p.hidden > 0 ? p.hidden : p.Ca;
+            if (tid < CG * 9) {
+                const int o = un.g * CG * 9 + tid;
+                float a = __bfloat162float(p.b_last[o]);
+                const __nv_bfloat16* wr = p.w_last + (size_t)o * n_in;
+                for (int c0 = 0; c0 < n_in; c0 += 16) {      // sixteen independent loads, FMAs in input order
+                    float wv[16];
+#pragma unroll
+                    for (int u = 0; u < 16; ++u) wv[u] = c0 + u < n_in ? __bfloat162float(wr[c0 + u]) : 0.f;
+#pragma unroll
+                    for (int u = 0; u < 16; ++u)
+                        if (c0 + u < n_in) a = fmaf(wv[u], vin[c0 + u], a);
+                }
+                f_dk[tid] = a;
+            }
+            dk_g = un.g;
+            mma_bar();
+        }
+    };
+
     for (long long k = 0; k < my_units; ++k) {
         const Unit un = decode(first + k * stride, p);
 
@@ -227,6 +377,7 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
 
         // ---- the NHWC tile has landed: transpose it into the 16 planes --------------------------------
         if (alive) alive = mbar_wait(full, (unsigned)(k & 1), p.ctrl, 0xA8000000u);
+        if (kFused && k == 0) tile_sum(first);               // (a second unit's tile is added up below, as soon as it can be)
         {
             // a step = 16 pixels of one staged row x 16 channels: four 8x8 matrices (pixel half, channel half)
             constexpr int STEPS = ROWS * (SW / 16);
@@ -293,9 +444,14 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         // a funnel shift by 0 or 16 lines them up.
         auto dk_all = [&](float (&d4)[NB][NA][4], const int c) {
             const uint32_t* plane32 = reinterpret_cast<const uint32_t*>(planes + (size_t)c * PLANE);
-            const float* dp = p.dk + ((size_t)un.b * p.Ca + un.g * CG + c) * 9;
+            if (kFused) {
 #pragma unroll
-            for (int v = 0; v < 9; ++v) dkv[v] = __ldcg(dp + v);
+                for (int v = 0; v < 9; ++v) dkv[v] = f_dk[c * 9 + v];
+            } else {
+                const float* dp = p.dk + ((size_t)un.b * p.Ca + un.g * CG + c) * 9;
+#pragma unroll
+                for (int v = 0; v < 9; ++v) dkv[v] = __ldcg(dp + v);
+            }
             const float bias = kBias ? __ldg(p.bias + (size_t)un.b * p.Ca + un.g * CG + c) : 0.f;
 #pragma unroll
             for (int q = 0; q < NB; ++q)
@@ -340,13 +496,31 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
                     }
         };
 
+        if (kFused && k == 0) {
+            // first unit: all tensor-core work first, and between the two channels the sum of the second unit's tile,
+            // which has landed meanwhile: every CTA has arrived for all its tiles well before dk is needed
+            float acc1[NB][NA][4];
+            mma_all(acc, warp * 2);
+            if (my_units > 1) {
+                if (alive) alive = mbar_wait(full, 1u, p.ctrl, 0xA9000000u);
+                tile_sum(first + stride);
+            }
+            mma_all(acc1, warp * 2 + 1);
+            obtain_dk(un, flag0[0]);
+            dk_all(dacc, warp * 2);
+            write_back(acc, dacc, warp * 2);
+            dk_all(dacc, warp * 2 + 1);
+            write_back(acc1, dacc, warp * 2 + 1);
+        } else {
+            if (kFused) obtain_dk(un, flag0[1]);
 #pragma unroll 1
-        for (int cc = 0; cc < 2; ++cc) {
-            const int c = warp * 2 + cc;
-            mma_all(acc, c);
-            if (!dk_ready) { pdl_wait_primary(); dk_ready = true; }
-            dk_all(dacc, c);
-            write_back(acc, dacc, c);
+            for (int cc = 0; cc < 2; ++cc) {
+                const int c = warp * 2 + cc;
+                mma_all(acc, c);
+                if (!kFused && !dk_ready) { pdl_wait_primary(); dk_ready = true; }
+                dk_all(dacc, c);
+                write_back(acc, dacc, c);
+            }
         }
         mma_bar();                                           // all 16 planes hold their results
 
@@ -381,10 +555,18 @@ inline long long units_of(int B, int Ca, int H, int W) {
     return (long long)B * (Ca / CG) * ((W + S::TW - 1) / S::TW) * ((H + S::TH - 1) / S::TH);
 }
 
-template <class S, bool kBias>
+// Stage 1 inside the stencil kernel: the estimator's weights and the scratch it needs (see Params).
+struct Fused {
+    const void *w_last, *b_last, *w_down, *b_down;
+    int hidden;
+    float* gpart;
+    unsigned *garr, *gflag;
+};
+
+template <class S, bool kBias, bool kFused>
 inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk,
                         const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches,
-                        std::string* err) {
+                        std::string* err, const Fused* fu = nullptr) {
     const int cc = C - Ca;
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -404,6 +586,13 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
     p.dk = dk; p.bias = bias; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
+    p.w_last = p.b_last = p.w_down = p.b_down = nullptr; p.hidden = 0; p.gpart = nullptr; p.garr = p.gflag = nullptr;
+    p.upi = p.groups * p.tiles_x * p.tiles_y;
+    if (kFused) {
+        p.w_last = static_cast<const __nv_bfloat16*>(fu->w_last); p.b_last = static_cast<const __nv_bfloat16*>(fu->b_last);
+        p.w_down = static_cast<const __nv_bfloat16*>(fu->w_down); p.b_down = static_cast<const __nv_bfloat16*>(fu->b_down);
+        p.hidden = fu->hidden; p.gpart = fu->gpart; p.garr = fu->garr; p.gflag = fu->gflag;
+    }
 
     CUtensorMap m_att, m_cin, m_cout;
     if (!make_map(&m_att, x, B, C, H, W, CG, S::SW, S::ROWS, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
@@ -413,13 +602,16 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     } else {
         m_cin = m_att; m_cout = m_att;
     }
-    const size_t smem = (size_t)S::STAGE_BYTES + (size_t)CG * S::PLANE_BYTES + PTAB_BYTES + (size_t)NSLOT * p.slot_stride + 64;
+    static_assert((S::STAGE_BYTES + CG * S::PLANE_BYTES + PTAB_BYTES) % 128 == 0 && (FUSED_SMEM_FLOATS * 4) % 128 == 0,
+                  "the copy ring is a TMA destination: 128-byte aligned");
+    const size_t smem = (size_t)S::STAGE_BYTES + (size_t)CG * S::PLANE_BYTES + PTAB_BYTES + (kFused ? FUSED_SMEM_FLOATS * 4 : 0) +
+                        (size_t)NSLOT * p.slot_stride + 64;   // 64: the mbarriers
     if (smem > 227 * 1024) return kNotApplicable;
     static bool attr_set[kMaxDevices] = {};
     const int dev = current_device();
     if (dev < 0) return kNotApplicable;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nhwc_bf16<S, kBias>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nhwc_bf16<S, kBias, kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
         attr_set[dev] = true;
     }
@@ -429,12 +621,15 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;             // fused stage 1: CTAs wait on one another, all must be resident
+    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias>, m_att, m_cin, m_cout, p);
+    cfg.numAttrs = kFused ? 2 : 1;
+    if (kFused && (grid > sm_count() || p.units > 2 * grid)) return kNotApplicable;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias, kFused>, m_att, m_cin, m_cout, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_toeplitz_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -455,8 +650,26 @@ inline int try_launch_toeplitz(int B, int C, int Ca, int H, int W, int K, int dt
                                cudaStream_t st, bool dependent, int* launches, std::string* err, int* tile_w) {
     if (!applies(C, Ca, K, dtype, layout) || sm_count() <= 0) return kNotApplicable;
     *tile_w = Shape64x16::TW;
-    return bias ? launch_shape<Shape64x16, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err)
-                : launch_shape<Shape64x16, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err);
+    return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err)
+                : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err);
+}
+
+// Whether the whole forward can be one launch of the tensor-core kernel with stage 1 inside: the kernel applies,
+// no CTA gets more than two units (a CTA adds up its tiles before it needs dk), the estimator fits the scratch.
+inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, int hidden) {
+    if (!applies(C, Ca, K, dtype, layout) || sm_count() <= 0) return false;
+    if (Ca > kFusedMaxCa || hidden > kMaxHidden) return false;
+    return units_of<Shape64x16>(B, Ca, H, W) <= 2LL * sm_count();
+}
+
+// The whole forward (stage 1 fused) as one launch; same return convention as try_launch_toeplitz.
+inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
+                            const void* w_large, const Fused& fu, void* out, unsigned* ctrl, cudaStream_t st,
+                            int* launches, std::string* err, int* tile_w) {
+    if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden)) return kNotApplicable;
+    *tile_w = Shape64x16::TW;
+    return launch_shape<Shape64x16, false, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
+                                                 launches, err, &fu);
 }
 
 }}}  // namespace esc::tma::toep
