@@ -39,6 +39,9 @@ FMA_LANES_PER_SM = 128
 L2_BYTES = 126 * 1024 * 1024
 SAMPLES = 11
 MIN_SAMPLE_S = 0.1
+PATH_NAMES = {1: "generic", 2: "tma-fp32", 3: "tensor-dense", 4: "tensor-toeplitz"}
+KERNEL_FILES = {1: "stencil_generic.cuh", 2: "stencil_tma.cuh", 3: "stencil_dense.cuh", 4: "stencil_toeplitz.cuh"}
+TOEPLITZ_DENSITY = 13.0 / 32.0               # useful share of the multiply-adds the banded-Toeplitz kernel issues
 PEAK_SRC = os.path.join(ROOT, "bench_fp32_peak.cu")
 PEAK_LIB = os.path.join(ROOT, "paper_2503_06671_b200", "lib", "libbench_fp32_peak.so")
 
@@ -352,7 +355,7 @@ def measure_config(pkg, torch, np, synth, wl, layout_name, steps, pk, sms, fp32_
     ms_step, ms_kernel = st_step["median_ms"], st_kernel["median_ms"]
     rec = {
         "workload": wl.name, "layout": layout_name, "storage": wl.dtype,
-        "stencil_path": {1: "generic", 2: "tma", 3: "tensor"}.get(path, str(path)), "tile_width": tile_w,
+        "stencil_path": PATH_NAMES.get(path, str(path)), "tile_width": tile_w, "launches_per_step": launches_per_step,
         "step_us": ms_step * 1e3, "step_us_min": st_step["min_ms"] * 1e3, "step_us_max": st_step["max_ms"] * 1e3,
         "stencil_us": ms_kernel * 1e3, "stencil_us_min": st_kernel["min_ms"] * 1e3, "stencil_us_max": st_kernel["max_ms"] * 1e3,
         "samples": st_step["samples"], "replays_per_sample": st_step["replays_per_sample"],
@@ -445,7 +448,7 @@ def main():
     wl_d, wd_d, bd_d, tensor_bytes = c["wl_d"], c["wd_d"], c["bd_d"], c["tensor_bytes"]
 
     flops, alg_bytes, peak_tflops, t_alu, t_hbm = (c[k] for k in ("flops", "alg_bytes", "peak_tflops", "t_alu", "t_hbm"))
-    kernel_file = {2: "stencil_tma.cuh", 1: "stencil_generic.cuh"}.get(c["path"], "stencil_tma.cuh")
+    kernel_file = KERNEL_FILES.get(c["path"], "stencil_tma.cuh")
     if t_alu >= t_hbm:
         ach = flops / (ms_step * 1e-3) / 1e12
         roof = {"bound": "alu", "achieved": ach, "peak": peak_tflops, "unit": "TFLOP/s", "frac": ach / peak_tflops,
@@ -461,7 +464,17 @@ def main():
         roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
                 "peak_source": f"{pk['source']} copy bandwidth"}
     roof["traffic"] = ncu_traffic(kernel_file, wl.name, args.layout)
-    roof.update({"frac_is": "whole step (both kernels of the forward), median", "kernel": "stencil (stage 2)",
+    if c["path"] == 4:
+        # the depth-wise stage runs on the tensor cores as banded-Toeplitz products: the fraction above is still
+        # the one of the FP32 roofline of the method's 169 multiply-adds per output (the contract's bound); beside
+        # it, what the tensor pipe was asked to do
+        issued = flops / TOEPLITZ_DENSITY
+        roof["engine"] = "tensor cores: mma.sync m16n8k16 bf16 x bf16 -> fp32, 13 of 32 issued multiply-adds useful"
+        roof["tensor_side"] = {"issued_TFLOPs_whole_step": issued / (ms_step * 1e-3) / 1e12,
+                               "issued_TFLOPs_stencil_stage": issued / (ms_kernel * 1e-3) / 1e12,
+                               "bf16_peak_TFLOPs": pk["bf16_tflops"],
+                               "stencil_stage_of_bf16_peak": issued / (ms_kernel * 1e-3) / 1e12 / pk["bf16_tflops"]}
+    roof.update({"frac_is": "whole step (all kernels of the forward), median", "kernel": "stencil (stage 2)",
                  "kernel_ms": ms_kernel, "stencil_stage_frac": max(t_alu, t_hbm) / (ms_kernel * 1e-3),
                  "whole_step_frac": max(t_alu, t_hbm) / (ms_step * 1e-3),
                  "fp32_peak_probe": fp32_meas,
@@ -479,6 +492,22 @@ def main():
         if 2 * c["tensor_bytes"] < L2_BYTES:
             st_hot, _ = timer.measure(lambda i: pkg.esc_convattn_stencil(xs[0], wl.C_a, wl.K, wl_d, dk, outs[0], lay_code, ws), samples=5)
             roof["kernel_ms_input_resident_in_l2"] = st_hot["median_ms"]
+        # the same workload with the depth-wise stage pinned to the FP32 pipe (the register-tiled TMA kernel)
+        if c["path"] == 4:
+            pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32)
+            try:
+                st_f, _ = timer.measure(c["step"], samples=5)
+                st_fk, _ = timer.measure(c["stencil"], samples=5)
+            finally:
+                pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
+            extras["fp32_engine"] = {"ms_per_step": st_f["median_ms"], "stencil_ms": st_fk["median_ms"],
+                                     "whole_step_frac": max(t_alu, t_hbm) / (st_f["median_ms"] * 1e-3)}
+            pkg.esc_convattn_set_fused_stage1(False)
+            try:
+                st_2, _ = timer.measure(c["step"], samples=5)
+            finally:
+                pkg.esc_convattn_set_fused_stage1(True)
+            extras["two_launch_forward_ms_per_step"] = st_2["median_ms"]
         # the whole step with the paper's two-layer estimator (hidden width 8, exact GELU)
         mlp_d = [torch.from_numpy(v).to(tdt).cuda() for v in synth.make_estimator_mlp(wl.C_a, 8, wl.dtype, wl.seed).values()]
         st, _ = timer.measure(lambda i: pkg.esc_convattn_forward_mlp(xs[i % n_rot], wl.C_a, wl.K, wl_d, *mlp_d, outs[i % n_rot], lay_code, ws), samples=5)
@@ -496,7 +525,7 @@ def main():
             extras["dense_large_kernel"] = {
                 "ms_per_step": ms_dense, "bound": "tensor", "achieved": fl / (ms_dense * 1e-3) / 1e12, "peak": pk["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": fl / (ms_dense * 1e-3) / 1e12 / pk["bf16_tflops"],
-                "path": {1: "generic", 3: "tensor"}.get(pkg.esc_convattn_last_path(), str(pkg.esc_convattn_last_path())),
+                "path": PATH_NAMES.get(pkg.esc_convattn_last_path(), str(pkg.esc_convattn_last_path())),
                 "note": "whole step (GAP kernel + dense stencil kernel with copy-through)"}
 
         # ---- end to end through the host-buffer entries (copies inside the timed region) ------------
