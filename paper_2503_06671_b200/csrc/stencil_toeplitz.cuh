@@ -43,6 +43,7 @@ struct Shape {
     static constexpr int ROWS = TH + K13 - 1;        // staged rows
     static constexpr int SW = 16 * (NB + 1);         // staged pixels per row (TW + 12, rounded up to whole input blocks)
     static constexpr int STAGE_BYTES = ROWS * SW * CG * 2;
+    static constexpr int BOX_BYTES = TH * TW * CG * 2;   // a tile's interior alone
     // A plane row holds SW bf16 and is padded to 8 * odd elements: the eight 16-byte rows of an ldmatrix
     // then fall in eight different groups of four banks.
     static constexpr int PP = ((SW / 8) | 1) * 8;
@@ -130,7 +131,8 @@ __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
 template <class S, bool kBias, bool kFused>
 __global__ void __launch_bounds__(kThreads, 1)
 stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
-                           const __grid_constant__ CUtensorMap map_cout, const Params p)
+                           const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_box,
+                           const Params p)
 {
     constexpr int NA = S::NA, NB = S::NB, TH = S::TH, TW = S::TW, ROWS = S::ROWS, SW = S::SW, PP = S::PP;
     constexpr int PLANE = S::PLANE_BYTES;
@@ -139,9 +141,10 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
     unsigned char* planes = smem + S::STAGE_BYTES;                 // 16 x [ROWS][PP] bf16
     uint32_t* ptab = reinterpret_cast<uint32_t*>(planes + CG * PLANE);   // [16][13][PT] packed tap pairs
     float* fsm = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(ptab) + PTAB_BYTES);   // fused stage 1 scratch
-    unsigned char* ring = reinterpret_cast<unsigned char*>(fsm) + (kFused ? FUSED_SMEM_FLOATS * 4 : 0);
+    unsigned char* sumbuf = reinterpret_cast<unsigned char*>(fsm) + FUSED_SMEM_FLOATS * 4;       // fused: interior of the second unit's tile
+    unsigned char* ring = reinterpret_cast<unsigned char*>(fsm) + (kFused ? FUSED_SMEM_FLOATS * 4 + S::BOX_BYTES : 0);
     u64* bars = reinterpret_cast<u64*>(ring + NSLOT * p.slot_stride);
-    const uint32_t full = smem_u32(bars), empty = full + 8, cfull0 = full + 16, sumdone = cfull0 + 8 * NSLOT;
+    const uint32_t full = smem_u32(bars), empty = full + 8, cfull0 = full + 16, sumdone = cfull0 + 8 * NSLOT, boxfull = sumdone + 8;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -149,6 +152,7 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         mbar_init(empty, kWarps);
         for (int s = 0; s < NSLOT; ++s) mbar_init(cfull0 + 8 * s, 1);
         mbar_init(sumdone, CG);
+        mbar_init(boxfull, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -160,25 +164,39 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
 
     if (warp >= kWarps) {
         if (lane != 0) return;
+        if (warp == kWarps && kFused) {
+            // ---- stage 1 fused: this lane starts the loads -- the first unit's halo tile and, for its sum alone, the
+            //      interior of the second unit's tile -- and performs the arrivals on the images' counters once the
+            //      working warps have written a unit's 16 sums (the atomic's round trip stays off their path).  The
+            //      second unit's halo tile is requested by the working warps when they have transposed the first.
+            bool alive = true;
+            const Unit u0 = decode(first, p), u1 = decode(first + (my_units > 1 ? stride : 0), p);
+            mbar_expect_tx(full, S::STAGE_BYTES);
+            tma_load_4d(smem_u32(stage), &map_att, full, u0.g * CG, u0.tx * TW - P6, u0.ty * TH - P6, u0.b);
+            if (my_units > 1) {
+                mbar_expect_tx(boxfull, S::BOX_BYTES);
+                tma_load_4d(smem_u32(sumbuf), &map_box, boxfull, u1.g * CG, u1.tx * TW, u1.ty * TH, u1.b);
+            }
+            // the flags as they stand before this CTA arrives anywhere: they cannot have advanced yet
+            const unsigned seen[2] = {ld_acquire(p.gflag + u0.b), ld_acquire(p.gflag + u1.b)};
+            for (int k = 0; k < (int)my_units; ++k) {
+                const Unit& un = k == 0 ? u0 : u1;
+                if (alive) alive = mbar_wait(sumdone, (unsigned)(k & 1), p.ctrl, 0xB9000000u);
+                // release: the 16 sums (seen through the barrier) are visible to whoever reads the counter or the flag
+                unsigned old;
+                asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.garr + un.b), "r"((unsigned)(p.upi - 1)) : "memory");
+                if (old == (unsigned)(p.upi - 1)) st_release(p.gflag + un.b, seen[k] + 1u);   // the counter has wrapped back to 0
+            }
+            return;
+        }
         if (warp == kWarps) {
-            // ---- tile producer: the staging buffer is free again once every warp has transposed its share.
-            //      With stage 1 fused this lane also performs the arrivals on the images' counters, once the
-            //      working warps have written a unit's 16 sums.
+            // ---- tile producer: the staging buffer is free again once every warp has transposed its share
             bool alive = true;
             for (long long k = 0; k < my_units; ++k) {
-                const Unit un = decode(first + k * stride, p);
-                unsigned seen = 0u;
-                if (kFused) seen = ld_acquire(p.gflag + un.b);       // before this CTA's arrival: the flag cannot have advanced yet
                 if (k >= 1 && alive) alive = mbar_wait(empty, (unsigned)((k - 1) & 1), p.ctrl, 0xB8000000u);
+                const Unit un = decode(first + k * stride, p);
                 mbar_expect_tx(full, S::STAGE_BYTES);
                 tma_load_4d(smem_u32(stage), &map_att, full, un.g * CG, un.tx * TW - P6, un.ty * TH - P6, un.b);
-                if (kFused) {
-                    if (alive) alive = mbar_wait(sumdone, (unsigned)(k & 1), p.ctrl, 0xB9000000u);
-                    // release: the 16 sums (seen through the barrier) are visible to whoever reads the counter or the flag
-                    unsigned old;
-                    asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.garr + un.b), "r"((unsigned)(p.upi - 1)) : "memory");
-                    if (old == (unsigned)(p.upi - 1)) st_release(p.gflag + un.b, seen + 1u);   // the counter has wrapped back to 0
-                }
             }
         } else if (p.copy_cc != 0) {
             // ---- copy-through of the untouched channels (same scheme as the FP32 kernel's copy warp)
@@ -261,15 +279,15 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
     }
     // Sum of the staged tile's interior per channel (the tiles' interiors partition the image; pixels outside
     // it are zero-filled), in a fixed order; 16 sums to the unit's slot, then the producer lane is told.
-    auto tile_sum = [&](const long long unit_index) {
+    auto tile_sum = [&](const long long unit_index, const unsigned char* src, const int pitch, const int origin) {
         const int gsub = lane >> 3, pr = lane & 7;           // pixel 4i + gsub of a row, channel pair pr: conflict-free
-        const uint32_t* st32 = reinterpret_cast<const uint32_t*>(stage);
+        const uint32_t* st32 = reinterpret_cast<const uint32_t*>(src) + origin * NPAIR;
         float s0 = 0.f, s1 = 0.f;
 #pragma unroll
         for (int rr = 0; rr < NA; ++rr)
 #pragma unroll
             for (int i = 0; i < TW / 4; ++i) {
-                const uint32_t v = st32[((P6 + warp * NA + rr) * SW + P6 + 4 * i + gsub) * NPAIR + pr];
+                const uint32_t v = st32[((warp * NA + rr) * pitch + 4 * i + gsub) * NPAIR + pr];
                 s0 += __uint_as_float(v << 16);
                 s1 += __uint_as_float(v & 0xffff0000u);
             }
@@ -304,12 +322,12 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
             if (sub < nsub) {
                 const float* src = p.gpart + ((size_t)un.b * p.upi + (size_t)(c / CG) * tpi) * CG + (c % CG);
                 float tsum = 0.f;
-                for (int tl = sub; tl < tpi; tl += 8 * nsub) {
-                    float v[8];
+                for (int tl = sub; tl < tpi; tl += 16 * nsub) {        // sixteen independent loads, added in order
+                    float v[16];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) v[u] = tl + u * nsub < tpi ? __ldcg(src + (size_t)(tl + u * nsub) * CG) : 0.f;
+                    for (int u = 0; u < 16; ++u) v[u] = tl + u * nsub < tpi ? __ldcg(src + (size_t)(tl + u * nsub) * CG) : 0.f;
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) tsum += v[u];
+                    for (int u = 0; u < 16; ++u) tsum += v[u];
                 }
                 f_sub[tid] = tsum;
             }
@@ -377,7 +395,15 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
 
         // ---- the NHWC tile has landed: transpose it into the 16 planes --------------------------------
         if (alive) alive = mbar_wait(full, (unsigned)(k & 1), p.ctrl, 0xA8000000u);
-        if (kFused && k == 0) tile_sum(first);               // (a second unit's tile is added up below, as soon as it can be)
+        if (kFused && k == 0) {
+            // both of this CTA's tiles are added up now, at the start, so that every image's flag advances long before
+            // any CTA needs dk: the first from the staging buffer, the second from the copy of its interior
+            tile_sum(first, stage, SW, P6 * SW + P6);
+            if (my_units > 1) {
+                if (alive) alive = mbar_wait(boxfull, 0u, p.ctrl, 0xA9000000u);
+                tile_sum(first + stride, sumbuf, TW, 0);
+            }
+        }
         {
             // a step = 16 pixels of one staged row x 16 channels: four 8x8 matrices (pixel half, channel half)
             constexpr int STEPS = ROWS * (SW / 16);
@@ -395,8 +421,13 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(empty);                   // staging may be refilled
+        if (!kFused && lane == 0) mbar_arrive(empty);        // staging may be refilled
         mma_bar();                                           // planes (and the tap table) complete
+        if (kFused && k == 0 && my_units > 1 && tid == 0) {  // every warp is past the staging buffer: the second unit's tile
+            const Unit nx = decode(first + stride, p);
+            mbar_expect_tx(full, S::STAGE_BYTES);
+            tma_load_4d(smem_u32(stage), &map_att, full, nx.g * CG, nx.tx * TW - P6, nx.ty * TH - P6, nx.b);
+        }
 
         // ---- two channels per warp --------------------------------------------------------------------
         // Per channel: 13 kernel rows of tensor-core work into acc, then the dynamic 3x3 kernel on the CUDA
@@ -497,14 +528,9 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         };
 
         if (kFused && k == 0) {
-            // first unit: all tensor-core work first, and between the two channels the sum of the second unit's tile,
-            // which has landed meanwhile: every CTA has arrived for all its tiles well before dk is needed
+            // first unit: all tensor-core work first; every CTA has arrived for all its tiles well before dk is needed
             float acc1[NB][NA][4];
             mma_all(acc, warp * 2);
-            if (my_units > 1) {
-                if (alive) alive = mbar_wait(full, 1u, p.ctrl, 0xA9000000u);
-                tile_sum(first + stride);
-            }
             mma_all(acc1, warp * 2 + 1);
             obtain_dk(un, flag0[0]);
             dk_all(dacc, warp * 2);
@@ -594,8 +620,9 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
         p.hidden = fu->hidden; p.gpart = fu->gpart; p.garr = fu->garr; p.gflag = fu->gflag;
     }
 
-    CUtensorMap m_att, m_cin, m_cout;
+    CUtensorMap m_att, m_cin, m_cout, m_box;
     if (!make_map(&m_att, x, B, C, H, W, CG, S::SW, S::ROWS, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
+    if (!make_map(&m_box, x, B, C, H, W, CG, S::TW, S::TH, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
     if (cc > 0) {
         if (!make_map(&m_cin, x, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
         if (!make_map(&m_cout, out, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
@@ -604,7 +631,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     }
     static_assert((S::STAGE_BYTES + CG * S::PLANE_BYTES + PTAB_BYTES) % 128 == 0 && (FUSED_SMEM_FLOATS * 4) % 128 == 0,
                   "the copy ring is a TMA destination: 128-byte aligned");
-    const size_t smem = (size_t)S::STAGE_BYTES + (size_t)CG * S::PLANE_BYTES + PTAB_BYTES + (kFused ? FUSED_SMEM_FLOATS * 4 : 0) +
+    const size_t smem = (size_t)S::STAGE_BYTES + (size_t)CG * S::PLANE_BYTES + PTAB_BYTES + (kFused ? FUSED_SMEM_FLOATS * 4 + S::BOX_BYTES : 0) +
                         (size_t)NSLOT * p.slot_stride + 64;   // 64: the mbarriers
     if (smem > 227 * 1024) return kNotApplicable;
     static bool attr_set[kMaxDevices] = {};
@@ -629,7 +656,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     cfg.attrs = attr;
     cfg.numAttrs = kFused ? 2 : 1;
     if (kFused && (grid > sm_count() || p.units > 2 * grid)) return kNotApplicable;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias, kFused>, m_att, m_cin, m_cout, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias, kFused>, m_att, m_cin, m_cout, m_box, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_toeplitz_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
