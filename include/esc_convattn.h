@@ -272,7 +272,7 @@ int esc_convattn_device_status(void* workspace, void* stream);
 /* Which stencil implementation the last esc_convattn_forward* / esc_convattn_stencil call on
  * this thread selected: 0 = none yet, 1 = guarded generic kernel, 2 = TMA-staged register-tiled
  * FP32 kernel, 3 = tensor-core kernel of the dense large kernel, 4 = tensor-core (banded Toeplitz)
- * kernel of the depth-wise large kernel.  For tests and benchmarks. */
+ * kernel of the depth-wise large kernel, 5 = tcgen05 kernel of the dense large kernel.  For tests and benchmarks. */
 int esc_convattn_last_path(void);
 
 /* Which arithmetic units evaluate the depth-wise 13x13 stage of Eq. 4 line 3 on NHWC bf16 tensors, for
@@ -298,6 +298,14 @@ int esc_convattn_set_stencil_engine(int engine);
  * instead of slabs: dk differs by fp32 rounding (about 1e-7 relative).  A workspace whose launch was cut short
  * must be zeroed again with esc_convattn_workspace_init before its next use.  For tests and tuning. */
 int esc_convattn_set_fused_stage1(int on);
+
+/* Which kernel evaluates the dense large kernel of Section 3.2 (esc_convattn_forward_dense / _stencil_dense /
+ * ESC_LK_DENSE) on NHWC bf16 tensors with 16 attention channels and K = 13, for later calls on this thread:
+ * 0 (default) = the tcgen05 kernel (accumulators in tensor memory, one instruction per input row and tap column
+ * with all 13 kernel rows stacked in N), 1 = the warp-level mma.sync kernel.  Both multiply exactly and accumulate
+ * in fp32; they differ in the order of the additions.  esc_convattn_last_path() reports 5 and 3.  Returns
+ * ESC_ERR_UNSUPPORTED for any other value.  For tests and comparisons. */
+int esc_convattn_set_dense_engine(int engine);
 
 /* Width in pixels of the output tile the TMA-staged kernel used in that call (FP32 kernel: 40 = 40x40
  * tiles, 64 = 64x16 tiles, chosen by the tile count's balance over the SMs; tensor-core kernel: 64 =

@@ -36,6 +36,7 @@ from .binding import (  # noqa: F401
     esc_convattn_set_tile_width,
     esc_convattn_set_stencil_engine,
     esc_convattn_set_fused_stage1,
+    esc_convattn_set_dense_engine,
     ESC_ENGINE_AUTO, ESC_ENGINE_FP32, ESC_ENGINE_TENSOR,
     esc_convattn_last_launches,
     esc_status_string,

@@ -63,12 +63,13 @@ def lib():
         L.esc_convattn_set_tile_width.argtypes = [i]
         L.esc_convattn_set_stencil_engine.argtypes = [i]
         L.esc_convattn_set_fused_stage1.argtypes = [i]
+        L.esc_convattn_set_dense_engine.argtypes = [i]
         L.esc_status_string.argtypes = [i]
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
                      "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
-                     "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_set_stencil_engine", "esc_convattn_set_fused_stage1", "esc_convattn_last_launches",
+                     "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_set_stencil_engine", "esc_convattn_set_fused_stage1", "esc_convattn_set_dense_engine", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
         _lib = L
@@ -138,6 +139,10 @@ def esc_convattn_set_tile_width(tile_width: int) -> None:
 
 
 ESC_ENGINE_AUTO, ESC_ENGINE_FP32, ESC_ENGINE_TENSOR = 0, 1, 2
+
+
+def esc_convattn_set_dense_engine(engine: int) -> None:
+    _check(lib().esc_convattn_set_dense_engine(int(engine)), "esc_convattn_set_dense_engine")
 
 
 def esc_convattn_set_fused_stage1(on: bool) -> None:

@@ -19,6 +19,7 @@
 #include "stencil_tma.cuh"
 #include "stencil_toeplitz.cuh"
 #include "stencil_dense.cuh"
+#include "stencil_dense_umma.cuh"
 #include "backward.cuh"
 
 namespace {
@@ -29,6 +30,7 @@ thread_local int g_last_tile_w = 0;
 thread_local int g_tile_policy = 0;      // 0 = by cost, else the tile width to use
 thread_local int g_engine_policy = 0;    // ESC_ENGINE_AUTO / _FP32 / _TENSOR for the depth-wise stencil
 thread_local int g_last_launches = 0;
+thread_local int g_dense_engine = 0;     // 0: tcgen05 kernel where it applies, 1: the mma.sync kernel
 thread_local bool g_fuse_stage1 = true;  // tensor-core kernel: stage 1 inside it where every CTA has at most two units
 
 int cuda_fail(cudaError_t e, const char* what) {
@@ -378,6 +380,14 @@ int launch_dense_generic_t(const Problem& p, const void* x, const void* w_dense,
 int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, const float* dk, void* out,
                          unsigned* ctrl, cudaStream_t st, bool dependent) {
     g_last_tile_w = 0;
+    if (g_dense_engine == 0) {
+        esc::CopyJob ujob = make_copy_job(p, x, out, 0, esc::tma::umma::kThreads);
+        if (ujob.blocks > (unsigned)sms_or_nominal()) ujob.blocks = (unsigned)sms_or_nominal();   // every block of that launch takes a whole SM
+        const int urc = esc::tma::umma::try_launch_dense_umma(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_dense, dk, out,
+                                                              ctrl, st, dependent, ujob, &g_last_launches, &g_last_error);
+        if (urc == ESC_OK) { g_last_path = 5; g_last_tile_w = esc::tma::umma::MW; return ESC_OK; }
+        if (urc != esc::tma::kNotApplicable) return urc;
+    }
     esc::CopyJob job = make_copy_job(p, x, out, 0, esc::tma::dense::kThreads);
     if (job.blocks > (unsigned)sms_or_nominal()) job.blocks = (unsigned)sms_or_nominal();   // every block of that launch takes a whole SM
     int rc = esc::tma::try_launch_dense(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_dense, dk, out, ctrl,
@@ -536,6 +546,11 @@ int esc_convattn_set_tile_width(int tile_width) {
 int esc_convattn_set_stencil_engine(int engine) {
     if (engine != ESC_ENGINE_AUTO && engine != ESC_ENGINE_FP32 && engine != ESC_ENGINE_TENSOR) return ESC_ERR_UNSUPPORTED;
     g_engine_policy = engine;
+    return ESC_OK;
+}
+int esc_convattn_set_dense_engine(int engine) {
+    if (engine != 0 && engine != 1) return ESC_ERR_UNSUPPORTED;
+    g_dense_engine = engine;
     return ESC_OK;
 }
 int esc_convattn_set_fused_stage1(int on) {

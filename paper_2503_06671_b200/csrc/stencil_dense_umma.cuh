@@ -1,0 +1,357 @@
+// Dense large kernel (ESC paper, Section 3.2: LK in R^{13x13x16x16}; Eq. 4 line 3 with that LK) for NHWC bf16
+// tensors with 16 attention channels on the fifth-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory):
+//
+//   out[b,n,y,x] = sum_{k,i,j} w_dense[n,k,i,j] x[b,k,y+i-6,x+j-6]  +  sum_{i,j} dk[b,n,i,j] x[b,n,y+i-1,x+j-1]
+//
+// Formulation.  One INPUT row of a 128-pixel-wide strip, shifted by a tap column j, is the A operand
+// (M = 128 pixels, K = 16 input channels) of ONE instruction whose B operand stacks all 13 kernel rows:
+// B_j[k][(12 - i) * 16 + n] = w_dense[n][k][i][j], N = 13 x 16 = 208.  Column block c of the result belongs to
+// output row (input row) - 6 + c, so the accumulators of 32 output rows live side by side in the 512 columns
+// of tensor memory (row y in columns (y mod 32) * 16 ..) and an input row is used once -- 13 instructions,
+// one per tap column -- and never again.  Per instruction 128 x 208 x 16 multiply-adds against 4 KB + 6.5 KB
+// of shared-memory operands: the tensor pipe, not shared memory, is the bound, and nothing is unfolded.
+// At the ends of a CTA's row range the instruction takes only the column blocks that exist (N = 16 .. 192).
+//
+// Operands are K-major without swizzle, where a row of 8 k-values is 16 contiguous bytes and rows are 16 bytes
+// apart, so a descriptor may start at ANY pixel: the staged row keeps the two channel halves apart
+// ([half][pixel][8 channels], two TMA loads per row with zero fill = the padding) and the tap column j is a
+// shift of the descriptor's start address by 16 * j bytes.
+//
+// Roles (192 threads, one CTA per SM, each CTA one range of rows of one strip):
+//   warp 0   lane 0 requests input rows by TMA into a ring of 16; the warp allocates and frees tensor memory
+//   warp 1   lane 0 issues the instructions and commits them to mbarriers (ring slot consumed / output row complete)
+//   warps 2-5  epilogue: tcgen05.ld of a finished row (one pixel per thread, 16 channels), the dynamic 3x3
+//            kernel in fp32 on the CUDA cores from the same ring, one rounding to bf16, 32-byte store;
+//            the row's columns are cleared for their next user.
+// The identity channels are copied by extra blocks at the end of the same grid.
+#pragma once
+#include "stencil_generic.cuh"
+#include "stencil_tma.cuh"
+
+namespace esc { namespace tma { namespace umma {
+
+constexpr int MW = 128;                       // output pixels per strip row = M of the instruction
+constexpr int SPX = 144;                      // staged pixels per row: 128 + 12, padded to keep half-rows 128-byte aligned
+constexpr int HALF_BYTES = SPX * 16;          // one row, one channel half
+constexpr int ROW_BYTES = 2 * HALF_BYTES;
+constexpr int NRING = 16;                     // input rows in flight / kept for the 3x3 part
+constexpr int NBLK = K13;                     // column blocks of 16 (kernel rows) in a B operand
+constexpr int BHALF_BYTES = NBLK * CG * 16;   // 3,328: one tap column, one channel half: [208 rows][8 k]
+constexpr int BJ_BYTES = 2 * BHALF_BYTES;
+constexpr int B_BYTES = K13 * BJ_BYTES;       // 86,528
+constexpr int SLOTS = 32;                     // output rows whose accumulators fit tensor memory (512 columns)
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr unsigned kPollLimit = 1u << 22;
+constexpr size_t kSmemBytes = (size_t)NRING * ROW_BYTES + B_BYTES + 1024 /* dk, progress, tmem base */ + (2 * NRING + SLOTS) * 8 + 64;
+static_assert(HALF_BYTES % 128 == 0, "TMA destinations are 128-byte aligned");
+
+struct Params {
+    int B, C, H, W;
+    int strips, segs, seg_rows;       // per image: strips of 128 pixels x row ranges of seg_rows rows
+    const __nv_bfloat16* w_dense;     // [16][16][13][13]  (output channel, input channel, row, column)
+    const float* dk;                  // [B][16][9]
+    __nv_bfloat16* out;
+    unsigned* ctrl;
+    int wait_first;
+};
+
+// Shared-memory matrix descriptor, K-major, no swizzle: 8 rows x 16 bytes are contiguous (rows 16 bytes apart),
+// the next 8 rows follow `sbo` bytes on, the second half of K (k = 8..15) `lbo` bytes on.
+__device__ __forceinline__ unsigned long long smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (unsigned long long)((addr >> 4) & 0x3FFFu) | ((unsigned long long)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((unsigned long long)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+// Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(MW >> 4) << 24);
+}
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, unsigned long long da, unsigned long long db, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 1, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_zero16(uint32_t taddr) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+                 ::"r"(taddr), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire_cta(const int* p) {
+    int v;
+    asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_cta(int* p, int v) {
+    asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    tma_load_4d(dst, map, bar, c0, c1, c2, c3);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const Params p, const CopyJob job)
+{
+    if (job.blocks != 0 && blockIdx.x >= job.first_block) {
+        if (p.wait_first) pdl_wait_primary();              // launched on its own: x may still be in the making
+        run_copy_job(job, blockIdx.x - job.first_block, threadIdx.x, kThreads);
+        return;
+    }
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char* ring = smem;                                             // [NRING][2 halves][SPX][16 bytes]
+    unsigned char* btab = smem + NRING * ROW_BYTES;                         // [13 tap columns][2 halves][208 rows][16 bytes]
+    float* dks = reinterpret_cast<float*>(btab + B_BYTES);                  // [9 taps][16 channels]
+    int* prog = reinterpret_cast<int*>(dks + 9 * CG);                       // output rows the epilogue has finished
+    int* aborted = prog + 1;
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(prog + 2);
+    u64* bars = reinterpret_cast<u64*>(btab + B_BYTES + 1024);
+    const uint32_t rowfull0 = smem_u32(bars), rowdone0 = rowfull0 + 8 * NRING, accfull0 = rowdone0 + 8 * NRING;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < NRING; ++s) { mbar_init(rowfull0 + 8 * s, 1); mbar_init(rowdone0 + 8 * s, 1); }
+        for (int s = 0; s < SLOTS; ++s) mbar_init(accfull0 + 8 * s, 1);
+        *prog = 0; *aborted = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {                                        // all 512 columns of this SM's tensor memory (one CTA per SM)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_base_slot;
+    if (p.wait_first) pdl_wait_primary();
+    pdl_launch_dependents();
+
+    // ---- this CTA's rows: image b, strip sx, rows [ya, yb) -------------------------------------------
+    unsigned u = blockIdx.x;
+    const int seg = (int)(u % (unsigned)p.segs); u /= (unsigned)p.segs;
+    const int sx = (int)(u % (unsigned)p.strips);
+    const int b = (int)(u / (unsigned)p.strips);
+    const int ya = seg * p.seg_rows, yb = min(p.H, ya + p.seg_rows), L = yb - ya;
+    const int x0 = sx * MW;
+    const int n_in = L + K13 - 1;                           // input rows ya - 6 .. yb + 5, index n = row - (ya - 6)
+
+    // ---- B operands: btab[j][half][(12 - i) * 16 + n][k % 8] = w_dense[n][half * 8 + k % 8][i][j] ------------
+    {
+        const unsigned short* w = reinterpret_cast<const unsigned short*>(p.w_dense);
+        uint4* bt = reinterpret_cast<uint4*>(btab);
+        for (int e = tid; e < K13 * 2 * NBLK * CG; e += kThreads) {          // one 16-byte row each
+            const int row = e % (NBLK * CG), h = (e / (NBLK * CG)) & 1, j = e / (2 * NBLK * CG);
+            const int i = (K13 - 1) - row / CG, n = row % CG;
+            unsigned v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = __ldg(w + ((size_t)(n * CG + h * 8 + q) * K13 + i) * K13 + j);
+            bt[e] = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
+        }
+    }
+    // clear the accumulators: every instruction accumulates, a row's columns are cleared again after it is read
+    if (warp >= 2) {
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        for (int s = 0; s < SLOTS; ++s) tmem_zero16(lane_base + (uint32_t)(s * CG));
+        tmem_wait_st();
+    }
+    fence_async_smem();                                     // the B table is read through the async proxy
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    if (warp == 0) {
+        // ======================= input rows by TMA ====================================================
+        if (lane == 0) {
+            bool alive = true;
+            for (int n = 0; n < n_in && alive; ++n) {
+                const int slot = n % NRING;
+                if (n >= NRING) {
+                    // the slot's previous row (n - 16) must have been consumed by the tensor cores and, if the 3x3
+                    // part of an output row reads it (rows n - 21 .. of this CTA's range), by the epilogue
+                    alive = mbar_wait(rowdone0 + 8 * slot, (unsigned)(((n - NRING) / NRING) & 1), p.ctrl, 0xD0000000u | (unsigned)n);
+                    const int need = min(n - 20, L);
+                    unsigned polls = 0;
+                    while (alive && ld_acquire_cta(prog) < need) {
+                        __nanosleep(64);
+                        if (++polls > kPollLimit || ld_acquire_cta(aborted)) alive = false;
+                    }
+                    if (!alive) { if (p.ctrl) { atomicExch(p.ctrl, kDevTimeout); atomicExch(p.ctrl + 1, 0xD1000000u | (unsigned)n); } st_release_cta(aborted, 1); break; }
+                }
+                const uint32_t dst = smem_u32(ring + (size_t)slot * ROW_BYTES), bar = rowfull0 + 8 * slot;
+                mbar_expect_tx(bar, ROW_BYTES);
+                tma_load_4d(dst, &map_half, bar, 0, x0 - P6, ya - P6 + n, b);
+                tma_load_4d(dst + HALF_BYTES, &map_half, bar, 8, x0 - P6, ya - P6 + n, b);
+            }
+        }
+    } else if (warp == 1) {
+        // ======================= tensor-core instructions =============================================
+        if (lane == 0) {
+            bool alive = true;
+            const uint32_t ring_a = smem_u32(ring), btab_a = smem_u32(btab);
+            for (int n = 0; n < n_in && alive; ++n) {
+                const int slot = n % NRING;
+                alive = mbar_wait(rowfull0 + 8 * slot, (unsigned)((n / NRING) & 1), p.ctrl, 0xD2000000u | (unsigned)n);
+                // the columns of the output row this input row opens (n, if it exists) were cleared by the epilogue of row n - 32
+                if (n >= SLOTS && n < L) {
+                    unsigned polls = 0;
+                    while (alive && ld_acquire_cta(prog) < n - SLOTS + 1) {
+                        __nanosleep(64);
+                        if (++polls > kPollLimit || ld_acquire_cta(aborted)) alive = false;
+                    }
+                }
+                if (!alive) { if (p.ctrl) { atomicExch(p.ctrl, kDevTimeout); atomicExch(p.ctrl + 1, 0xD3000000u | (unsigned)n); } st_release_cta(aborted, 1); break; }
+                tc_fence_after();
+                // input row n feeds output rows n - 12 + c, c = 0 .. 12 (kernel row 12 - c), those inside [0, L)
+                const int c_lo = max(0, (K13 - 1) - n), c_hi = min(K13 - 1, L - 1 - n + (K13 - 1));
+                if (c_lo <= c_hi) {
+                    const int cnt = c_hi - c_lo + 1, s0 = (n - (K13 - 1) + c_lo) % SLOTS;
+                    const int cnt1 = min(cnt, SLOTS - s0), cnt2 = cnt - cnt1;      // the row slots wrap around at 32
+                    for (int j = 0; j < K13; ++j) {
+                        const unsigned long long da = smem_desc(ring_a + (uint32_t)(slot * ROW_BYTES + 16 * j), HALF_BYTES, 128);
+                        const uint32_t bj = btab_a + (uint32_t)(j * BJ_BYTES + c_lo * CG * 16);
+                        mma_f16(tmem + (uint32_t)(s0 * CG), da, smem_desc(bj, BHALF_BYTES, 128), instr_desc(cnt1 * CG));
+                        if (cnt2 > 0)
+                            mma_f16(tmem, da, smem_desc(bj + (uint32_t)(cnt1 * CG * 16), BHALF_BYTES, 128), instr_desc(cnt2 * CG));
+                    }
+                }
+                mma_commit(rowdone0 + 8 * slot);                           // arrives when the instructions above have read the row
+                if (n >= K13 - 1) mma_commit(accfull0 + 8 * ((n - (K13 - 1)) % SLOTS));   // output row n - 12 is complete
+            }
+        }
+    } else {
+        // ======================= epilogue: one pixel per thread =======================================
+        const int et = tid - 64, m = ((warp & 3) * 32) + lane;              // tensor-memory lane = pixel of the strip row
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        if (!p.wait_first) pdl_wait_primary();                               // dk comes from the kernel before this one
+        for (int e = et; e < 9 * CG; e += kEpiThreads) dks[e] = __ldcg(p.dk + ((size_t)b * CG + (e % CG)) * 9 + e / CG);
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        bool alive = true;
+        const int x = x0 + m;
+        for (int yr = 0; yr < L; ++yr) {
+            const int slot = yr % SLOTS;
+            if (alive) alive = mbar_wait(accfull0 + 8 * slot, (unsigned)((yr / SLOTS) & 1), p.ctrl, 0xD4000000u | (unsigned)yr);
+            if (!alive) st_release_cta(aborted, 1);
+            tc_fence_after();
+            uint32_t r[16];
+            tmem_ld16(lane_base + (uint32_t)(slot * CG), r);
+            tmem_zero16(lane_base + (uint32_t)(slot * CG));
+            float acc[CG];
+#pragma unroll
+            for (int c = 0; c < CG; ++c) acc[c] = __uint_as_float(r[c]);
+            // dynamic 3x3 kernel, depth-wise, fp32 (Eq. 4 line 3, second term): input rows yr + 5 .. yr + 7 of the ring,
+            // pixels m + 5 .. m + 7 of the staged row
+#pragma unroll
+            for (int a = 0; a < 3; ++a) {
+                const unsigned char* rowp = ring + (size_t)((yr + 5 + a) % NRING) * ROW_BYTES;
+#pragma unroll
+                for (int bb = 0; bb < 3; ++bb) {
+                    const uint4 lo = *reinterpret_cast<const uint4*>(rowp + (size_t)(m + 5 + bb) * 16);
+                    const uint4 hi = *reinterpret_cast<const uint4*>(rowp + HALF_BYTES + (size_t)(m + 5 + bb) * 16);
+                    float f[16];
+                    unpack16<__nv_bfloat16>(lo, f);
+                    unpack16<__nv_bfloat16>(hi, f + 8);
+                    const float4* d4 = reinterpret_cast<const float4*>(dks + (a * 3 + bb) * CG);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 d = d4[q];
+                        acc[4 * q] = fmaf(d.x, f[4 * q], acc[4 * q]);
+                        acc[4 * q + 1] = fmaf(d.y, f[4 * q + 1], acc[4 * q + 1]);
+                        acc[4 * q + 2] = fmaf(d.z, f[4 * q + 2], acc[4 * q + 2]);
+                        acc[4 * q + 3] = fmaf(d.w, f[4 * q + 3], acc[4 * q + 3]);
+                    }
+                }
+            }
+            if (x < p.W) {
+                uint32_t o[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[2 * q], acc[2 * q + 1]);
+                    o[q] = *reinterpret_cast<const uint32_t*>(&h2);
+                }
+                uint4* dst = reinterpret_cast<uint4*>(p.out + (((size_t)b * p.H + ya + yr) * p.W + x) * p.C);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+            tmem_wait_st();                                                   // the row's columns are cleared
+            tc_fence_before();
+            asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+            if (et == 0) st_release_cta(prog, yr + 1);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+// [B][H][W][C] bf16 as a 4-D map {C, W, H, B} with a box of 8 channels x SPX pixels x 1 row.
+inline int try_launch_dense_umma(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
+                                 const void* w_dense, const float* dk, void* out, unsigned* ctrl, cudaStream_t st,
+                                 bool dependent, CopyJob job, int* launches, std::string* err) {
+    if (K != K13 || dtype != 1 /*bf16*/ || layout != kNHWC || Ca != CG || C % 8 != 0) return kNotApplicable;
+    if ((reinterpret_cast<uintptr_t>(w_dense) & 1) != 0) return kNotApplicable;
+    const int sms = sm_count();
+    if (sms <= 0) return kNotApplicable;
+    Params p;
+    p.B = B; p.C = C; p.H = H; p.W = W;
+    p.strips = (W + MW - 1) / MW;
+    // row ranges: about one CTA per SM, at least 8 rows each (12 more are read above and below a range)
+    long long want = (long long)sms / ((long long)B * p.strips);
+    if (want < 1) want = 1;
+    int rows = (int)((H + want - 1) / want);
+    if (rows < 8) rows = H < 8 ? H : 8;
+    p.seg_rows = rows;
+    p.segs = (H + rows - 1) / rows;
+    const long long ctas = (long long)B * p.strips * p.segs;
+    if (ctas > 0x3fffffffLL) return kNotApplicable;
+    p.w_dense = static_cast<const __nv_bfloat16*>(w_dense);
+    p.dk = dk; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
+    p.wait_first = dependent ? 0 : 1;
+    CUtensorMap m_half;
+    if (!make_map(&m_half, x, B, C, H, W, 8, SPX, 1, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
+    static bool attr_set[kMaxDevices] = {};
+    const int dev = current_device();
+    if (dev < 0) return kNotApplicable;
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(stencil_dense_umma_nhwc_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
+        attr_set[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    if (job.blocks != 0) job.first_block = (unsigned)ctas;
+    cfg.gridDim = dim3((unsigned)ctas + job.blocks);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_dense_umma_nhwc_bf16, m_half, p, job);
+    if (e != cudaSuccess) {
+        char buf[256];
+        snprintf(buf, sizeof buf, "stencil_dense_umma_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
+        *err = buf;
+        return 7;  // ESC_ERR_CUDA
+    }
+    ++*launches;
+    return 0;
+}
+
+}}}  // namespace esc::tma::umma

@@ -48,6 +48,10 @@ TENSOR_SHAPES = [
     (1, 64, 16, 150, 1),      # single column
     (40, 32, 16, 40, 40),     # 120 tiles: one per CTA, many images
     (1, 64, 16, 360, 640),    # 230 tiles of 64x16: two per CTA on 148 SMs (the benchmark's launch)
+    (1, 64, 16, 700, 130),    # tcgen05 kernel: two strips of 128 pixels (the second two pixels wide), 70 row ranges of 10 rows
+    (60, 32, 16, 100, 40),    # tcgen05 kernel: row ranges of 50 rows -- the 32 row slots of tensor memory and the ring of 16 input
+                              # rows are re-used inside a CTA, the issuing thread waits for the epilogue's progress
+    (150, 16, 16, 70, 20),    # more images than SMs: one CTA per image, 70 rows each (two wraps of the row slots)
     (50, 32, 16, 96, 128),    # 600 tiles: four or five per CTA -- both buffers re-used, the barrier phase wraps,
                               # the image (and its dk) changes inside a CTA's walk
 ]
@@ -55,7 +59,10 @@ TENSOR_SHAPES = [
 
 @pytest.mark.parametrize("shape", TENSOR_SHAPES, ids=lambda s: "x".join(map(str, s)))
 @pytest.mark.parametrize("forward", [True, False], ids=["forward", "stencil"])
-def test_dense_tensor_core_kernel(pkg, oracle, shape, forward):
+@pytest.mark.parametrize("engine", [0, 1], ids=["tcgen05", "mma_sync"])
+def test_dense_tensor_core_kernel(pkg, oracle, shape, forward, engine):
+    """Both tensor-core kernels of the dense large kernel (tcgen05 with accumulators in tensor memory, path 5;
+    warp-level mma.sync, path 3) on every shape, every output compared with the oracle."""
     import torch
 
     B, C, C_a, H, W = shape
@@ -69,15 +76,19 @@ def test_dense_tensor_core_kernel(pkg, oracle, shape, forward):
     buf = torch.full((n + 2048,), 7.0, dtype=x.dtype, device="cuda")
     out = buf[1024:1024 + n].view(x.shape)
     ws = pkg.new_workspace(B, C_a, H, W, K)
-    for _ in range(2):                                     # twice: barriers and the ring start clean each launch
-        if forward:
-            pkg.esc_convattn_forward_dense(x, C_a, K, wd_d, wdyn, bdyn, out, pkg.ESC_NHWC, ws)
-        else:
-            dk = np.random.default_rng(7).uniform(-0.5, 0.5, size=(B, C_a, 3, 3)).astype(np.float32)
-            pkg.esc_convattn_stencil_dense(x, C_a, K, wd_d, torch.from_numpy(dk).cuda(), out, pkg.ESC_NHWC, ws)
-    torch.cuda.synchronize()
+    pkg.esc_convattn_set_dense_engine(engine)
+    try:
+        for _ in range(2):                                 # twice: barriers, rings and tensor memory start clean each launch
+            if forward:
+                pkg.esc_convattn_forward_dense(x, C_a, K, wd_d, wdyn, bdyn, out, pkg.ESC_NHWC, ws)
+            else:
+                dk = np.random.default_rng(7).uniform(-0.5, 0.5, size=(B, C_a, 3, 3)).astype(np.float32)
+                pkg.esc_convattn_stencil_dense(x, C_a, K, wd_d, torch.from_numpy(dk).cuda(), out, pkg.ESC_NHWC, ws)
+        torch.cuda.synchronize()
+    finally:
+        pkg.esc_convattn_set_dense_engine(0)
     assert pkg.esc_convattn_device_status(ws) == 0
-    assert pkg.esc_convattn_last_path() == 3
+    assert pkg.esc_convattn_last_path() == (5 if engine == 0 else 3)
     assert bool((buf[:1024] == 7.0).all()) and bool((buf[1024 + n:] == 7.0).all()), "write outside out"
     if forward:
         ref, mag = oracle.forward_dense(d["x"], C_a, wd, d["w_dyn"], d["b_dyn"], want_mag=True)
@@ -112,7 +123,7 @@ def test_dense_every_type_and_layout(pkg, oracle, shape, dtype, layout):
     torch.cuda.synchronize()
     assert pkg.esc_convattn_device_status(ws) == 0
     fast = dtype == synth.BF16 and layout == synth.NHWC and K == 13 and C_a == 16
-    assert pkg.esc_convattn_last_path() == (3 if fast else 1)
+    assert pkg.esc_convattn_last_path() == (5 if fast else 1)
     ref, mag = oracle.forward_dense(d["x"], C_a, wd, d["w_dyn"], d["b_dyn"], want_mag=True)
     _check(util.to_host_nchw(out, layout), ref, mag, dtype, C_a, f"dense {shape} {dtype} {layout}")
 

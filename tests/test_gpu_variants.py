@@ -71,7 +71,7 @@ def test_model_variants(pkg, oracle, variant, dtype, layout):
         fast_pw = kind == "decomposed" and pkg.esc_convattn_last_path() == 2
         bar = 2.0 ** -8 * np.abs(ref[:, :C_a]) * 1.001 + (2.0 ** -8 * mag if fast_pw else 0.0) \
             + (5e-5 if kind == "dense" else 1e-5) * mag + 1e-30
-        assert pkg.esc_convattn_last_path() == (3 if kind == "dense" else 2 if kind == "decomposed" else 4)
+        assert pkg.esc_convattn_last_path() == (5 if kind == "dense" else 2 if kind == "decomposed" else 4)
     assert (err <= bar).all(), f"{variant[0]}: {int((err > bar).sum())} outputs beyond the bound"
     assert np.array_equal(got[:, C_a:], ref[:, C_a:])
 
