@@ -381,10 +381,8 @@ int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, c
                          unsigned* ctrl, cudaStream_t st, bool dependent) {
     g_last_tile_w = 0;
     if (g_dense_engine == 0) {
-        esc::CopyJob ujob = make_copy_job(p, x, out, 0, esc::tma::umma::kThreads);
-        if (ujob.blocks > (unsigned)sms_or_nominal()) ujob.blocks = (unsigned)sms_or_nominal();   // every block of that launch takes a whole SM
         const int urc = esc::tma::umma::try_launch_dense_umma(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_dense, dk, out,
-                                                              ctrl, st, dependent, ujob, &g_last_launches, &g_last_error);
+                                                              ctrl, st, dependent, &g_last_launches, &g_last_error);
         if (urc == ESC_OK) { g_last_path = 5; g_last_tile_w = esc::tma::umma::MW; return ESC_OK; }
         if (urc != esc::tma::kNotApplicable) return urc;
     }

@@ -18,13 +18,13 @@
 // ([half][pixel][8 channels], two TMA loads per row with zero fill = the padding) and the tap column j is a
 // shift of the descriptor's start address by 16 * j bytes.
 //
-// Roles (192 threads, one CTA per SM, each CTA one range of rows of one strip):
+// Roles (224 threads, one CTA per SM, each CTA one range of rows of one strip):
 //   warp 0   lane 0 requests input rows by TMA into a ring of 16; the warp allocates and frees tensor memory
 //   warp 1   lane 0 issues the instructions and commits them to mbarriers (ring slot consumed / output row complete)
 //   warps 2-5  epilogue: tcgen05.ld of a finished row (one pixel per thread, 16 channels), the dynamic 3x3
 //            kernel in fp32 on the CUDA cores from the same ring, one rounding to bf16, 32-byte store;
 //            the row's columns are cleared for their next user.
-// The identity channels are copied by extra blocks at the end of the same grid.
+//   warp 6   lane 0 copies the identity channels of the CTA's rows, TMA in / TMA out through a ring of two slots.
 #pragma once
 #include "stencil_generic.cuh"
 #include "stencil_tma.cuh"
@@ -41,10 +41,15 @@ constexpr int BHALF_BYTES = NBLK * CG * 16;   // 3,328: one tap column, one chan
 constexpr int BJ_BYTES = 2 * BHALF_BYTES;
 constexpr int B_BYTES = K13 * BJ_BYTES;       // 86,528
 constexpr int SLOTS = 32;                     // output rows whose accumulators fit tensor memory (512 columns)
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;                 // producer, issuer, four epilogue warps, copy-through warp
 constexpr int kEpiThreads = 128;
+constexpr int kCopySlotBytes = 16384, kCopySlots = 2;
 constexpr unsigned kPollLimit = 1u << 22;
-constexpr size_t kSmemBytes = (size_t)NRING * ROW_BYTES + B_BYTES + 1024 /* dk, progress, tmem base */ + (2 * NRING + SLOTS) * 8 + 64;
+constexpr int kMiscBytes = 1024;               // dk, progress word, tensor-memory base
+constexpr int kBarBytes = 1024;                // 2 * NRING + SLOTS + kCopySlots mbarriers
+constexpr int kCopyRingOffset = NRING * ROW_BYTES + B_BYTES + kMiscBytes + kBarBytes;
+constexpr size_t kSmemBytes = (size_t)kCopyRingOffset + kCopySlots * kCopySlotBytes;
+static_assert((2 * NRING + SLOTS + kCopySlots) * 8 <= kBarBytes && kCopyRingOffset % 128 == 0, "barriers fit; the copy ring is a TMA destination");
 static_assert(HALF_BYTES % 128 == 0, "TMA destinations are 128-byte aligned");
 
 struct Params {
@@ -55,6 +60,8 @@ struct Params {
     __nv_bfloat16* out;
     unsigned* ctrl;
     int wait_first;
+    int w_aligned;                    // w_dense is 16-byte aligned: the B operands are built from a staged copy
+    int copy_cc, copy_pw;             // identity channels; pixels of a strip row per copy chunk (0: nothing to copy)
 };
 
 // Shared-memory matrix descriptor, K-major, no swizzle: 8 rows x 16 bytes are contiguous (rows 16 bytes apart),
@@ -103,13 +110,9 @@ __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const Params p, const CopyJob job)
+stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const __grid_constant__ CUtensorMap map_cin,
+                             const __grid_constant__ CUtensorMap map_cout, const Params p)
 {
-    if (job.blocks != 0 && blockIdx.x >= job.first_block) {
-        if (p.wait_first) pdl_wait_primary();              // launched on its own: x may still be in the making
-        run_copy_job(job, blockIdx.x - job.first_block, threadIdx.x, kThreads);
-        return;
-    }
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* ring = smem;                                             // [NRING][2 halves][SPX][16 bytes]
     unsigned char* btab = smem + NRING * ROW_BYTES;                         // [13 tap columns][2 halves][208 rows][16 bytes]
@@ -118,12 +121,15 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
     int* aborted = prog + 1;
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(prog + 2);
     u64* bars = reinterpret_cast<u64*>(btab + B_BYTES + 1024);
-    const uint32_t rowfull0 = smem_u32(bars), rowdone0 = rowfull0 + 8 * NRING, accfull0 = rowdone0 + 8 * NRING;
+    const uint32_t rowfull0 = smem_u32(bars), rowdone0 = rowfull0 + 8 * NRING, accfull0 = rowdone0 + 8 * NRING,
+                   cfull0 = accfull0 + 8 * SLOTS;
+    unsigned char* cring = smem + kCopyRingOffset;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < NRING; ++s) { mbar_init(rowfull0 + 8 * s, 1); mbar_init(rowdone0 + 8 * s, 1); }
         for (int s = 0; s < SLOTS; ++s) mbar_init(accfull0 + 8 * s, 1);
+        for (int s = 0; s < kCopySlots; ++s) mbar_init(cfull0 + 8 * s, 1);
         *prog = 0; *aborted = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -148,16 +154,34 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
     const int n_in = L + K13 - 1;                           // input rows ya - 6 .. yb + 5, index n = row - (ya - 6)
 
     // ---- B operands: btab[j][half][(12 - i) * 16 + n][k % 8] = w_dense[n][half * 8 + k % 8][i][j] ------------
+    // The weights are gathered with a stride of 169 elements.  From global memory that is 28 rounds of dependent
+    // 2-byte loads per thread; instead half of w_dense at a time (8 output channels, 43 KB) is copied, coalesced,
+    // into the still empty input ring and the rows are gathered from there.
     {
-        const unsigned short* w = reinterpret_cast<const unsigned short*>(p.w_dense);
         uint4* bt = reinterpret_cast<uint4*>(btab);
-        for (int e = tid; e < K13 * 2 * NBLK * CG; e += kThreads) {          // one 16-byte row each
-            const int row = e % (NBLK * CG), h = (e / (NBLK * CG)) & 1, j = e / (2 * NBLK * CG);
-            const int i = (K13 - 1) - row / CG, n = row % CG;
-            unsigned v[8];
+        constexpr int HALF_W = 8 * CG * K13 * K13;                              // elements of 8 output channels
+        static_assert(HALF_W * 2 <= NRING * ROW_BYTES && (HALF_W * 2) % 16 == 0, "staging fits the ring");
+        for (int nh = 0; nh < 2; ++nh) {
+            const unsigned short* w;
+            if (p.w_aligned) {
+                const uint4* src = reinterpret_cast<const uint4*>(p.w_dense + (size_t)nh * HALF_W);
+                uint4* dst = reinterpret_cast<uint4*>(ring);
+                for (int e = tid; e < HALF_W * 2 / 16; e += kThreads) dst[e] = __ldg(src + e);
+                __syncthreads();
+                w = reinterpret_cast<const unsigned short*>(ring);
+            } else {
+                w = reinterpret_cast<const unsigned short*>(p.w_dense) + (size_t)nh * HALF_W;
+            }
+            for (int e = tid; e < K13 * 2 * NBLK * 8; e += kThreads) {           // one 16-byte row each: (j, half, i, n % 8)
+                const int n8 = e & 7, ii = (e >> 3) % NBLK, h = ((e >> 3) / NBLK) & 1, j = (e >> 3) / (2 * NBLK);
+                const int i = (K13 - 1) - ii;
+                unsigned v[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = __ldg(w + ((size_t)(n * CG + h * 8 + q) * K13 + i) * K13 + j);
-            bt[e] = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
+                for (int q = 0; q < 8; ++q) v[q] = w[((size_t)(n8 * CG + h * 8 + q) * K13 + i) * K13 + j];
+                bt[(j * 2 + h) * (NBLK * CG) + ii * CG + nh * 8 + n8] =
+                    make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
+            }
+            __syncthreads();                                                     // the staging area is re-used
         }
     }
     // clear the accumulators: every instruction accumulates, a row's columns are cleared again after it is read
@@ -229,6 +253,41 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
                 mma_commit(rowdone0 + 8 * slot);                           // arrives when the instructions above have read the row
                 if (n >= K13 - 1) mma_commit(accfull0 + 8 * ((n - (K13 - 1)) % SLOTS));   // output row n - 12 is complete
             }
+        }
+    } else if (warp == 6) {
+        // ======================= copy-through of the identity channels: TMA in, TMA out ================
+        // this CTA's rows of its strip, a strip row (or a part of it) per chunk, through a ring of two slots
+        if (lane == 0 && p.copy_cc != 0) {
+            bool alive = true;
+            const int per_row = MW / p.copy_pw, chunks = L * per_row;
+            const unsigned bytes = (unsigned)(p.copy_cc * p.copy_pw * 2);
+            auto coords = [&](int ch, int& cx, int& cy) { cy = ya + ch / per_row; cx = x0 + (ch % per_row) * p.copy_pw; };
+            auto issue = [&](int ch) {
+                int cx, cy; coords(ch, cx, cy);
+                const int slot = ch % kCopySlots;
+                mbar_expect_tx(cfull0 + 8 * slot, bytes);
+                tma_load_4d(smem_u32(cring + slot * kCopySlotBytes), &map_cin, cfull0 + 8 * slot, CG, cx, cy, b);
+            };
+            // chunks wholly outside the image (right of W) are skipped by both cursors alike
+            auto inside = [&](int ch) { int cx, cy; coords(ch, cx, cy); return cx < p.W; };
+            int next = 0;
+            while (next < chunks && !inside(next)) ++next;
+            if (next < chunks) issue(next);
+            int cur = next;
+            while (cur < chunks) {
+                int nx = cur + 1;
+                while (nx < chunks && !inside(nx)) ++nx;
+                if (nx < chunks) {
+                    bulk_wait_read<0>();                                    // the store that last used the other slot has read it
+                    issue(nx);
+                }
+                if (alive) alive = mbar_wait(cfull0 + 8 * (cur % kCopySlots), (unsigned)((cur / kCopySlots) & 1), p.ctrl, 0xD6000000u | (unsigned)cur);
+                int cx, cy; coords(cur, cx, cy);
+                tma_store_4d(&map_cout, smem_u32(cring + (cur % kCopySlots) * kCopySlotBytes), CG, cx, cy, b);
+                bulk_commit();
+                cur = nx;
+            }
+            bulk_wait_all<0>();
         }
     } else {
         // ======================= epilogue: one pixel per thread =======================================
@@ -302,7 +361,7 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
 // [B][H][W][C] bf16 as a 4-D map {C, W, H, B} with a box of 8 channels x SPX pixels x 1 row.
 inline int try_launch_dense_umma(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
                                  const void* w_dense, const float* dk, void* out, unsigned* ctrl, cudaStream_t st,
-                                 bool dependent, CopyJob job, int* launches, std::string* err) {
+                                 bool dependent, int* launches, std::string* err) {
     if (K != K13 || dtype != 1 /*bf16*/ || layout != kNHWC || Ca != CG || C % 8 != 0) return kNotApplicable;
     if ((reinterpret_cast<uintptr_t>(w_dense) & 1) != 0) return kNotApplicable;
     const int sms = sm_count();
@@ -322,8 +381,24 @@ inline int try_launch_dense_umma(int B, int C, int Ca, int H, int W, int K, int 
     p.w_dense = static_cast<const __nv_bfloat16*>(w_dense);
     p.dk = dk; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
-    CUtensorMap m_half;
+    p.w_aligned = (reinterpret_cast<uintptr_t>(w_dense) & 15) == 0 ? 1 : 0;
+    const int cc = C - Ca;
+    p.copy_cc = cc; p.copy_pw = 0;
+    if (cc > 256) return kNotApplicable;
+    if (cc > 0) {
+        int pw = MW;
+        while (pw > 8 && cc * 2 * pw > kCopySlotBytes) pw >>= 1;
+        if (cc * 2 * pw > kCopySlotBytes) return kNotApplicable;
+        p.copy_pw = pw;
+    }
+    CUtensorMap m_half, m_cin, m_cout;
     if (!make_map(&m_half, x, B, C, H, W, 8, SPX, 1, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
+    if (cc > 0) {
+        if (!make_map(&m_cin, x, B, C, H, W, cc, p.copy_pw, 1)) return kNotApplicable;
+        if (!make_map(&m_cout, out, B, C, H, W, cc, p.copy_pw, 1)) return kNotApplicable;
+    } else {
+        m_cin = m_half; m_cout = m_half;
+    }
     static bool attr_set[kMaxDevices] = {};
     const int dev = current_device();
     if (dev < 0) return kNotApplicable;
@@ -333,8 +408,7 @@ inline int try_launch_dense_umma(int B, int C, int Ca, int H, int W, int K, int 
         attr_set[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
-    if (job.blocks != 0) job.first_block = (unsigned)ctas;
-    cfg.gridDim = dim3((unsigned)ctas + job.blocks);
+    cfg.gridDim = dim3((unsigned)ctas);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = st;
@@ -343,7 +417,7 @@ inline int try_launch_dense_umma(int B, int C, int Ca, int H, int W, int K, int 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_dense_umma_nhwc_bf16, m_half, p, job);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_dense_umma_nhwc_bf16, m_half, m_cin, m_cout, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_dense_umma_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
