@@ -18,6 +18,8 @@ from .convattn_oracle import (  # noqa: F401
     stencil_pw,
     forward_pw,
     points,
+    fuse,
+    forward_fused,
     set_threads,
     max_threads,
 )

@@ -282,3 +282,34 @@ def points(x, C_a, w_large, w_dyn, b_dyn, flat_idx, want_mag=False):
         idx.ctypes.data_as(_i64p), vals.ctypes.data_as(_f64p), mags.ctypes.data_as(_f64p),
     )
     return (vals, mags) if want_mag else vals
+
+
+def fuse(cat, w_fuse, b_fuse=None, residual=None, want_mag=False):
+    """Conv_fuse (1x1 over all C channels, Eq. 4 line 4) of a concatenated map cat[B,C,H,W] (fp64), plus bias and the
+    block's residual (Eq. 3 line 3) when given."""
+    cat = np.ascontiguousarray(cat, dtype=np.float64)
+    B, C, H, W = cat.shape
+    w_fuse, wp = _f64(w_fuse)
+    assert w_fuse.shape == (C, C)
+    bp = None
+    if b_fuse is not None:
+        b_fuse, bp = _f64(b_fuse)
+        assert b_fuse.shape == (C,)
+    rp = None
+    if residual is not None:
+        residual, rp = _f32(residual)
+        assert residual.shape == cat.shape
+    out = np.empty_like(cat)
+    mag = np.empty_like(cat) if want_mag else None
+    _load().convattn_ref_fuse(cat.ctypes.data_as(_f64p), B, C, H, W, wp, bp, rp, out.ctypes.data_as(_f64p),
+                              mag.ctypes.data_as(_f64p) if want_mag else None)
+    return (out, mag) if want_mag else out
+
+
+def forward_fused(x, C_a, w_large, w_dyn, b_dyn, w_fuse, b_fuse=None, residual=None, want_mag=False, want_cat=False):
+    """The whole module of Eq. 4 including its last line: ConvAttn stages, then Conv_fuse (+ residual)."""
+    cat = forward(x, C_a, w_large, w_dyn, b_dyn)
+    res = fuse(cat, w_fuse, b_fuse, residual, want_mag=want_mag)
+    if want_cat:
+        return (*res, cat) if want_mag else (res, cat)
+    return res

@@ -28,6 +28,9 @@
  * convattn_ref_stencil_dense is Eq. 4 line 3 with the dense large kernel of Section 3.2
  * (13x13x16x16: every output channel sums over all attention input channels).
  *
+ * convattn_ref_fuse is the module's last step, Conv_fuse over the concatenated channels (Eq. 4 line 4),
+ * with the block's residual connection (Eq. 3 line 3).
+ *
  * convattn_ref_backward is the gradient of the first form above with respect to x, LK, W_dyn and
  * b_dyn, by the chain rule written out.
  *
@@ -188,6 +191,35 @@ void convattn_ref_forward(const float *x, int B, int C, int C_a, int H, int W, i
     convattn_ref_gap(x, B, C, C_a, H, W, g_out);
     convattn_ref_dynkernel(g_out, B, C_a, w_dyn, b_dyn, dk_out);
     convattn_ref_stencil(x, B, C, C_a, H, W, K, w_large, dk_out, 0, H, out, mag);
+}
+
+/* The module's last step (Eq. 4 line 4): F_fuse = Conv_fuse(Concat(F_res, F_idt)), a 1x1 convolution over all C
+ * channels of the concatenated map `cat` [B,C,H,W] (the output of the stages above), with bias, and the residual
+ * connection of the ESC block around the module (Eq. 3 line 3: F_{i,j} = F_{i,j-1} + ConvAttn(...)):
+ *   out[b,n,y,x] = b_fuse[n] + sum_c w_fuse[n,c] * cat[b,c,y,x]  ( + residual[b,n,y,x] )
+ * b_fuse and residual may be NULL.  mag (optional) [B,C,H,W] receives |b_fuse[n]| + sum_c |w_fuse[n,c] * cat| + |residual|. */
+void convattn_ref_fuse(const double *cat, int B, int C, int H, int W, const double *w_fuse, const double *b_fuse,
+                       const float *residual, double *out, double *mag)
+{
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < C; ++n)
+            for (int y = 0; y < H; ++y)
+                for (int xx = 0; xx < W; ++xx) {
+                    double s = b_fuse ? b_fuse[n] : 0.0, m = fabs(s);
+                    for (int c = 0; c < C; ++c) {
+                        double t = w_fuse[(size_t)n * C + c] * cat[IDX4(b, c, y, xx, C, H, W)];
+                        s += t;
+                        m += fabs(t);
+                    }
+                    if (residual) {
+                        double r = (double)residual[IDX4(b, n, y, xx, C, H, W)];
+                        s += r;
+                        m += fabs(r);
+                    }
+                    out[IDX4(b, n, y, xx, C, H, W)] = s;
+                    if (mag) mag[IDX4(b, n, y, xx, C, H, W)] = m;
+                }
 }
 
 /* Point-wise large-kernel filter LK^c of the decomposed form (Eq. 5, first factor F_att (*) LK^c):

@@ -152,6 +152,13 @@ def make_pointwise(C_a, dtype=F32, seed=0):
     return round_to(w, dtype)
 
 
+def make_fuse(C, dtype=F32, seed=0):
+    """w_fuse [C,C] (row = output channel) and b_fuse [C] of the module's closing 1x1 convolution, kaiming-uniform
+    with fan_in C, float32 rounded to `dtype`."""
+    rng = np.random.default_rng(11000027 * (seed + 1) + C)
+    return {"w_fuse": round_to(_kaiming_uniform(rng, (C, C), C), dtype), "b_fuse": round_to(_kaiming_uniform(rng, (C,), C), dtype)}
+
+
 def make_dense_kernel(C_a, K=13, dtype=F32, seed=0):
     """w_dense [C_a,C_a,K,K] (output channel, input channel, row, column): the dense large kernel of the main
     model, kaiming-uniform with fan_in C_a*K*K, float32 rounded to `dtype`."""
