@@ -245,6 +245,26 @@ int esc_convattn_forward_variant(const void* x, int B, int C, int C_a, int H, in
                                  void* out, int dtype, int layout,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
+/* The whole module including its last step (Section 3.3, Eq. 4 lines 1-4) and the residual connection of the ESC
+ * block around it (Eq. 3 line 3), for the depth-wise large kernel with the one-layer estimator:
+ *   cat = esc_convattn_forward_ex(x)                                   (F_res | F_idt)
+ *   out[b,n,y,x] = b_fuse[n] + sum_c w_fuse[n,c] * cat[b,c,y,x]  ( + residual[b,n,y,x] )
+ *   w_fuse     [C,C]        same dtype as x, row = output channel (Conv_fuse, 1x1)
+ *   b_fuse     [C]          same dtype, may be NULL
+ *   residual   [B,C,H,W]    same dtype and layout as x, 16-byte aligned, may be NULL, may be x itself; must not overlap out
+ * Everything else as for esc_convattn_forward_ex.  Asynchronous on `stream`.
+ * NHWC bf16 with C in {32, 48, 64, 96, 128}, C_a a multiple of 16, K = 13 and 16-byte aligned w_fuse: the stencil kernel
+ * writes only the attention channels, and a tensor-core 1x1 kernel reads them back together with the identity channels
+ * straight from x -- the concatenation is never copied (2 or 3 launches).  F_res passes through out as bf16 there, so it
+ * is rounded once before Conv_fuse, as it would be between two layers of a bf16 network; all sums are fp32 and the result
+ * is rounded once.  Every other configuration runs esc_convattn_forward_ex into out and a guarded 1x1 kernel in place
+ * (C * 128 bytes of shared memory per block: ESC_ERR_UNSUPPORTED beyond C = 384). */
+int esc_convattn_forward_fused(const void* x, int B, int C, int C_a, int H, int W, int K,
+                               const void* w_large, const void* w_dyn, const void* b_dyn,
+                               const void* w_fuse, const void* b_fuse, const void* residual,
+                               void* out, int dtype, int layout,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
 /*
  * Backward pass of esc_convattn_forward_ex (one-layer estimator, depth-wise LK; the chain rule applied to
  * Eq. 4): given grad_out = dL/dout, writes

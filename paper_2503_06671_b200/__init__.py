@@ -28,6 +28,7 @@ from .binding import (  # noqa: F401
     esc_convattn_backward_workspace_bytes,
     new_backward_workspace,
     esc_convattn_forward_mlp,
+    esc_convattn_forward_fused,
     esc_convattn_forward_pw,
     esc_convattn_stencil_pw,
     esc_convattn_dynkernel_mlp,

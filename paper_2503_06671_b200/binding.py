@@ -40,6 +40,7 @@ def lib():
         vp, i, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
         L.esc_convattn_forward.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp]
         L.esc_convattn_forward_ex.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_forward_fused.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_workspace_bytes.argtypes = [i, i, i, i, i]
         L.esc_convattn_workspace_bytes.restype = sz
         L.esc_convattn_workspace_init.argtypes = [vp, sz, vp]
@@ -67,7 +68,7 @@ def lib():
         L.esc_status_string.argtypes = [i]
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
-        for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_workspace_init",
+        for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_forward_fused", "esc_convattn_workspace_init",
                      "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_set_stencil_engine", "esc_convattn_set_fused_stage1", "esc_convattn_set_dense_engine", "esc_convattn_last_launches",
                      "esc_version"):
@@ -192,6 +193,15 @@ def esc_convattn_forward_ex(x, C_a, K, w_large, w_dyn, b_dyn, out, layout, works
                                          _ptr(out), _dtype_code(x), layout, _ptr(workspace),
                                          workspace.numel() * workspace.element_size(), _stream(stream)),
            "esc_convattn_forward_ex")
+    return out
+
+
+def esc_convattn_forward_fused(x, C_a, K, w_large, w_dyn, b_dyn, w_fuse, b_fuse, residual, out, layout, workspace, stream=None):
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_forward_fused(_ptr(x), B, C, C_a, H, W, K, _ptr(w_large), _ptr(w_dyn), _ptr(b_dyn), _ptr(w_fuse),
+                                            _ptr(b_fuse), _ptr(residual), _ptr(out), _dtype_code(x), layout, _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_forward_fused")
     return out
 
 

@@ -21,6 +21,7 @@
 #include "stencil_dense.cuh"
 #include "stencil_dense_umma.cuh"
 #include "backward.cuh"
+#include "conv_fuse.cuh"
 
 namespace {
 
@@ -52,6 +53,7 @@ struct Problem {
     const void* w_point = nullptr;   // [Ca][Ca] point-wise filter LK^c of the decomposed form (Eq. 5), or none
     bool dense = false;              // w_large is the dense kernel [Ca][Ca][K][K] of Section 3.2
     const float* bias = nullptr;     // [B][Ca] constant per (image, channel) added to the attention outputs (backward pass)
+    bool skip_copy = false;          // the identity channels are not written (the fused 1x1 convolution reads them from x)
     size_t es() const { return elem_size(dtype); }
     size_t elems() const { return (size_t)B * C * H * W; }
 };
@@ -314,10 +316,11 @@ int launch_stencil(const Problem& p, const void* x, const void* w_large, const f
     if (!p.w_point && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0) {
         int tw = 0;
         const int rc = esc::tma::toep::try_launch_toeplitz(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, p.bias,
-                                                           out, ctrl, st, dependent, &g_last_launches, &g_last_error, &tw);
+                                                           out, ctrl, st, dependent, &g_last_launches, &g_last_error, &tw, p.skip_copy);
         if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
         if (rc != esc::tma::kNotApplicable) return rc;
     }
+    if (p.skip_copy) return ESC_ERR_UNSUPPORTED;           // only the tensor-core kernel can leave the identity channels out
     if (g_engine_policy == ESC_ENGINE_TENSOR) return launch_generic(p, x, w_large, dk, out, st, dependent);
     int tile_w = g_tile_policy;
     int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, p.w_point, dk, p.bias, out,
@@ -415,7 +418,7 @@ int forward_impl(const Problem& p, const void* x, const void* w_large, const Est
         const esc::tma::toep::Fused fu{est.w_last, est.b_last, est.w_down, est.b_down, est.hidden, w.unit_sums, w.arrivals, w.flags};
         int tw = 0;
         const int rc = esc::tma::toep::try_launch_fused(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, fu, out,
-                                                        w.ctrl, st, &g_last_launches, &g_last_error, &tw);
+                                                        w.ctrl, st, &g_last_launches, &g_last_error, &tw, p.skip_copy);
         if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
         if (rc != esc::tma::kNotApplicable) {
             // a cooperative launch can be refused (SMs held by another context): fall back to two kernels
@@ -824,6 +827,61 @@ int esc_convattn_forward_variant(const void* x, int B, int C, int C_a, int H, in
     if (large_kernel == ESC_LK_DECOMPOSED) p.w_point = w_point;
     p.dense = large_kernel == ESC_LK_DENSE;
     return forward_impl(p, x, w_large, est, out, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int esc_convattn_forward_fused(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                               const void* w_dyn, const void* b_dyn, const void* w_fuse, const void* b_fuse,
+                               const void* residual, void* out, int dtype, int layout, void* workspace,
+                               size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    Problem p{B, C, C_a, H, W, K, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!w_large || !w_dyn || !b_dyn || !w_fuse) return ESC_ERR_NULL;
+    rc = check_tensors(p, x, out);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(w_large, p.es()) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es()) || !aligned(w_fuse, p.es()) ||
+        (b_fuse && !aligned(b_fuse, p.es())))
+        return ESC_ERR_ALIGN;
+    if (residual) {
+        if (!aligned(residual, 16)) return ESC_ERR_ALIGN;
+        const uintptr_t ra = reinterpret_cast<uintptr_t>(residual), oa = reinterpret_cast<uintptr_t>(out);
+        const size_t bytes = p.elems() * p.es();
+        if (ra < oa + bytes && oa < ra + bytes) return ESC_ERR_ALIAS;        // out is rewritten pixel block by pixel block
+    }
+    rc = check_workspace(p, workspace, workspace_bytes_);
+    if (rc != ESC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Estimator est{w_dyn, b_dyn, nullptr, nullptr, 0};
+    const long long pixels = (long long)B * H * W;
+    // Fast path: the tensor-core stencil writes only the attention channels; the 1x1 kernel takes the identity
+    // channels straight from x, so they are never copied.
+    if (esc::fuse::fast_applies(C, C_a, dtype, layout) && aligned(w_fuse, 16) && tensor_stencil_follows(p)) {
+        p.skip_copy = true;
+        rc = forward_impl(p, x, w_large, est, out, workspace, st);
+        if (rc != ESC_OK) return rc;
+        esc::fuse::Params fp;
+        fp.att = static_cast<const __nv_bfloat16*>(out); fp.idt = static_cast<const __nv_bfloat16*>(x);
+        fp.w = static_cast<const __nv_bfloat16*>(w_fuse); fp.bias = static_cast<const __nv_bfloat16*>(b_fuse);
+        fp.residual = static_cast<const __nv_bfloat16*>(residual); fp.out = static_cast<__nv_bfloat16*>(out);
+        fp.pixels = pixels; fp.C = C; fp.Ca = C_a;
+        ESC_CUDA(esc::fuse::launch_fast(fp, st));
+        ++g_last_launches;
+        return ESC_OK;
+    }
+    rc = forward_impl(p, x, w_large, est, out, workspace, st);
+    if (rc != ESC_OK) return rc;
+    const size_t smem = (size_t)esc::fuse::kGenPix * C * sizeof(float);
+    if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
+    const unsigned blocks = (unsigned)((pixels + esc::fuse::kGenPix - 1) / esc::fuse::kGenPix);
+#define ESC_FUSE_GENERIC(T, L) esc::fuse::conv_fuse_generic<T, L><<<blocks, esc::fuse::kGenThreads, smem, st>>>( \
+        static_cast<T*>(out), static_cast<const T*>(w_fuse), static_cast<const T*>(b_fuse), static_cast<const T*>(residual), B, C, H, W)
+    if (dtype == ESC_F32) { if (layout == ESC_NCHW) ESC_FUSE_GENERIC(float, esc::kNCHW); else ESC_FUSE_GENERIC(float, esc::kNHWC); }
+    else { if (layout == ESC_NCHW) ESC_FUSE_GENERIC(__nv_bfloat16, esc::kNCHW); else ESC_FUSE_GENERIC(__nv_bfloat16, esc::kNHWC); }
+#undef ESC_FUSE_GENERIC
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
 }
 
 size_t esc_convattn_backward_workspace_bytes(int B, int C_a, int H, int W, int K) {

@@ -592,8 +592,8 @@ struct Fused {
 template <class S, bool kBias, bool kFused>
 inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk,
                         const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches,
-                        std::string* err, const Fused* fu = nullptr) {
-    const int cc = C - Ca;
+                        std::string* err, const Fused* fu = nullptr, bool skip_copy = false) {
+    const int cc = skip_copy ? 0 : C - Ca;                 // skip_copy: the identity channels are consumed elsewhere (fused 1x1)
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
     p.tiles_x = (W + S::TW - 1) / S::TW; p.tiles_y = (H + S::TH - 1) / S::TH; p.groups = Ca / CG;
@@ -674,11 +674,12 @@ inline bool applies(int C, int Ca, int K, int dtype, int layout) {
 // Launches the tensor-core stencil if the problem fits it: 0 on success, kNotApplicable otherwise, or an ESC_ERR_* code.
 inline int try_launch_toeplitz(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
                                const void* w_large, const float* dk, const float* bias, void* out, unsigned* ctrl,
-                               cudaStream_t st, bool dependent, int* launches, std::string* err, int* tile_w) {
+                               cudaStream_t st, bool dependent, int* launches, std::string* err, int* tile_w,
+                               bool skip_copy = false) {
     if (!applies(C, Ca, K, dtype, layout) || sm_count() <= 0) return kNotApplicable;
     *tile_w = Shape64x16::TW;
-    return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err)
-                : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err);
+    return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy)
+                : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy);
 }
 
 // Whether the whole forward can be one launch of the tensor-core kernel with stage 1 inside: the kernel applies,
@@ -692,11 +693,11 @@ inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, 
 // The whole forward (stage 1 fused) as one launch; same return convention as try_launch_toeplitz.
 inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
                             const void* w_large, const Fused& fu, void* out, unsigned* ctrl, cudaStream_t st,
-                            int* launches, std::string* err, int* tile_w) {
+                            int* launches, std::string* err, int* tile_w, bool skip_copy = false) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden)) return kNotApplicable;
     *tile_w = Shape64x16::TW;
     return launch_shape<Shape64x16, false, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
-                                                 launches, err, &fu);
+                                                 launches, err, &fu, skip_copy);
 }
 
 }}}  // namespace esc::tma::toep
