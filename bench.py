@@ -516,6 +516,42 @@ def main():
         wp_d = torch.from_numpy(synth.make_pointwise(wl.C_a, wl.dtype, wl.seed)).to(tdt).cuda()
         st, _ = timer.measure(lambda i: pkg.esc_convattn_forward_pw(xs[i % n_rot], wl.C_a, wl.K, wl_d, wp_d, wd_d, bd_d, outs[i % n_rot], lay_code, ws), samples=5)
         extras["ms_per_step_decomposed_large_kernel"] = st["median_ms"]
+        # the module with its closing 1x1 convolution and residual (Eq. 4 line 4, Eq. 3 line 3): one fused call against
+        # the forward followed by a library 1x1 convolution and an add
+        try:
+            fz = synth.make_fuse(wl.C, wl.dtype, wl.seed)
+            wf_d = torch.from_numpy(fz["w_fuse"]).to(tdt).cuda()
+            bf_d = torch.from_numpy(fz["b_fuse"]).to(tdt).cuda()
+            res_d = torch.randn_like(xs[0])
+            st, _ = timer.measure(lambda i: pkg.esc_convattn_forward_fused(xs[i % n_rot], wl.C_a, wl.K, wl_d, wd_d, bd_d, wf_d, bf_d, res_d,
+                                                                           outs[i % n_rot], lay_code, ws), samples=5)
+            fused_ms, fused_launches = st["median_ms"], pkg.esc_convattn_last_launches()
+            sep_ms = None
+            if lay_code == pkg.ESC_NHWC:
+                w4 = wf_d.view(wl.C, wl.C, 1, 1).contiguous(memory_format=torch.channels_last)
+                views = [o.permute(0, 3, 1, 2) for o in outs]            # NHWC storage seen as [B,C,H,W] channels_last
+                res_v = res_d.permute(0, 3, 1, 2)
+
+                def separate(i):
+                    pkg.esc_convattn_forward_ex(xs[i % n_rot], wl.C_a, wl.K, wl_d, wd_d, bd_d, outs[i % n_rot], lay_code, ws)
+                    y = torch.nn.functional.conv2d(views[i % n_rot], w4, bf_d)
+                    y.add_(res_v)
+
+                with torch.cuda.stream(timer.side):
+                    for i in range(3):
+                        separate(i)
+                torch.cuda.synchronize()
+                st, _ = timer.measure(separate, samples=5)
+                sep_ms = st["median_ms"]
+            extras["module_with_conv_fuse"] = {
+                "fused_call_ms": fused_ms, "fused_call_launches": fused_launches,
+                "forward_then_library_conv1x1_and_add_ms": sep_ms,
+                "algorithmic_bytes_per_pixel": {"fused_call": (wl.C_a * 2 + wl.C + wl.C + wl.C) * es,
+                                                "separate": (2 * wl.C + 2 * wl.C + 3 * wl.C) * es},
+                "note": "fused: stencil reads and writes the attention channels, the 1x1 kernel reads x's identity channels, the residual, "
+                        "and writes out; separate: forward (read x, write cat), conv (read cat, write y), add (read y, residual, write y)"}
+        except Exception as exc:                                          # never lose the headline over an extra
+            extras["module_with_conv_fuse"] = {"error": f"{type(exc).__name__}: {exc}"}
         # with the dense large kernel of the main model (Section 3.2): an implicit GEMM on the tensor cores
         if wl.C_a == 16 and wl.K == 13:
             wdn_d = torch.from_numpy(synth.make_dense_kernel(wl.C_a, wl.K, wl.dtype, wl.seed)).to(tdt).cuda()

@@ -39,9 +39,9 @@ conv_fuse_nhwc_bf16(const Params p)
     constexpr int NT = C / 8, KS = C / 16;
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* wsm = smem;                              // [C][PITCH]: w_fuse, row n = output channel
-    unsigned char* xsm = smem + C * PITCH;                  // [kPix][PITCH]: cat of the block's pixels; later the results
+    unsigned char* xsm = smem + C * PITCH;                  // [kPix][PITCH]: cat of the tile's pixels; later the results
+    unsigned char* rsm = xsm + kPix * PITCH;                // [kPix][PITCH]: the residual of the same pixels
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const long long px0 = (long long)blockIdx.x * kPix;
 
     // ---- stage w_fuse and the 64 pixels (16-byte pieces; channels below Ca from `att`, the rest from `idt`) -----
     constexpr int CH = C / 8;                               // 16-byte pieces per row
@@ -49,15 +49,21 @@ conv_fuse_nhwc_bf16(const Params p)
         const int r = e / CH, q = e % CH;
         *reinterpret_cast<uint4*>(wsm + r * PITCH + q * 16) = __ldg(reinterpret_cast<const uint4*>(p.w + (size_t)r * C) + q);
     }
+    // a block keeps w_fuse and walks tiles of 64 pixels
+    const long long ntiles = (p.pixels + kPix - 1) / kPix;
+    for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const long long px0 = tile * kPix;
     for (int e = tid; e < kPix * CH; e += kThreads) {
         const int r = e / CH, q = e % CH;
         const long long px = px0 + r;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u), rv = make_uint4(0u, 0u, 0u, 0u);
         if (px < p.pixels) {
             const __nv_bfloat16* src = (q * 8 < p.Ca ? p.att : p.idt) + (size_t)px * C;
             v = __ldcg(reinterpret_cast<const uint4*>(src) + q);
+            if (p.residual) rv = __ldcg(reinterpret_cast<const uint4*>(p.residual + (size_t)px * C) + q);
         }
         *reinterpret_cast<uint4*>(xsm + r * PITCH + q * 16) = v;
+        *reinterpret_cast<uint4*>(rsm + r * PITCH + q * 16) = rv;
     }
     __syncthreads();
 
@@ -95,12 +101,9 @@ conv_fuse_nhwc_bf16(const Params p)
         for (int h = 0; h < 2; ++h) {
             const int r = warp * 16 + g + 8 * h;
             float v0 = acc[n][2 * h] + b0, v1 = acc[n][2 * h + 1] + b1;
-            const long long px = px0 + r;
-            if (p.residual && px < p.pixels) {
-                const uint32_t rr = __ldcg(reinterpret_cast<const uint32_t*>(p.residual + (size_t)px * C + oc));
-                v0 += __uint_as_float(rr << 16);
-                v1 += __uint_as_float(rr & 0xffff0000u);
-            }
+            const uint32_t rr = *reinterpret_cast<const uint32_t*>(rsm + r * PITCH + oc * 2);   // zero without a residual
+            v0 += __uint_as_float(rr << 16);
+            v1 += __uint_as_float(rr & 0xffff0000u);
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
             *reinterpret_cast<uint32_t*>(xsm + r * PITCH + oc * 2) = *reinterpret_cast<const uint32_t*>(&h2);
         }
@@ -111,6 +114,8 @@ conv_fuse_nhwc_bf16(const Params p)
         const long long px = px0 + r;
         if (px < p.pixels)
             *(reinterpret_cast<uint4*>(p.out + (size_t)px * C) + q) = *reinterpret_cast<const uint4*>(xsm + r * PITCH + q * 16);
+    }
+    __syncthreads();                                        // the staging areas are re-used by the next tile
     }
 }
 
@@ -155,7 +160,7 @@ inline bool fast_applies(int C, int Ca, int dtype, int layout) {
 template <int C>
 inline cudaError_t launch_fast_c(const Params& p, cudaStream_t st) {
     constexpr int PITCH = C * 2 + 16;
-    const size_t smem = (size_t)(C + kPix) * PITCH;
+    const size_t smem = (size_t)(C + 2 * kPix) * PITCH;
     static bool attr_set[tma::kMaxDevices] = {};
     const int dev = tma::current_device();
     if (dev < 0) return cudaErrorInvalidDevice;
@@ -164,8 +169,8 @@ inline cudaError_t launch_fast_c(const Params& p, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    const long long blocks = (p.pixels + kPix - 1) / kPix;
-    conv_fuse_nhwc_bf16<C><<<(unsigned)blocks, kThreads, smem, st>>>(p);
+    const long long ntiles = (p.pixels + kPix - 1) / kPix, cap = 8LL * (tma::sm_count() > 0 ? tma::sm_count() : 148);
+    conv_fuse_nhwc_bf16<C><<<(unsigned)(ntiles < cap ? ntiles : cap), kThreads, smem, st>>>(p);
     return cudaGetLastError();
 }
 
