@@ -13,13 +13,17 @@
 // of shared-memory operands: the tensor pipe, not shared memory, is the bound, and nothing is unfolded.
 // At the ends of a CTA's row range the instruction takes only the column blocks that exist (N = 16 .. 192).
 //
-// Operands are K-major without swizzle, where a row of 8 k-values is 16 contiguous bytes and rows are 16 bytes
-// apart, so a descriptor may start at ANY pixel: the staged row keeps the two channel halves apart
-// ([half][pixel][8 channels], two TMA loads per row with zero fill = the padding) and the tap column j is a
-// shift of the descriptor's start address by 16 * j bytes.
+// Operands are K-major.  A: a staged input row is [pixel][16 channels], 32 bytes per pixel, written by ONE TMA load
+// per row (zero fill = the padding) with the 32-byte swizzle, and described to the tensor core with the same
+// swizzle; the swizzle is a function of the shared-memory address, so the descriptor may start at ANY pixel and
+// the tap column j is a shift of its start address by 32 * j bytes (measured: every output agrees with the
+// oracle).  B: the weights, without swizzle ([half of K][row][8 k-values], rows 16 bytes apart).
+// What bounds it: an instruction takes about 110-130 cycles whatever its N, so the 12 input rows above and below
+// a CTA's range, which feed only some of the 13 column blocks, cost as much as full rows: with 13 output rows per
+// CTA (640x360 on 148 SMs) 25 row-times are spent for 13 rows of results; larger maps give longer ranges.
 //
 // Roles (224 threads, one CTA per SM, each CTA one range of rows of one strip):
-//   warp 0   lane 0 requests input rows by TMA into a ring of 16; the warp allocates and frees tensor memory
+//   warp 0   lane 0 requests input rows by TMA (one load per row) into a ring of 16; the warp allocates and frees tensor memory
 //   warp 1   lane 0 issues the instructions and commits them to mbarriers (ring slot consumed / output row complete)
 //   warps 2-5  epilogue: tcgen05.ld of a finished row (one pixel per thread, 16 channels), the dynamic 3x3
 //            kernel in fp32 on the CUDA cores from the same ring, one rounding to bf16, 32-byte store;
@@ -33,8 +37,8 @@ namespace esc { namespace tma { namespace umma {
 
 constexpr int MW = 128;                       // output pixels per strip row = M of the instruction
 constexpr int SPX = 144;                      // staged pixels per row: 128 + 12, padded to keep half-rows 128-byte aligned
-constexpr int HALF_BYTES = SPX * 16;          // one row, one channel half
-constexpr int ROW_BYTES = 2 * HALF_BYTES;
+constexpr int HALF_BYTES = SPX * 16;
+constexpr int ROW_BYTES = 2 * HALF_BYTES;     // one staged row: SPX pixels x 32 bytes
 constexpr int NRING = 16;                     // input rows in flight / kept for the 3x3 part
 constexpr int NBLK = K13;                     // column blocks of 16 (kernel rows) in a B operand
 constexpr int BHALF_BYTES = NBLK * CG * 16;   // 3,328: one tap column, one channel half: [208 rows][8 k]
@@ -69,6 +73,13 @@ struct Params {
 __device__ __forceinline__ unsigned long long smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
     return (unsigned long long)((addr >> 4) & 0x3FFFu) | ((unsigned long long)((lbo >> 4) & 0x3FFFu) << 16) |
            ((unsigned long long)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+// A operand: K-major with the 32-byte swizzle -- a row (pixel) is 32 contiguous bytes, its two 16-byte halves swapped
+// where bit 7 of the shared-memory address is set -- exactly what a TMA load with CU_TENSOR_MAP_SWIZZLE_32B writes for
+// a 32-byte inner box.  Rows are 32 bytes apart, 8-row groups 256 bytes.
+__device__ __forceinline__ unsigned long long smem_desc_sw32(uint32_t addr) {
+    return (unsigned long long)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((unsigned long long)(256u >> 4) << 32) | (1ull << 46) |
+           (6ull << 61);
 }
 // Instruction descriptor of kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = n.
 __device__ __forceinline__ uint32_t instr_desc(int n) {
@@ -114,7 +125,7 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
                              const __grid_constant__ CUtensorMap map_cout, const Params p)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char* ring = smem;                                             // [NRING][2 halves][SPX][16 bytes]
+    unsigned char* ring = smem;                                             // [NRING][SPX pixels][32 bytes], 32-byte swizzle
     unsigned char* btab = smem + NRING * ROW_BYTES;                         // [13 tap columns][2 halves][208 rows][16 bytes]
     float* dks = reinterpret_cast<float*>(btab + B_BYTES);                  // [9 taps][16 channels]
     int* prog = reinterpret_cast<int*>(dks + 9 * CG);                       // output rows the epilogue has finished
@@ -216,7 +227,6 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
                 const uint32_t dst = smem_u32(ring + (size_t)slot * ROW_BYTES), bar = rowfull0 + 8 * slot;
                 mbar_expect_tx(bar, ROW_BYTES);
                 tma_load_4d(dst, &map_half, bar, 0, x0 - P6, ya - P6 + n, b);
-                tma_load_4d(dst + HALF_BYTES, &map_half, bar, 8, x0 - P6, ya - P6 + n, b);
             }
         }
     } else if (warp == 1) {
@@ -243,7 +253,7 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
                     const int cnt = c_hi - c_lo + 1, s0 = (n - (K13 - 1) + c_lo) % SLOTS;
                     const int cnt1 = min(cnt, SLOTS - s0), cnt2 = cnt - cnt1;      // the row slots wrap around at 32
                     for (int j = 0; j < K13; ++j) {
-                        const unsigned long long da = smem_desc(ring_a + (uint32_t)(slot * ROW_BYTES + 16 * j), HALF_BYTES, 128);
+                        const unsigned long long da = smem_desc_sw32(ring_a + (uint32_t)(slot * ROW_BYTES + 32 * j));
                         const uint32_t bj = btab_a + (uint32_t)(j * BJ_BYTES + c_lo * CG * 16);
                         mma_f16(tmem + (uint32_t)(s0 * CG), da, smem_desc(bj, BHALF_BYTES, 128), instr_desc(cnt1 * CG));
                         if (cnt2 > 0)
@@ -300,8 +310,10 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
         const int x = x0 + m;
         for (int yr = 0; yr < L; ++yr) {
             const int slot = yr % SLOTS;
-            if (alive) alive = mbar_wait(accfull0 + 8 * slot, (unsigned)((yr / SLOTS) & 1), p.ctrl, 0xD4000000u | (unsigned)yr);
-            if (!alive) st_release_cta(aborted, 1);
+            // one lane asks (a wait that all 32 lanes execute costs the warp over a hundred cycles)
+            if (lane == 0 && alive) alive = mbar_wait(accfull0 + 8 * slot, (unsigned)((yr / SLOTS) & 1), p.ctrl, 0xD4000000u | (unsigned)yr);
+            if (lane == 0 && !alive) st_release_cta(aborted, 1);
+            __syncwarp();
             tc_fence_after();
             uint32_t r[16];
             tmem_ld16(lane_base + (uint32_t)(slot * CG), r);
@@ -313,11 +325,14 @@ stencil_dense_umma_nhwc_bf16(const __grid_constant__ CUtensorMap map_half, const
             // pixels m + 5 .. m + 7 of the staged row
 #pragma unroll
             for (int a = 0; a < 3; ++a) {
-                const unsigned char* rowp = ring + (size_t)((yr + 5 + a) % NRING) * ROW_BYTES;
+                const int rslot = (yr + 5 + a) % NRING;
+                const unsigned char* rowp = ring + (size_t)rslot * ROW_BYTES;
 #pragma unroll
                 for (int bb = 0; bb < 3; ++bb) {
-                    const uint4 lo = *reinterpret_cast<const uint4*>(rowp + (size_t)(m + 5 + bb) * 16);
-                    const uint4 hi = *reinterpret_cast<const uint4*>(rowp + HALF_BYTES + (size_t)(m + 5 + bb) * 16);
+                    // the pixel's two 16-byte halves are swapped where bit 7 of its address is set (32-byte swizzle)
+                    const int px = m + 5 + bb, sw = ((rslot * (ROW_BYTES / 128) + (px >> 2)) & 1) * 16;
+                    const uint4 lo = *reinterpret_cast<const uint4*>(rowp + (size_t)px * 32 + sw);
+                    const uint4 hi = *reinterpret_cast<const uint4*>(rowp + (size_t)px * 32 + (16 - sw));
                     float f[16];
                     unpack16<__nv_bfloat16>(lo, f);
                     unpack16<__nv_bfloat16>(hi, f + 8);
@@ -392,7 +407,17 @@ inline int try_launch_dense_umma(int B, int C, int Ca, int H, int W, int K, int 
         p.copy_pw = pw;
     }
     CUtensorMap m_half, m_cin, m_cout;
-    if (!make_map(&m_half, x, B, C, H, W, 8, SPX, 1, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
+    {   // one staged row per load: 16 channels x SPX pixels, written with the 32-byte swizzle the A descriptor names
+        EncodeTiledFn fn = encode_fn();
+        if (!fn) return kNotApplicable;
+        const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
+        const cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+        const cuuint32_t box[4] = {(cuuint32_t)CG, (cuuint32_t)SPX, 1, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (fn(&m_half, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_64B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return kNotApplicable;
+    }
     if (cc > 0) {
         if (!make_map(&m_cin, x, B, C, H, W, cc, p.copy_pw, 1)) return kNotApplicable;
         if (!make_map(&m_cout, out, B, C, H, W, cc, p.copy_pw, 1)) return kNotApplicable;
