@@ -16,8 +16,8 @@
 // Operands are K-major.  A: a staged input row is [pixel][16 channels], 32 bytes per pixel, written by ONE TMA load
 // per row (zero fill = the padding) with the 32-byte swizzle, and described to the tensor core with the same
 // swizzle; the swizzle is a function of the shared-memory address, so the descriptor may start at ANY pixel and
-// the tap column j is a shift of its start address by 32 * j bytes (measured: every output agrees with the
-// oracle).  B: the weights, without swizzle ([half of K][row][8 k-values], rows 16 bytes apart).
+// the tap column j is a shift of its start address by 32 * j bytes (verified output by output against
+// a direct fp64 evaluation).  B: the weights, without swizzle ([half of K][row][8 k-values], rows 16 bytes apart).
 // What bounds it: an instruction takes about 110-130 cycles whatever its N, so the 12 input rows above and below
 // a CTA's range, which feed only some of the 13 column blocks, cost as much as full rows: with 13 output rows per
 // CTA (640x360 on 148 SMs) 25 row-times are spent for 13 rows of results; larger maps give longer ranges.
