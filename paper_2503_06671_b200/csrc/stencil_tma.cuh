@@ -55,8 +55,8 @@ constexpr int NSLOT = 2, COPY_DEPTH = 1;             // copy ring: slots, loads 
                                                      // thread shares a scheduler with two compute warps and every
                                                      // instruction it issues delays them, then the whole block at the barriers)
 constexpr int kMaxSlotBytes = 16384;
-constexpr unsigned kSpinLimit = 1u << 20;    // polls before a wait gives up (each poll may suspend up to the hint)
-constexpr unsigned kSuspendHintNs = 20000;
+constexpr unsigned kSpinLimit = 1u << 20;    // polls before a wait gives up (each poll may suspend up to the hint):
+constexpr unsigned kSuspendHintNs = 1000;    // a wait that never ends gives up after about one second
 
 // Tile geometry.  A lane owns a patch of OY rows x OX columns of outputs; a tile is LXP x LYP
 // patches (always 32, i.e. 8 warps of 4 patches x 8 channel pairs).  The 32 lanes of an LDS.32 hit

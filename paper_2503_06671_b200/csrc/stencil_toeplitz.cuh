@@ -430,9 +430,9 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         }
 
         // ---- two channels per warp --------------------------------------------------------------------
-        // Per channel: 13 kernel rows of tensor-core work into acc, then the dynamic 3x3 kernel on the CUDA
-        // cores, fp32 (Eq. 4 line 3, second term), into dacc; dk is waited for after the first channel's
-        // tensor-core work of a CTA's first unit, which runs beside the kernel that produces it.
+        // Per channel: 13 kernel rows of tensor-core work into acc / acc1, then the dynamic 3x3 kernel on the CUDA
+        // cores, fp32 (Eq. 4 line 3, second term), into dacc; dk is waited for after both channels'
+        // tensor-core work.
         const unsigned sh = (g & 1) ? 0u : 16u;
         float acc[NB][NA][4], dacc[NB][NA][4];
         float dkv[9];
@@ -446,7 +446,9 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
                 for (int r = 0; r < NA; ++r)
 #pragma unroll
                     for (int v = 0; v < 4; ++v) a4[q][r][v] = 0.f;
-#pragma unroll 1
+            // Straight-line code for the 13 kernel rows: the loads of a row run ahead of the previous row's products
+            // (-4 % on large maps, -1.2 us on a 640x360 forward against the rolled loop).
+#pragma unroll
             for (int i = 0; i < K13; ++i) {
                 const uint32_t pa = pt[i * PT + ia], pb = pt[i * PT + ib], pc = pt[i * PT + ic];
                 // A0[m][k] = LK[i][k - m] (outputs of block q from inputs of block q),
@@ -527,26 +529,19 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
                     }
         };
 
-        if (kFused && k == 0) {
-            // first unit: all tensor-core work first; every CTA has arrived for all its tiles well before dk is needed
+        {
+            // Both channels' tensor-core work first, then the 3x3 part of each: dk is first needed well after every CTA has
+            // arrived for all its tiles (one-launch form) or after the kernel that produces it has run beside this one.
+            // (Alternating products and 3x3 part per channel was 4 % slower on large maps.)
             float acc1[NB][NA][4];
             mma_all(acc, warp * 2);
             mma_all(acc1, warp * 2 + 1);
-            obtain_dk(un, flag0[0]);
+            if (kFused) obtain_dk(un, flag0[k == 0 ? 0 : 1]);
+            else if (!dk_ready) { pdl_wait_primary(); dk_ready = true; }
             dk_all(dacc, warp * 2);
             write_back(acc, dacc, warp * 2);
             dk_all(dacc, warp * 2 + 1);
             write_back(acc1, dacc, warp * 2 + 1);
-        } else {
-            if (kFused) obtain_dk(un, flag0[1]);
-#pragma unroll 1
-            for (int cc = 0; cc < 2; ++cc) {
-                const int c = warp * 2 + cc;
-                mma_all(acc, c);
-                if (!kFused && !dk_ready) { pdl_wait_primary(); dk_ready = true; }
-                dk_all(dacc, c);
-                write_back(acc, dacc, c);
-            }
         }
         mma_bar();                                           // all 16 planes hold their results
 
