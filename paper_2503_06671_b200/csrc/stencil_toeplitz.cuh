@@ -599,7 +599,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
         const int shapes[6][2] = {{S::TW, 4}, {S::TW, 2}, {S::TW, 1}, {S::TW / 2, 1}, {S::TW / 4, 1}, {S::TW / 8, 1}};
         int pick = -1;
         for (int s = 0; s < 6 && pick < 0; ++s)
-            if (S::TH % shapes[s][1] == 0 && cc * 2 * shapes[s][0] * shapes[s][1] <= kMaxSlotBytes) pick = s;
+            if (S::TH % shapes[s][1] == 0 && cc * 2 * shapes[s][0] * shapes[s][1] <= (kFused ? 12288 : kMaxSlotBytes)) pick = s;   // one-launch form: its scratch leaves 12 KB per slot
         if (pick < 0) return kNotApplicable;
         p.copy_cw = shapes[pick][0]; p.copy_cr = shapes[pick][1];
         p.slot_stride = (cc * 2 * p.copy_cw * p.copy_cr + 127) / 128 * 128;

@@ -96,3 +96,44 @@ def test_stencil_stage_explicit_dk_and_determinism(pkg, oracle):
     util.check_attention(got[:, :C_a], ref[:, :C_a], mag, synth.BF16, "stencil stage, tensor engine", unit_variance=True)
     assert np.array_equal(got[:, C_a:], ref[:, C_a:])
     assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16)) and torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
+
+
+@pytest.mark.parametrize("shape", [(1, 64, 16, 300, 640), (70, 32, 16, 40, 64), (16, 64, 32, 33, 70), (14, 48, 48, 30, 90), (1, 64, 16, 100, 150)],
+                         ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("mode", ["one_launch", "unaligned", "two_launches"])
+def test_one_launch_forward_estimator_inputs(pkg, oracle, shape, mode):
+    """The one-launch forward (stage 1 inside the stencil kernel; a CTA evaluates the estimator for both of its
+    units at once), the same with the estimator's weights at an address that is only 2-byte aligned, and
+    "two_launches": the same forward with stage 1 as its own kernel.
+    Shapes: one image with two units per CTA (190 units), 210 / 192 / 168 units whose image and channel group change
+    between a CTA's two units (one, two, three groups), and a launch with fewer units than SMs.  All outputs compared with the oracle, twice (the counters and flags are re-used)."""
+    import torch
+
+    B, C, C_a, H, W = shape
+    K = 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=sum(shape) + 9, per_image_scale=True, channel_means=True)
+    x = util.to_device(d["x"], synth.BF16, synth.NHWC)
+    wl, wd, bd = util.weights_to_device(d, synth.BF16)
+    if mode == "unaligned":
+        hold_w = torch.empty(wd.numel() + 8, dtype=wd.dtype, device="cuda")
+        hold_b = torch.empty(bd.numel() + 8, dtype=bd.dtype, device="cuda")
+        hold_w[1:1 + wd.numel()] = wd.reshape(-1)
+        hold_b[1:1 + bd.numel()] = bd.reshape(-1)
+        wd, bd = hold_w[1:1 + wd.numel()].view(wd.shape), hold_b[1:1 + bd.numel()].view(bd.shape)
+        assert wd.data_ptr() % 16 == 2
+    ws = pkg.new_workspace(B, C_a, H, W, K)
+    out = torch.full_like(x, 7.0)
+    pkg.esc_convattn_set_fused_stage1(mode != "two_launches")
+    try:
+        for _ in range(2):
+            pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, out, pkg.ESC_NHWC, ws)
+        torch.cuda.synchronize()
+    finally:
+        pkg.esc_convattn_set_fused_stage1(True)
+    assert pkg.esc_convattn_device_status(ws) == 0
+    assert pkg.esc_convattn_last_path() == 4
+    assert pkg.esc_convattn_last_launches() == (2 if mode == "two_launches" else 1)
+    ref, mag = oracle.forward(d["x"], C_a, d["w_large"], d["w_dyn"], d["b_dyn"], want_mag=True)
+    got = util.to_host_nchw(out, synth.NHWC)
+    util.check_attention(got[:, :C_a], ref[:, :C_a], mag, synth.BF16, f"{shape} {mode}")
+    assert np.array_equal(got[:, C_a:], ref[:, C_a:])
