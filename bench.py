@@ -39,8 +39,8 @@ FMA_LANES_PER_SM = 128
 L2_BYTES = 126 * 1024 * 1024
 SAMPLES = 11
 MIN_SAMPLE_S = 0.1
-PATH_NAMES = {1: "generic", 2: "tma-fp32", 3: "tensor-dense-mma.sync", 4: "tensor-toeplitz", 5: "tensor-dense-tcgen05"}
-KERNEL_FILES = {1: "stencil_generic.cuh", 2: "stencil_tma.cuh", 3: "stencil_dense.cuh", 4: "stencil_toeplitz.cuh", 5: "stencil_dense_umma.cuh"}
+PATH_NAMES = {1: "generic", 2: "tma-fp32", 3: "tensor-dense-mma.sync", 4: "tensor-toeplitz", 5: "tensor-dense-tcgen05", 6: "tensor-toeplitz-nchw"}
+KERNEL_FILES = {1: "stencil_generic.cuh", 2: "stencil_tma.cuh", 3: "stencil_dense.cuh", 4: "stencil_toeplitz.cuh", 5: "stencil_dense_umma.cuh", 6: "stencil_toeplitz_nchw.cuh"}
 TOEPLITZ_DENSITY = 13.0 / 32.0               # useful share of the multiply-adds the banded-Toeplitz kernel issues
 PEAK_SRC = os.path.join(ROOT, "bench_fp32_peak.cu")
 PEAK_LIB = os.path.join(ROOT, "paper_2503_06671_b200", "lib", "libbench_fp32_peak.so")

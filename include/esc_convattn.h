@@ -292,7 +292,8 @@ int esc_convattn_device_status(void* workspace, void* stream);
 /* Which stencil implementation the last esc_convattn_forward* / esc_convattn_stencil call on
  * this thread selected: 0 = none yet, 1 = guarded generic kernel, 2 = TMA-staged register-tiled
  * FP32 kernel, 3 = tensor-core kernel of the dense large kernel, 4 = tensor-core (banded Toeplitz)
- * kernel of the depth-wise large kernel, 5 = tcgen05 kernel of the dense large kernel.  For tests and benchmarks. */
+ * kernel of the depth-wise large kernel on NHWC tensors, 5 = tcgen05 kernel of the dense large kernel,
+ * 6 = the tensor-core (banded Toeplitz) kernel on NCHW tensors.  For tests and benchmarks. */
 int esc_convattn_last_path(void);
 
 /* Which arithmetic units evaluate the depth-wise 13x13 stage of Eq. 4 line 3 on NHWC bf16 tensors, for

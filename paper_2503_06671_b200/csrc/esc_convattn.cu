@@ -18,6 +18,7 @@
 #include "stencil_generic.cuh"
 #include "stencil_tma.cuh"
 #include "stencil_toeplitz.cuh"
+#include "stencil_toeplitz_nchw.cuh"
 #include "stencil_dense.cuh"
 #include "stencil_dense_umma.cuh"
 #include "backward.cuh"
@@ -319,6 +320,12 @@ int launch_stencil(const Problem& p, const void* x, const void* w_large, const f
                                                            out, ctrl, st, dependent, &g_last_launches, &g_last_error, &tw, p.skip_copy);
         if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
         if (rc != esc::tma::kNotApplicable) return rc;
+        if (!p.skip_copy) {                                  // the same arithmetic on NCHW tensors
+            const int rn = esc::tma::toepn::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, p.bias, out,
+                                                       ctrl, st, dependent, &g_last_launches, &g_last_error);
+            if (rn == ESC_OK) { g_last_path = 6; g_last_tile_w = esc::tma::toepn::TW; return ESC_OK; }
+            if (rn != esc::tma::kNotApplicable) return rn;
+        }
     }
     if (p.skip_copy) return ESC_ERR_UNSUPPORTED;           // only the tensor-core kernel can leave the identity channels out
     if (g_engine_policy == ESC_ENGINE_TENSOR) return launch_generic(p, x, w_large, dk, out, st, dependent);
@@ -426,7 +433,16 @@ int forward_impl(const Problem& p, const void* x, const void* w_large, const Est
             g_last_error.clear();
         }
     }
-    int rc = launch_gap(p, x, est, w, w.dk, st, tensor_stencil_follows(p));
+    if (g_fuse_stage1 && !p.dense && !p.w_point && !p.bias && !p.skip_copy && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0) {
+        const esc::tma::toep::Fused fu{est.w_last, est.b_last, est.w_down, est.b_down, est.hidden, w.unit_sums, w.arrivals, w.flags};
+        const int rc = esc::tma::toepn::try_launch_fused(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, fu, out, w.ctrl, st,
+                                                         &g_last_launches, &g_last_error);
+        if (rc == ESC_OK) { g_last_path = 6; g_last_tile_w = esc::tma::toepn::TW; return ESC_OK; }
+        if (rc != esc::tma::kNotApplicable) { (void)cudaGetLastError(); g_last_error.clear(); }
+    }
+    const bool tensor_nchw = !p.dense && !p.w_point && !p.bias && !p.skip_copy && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
+                             esc::tma::toepn::applies(p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, out);
+    int rc = launch_gap(p, x, est, w, w.dk, st, tensor_stencil_follows(p) || tensor_nchw);
     if (rc != ESC_OK) return rc;
     if (p.dense) return launch_stencil_dense(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
     return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
