@@ -31,91 +31,156 @@ struct Params {
     int C, Ca;
 };
 
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+    // 16 bytes global -> shared without a register in between; an invalid piece is zero-filled (source size 0)
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(valid ? 16 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+template <int C> struct Stages { static constexpr int N = C <= 64 ? 3 : 2; };   // tiles resident per block (one worked on, the rest in flight)
+
 template <int C>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, C <= 64 ? 4 : 2)
 conv_fuse_nhwc_bf16(const Params p)
 {
     constexpr int PITCH = C * 2 + 16;                       // bytes per staged row: 16-byte rows of an ldmatrix fall in different banks
     constexpr int NT = C / 8, KS = C / 16;
+    constexpr bool kRegB = C <= 64;                         // w_fuse as tensor-core fragments in registers (C <= 64), else in shared memory
+    constexpr int STAGE = 2 * kPix * PITCH;                 // a tile's cat rows, then its residual rows
     extern __shared__ __align__(16) unsigned char smem[];
-    unsigned char* wsm = smem;                              // [C][PITCH]: w_fuse, row n = output channel
-    unsigned char* xsm = smem + C * PITCH;                  // [kPix][PITCH]: cat of the tile's pixels; later the results
-    unsigned char* rsm = xsm + kPix * PITCH;                // [kPix][PITCH]: the residual of the same pixels
+    constexpr int NS = Stages<C>::N;
+    // [C][PITCH]: w_fuse, row n = output channel; where it goes to registers, it passes through the last stage, which the
+    // pipeline fills only after the first barrier of the tile loop
+    unsigned char* wsm = smem + (kRegB ? (NS - 1) * STAGE : NS * STAGE);
+    static_assert(!kRegB || C * PITCH <= STAGE, "w_fuse fits a stage");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-
-    // ---- stage w_fuse and the 64 pixels (16-byte pieces; channels below Ca from `att`, the rest from `idt`) -----
     constexpr int CH = C / 8;                               // 16-byte pieces per row
-    for (int e = tid; e < C * CH; e += kThreads) {
+
+    // ---- w_fuse: B fragments of mma.m16n8k16 (k = input channel, n = output channel): b0 = W[8 nt + g][16 ks + 2t, + 1],
+    //      b1 = the same row, eight input channels on
+    uint32_t bw[kRegB ? KS : 1][kRegB ? NT : 1][2];
+    for (int e = tid; e < C * CH; e += kThreads) {          // coalesced, 16 bytes per thread
         const int r = e / CH, q = e % CH;
         *reinterpret_cast<uint4*>(wsm + r * PITCH + q * 16) = __ldg(reinterpret_cast<const uint4*>(p.w + (size_t)r * C) + q);
     }
-    // a block keeps w_fuse and walks tiles of 64 pixels
-    const long long ntiles = (p.pixels + kPix - 1) / kPix;
-    for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-    const long long px0 = tile * kPix;
-    for (int e = tid; e < kPix * CH; e += kThreads) {
-        const int r = e / CH, q = e % CH;
-        const long long px = px0 + r;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u), rv = make_uint4(0u, 0u, 0u, 0u);
-        if (px < p.pixels) {
-            const __nv_bfloat16* src = (q * 8 < p.Ca ? p.att : p.idt) + (size_t)px * C;
-            v = __ldcg(reinterpret_cast<const uint4*>(src) + q);
-            if (p.residual) rv = __ldcg(reinterpret_cast<const uint4*>(p.residual + (size_t)px * C) + q);
-        }
-        *reinterpret_cast<uint4*>(xsm + r * PITCH + q * 16) = v;
-        *reinterpret_cast<uint4*>(rsm + r * PITCH + q * 16) = rv;
+    if (kRegB) {
+        __syncthreads();
+        const int wmi = lane >> 3, wmr = lane & 7;
+        const uint32_t w_lane = tma::smem_u32(wsm) + (uint32_t)(((wmi >> 1) * 8 + wmr) * PITCH + (wmi & 1) * 16);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int n2 = 0; n2 < NT / 2; ++n2) {
+                uint32_t b[4];                              // output channels 16 n2 .. + 7 (k halves), then + 8 .. + 15
+                tma::toep::ldsm_x4(w_lane + (uint32_t)(n2 * 16 * PITCH) + ks * 32, b);
+                bw[kRegB ? ks : 0][kRegB ? 2 * n2 : 0][0] = b[0]; bw[kRegB ? ks : 0][kRegB ? 2 * n2 : 0][1] = b[1];
+                bw[kRegB ? ks : 0][kRegB ? 2 * n2 + 1 : 0][0] = b[2]; bw[kRegB ? ks : 0][kRegB ? 2 * n2 + 1 : 0][1] = b[3];
+            }
     }
-    __syncthreads();
-
-    // ---- D (16 pixels x C) = A (16 x C) x B (C x C) per warp ------------------------------------------------
-    float acc[NT][4];
-#pragma unroll
-    for (int n = 0; n < NT; ++n)
-#pragma unroll
-        for (int v = 0; v < 4; ++v) acc[n][v] = 0.f;
-    const int mi = lane >> 3, mr = lane & 7;
-    const uint32_t a_lane = tma::smem_u32(xsm) + (uint32_t)((warp * 16 + (mi & 1) * 8 + mr) * PITCH + (mi >> 1) * 16);
-    const uint32_t b_lane = tma::smem_u32(wsm) + (uint32_t)(((mi >> 1) * 8 + mr) * PITCH + (mi & 1) * 16);
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-        uint32_t a[4];
-        tma::toep::ldsm_x4(a_lane + ks * 32, a);            // rows 0-7 / 8-15 of the warp's pixels, k halves 0 / 1
-#pragma unroll
-        for (int n2 = 0; n2 < NT / 2; ++n2) {
-            uint32_t b[4];                                  // output channels 16 n2 .. + 7 (k halves), then + 8 .. + 15
-            tma::toep::ldsm_x4(b_lane + (uint32_t)(n2 * 16 * PITCH) + ks * 32, b);
-            tma::toep::mma_bf16(acc[2 * n2], a[0], a[1], a[2], a[3], b[0], b[1]);
-            tma::toep::mma_bf16(acc[2 * n2 + 1], a[0], a[1], a[2], a[3], b[2], b[3]);
-        }
-    }
-    __syncthreads();                                        // everybody has read the staged pixels
-
-    // ---- bias and residual are added in fp32; one rounding to bf16; results staged over the block's pixels -------
-    // acc[n]: [0], [1] = pixel g, output channels 8n + 2t, + 1; [2], [3] = pixel g + 8
+    float bs[NT][2];                                        // this lane's output channels 8n + 2t, + 1
 #pragma unroll
     for (int n = 0; n < NT; ++n) {
-        const int oc = 8 * n + 2 * t;
-        float b0 = 0.f, b1 = 0.f;
-        if (p.bias) { b0 = __bfloat162float(p.bias[oc]); b1 = __bfloat162float(p.bias[oc + 1]); }
+        bs[n][0] = p.bias ? __bfloat162float(p.bias[8 * n + 2 * t]) : 0.f;
+        bs[n][1] = p.bias ? __bfloat162float(p.bias[8 * n + 2 * t + 1]) : 0.f;
+    }
+    // the weights do not depend on the kernel before this one; the attention channels do
+    pdl_wait_primary();
+
+    // a tile's 64 pixels: channels below Ca from `att`, the rest from `idt`, and the residual, 16 bytes per copy
+    const long long ntiles = (p.pixels + kPix - 1) / kPix;
+    auto stage = [&](long long tile, int buf) {
+        const uint32_t xs = tma::smem_u32(smem + buf * STAGE), rs = xs + kPix * PITCH;
+        const long long px0 = tile * kPix;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int r = warp * 16 + g + 8 * h;
-            float v0 = acc[n][2 * h] + b0, v1 = acc[n][2 * h + 1] + b1;
-            const uint32_t rr = *reinterpret_cast<const uint32_t*>(rsm + r * PITCH + oc * 2);   // zero without a residual
-            v0 += __uint_as_float(rr << 16);
-            v1 += __uint_as_float(rr & 0xffff0000u);
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-            *reinterpret_cast<uint32_t*>(xsm + r * PITCH + oc * 2) = *reinterpret_cast<const uint32_t*>(&h2);
+        for (int u = 0; u < kPix * CH / kThreads; ++u) {
+            const int e = tid + u * kThreads, r = e / CH, q = e % CH;
+            const long long px = px0 + r;
+            const bool ok = px < p.pixels;
+            const size_t at = (size_t)(ok ? px : 0) * C;
+            cp_async16(xs + r * PITCH + q * 16, reinterpret_cast<const uint4*>((q * 8 < p.Ca ? p.att : p.idt) + at) + q, ok);
+            if (p.residual) cp_async16(rs + r * PITCH + q * 16, reinterpret_cast<const uint4*>(p.residual + at) + q, ok);
         }
+        cp_async_commit();
+    };
+    static_assert(kPix * CH % kThreads == 0, "pieces per thread");
+
+    long long tile = blockIdx.x;
+    int buf = 0;
+    // one group per tile, empty where there is no tile, so that "all but the NS - 2 newest groups" is always this tile
+#pragma unroll
+    for (int j = 0; j < NS - 1; ++j) {
+        if (tile + j * (long long)gridDim.x < ntiles) stage(tile + j * (long long)gridDim.x, j);
+        else cp_async_commit();
     }
-    __syncthreads();
-    for (int e = tid; e < kPix * CH; e += kThreads) {
-        const int r = e / CH, q = e % CH;
-        const long long px = px0 + r;
-        if (px < p.pixels)
-            *(reinterpret_cast<uint4*>(p.out + (size_t)px * C) + q) = *reinterpret_cast<const uint4*>(xsm + r * PITCH + q * 16);
-    }
-    __syncthreads();                                        // the staging areas are re-used by the next tile
+    for (; tile < ntiles; tile += gridDim.x, buf = buf + 1 == NS ? 0 : buf + 1) {
+        const long long px0 = tile * kPix;
+        unsigned char* xsm = smem + buf * STAGE;            // cat of the tile's pixels; later the results
+        unsigned char* rsm = xsm + kPix * PITCH;            // the residual of the same pixels
+        cp_async_wait<NS - 2>();
+        __syncthreads();                                    // the tile is there for everybody; everybody is done with the tile before
+        {
+            const long long nx = tile + (NS - 1) * (long long)gridDim.x;       // into the buffer of the tile before this one
+            if (nx < ntiles) stage(nx, buf == 0 ? NS - 1 : buf - 1);
+            else cp_async_commit();
+        }
+
+        // ---- D (16 pixels x C) = A (16 x C) x B (C x C) per warp ------------------------------------------------
+        float acc[NT][4];
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[n][v] = 0.f;
+        const int mi = lane >> 3, mr = lane & 7;
+        const uint32_t a_lane = tma::smem_u32(xsm) + (uint32_t)((warp * 16 + (mi & 1) * 8 + mr) * PITCH + (mi >> 1) * 16);
+        const uint32_t b_lane = tma::smem_u32(wsm) + (uint32_t)(((mi >> 1) * 8 + mr) * PITCH + (mi & 1) * 16);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t a[4];
+            tma::toep::ldsm_x4(a_lane + ks * 32, a);        // rows 0-7 / 8-15 of the warp's pixels, k halves 0 / 1
+            if (kRegB) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+                    tma::toep::mma_bf16(acc[nt], a[0], a[1], a[2], a[3], bw[kRegB ? ks : 0][kRegB ? nt : 0][0], bw[kRegB ? ks : 0][kRegB ? nt : 0][1]);
+            } else {
+#pragma unroll
+                for (int n2 = 0; n2 < NT / 2; ++n2) {
+                    uint32_t b[4];                          // output channels 16 n2 .. + 7 (k halves), then + 8 .. + 15
+                    tma::toep::ldsm_x4(b_lane + (uint32_t)(n2 * 16 * PITCH) + ks * 32, b);
+                    tma::toep::mma_bf16(acc[2 * n2], a[0], a[1], a[2], a[3], b[0], b[1]);
+                    tma::toep::mma_bf16(acc[2 * n2 + 1], a[0], a[1], a[2], a[3], b[2], b[3]);
+                }
+            }
+        }
+        __syncwarp();                                       // a warp's 16 staged pixels are read by that warp alone
+
+        // ---- bias and residual are added in fp32; one rounding to bf16; results staged over the warp's own pixels ----
+        // acc[n]: [0], [1] = pixel g, output channels 8n + 2t, + 1; [2], [3] = pixel g + 8
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+            const int oc = 8 * n + 2 * t;
+            const float b0 = bs[n][0], b1 = bs[n][1];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int r = warp * 16 + g + 8 * h;
+                float v0 = acc[n][2 * h] + b0, v1 = acc[n][2 * h + 1] + b1;
+                if (p.residual) {
+                    const uint32_t rr = *reinterpret_cast<const uint32_t*>(rsm + r * PITCH + oc * 2);
+                    v0 += __uint_as_float(rr << 16);
+                    v1 += __uint_as_float(rr & 0xffff0000u);
+                }
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                *reinterpret_cast<uint32_t*>(xsm + r * PITCH + oc * 2) = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+        }
+        __syncwarp();
+        // the warp's 16 pixels are 32 C contiguous bytes of the output
+#pragma unroll
+        for (int u = 0; u < 16 * CH / 32; ++u) {
+            const int e = lane + u * 32, r = warp * 16 + e / CH, q = e % CH;
+            const long long px = px0 + r;
+            if (px < p.pixels)
+                *(reinterpret_cast<uint4*>(p.out + (size_t)px * C) + q) = *reinterpret_cast<const uint4*>(xsm + r * PITCH + q * 16);
+        }
     }
 }
 
@@ -160,7 +225,7 @@ inline bool fast_applies(int C, int Ca, int dtype, int layout) {
 template <int C>
 inline cudaError_t launch_fast_c(const Params& p, cudaStream_t st) {
     constexpr int PITCH = C * 2 + 16;
-    const size_t smem = (size_t)(C + 2 * kPix) * PITCH;
+    const size_t smem = (size_t)(2 * Stages<C>::N * kPix + (C <= 64 ? 0 : C)) * PITCH;   // stages of (cat, residual); w_fuse where it is not in registers
     static bool attr_set[tma::kMaxDevices] = {};
     const int dev = tma::current_device();
     if (dev < 0) return cudaErrorInvalidDevice;
@@ -169,9 +234,18 @@ inline cudaError_t launch_fast_c(const Params& p, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    const long long ntiles = (p.pixels + kPix - 1) / kPix, cap = 8LL * (tma::sm_count() > 0 ? tma::sm_count() : 148);
-    conv_fuse_nhwc_bf16<C><<<(unsigned)(ntiles < cap ? ntiles : cap), kThreads, smem, st>>>(p);
-    return cudaGetLastError();
+    const long long ntiles = (p.pixels + kPix - 1) / kPix, cap = (C <= 64 ? 4LL : 2LL) * (tma::sm_count() > 0 ? tma::sm_count() : 148);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(ntiles < cap ? ntiles : cap));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];                             // may start (and stage w_fuse) while the stencil kernel drains
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, conv_fuse_nhwc_bf16<C>, p);
 }
 
 inline cudaError_t launch_fast(const Params& p, cudaStream_t st) {
