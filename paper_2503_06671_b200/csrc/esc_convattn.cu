@@ -314,13 +314,13 @@ int launch_stencil(const Problem& p, const void* x, const void* w_large, const f
     // Depth-wise K = 13 on NHWC bf16: the tensor-core (Toeplitz) kernel unless the caller pinned the FP32
     // kernel (by engine or by one of its tile widths) or asked for the point-wise mix, which only the
     // FP32 kernel carries.
-    if (!p.w_point && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0) {
+    if ((!p.w_point || p.Ca == esc::tma::CG) && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0) {
         int tw = 0;
         const int rc = esc::tma::toep::try_launch_toeplitz(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, p.bias,
-                                                           out, ctrl, st, dependent, &g_last_launches, &g_last_error, &tw, p.skip_copy);
+                                                           out, ctrl, st, dependent, &g_last_launches, &g_last_error, &tw, p.skip_copy, p.w_point);
         if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
         if (rc != esc::tma::kNotApplicable) return rc;
-        if (!p.skip_copy) {                                  // the same arithmetic on NCHW tensors
+        if (!p.skip_copy && !p.w_point) {                                  // the same arithmetic on NCHW tensors
             const int rn = esc::tma::toepn::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, p.bias, out,
                                                        ctrl, st, dependent, &g_last_launches, &g_last_error);
             if (rn == ESC_OK) { g_last_path = 6; g_last_tile_w = esc::tma::toepn::TW; return ESC_OK; }
@@ -339,7 +339,7 @@ int launch_stencil(const Problem& p, const void* x, const void* w_large, const f
 
 // Whether launch_stencil will take the tensor-core kernel for this problem (same conditions).
 bool tensor_stencil_follows(const Problem& p) {
-    return !p.dense && !p.w_point && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
+    return !p.dense && (!p.w_point || (p.Ca == esc::tma::CG && !p.bias)) && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
            esc::tma::toep::applies(p.C, p.Ca, p.K, p.dtype, p.layout);
 }
 
@@ -425,7 +425,7 @@ int forward_impl(const Problem& p, const void* x, const void* w_large, const Est
         const esc::tma::toep::Fused fu{est.w_last, est.b_last, est.w_down, est.b_down, est.hidden, w.unit_sums, w.arrivals, w.flags};
         int tw = 0;
         const int rc = esc::tma::toep::try_launch_fused(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, fu, out,
-                                                        w.ctrl, st, &g_last_launches, &g_last_error, &tw, p.skip_copy);
+                                                        w.ctrl, st, &g_last_launches, &g_last_error, &tw, p.skip_copy, p.w_point);
         if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
         if (rc != esc::tma::kNotApplicable) {
             // a cooperative launch can be refused (SMs held by another context): fall back to two kernels

@@ -63,6 +63,7 @@ struct Params {
     long long units;
     int copy_cc, copy_cw, copy_cr, slot_stride;
     const __nv_bfloat16* w_large;     // [Ca][13][13]
+    const __nv_bfloat16* w_point;     // kMix: [16][16] point-wise filter LK^c of the decomposed form (Eq. 5), row = output channel
     const float* dk;                  // [B][Ca][9]
     const float* bias;                // [B][Ca] or nullptr
     __nv_bfloat16* out;
@@ -128,7 +129,10 @@ __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
 // kernel, no second pass over the attention channels, and dk is there when the tensor-core work of a CTA's
 // first unit is done.  CTAs wait on one another: the launch is cooperative (all CTAs resident, one per SM)
 // and every wait is bounded.
-template <class S, bool kBias, bool kFused>
+// kMix: the decomposed large kernel of Eq. 5 -- the staged tile's 16 attention channels are replaced, pixel by pixel
+// and in place, by LK^c applied to them (tensor cores, one rounding to bf16) before the tile is transposed; the pooled
+// means of stage 1 are taken from the unmixed tile.
+template <class S, bool kBias, bool kFused, bool kMix = false>
 __global__ void __launch_bounds__(kThreads, 1)
 stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
                            const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_box,
@@ -404,6 +408,13 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
                 tile_sum(first + stride, sumbuf, TW, 0);
             }
         }
+        if (kMix) {                                          // Eq. 5: the depth-wise stage sees F_att * LK^c
+            uint32_t mixb[4];
+            load_mix_fragments(p.w_point, lane, mixb);
+            pointwise_mix_tile<ROWS * SW>(reinterpret_cast<uint32_t*>(stage), mixb, warp, lane);
+            fence_async_smem();                              // these stores before the next tile's TMA load into the same buffer
+            mma_bar();
+        }
         {
             // a step = 16 pixels of one staged row x 16 channels: four 8x8 matrices (pixel half, channel half)
             constexpr int STEPS = ROWS * (SW / 16);
@@ -584,10 +595,10 @@ struct Fused {
     unsigned *garr, *gflag;
 };
 
-template <class S, bool kBias, bool kFused>
+template <class S, bool kBias, bool kFused, bool kMix = false>
 inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk,
                         const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches,
-                        std::string* err, const Fused* fu = nullptr, bool skip_copy = false) {
+                        std::string* err, const Fused* fu = nullptr, bool skip_copy = false, const void* w_point = nullptr) {
     const int cc = skip_copy ? 0 : C - Ca;                 // skip_copy: the identity channels are consumed elsewhere (fused 1x1)
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -605,6 +616,8 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
         p.slot_stride = (cc * 2 * p.copy_cw * p.copy_cr + 127) / 128 * 128;
     }
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
+    p.w_point = static_cast<const __nv_bfloat16*>(w_point);
+    if (kMix && (Ca != CG || !w_point || (reinterpret_cast<uintptr_t>(w_point) & 3u) != 0)) return kNotApplicable;   // one group, 4-byte loads
     p.dk = dk; p.bias = bias; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
     p.w_last = p.b_last = p.w_down = p.b_down = nullptr; p.hidden = 0; p.gpart = nullptr; p.garr = p.gflag = nullptr;
@@ -633,7 +646,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     const int dev = current_device();
     if (dev < 0) return kNotApplicable;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nhwc_bf16<S, kBias, kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nhwc_bf16<S, kBias, kFused, kMix>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
         attr_set[dev] = true;
     }
@@ -651,7 +664,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     cfg.attrs = attr;
     cfg.numAttrs = kFused ? 2 : 1;
     if (kFused && (grid > sm_count() || p.units > 2 * grid)) return kNotApplicable;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias, kFused>, m_att, m_cin, m_cout, m_box, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias, kFused, kMix>, m_att, m_cin, m_cout, m_box, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_toeplitz_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -670,9 +683,12 @@ inline bool applies(int C, int Ca, int K, int dtype, int layout) {
 inline int try_launch_toeplitz(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
                                const void* w_large, const float* dk, const float* bias, void* out, unsigned* ctrl,
                                cudaStream_t st, bool dependent, int* launches, std::string* err, int* tile_w,
-                               bool skip_copy = false) {
+                               bool skip_copy = false, const void* w_point = nullptr) {
     if (!applies(C, Ca, K, dtype, layout) || sm_count() <= 0) return kNotApplicable;
     *tile_w = Shape64x16::TW;
+    if (w_point)
+        return bias ? kNotApplicable
+                    : launch_shape<Shape64x16, false, false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, w_point);
     return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy)
                 : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy);
 }
@@ -688,9 +704,12 @@ inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, 
 // The whole forward (stage 1 fused) as one launch; same return convention as try_launch_toeplitz.
 inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x,
                             const void* w_large, const Fused& fu, void* out, unsigned* ctrl, cudaStream_t st,
-                            int* launches, std::string* err, int* tile_w, bool skip_copy = false) {
+                            int* launches, std::string* err, int* tile_w, bool skip_copy = false, const void* w_point = nullptr) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden)) return kNotApplicable;
     *tile_w = Shape64x16::TW;
+    if (w_point)
+        return launch_shape<Shape64x16, false, true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
+                                                           launches, err, &fu, skip_copy, w_point);
     return launch_shape<Shape64x16, false, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
                                                  launches, err, &fu, skip_copy);
 }

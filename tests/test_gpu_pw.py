@@ -36,7 +36,7 @@ SHAPES = [
 ]
 
 
-def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True):
+def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True, engine=None):
     import torch
 
     B, C, C_a, H, W, K = shape
@@ -48,6 +48,8 @@ def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True):
     out = torch.full_like(x, 7.0)
     ws = pkg.new_workspace(B, C_a, H, W, K)
     pkg.esc_convattn_set_tile_width(width)
+    if engine is not None:
+        pkg.esc_convattn_set_stencil_engine(engine)
     try:
         if forward:
             pkg.esc_convattn_forward_pw(x, C_a, K, wl, wp_d, wd, bd, out, util.layout_code(layout), ws)
@@ -59,11 +61,12 @@ def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True):
         torch.cuda.synchronize()
     finally:
         pkg.esc_convattn_set_tile_width(0)
+        pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
     assert pkg.esc_convattn_device_status(ws) == 0
     got = util.to_host_nchw(out, layout)
     path = pkg.esc_convattn_last_path()
-    if dtype == synth.BF16 and path == 2:
-        # The fast kernel keeps the mixed features in its bf16 tile: one rounding of F_att * LK^c, as a
+    if dtype == synth.BF16 and path in (2, 4):
+        # The fast kernels keep the mixed features in its bf16 tile: one rounding of F_att * LK^c, as a
         # bf16 network stores that tensor.  (a) Against the exact oracle the error is bounded by the two
         # roundings: 2^-9 * sum|w||mixed| for the intermediate plus 2^-9 * |out| for the result, both
         # <= 2^-9 * mag.  (b) Against the oracle fed with the same rounded intermediate the usual bf16
@@ -75,7 +78,9 @@ def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True):
         dk_used = dk if not forward else oracle.dynkernel(oracle.gap(d["x"], C_a), d["w_dyn"], d["b_dyn"])
         ref2, mag2 = oracle.stencil(x2, C_a, d["w_large"], dk_used, want_mag=True)
         err2 = np.abs(got[:, :C_a] - ref2[:, :C_a])
-        assert (err2 / np.maximum(np.abs(ref2[:, :C_a]), 1.0)).max() <= util.BF16_REL
+        # (the rare outputs whose intermediate rounds to the other bf16 neighbour -- see below -- may also exceed the
+        # relative bar; (a) above still bounds every one of them)
+        assert ((err2 / np.maximum(np.abs(ref2[:, :C_a]), 1.0)) > util.BF16_REL).mean() <= 1e-5
         # one bf16 rounding of the result plus fp32 noise -- except where the fp32-accumulated mix and the
         # oracle's fp64 mix round a value to different bf16 neighbours, which moves an output by one
         # tap's worth; that may happen to a few outputs in a hundred thousand, not more
@@ -93,7 +98,21 @@ def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True):
 def test_forward_pw(pkg, oracle, shape, dtype, layout):
     path, _ = _run(pkg, oracle, shape, dtype, layout)
     fast = dtype == synth.BF16 and layout == synth.NHWC and shape[5] == 13 and shape[2] == 16
-    assert path == (2 if fast else 1)
+    assert path == (4 if fast else 1)                      # the mix inside the tensor-core depth-wise kernel
+
+
+@pytest.mark.parametrize("forward", [True, False], ids=["forward", "stencil"])
+@pytest.mark.parametrize("shape", [s for s in SHAPES if s[2] == 16 and s[5] == 13] + [(1, 64, 16, 300, 640, 13), (70, 32, 16, 40, 64, 13)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_pw_on_either_engine(pkg, oracle, shape, forward):
+    """The mix inside the tensor-core kernel (one launch for the forward where at most two units fall to a CTA:
+    the last two shapes give CTAs two units, of one image and of two) and inside the FP32 kernel."""
+    import paper_2503_06671_b200 as p
+
+    path, _ = _run(pkg, oracle, shape, synth.BF16, synth.NHWC, forward=forward, engine=p.ESC_ENGINE_AUTO)
+    assert path == 4
+    path, _ = _run(pkg, oracle, shape, synth.BF16, synth.NHWC, forward=forward, engine=p.ESC_ENGINE_FP32)
+    assert path == 2
 
 
 @pytest.mark.parametrize("width", [40, 64])
@@ -104,9 +123,10 @@ def test_stencil_pw_both_tile_geometries(pkg, oracle, shape, width):
     assert path == 2 and used == width
 
 
-def test_identity_mix_reproduces_the_plain_forward_bit_for_bit(pkg):
+@pytest.mark.parametrize("which", ["tensor", "fp32"])
+def test_identity_mix_reproduces_the_plain_forward_bit_for_bit(pkg, which):
     """With LK^c = I the tensor-core mix returns every bf16 value unchanged, so the result equals the
-    depth-wise forward of the same (FP32) stencil kernel exactly."""
+    depth-wise forward of the same stencil kernel exactly (either engine: compare like with like)."""
     import torch
 
     B, C, C_a, H, W, K = 2, 64, 16, 70, 100, 13
@@ -116,12 +136,12 @@ def test_identity_mix_reproduces_the_plain_forward_bit_for_bit(pkg):
     eye = torch.eye(C_a, dtype=torch.bfloat16, device="cuda")
     ws = pkg.new_workspace(B, C_a, H, W, K)
     a, b = torch.empty_like(x), torch.empty_like(x)
-    pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32)      # the mix lives in the FP32 kernel: compare like with like
+    pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32 if which == "fp32" else pkg.ESC_ENGINE_AUTO)
     try:
         pkg.esc_convattn_forward_ex(x, C_a, K, wl, wd, bd, a, pkg.ESC_NHWC, ws)
+        pkg.esc_convattn_forward_pw(x, C_a, K, wl, eye, wd, bd, b, pkg.ESC_NHWC, ws)
+        torch.cuda.synchronize()
     finally:
         pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
-    pkg.esc_convattn_forward_pw(x, C_a, K, wl, eye, wd, bd, b, pkg.ESC_NHWC, ws)
-    torch.cuda.synchronize()
-    assert pkg.esc_convattn_last_path() == 2
+    assert pkg.esc_convattn_last_path() == (2 if which == "fp32" else 4)
     assert torch.equal(a.view(torch.int16), b.view(torch.int16))
