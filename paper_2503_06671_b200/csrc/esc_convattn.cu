@@ -19,6 +19,7 @@
 #include "stencil_tma.cuh"
 #include "stencil_toeplitz.cuh"
 #include "stencil_toeplitz_nchw.cuh"
+#include "backward_toeplitz.cuh"
 #include "stencil_dense.cuh"
 #include "stencil_dense_umma.cuh"
 #include "backward.cuh"
@@ -458,8 +459,9 @@ struct BackwardWs {
     size_t bytes;
 };
 BackwardWs carve_backward(void* ws, const Problem& p) {
-    // sized for the finer of the two tilings the tap-gradient kernels use (32x32)
-    const int tiles = ((p.W + esc::bwd::n8::TX - 1) / esc::bwd::n8::TX) * ((p.H + esc::bwd::n8::TY - 1) / esc::bwd::n8::TY);
+    // sized for whichever tiling of the tap-gradient kernels has more tiles (32x32, or 64x16 on the tensor cores)
+    const int tiles = std::max(((p.W + esc::bwd::n8::TX - 1) / esc::bwd::n8::TX) * ((p.H + esc::bwd::n8::TY - 1) / esc::bwd::n8::TY),
+                               esc::bwd::toep::tiles_of(p.H, p.W));
     BackwardWs w;
     char* base = static_cast<char*>(ws);
     size_t off = 256;
@@ -476,13 +478,23 @@ BackwardWs carve_backward(void* ws, const Problem& p) {
 template <typename T, int LAYOUT>
 int backward_t(const Problem& p, const void* x, const void* go, const void* w_large, const void* w_dyn,
                const void* b_dyn, const BackwardWs& w, float* g_lk, float* g_w, float* g_b, cudaStream_t st) {
+    // bf16 NHWC with whole groups of 16 channels: the tensor-core kernel
+    int tiles_done = 0;
+    if (g_engine_policy != ESC_ENGINE_FP32) {
+        const int rt = esc::bwd::toep::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, go, w.part, w.ctrl, st,
+                                                  &g_last_launches, &g_last_error);
+        if (rt == ESC_OK) tiles_done = esc::bwd::toep::tiles_of(p.H, p.W);
+        else if (rt != esc::tma::kNotApplicable) return rt;
+    }
     // NHWC with whole octets of channels: eight channels per block, 16-byte loads; else a block per channel
     const bool oct = LAYOUT == esc::kNHWC && p.Ca % 8 == 0 && p.C % 8 == 0;
     const int TXs = oct ? esc::bwd::n8::TX : esc::bwd::TX, TYs = oct ? esc::bwd::n8::TY : esc::bwd::TY;
     const int tiles_x = (p.W + TXs - 1) / TXs, tiles_y = (p.H + TYs - 1) / TYs;
     const long long blocks = (long long)p.B * (oct ? p.Ca / 8 : p.Ca) * tiles_x * tiles_y;
     if (blocks > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
-    if (oct) {
+    if (tiles_done > 0) {
+        // done above
+    } else if (oct) {
         static bool attr_set[esc::tma::kMaxDevices] = {};
         const int dev = esc::tma::current_device();
         if (dev < 0) return ESC_ERR_UNSUPPORTED;
@@ -498,13 +510,14 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
             static_cast<const T*>(x), static_cast<const T*>(go), p.C, p.Ca, p.H, p.W, tiles_x, tiles_y, w.part);
     }
     ESC_CUDA(cudaGetLastError());
-    esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), 192, 0, st>>>(w.part, tiles_x * tiles_y, w.gtap);
+    if (tiles_done == 0) ++g_last_launches;
+    esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), 192, 0, st>>>(w.part, tiles_done > 0 ? tiles_done : tiles_x * tiles_y, w.gtap);
     ESC_CUDA(cudaGetLastError());
     esc::bwd::finish<T><<<64, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, static_cast<const T*>(w_large),
                                             static_cast<const T*>(w_dyn), static_cast<const T*>(b_dyn), g_lk, g_w, g_b,
                                             static_cast<T*>(w.w_flip), w.dk_flip, w.bias);
     ESC_CUDA(cudaGetLastError());
-    g_last_launches += 3;
+    g_last_launches += 2;
     return ESC_OK;
 }
 

@@ -78,6 +78,50 @@ def test_backward(pkg, oracle, shape, dtype, layout):
     assert (err <= bar).all(), f"grad x: {int((err > bar).sum())} values beyond the bound"
 
 
+def _run_backward(pkg, d, go, C_a, K, dtype, layout):
+    import torch
+
+    x = util.to_device(d["x"], dtype, layout)
+    go_d = util.to_device(go, dtype, layout)
+    wl, wd, bd = util.weights_to_device(d, dtype)
+    B, _, H, W = d["x"].shape
+    gx = torch.full_like(x, 7.0)
+    g_lk = torch.full((C_a, K, K), float("nan"), device="cuda")
+    g_w = torch.full((9 * C_a, C_a), float("nan"), device="cuda")
+    g_b = torch.full((9 * C_a,), float("nan"), device="cuda")
+    ws = pkg.new_backward_workspace(B, C_a, H, W, K)
+    for _ in range(2):
+        pkg.esc_convattn_backward(x, go_d, C_a, K, wl, wd, bd, gx, g_lk, g_w, g_b, util.layout_code(layout), ws)
+    torch.cuda.synchronize()
+    assert pkg.esc_convattn_device_status(ws) == 0
+    return gx, g_lk, g_w, g_b
+
+
+@pytest.mark.parametrize("shape", [(1, 64, 16, 300, 640), (6, 32, 32, 130, 200), (40, 16, 16, 64, 64)], ids=lambda s: "x".join(map(str, s)))
+def test_backward_weight_gradients_many_units(pkg, oracle, shape):
+    """bf16 NHWC, where the tap gradients run on the tensor cores: 190, 432 and 160 units of 64x16 on 148 SMs, so CTAs
+    walk two or three units (staging buffers, planes and barriers are re-used; image and channel group change inside
+    a walk); the three weight gradients against the oracle, and against the FP32-pipe kernels."""
+    B, C, C_a, H, W = shape
+    K = 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=sum(shape) + 3, per_image_scale=True, channel_means=True)
+    go = synth.round_to(np.random.default_rng(sum(shape) + 4).standard_normal(size=d["x"].shape).astype(np.float32), synth.BF16)
+    _, g_lk, g_w, g_b = _run_backward(pkg, d, go, C_a, K, synth.BF16, synth.NHWC)
+    _, rlk, rw, rb = oracle.backward(d["x"], go, C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    _, alk, aw, ab = oracle.backward(np.abs(d["x"]), np.abs(go), C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    for name, got, ref, scale in (("w_large", g_lk, rlk, alk), ("w_dyn", g_w, rw, aw), ("b_dyn", g_b, rb, ab)):
+        err = np.abs(got.cpu().numpy().astype(np.float64) - ref)
+        assert (err <= 1e-5 * scale + 1e-30).all(), f"grad {name}: worst {(err / np.maximum(scale, 1e-30)).max():.3e} of its scale"
+    pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32)
+    try:
+        _, f_lk, f_w, f_b = _run_backward(pkg, d, go, C_a, K, synth.BF16, synth.NHWC)
+    finally:
+        pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
+    for name, a, b, scale in (("w_large", g_lk, f_lk, alk), ("w_dyn", g_w, f_w, aw), ("b_dyn", g_b, f_b, ab)):
+        err = np.abs(a.cpu().numpy().astype(np.float64) - b.cpu().numpy().astype(np.float64))
+        assert (err <= 2e-5 * scale + 1e-30).all(), f"grad {name}: the two kernels differ by {(err / np.maximum(scale, 1e-30)).max():.3e} of its scale"
+
+
 def test_backward_rejections(pkg):
     import torch
 
