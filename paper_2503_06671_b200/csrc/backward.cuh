@@ -240,71 +240,106 @@ tap_grad_nhwc8(const T* __restrict__ x, const T* __restrict__ go, int C, int Ca,
     if (lane == 0) slot[TAPS] = sx;
 }
 
-// ---- kernel 2a: add the tiles of one (image, channel) in order ---------------------------------------------
-__global__ void __launch_bounds__(192)
+// ---- kernel 2a: add the tiles of one (image, channel) in a fixed order -----------------------------------------
+// Block = (image, channel); kSumGroups groups of 192 threads take every kSumGroups-th tile each (eight loads in
+// flight, added in order), then the groups' sums are added in group order.
+constexpr int kSumGroups = 4, kSumThreads = 192 * kSumGroups;
+__global__ void __launch_bounds__(kSumThreads)
 sum_tiles(const float* __restrict__ part, int tiles, float* __restrict__ gtap)   // gtap [B*Ca][kSlot]
 {
+    __shared__ float acc[kSumGroups][192];
     const size_t bc = blockIdx.x;
-    const int t = threadIdx.x;
-    if (t > TAPS) return;
-    const float* p = part + bc * tiles * kSlot + t;
-    float s = 0.f;
-    for (int k = 0; k < tiles; ++k) s += p[(size_t)k * kSlot];
-    gtap[bc * kSlot + t] = s;
+    const int t = threadIdx.x % 192, grp = threadIdx.x / 192;
+    if (t <= TAPS) {
+        const float* p = part + bc * tiles * kSlot + t;
+        float s = 0.f;
+#pragma unroll 8
+        for (int k = grp; k < tiles; k += kSumGroups) s += p[(size_t)k * kSlot];
+        acc[grp][t] = s;
+    }
+    __syncthreads();
+    if (grp == 0 && t <= TAPS) {
+        float s = acc[0][t];
+#pragma unroll
+        for (int q = 1; q < kSumGroups; ++q) s += acc[q][t];
+        gtap[bc * kSlot + t] = s;
+    }
 }
 
 // ---- kernel 2b: everything small; every output element is independent, a few blocks share them ------------
 // From g_tap [B][Ca][169 + sum x]: g_lk, g_b, g_W (fp32 outputs), and for the stencil pass that follows the
 // kernels rotated by 180 degrees -- w_flip (element type T), dk_flip [B][Ca][9] -- and the constants
 // bias[b][c] = g_g[b,c] / (H W).  g[b,k] = sum x / (H W) and dk = b_dyn + W g are recomputed here.
+constexpr int kFinishRoles = 6, kFinishBlocks = 32 * kFinishRoles;
 template <typename T>
 __global__ void __launch_bounds__(256)
 finish(const float* __restrict__ gtap, int B, int Ca, int H, int W, const T* __restrict__ w_large,
        const T* __restrict__ w_dyn, const T* __restrict__ b_dyn, float* __restrict__ g_lk, float* __restrict__ g_w,
        float* __restrict__ g_b, T* __restrict__ w_flip, float* __restrict__ dk_flip, float* __restrict__ bias)
 {
-    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+    // Six independent jobs; each takes a sixth of the grid, so that their chains of dependent loads run side by side
+    // instead of one after the other in every thread.
+    const int per_role = gridDim.x / kFinishRoles, role = blockIdx.x / per_role;
+    const int tid = (blockIdx.x % per_role) * blockDim.x + threadIdx.x, nth = per_role * blockDim.x;
     const float inv_hw = 1.0f / ((float)H * (float)W);
     auto gdk = [&](int b, int o) {                        // o = c*9 + i*3 + j -> central 3x3 of the tap gradient
         const int c = o / 9, i = (o % 9) / 3, j = o % 3;
         return gtap[((size_t)b * Ca + c) * kSlot + (i + P - 1) * K + (j + P - 1)];
     };
     auto gmean = [&](int b, int k) { return gtap[((size_t)b * Ca + k) * kSlot + TAPS] * inv_hw; };
-    if (g_lk)
+    if (role == 0 && g_lk)
         for (int e = tid; e < Ca * TAPS; e += nth) {
             const int c = e / TAPS, t = e % TAPS;
             float s = 0.f;
+#pragma unroll 8
             for (int b = 0; b < B; ++b) s += gtap[((size_t)b * Ca + c) * kSlot + t];
             g_lk[e] = s;
         }
-    if (g_b)
+    if (role == 1 && g_b)
         for (int o = tid; o < 9 * Ca; o += nth) {
             float s = 0.f;
+#pragma unroll 8
             for (int b = 0; b < B; ++b) s += gdk(b, o);
             g_b[o] = s;
         }
-    if (g_w)
+    if (role == 2 && g_w)
         for (int e = tid; e < 9 * Ca * Ca; e += nth) {
             const int o = e / Ca, k = e % Ca;
             float s = 0.f;
+#pragma unroll 8
             for (int b = 0; b < B; ++b) s = fmaf(gdk(b, o), gmean(b, k), s);
             g_w[e] = s;
         }
+    if (role == 3)
     for (int e = tid; e < Ca * TAPS; e += nth) {
         const int c = e / TAPS, t = e % TAPS;
         w_flip[(size_t)c * TAPS + (TAPS - 1 - t)] = w_large[e];
     }
+    if (role == 4)
     for (int e = tid; e < B * Ca * 9; e += nth) {
         const int b = e / (9 * Ca), o = e % (9 * Ca), c = o / 9, t = o % 9;
         float s = Elem<T>::to_f32(b_dyn[o]);
+#pragma unroll 8
         for (int k = 0; k < Ca; ++k) s = fmaf(Elem<T>::to_f32(w_dyn[(size_t)o * Ca + k]), gmean(b, k), s);
         dk_flip[((size_t)b * Ca + c) * 9 + (8 - t)] = s;
     }
-    for (int e = tid; e < B * Ca; e += nth) {
-        const int b = e / Ca, k = e % Ca;
-        float s = 0.f;
-        for (int o = 0; o < 9 * Ca; ++o) s = fmaf(Elem<T>::to_f32(w_dyn[(size_t)o * Ca + k]), gdk(b, o), s);
-        bias[e] = s * inv_hw;
+    if (role == 5) {
+        // bias[b][k] = sum_o W[o][k] g_dk[b][o] / (H W): a warp per element, lane = channel c (nine taps each, all loads
+        // independent), then a fixed butterfly over the lanes
+        const int lane = threadIdx.x & 31, wid = tid >> 5, nw = nth >> 5;
+        for (int e = wid; e < B * Ca; e += nw) {
+            const int b = e / Ca, k = e % Ca;
+            float s = 0.f;
+            for (int c = lane; c < Ca; c += 32) {
+                const float* gt = gtap + ((size_t)b * Ca + c) * kSlot + (P - 1) * K + (P - 1);
+#pragma unroll
+                for (int ij = 0; ij < 9; ++ij)
+                    s = fmaf(Elem<T>::to_f32(w_dyn[(size_t)(c * 9 + ij) * Ca + k]), gt[(ij / 3) * K + ij % 3], s);
+            }
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane == 0) bias[e] = s * inv_hw;
+        }
     }
 }
 

@@ -511,9 +511,9 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
     }
     ESC_CUDA(cudaGetLastError());
     if (tiles_done == 0) ++g_last_launches;
-    esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), 192, 0, st>>>(w.part, tiles_done > 0 ? tiles_done : tiles_x * tiles_y, w.gtap);
+    esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), esc::bwd::kSumThreads, 0, st>>>(w.part, tiles_done > 0 ? tiles_done : tiles_x * tiles_y, w.gtap);
     ESC_CUDA(cudaGetLastError());
-    esc::bwd::finish<T><<<64, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, static_cast<const T*>(w_large),
+    esc::bwd::finish<T><<<esc::bwd::kFinishBlocks, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, static_cast<const T*>(w_large),
                                             static_cast<const T*>(w_dyn), static_cast<const T*>(b_dyn), g_lk, g_w, g_b,
                                             static_cast<T*>(w.w_flip), w.dk_flip, w.bias);
     ESC_CUDA(cudaGetLastError());
