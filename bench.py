@@ -573,6 +573,23 @@ def main():
                         "and writes out; separate: forward (read x, write cat), conv (read cat, write y), add (read y, residual, write y)"}
         except Exception as exc:                                          # never lose the headline over an extra
             extras["module_with_conv_fuse"] = {"error": f"{type(exc).__name__}: {exc}"}
+        # the backward pass of the same module (gradients of x, LK, W_dyn, b_dyn): tap gradients and the stencil on
+        # grad_out, 2 x K x K multiply-adds per attention pixel-channel
+        try:
+            go_d = torch.randn_like(xs[0])
+            gx_d = torch.empty_like(xs[0])
+            g_lk = torch.zeros(wl.C_a, wl.K, wl.K, device="cuda")
+            g_w = torch.zeros(9 * wl.C_a, wl.C_a, device="cuda")
+            g_b = torch.zeros(9 * wl.C_a, device="cuda")
+            bws = pkg.new_backward_workspace(wl.B, wl.C_a, wl.H, wl.W, wl.K)
+            st, _ = timer.measure(lambda i: pkg.esc_convattn_backward(xs[i % n_rot], go_d, wl.C_a, wl.K, wl_d, wd_d, bd_d, gx_d, g_lk, g_w, g_b,
+                                                                      lay_code, bws), samples=5)
+            t_fma = 2.0 * 2.0 * wl.K * wl.K * wl.C_a * wl.pixels / (sms * FMA_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6)
+            extras["backward"] = {"ms_per_step": st["median_ms"], "launches": pkg.esc_convattn_last_launches(),
+                                  "frac_of_fp32_roofline": t_fma / (st["median_ms"] * 1e-3),
+                                  "note": "roofline: 2 x K x K multiply-adds per attention pixel-channel on the FP32 pipe"}
+        except Exception as exc:
+            extras["backward"] = {"error": f"{type(exc).__name__}: {exc}"}
         # with the dense large kernel of the main model (Section 3.2): an implicit GEMM on the tensor cores
         if wl.C_a == 16 and wl.K == 13:
             wdn_d = torch.from_numpy(synth.make_dense_kernel(wl.C_a, wl.K, wl.dtype, wl.seed)).to(tdt).cuda()
