@@ -12,6 +12,7 @@ from .convattn_oracle import (  # noqa: F401
     forward_mlp,
     stencil,
     backward,
+    backward_mlp,
     stencil_dense,
     forward_dense,
     pointwise,

@@ -220,6 +220,33 @@ def backward(x, grad_out, C_a, w_large, w_dyn, b_dyn):
     return gx, glk, gw, gb
 
 
+def backward_mlp(x, grad_out, C_a, w_large, w_down, b_down, w_up, b_up):
+    """Gradients of forward_mlp(x, ...) contracted with grad_out: returns (gx [B,C,H,W], g_w_large [C_a,K,K],
+    g_w_down [h,C_a], g_b_down [h], g_w_up [9*C_a,h], g_b_up [9*C_a])."""
+    x, xp = _f32(x)
+    go, gp = _f32(grad_out)
+    assert go.shape == x.shape
+    w_large, wp = _f64(w_large)
+    K = int(w_large.shape[-1])
+    assert K >= 3
+    B, C, H, W = _dims(x, C_a, K)
+    w_down, wdp = _f64(w_down)
+    b_down, bdp = _f64(b_down)
+    w_up, wup = _f64(w_up)
+    b_up, bup = _f64(b_up)
+    h = int(w_down.shape[0])
+    assert w_down.shape == (h, C_a) and b_down.shape == (h,) and w_up.shape == (9 * C_a, h) and b_up.shape == (9 * C_a,)
+    gx = np.empty((B, C, H, W), dtype=np.float64)
+    glk = np.empty((C_a, K, K), dtype=np.float64)
+    gwd = np.empty((h, C_a), dtype=np.float64)
+    gbd = np.empty((h,), dtype=np.float64)
+    gwu = np.empty((9 * C_a, h), dtype=np.float64)
+    gbu = np.empty((9 * C_a,), dtype=np.float64)
+    _load().convattn_ref_backward_mlp(xp, gp, B, C, C_a, H, W, K, wp, h, wdp, bdp, wup, bup, *(a.ctypes.data_as(_f64p)
+                                      for a in (gx, glk, gwd, gbd, gwu, gbu)))
+    return gx, glk, gwd, gbd, gwu, gbu
+
+
 def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
     """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
     x, xp = _f32(x)

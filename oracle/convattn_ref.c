@@ -32,7 +32,8 @@
  * with the block's residual connection (Eq. 3 line 3).
  *
  * convattn_ref_backward is the gradient of the first form above with respect to x, LK, W_dyn and
- * b_dyn, by the chain rule written out.
+ * b_dyn, by the chain rule written out; convattn_ref_backward_mlp the same with the two-layer estimator
+ * (gradients with respect to x, LK, W_down, b_down, W_up, b_up).
  *
  * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
  * Everything is accumulated in double precision with direct nested loops in
@@ -57,7 +58,9 @@
  * convolution, the depth-wise-then-point-wise factorisation and a brute force; the
  * backward pass by central differences of the pinned forward (exact for this
  * function, which is quadratic in x and bilinear in weights and x) and the
- * adjoint identity.
+ * adjoint identity; the backward pass with the two-layer estimator by central differences of
+ * the pinned forward and by its linear limit, where it must equal the pinned one-layer backward
+ * with composed weights.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -446,6 +449,148 @@ void convattn_ref_backward(const float *x, const float *go, int B, int C, int C_
                     }
     }
     free(g); free(dk); free(gtap); free(gg); free(gdk);
+}
+
+/* Derivative of the Gaussian error linear unit phi(t) = t * Phi(t): phi'(t) = Phi(t) + t * n(t), n the standard
+ * normal density. */
+static double gelu_prime(double t)
+{
+    return 0.5 * erfc(-t / sqrt(2.0)) + t * exp(-0.5 * t * t) / sqrt(2.0 * 3.14159265358979323846);
+}
+
+/* Backward pass of the forward with the estimator as Eq. 4 line 2 writes it (two layers, GELU between them; depth-wise
+ * LK), by the chain rule written out.  With g = GAP(x), t = W_down g + b_down, a = phi(t), dk = W_up a + b_up, and
+ * g_tap, g_lk, g_dk as in convattn_ref_backward:
+ *   g_bu[o]   = sum_b g_dk[b,o]                   g_Wu[o,m] = sum_b g_dk[b,o] * a[b,m]
+ *   g_a[b,m]  = sum_o W_up[o,m] * g_dk[b,o]       g_t[b,m]  = g_a[b,m] * phi'(t[b,m])
+ *   g_bd[m]   = sum_b g_t[b,m]                    g_Wd[m,k] = sum_b g_t[b,m] * g[b,k]
+ *   g_g[b,k]  = sum_m W_down[m,k] * g_t[b,m]
+ *   g_x[b,c,y,x] = sum_{i,j} Wm[b,c,i,j] * go~[b,c,y-(i-P),x-(j-P)] + g_g[b,c] / (H*W)   (c < C_a);   g_x[b,c] = go[b,c]  (c >= C_a)
+ * Outputs: gx [B,C,H,W], glk [C_a,K,K], gwd [h,C_a], gbd [h], gwu [9*C_a,h], gbu [9*C_a]; any may be NULL.  K >= 3. */
+void convattn_ref_backward_mlp(const float *x, const float *go, int B, int C, int C_a, int H, int W, int K,
+                               const double *w_large, int h, const double *w_down, const double *b_down,
+                               const double *w_up, const double *b_up,
+                               double *gx, double *glk, double *gwd, double *gbd, double *gwu, double *gbu)
+{
+    const int P = (K - 1) / 2;
+    double *g = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    double *t = (double *)malloc(sizeof(double) * (size_t)B * h);
+    double *a = (double *)malloc(sizeof(double) * (size_t)B * h);
+    double *dk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    double *gtap = (double *)malloc(sizeof(double) * (size_t)B * C_a * K * K);
+    double *gdk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    double *gt = (double *)malloc(sizeof(double) * (size_t)B * h);
+    double *gg = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    /* forward quantities */
+    convattn_ref_gap(x, B, C, C_a, H, W, g);
+    for (int b = 0; b < B; ++b) {
+        for (int m = 0; m < h; ++m) {
+            double s = b_down[m];
+            for (int k = 0; k < C_a; ++k) s += w_down[(size_t)m * C_a + k] * g[(size_t)b * C_a + k];
+            t[(size_t)b * h + m] = s;
+            a[(size_t)b * h + m] = gelu(s);
+        }
+        for (int o = 0; o < 9 * C_a; ++o) {
+            double s = b_up[o];
+            for (int m = 0; m < h; ++m) s += w_up[(size_t)o * h + m] * a[(size_t)b * h + m];
+            dk[(size_t)b * 9 * C_a + o] = s;
+        }
+    }
+    /* per-image tap gradients */
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C_a; ++c)
+            for (int i = 0; i < K; ++i)
+                for (int j = 0; j < K; ++j) {
+                    double s = 0.0;
+                    for (int y = 0; y < H; ++y)
+                        for (int xx = 0; xx < W; ++xx) {
+                            int yy = y + i - P, xc = xx + j - P;
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                s += (double)go[IDX4(b, c, y, xx, C, H, W)] * (double)x[IDX4(b, c, yy, xc, C, H, W)];
+                        }
+                    gtap[(((size_t)b * C_a + c) * K + i) * K + j] = s;
+                }
+    if (glk)
+        for (int c = 0; c < C_a; ++c)
+            for (int q = 0; q < K * K; ++q) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gtap[((size_t)b * C_a + c) * K * K + q];
+                glk[(size_t)c * K * K + q] = s;
+            }
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C_a; ++c)
+            for (int i = 0; i < 3; ++i)
+                for (int j = 0; j < 3; ++j)
+                    gdk[((size_t)b * C_a + c) * 9 + i * 3 + j] = gtap[(((size_t)b * C_a + c) * K + i + P - 1) * K + j + P - 1];
+    /* second layer */
+    if (gbu)
+        for (int o = 0; o < 9 * C_a; ++o) {
+            double s = 0.0;
+            for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o];
+            gbu[o] = s;
+        }
+    if (gwu)
+        for (int o = 0; o < 9 * C_a; ++o)
+            for (int m = 0; m < h; ++m) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o] * a[(size_t)b * h + m];
+                gwu[(size_t)o * h + m] = s;
+            }
+    /* through the activation */
+    for (int b = 0; b < B; ++b)
+        for (int m = 0; m < h; ++m) {
+            double s = 0.0;
+            for (int o = 0; o < 9 * C_a; ++o) s += w_up[(size_t)o * h + m] * gdk[(size_t)b * 9 * C_a + o];
+            gt[(size_t)b * h + m] = s * gelu_prime(t[(size_t)b * h + m]);
+        }
+    /* first layer */
+    if (gbd)
+        for (int m = 0; m < h; ++m) {
+            double s = 0.0;
+            for (int b = 0; b < B; ++b) s += gt[(size_t)b * h + m];
+            gbd[m] = s;
+        }
+    if (gwd)
+        for (int m = 0; m < h; ++m)
+            for (int k = 0; k < C_a; ++k) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gt[(size_t)b * h + m] * g[(size_t)b * C_a + k];
+                gwd[(size_t)m * C_a + k] = s;
+            }
+    for (int b = 0; b < B; ++b)
+        for (int k = 0; k < C_a; ++k) {
+            double s = 0.0;
+            for (int m = 0; m < h; ++m) s += w_down[(size_t)m * C_a + k] * gt[(size_t)b * h + m];
+            gg[(size_t)b * C_a + k] = s;
+        }
+    if (gx) {
+#pragma omp parallel for collapse(3) schedule(static)
+        for (int b = 0; b < B; ++b)
+            for (int c = 0; c < C; ++c)
+                for (int y = 0; y < H; ++y)
+                    for (int xx = 0; xx < W; ++xx) {
+                        if (c >= C_a) {
+                            gx[IDX4(b, c, y, xx, C, H, W)] = (double)go[IDX4(b, c, y, xx, C, H, W)];
+                            continue;
+                        }
+                        double s = 0.0;
+                        for (int i = 0; i < K; ++i)
+                            for (int j = 0; j < K; ++j) {
+                                int yy = y - (i - P), xc = xx - (j - P);
+                                if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                    s += w_large[((size_t)c * K + i) * K + j] * (double)go[IDX4(b, c, yy, xc, C, H, W)];
+                            }
+                        for (int i = 0; i < 3; ++i)
+                            for (int j = 0; j < 3; ++j) {
+                                int yy = y - (i - 1), xc = xx - (j - 1);
+                                if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                    s += dk[((size_t)b * C_a + c) * 9 + i * 3 + j] * (double)go[IDX4(b, c, yy, xc, C, H, W)];
+                            }
+                        gx[IDX4(b, c, y, xx, C, H, W)] = s + gg[(size_t)b * C_a + c] / ((double)H * (double)W);
+                    }
+    }
+    free(g); free(t); free(a); free(dk); free(gtap); free(gdk); free(gt); free(gg);
 }
 
 /* Selected outputs, one by one: idx[n] are flat indices into out[B,C,H,W]; dk is
