@@ -285,6 +285,24 @@ int esc_convattn_backward(const void* x, const void* grad_out, int B, int C, int
                           int dtype, int layout,
                           void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Backward pass of esc_convattn_forward_mlp: the same with the estimator as Eq. 4 line 2 writes it,
+ * dk = W_up phi(W_down g + b_down) + b_up with phi(t) = t Phi(t) (exact GELU), differentiated through
+ * phi'(t) = Phi(t) + t n(t) (n the standard normal density).  Weight layouts as in esc_convattn_forward_mlp:
+ * w_down [hidden,C_a], b_down [hidden], w_up [9*C_a,hidden], b_up [9*C_a], element type of x; 1 <= hidden <= 128.
+ *   grad_x        [B,C,H,W]        as above
+ *   grad_w_large  [C_a,K,K]        fp32   (may be NULL)
+ *   grad_w_down   [hidden,C_a]     fp32   (may be NULL)        grad_b_down [hidden]   fp32 (may be NULL)
+ *   grad_w_up     [9*C_a,hidden]   fp32   (may be NULL)        grad_b_up   [9*C_a]    fp32 (may be NULL)
+ * Same workspace, restrictions and error codes as esc_convattn_backward; ESC_ERR_SHAPE for hidden out of range.
+ */
+int esc_convattn_backward_mlp(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                              const void* w_large, const void* w_down, const void* b_down,
+                              const void* w_up, const void* b_up, int hidden,
+                              void* grad_x, float* grad_w_large, float* grad_w_down, float* grad_b_down,
+                              float* grad_w_up, float* grad_b_up, int dtype, int layout,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

@@ -1,5 +1,5 @@
-// Backward pass of the ConvAttn forward (ESC paper, Section 3.3, Eq. 4, one-layer estimator, depth-wise LK),
-// the chain rule written out.  With go = dL/dout and Wm[b,c] = LK[c] + ZP(dk[b,c]):
+// Backward pass of the ConvAttn forward (ESC paper, Section 3.3, Eq. 4, depth-wise LK; one-layer estimator, or the
+// two-layer estimator of Eq. 4 line 2 at the end of this file), the chain rule written out.  With go = dL/dout and Wm[b,c] = LK[c] + ZP(dk[b,c]):
 //
 //   g_tap[b,c,i,j] = sum_{y,x} go[b,c,y,x] * x~[b,c,y+i-6,x+j-6]      per-image tap gradient  (kernel tap_grad)
 //   g_lk = sum_b g_tap;   g_dk = central 3x3 of g_tap;   g_b = sum_b g_dk;   g_W[o,k] = sum_b g_dk[b,o] g[b,k]
@@ -12,6 +12,7 @@
 #pragma once
 #include "common.cuh"
 #include "stencil_generic.cuh"
+#include "gap_dynkernel.cuh"
 
 namespace esc { namespace bwd {
 
@@ -341,6 +342,125 @@ finish(const float* __restrict__ gtap, int B, int Ca, int H, int W, const T* __r
             if (lane == 0) bias[e] = s * inv_hw;
         }
     }
+}
+
+// ---- the estimator as Eq. 4 line 2 writes it: two layers with the exact GELU between them ---------------------
+//   t = W_down g + b_down,  a = phi(t),  dk = W_up a + b_up;   phi'(t) = Phi(t) + t n(t)
+//   g_a[b,m] = sum_o W_up[o,m] g_dk[b,o],   g_t = g_a * phi'(t),   g_g[b,k] = sum_m W_down[m,k] g_t[b,m]
+//   g_b_up = sum_b g_dk,  g_W_up[o,m] = sum_b g_dk[b,o] a[b,m],  g_b_down = sum_b g_t,  g_W_down[m,k] = sum_b g_t[b,m] g[b,k]
+__device__ __forceinline__ float gelu_exact_prime(float t) {
+    return 0.5f * erfcf(-0.70710678118654752f * t) + t * 0.3989422804014327f * expf(-0.5f * t * t);
+}
+
+// kernel 2c: one block per image -- the estimator's forward values and the part of the chain that belongs to one
+// image: a and g_t go to the workspace for the sums over images, dk (rotated) and the GAP-path constant to the
+// stencil pass that follows.  Dynamic shared memory: (10 Ca + 3 hidden) floats.
+template <typename T>
+__global__ void __launch_bounds__(256)
+mlp_image(const float* __restrict__ gtap, int Ca, int hidden, int H, int W, const T* __restrict__ w_down,
+          const T* __restrict__ b_down, const T* __restrict__ w_up, const T* __restrict__ b_up,
+          float* __restrict__ act, float* __restrict__ gt, float* __restrict__ dk_flip, float* __restrict__ bias)
+{
+    extern __shared__ float sm[];
+    float* gm = sm;                    // [Ca] pooled means
+    float* gd = gm + Ca;               // [9 Ca] g_dk of this image
+    float* tt = gd + 9 * Ca;           // [hidden] pre-activations
+    float* aa = tt + hidden;           // [hidden] activations
+    float* gs = aa + hidden;           // [hidden] g_t
+    const int b = blockIdx.x, tid = threadIdx.x, nth = blockDim.x;
+    const float inv_hw = 1.0f / ((float)H * (float)W);
+    for (int k = tid; k < Ca; k += nth) gm[k] = gtap[((size_t)b * Ca + k) * kSlot + TAPS] * inv_hw;
+    for (int o = tid; o < 9 * Ca; o += nth) {
+        const int c = o / 9, i = (o % 9) / 3, j = o % 3;
+        gd[o] = gtap[((size_t)b * Ca + c) * kSlot + (i + P - 1) * K + (j + P - 1)];
+    }
+    __syncthreads();
+    for (int m = tid; m < hidden; m += nth) {
+        float t = Elem<T>::to_f32(b_down[m]);
+        for (int k = 0; k < Ca; ++k) t = fmaf(Elem<T>::to_f32(w_down[(size_t)m * Ca + k]), gm[k], t);
+        tt[m] = t;
+        aa[m] = gelu_exact(t);
+        act[(size_t)b * hidden + m] = aa[m];
+    }
+    __syncthreads();
+    for (int o = tid; o < 9 * Ca; o += nth) {
+        float s = Elem<T>::to_f32(b_up[o]);
+        for (int m = 0; m < hidden; ++m) s = fmaf(Elem<T>::to_f32(w_up[(size_t)o * hidden + m]), aa[m], s);
+        dk_flip[(size_t)b * Ca * 9 + (o / 9) * 9 + (8 - o % 9)] = s;
+    }
+    for (int m = tid; m < hidden; m += nth) {
+        float s = 0.f;
+        for (int o = 0; o < 9 * Ca; ++o) s = fmaf(Elem<T>::to_f32(w_up[(size_t)o * hidden + m]), gd[o], s);
+        s *= gelu_exact_prime(tt[m]);
+        gs[m] = s;
+        gt[(size_t)b * hidden + m] = s;
+    }
+    __syncthreads();
+    for (int k = tid; k < Ca; k += nth) {
+        float s = 0.f;
+        for (int m = 0; m < hidden; ++m) s = fmaf(Elem<T>::to_f32(w_down[(size_t)m * Ca + k]), gs[m], s);
+        bias[(size_t)b * Ca + k] = s * inv_hw;
+    }
+}
+
+// kernel 2d: the sums over images (fixed order) and the rotated LK; six jobs on separate blocks.
+constexpr int kMlpRoles = 6, kMlpBlocks = 32 * kMlpRoles;
+template <typename T>
+__global__ void __launch_bounds__(256)
+mlp_weights(const float* __restrict__ gtap, const float* __restrict__ act, const float* __restrict__ gt, int B, int Ca,
+            int hidden, int H, int W, const T* __restrict__ w_large, float* __restrict__ g_lk, float* __restrict__ g_wd,
+            float* __restrict__ g_bd, float* __restrict__ g_wu, float* __restrict__ g_bu, T* __restrict__ w_flip)
+{
+    const int per_role = gridDim.x / kMlpRoles, role = blockIdx.x / per_role;
+    const int tid = (blockIdx.x % per_role) * blockDim.x + threadIdx.x, nth = per_role * blockDim.x;
+    const float inv_hw = 1.0f / ((float)H * (float)W);
+    auto gdk = [&](int b, int o) {
+        const int c = o / 9, i = (o % 9) / 3, j = o % 3;
+        return gtap[((size_t)b * Ca + c) * kSlot + (i + P - 1) * K + (j + P - 1)];
+    };
+    if (role == 0 && g_lk)
+        for (int e = tid; e < Ca * TAPS; e += nth) {
+            const int c = e / TAPS, t = e % TAPS;
+            float s = 0.f;
+#pragma unroll 8
+            for (int b = 0; b < B; ++b) s += gtap[((size_t)b * Ca + c) * kSlot + t];
+            g_lk[e] = s;
+        }
+    if (role == 1)
+        for (int e = tid; e < Ca * TAPS; e += nth) {
+            const int c = e / TAPS, t = e % TAPS;
+            w_flip[(size_t)c * TAPS + (TAPS - 1 - t)] = w_large[e];
+        }
+    if (role == 2 && g_bu)
+        for (int o = tid; o < 9 * Ca; o += nth) {
+            float s = 0.f;
+#pragma unroll 8
+            for (int b = 0; b < B; ++b) s += gdk(b, o);
+            g_bu[o] = s;
+        }
+    if (role == 3 && g_wu)
+        for (int e = tid; e < 9 * Ca * hidden; e += nth) {
+            const int o = e / hidden, m = e % hidden;
+            float s = 0.f;
+#pragma unroll 8
+            for (int b = 0; b < B; ++b) s = fmaf(gdk(b, o), act[(size_t)b * hidden + m], s);
+            g_wu[e] = s;
+        }
+    if (role == 4 && g_bd)
+        for (int m = tid; m < hidden; m += nth) {
+            float s = 0.f;
+#pragma unroll 8
+            for (int b = 0; b < B; ++b) s += gt[(size_t)b * hidden + m];
+            g_bd[m] = s;
+        }
+    if (role == 5 && g_wd)
+        for (int e = tid; e < hidden * Ca; e += nth) {
+            const int m = e / Ca, k = e % Ca;
+            float s = 0.f;
+#pragma unroll 8
+            for (int b = 0; b < B; ++b) s = fmaf(gt[(size_t)b * hidden + m], gtap[((size_t)b * Ca + k) * kSlot + TAPS] * inv_hw, s);
+            g_wd[e] = s;
+        }
 }
 
 }}  // namespace esc::bwd

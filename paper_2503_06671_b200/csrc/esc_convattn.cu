@@ -455,6 +455,7 @@ int forward_impl(const Problem& p, const void* x, const void* w_large, const Est
 struct BackwardWs {
     unsigned* ctrl;
     float *part, *gtap, *dk_flip, *bias;
+    float *act, *gt;                 // two-layer estimator: activations and g_t, [B][kMaxHidden] each
     void* w_flip;
     size_t bytes;
 };
@@ -471,13 +472,21 @@ BackwardWs carve_backward(void* ws, const Problem& p) {
     w.w_flip = base + off;                          off += round_up((size_t)p.Ca * esc::bwd::TAPS * 4, 256);
     w.dk_flip = reinterpret_cast<float*>(base + off); off += round_up((size_t)p.B * p.Ca * 9 * 4, 256);
     w.bias = reinterpret_cast<float*>(base + off);  off += round_up((size_t)p.B * p.Ca * 4, 256);
+    w.act = reinterpret_cast<float*>(base + off);   off += round_up((size_t)p.B * esc::kMaxHidden * 4, 256);
+    w.gt = reinterpret_cast<float*>(base + off);    off += round_up((size_t)p.B * esc::kMaxHidden * 4, 256);
     w.bytes = off;
     return w;
 }
 
+// Weight gradients the caller asked for (fp32, any may be null): of LK, and of the estimator's layers -- last layer
+// (W_dyn, b_dyn, or W_up, b_up) and, for the two-layer estimator, W_down, b_down.
+struct BackwardGrads {
+    float *g_lk, *g_w_last, *g_b_last, *g_w_down, *g_b_down;
+};
+
 template <typename T, int LAYOUT>
-int backward_t(const Problem& p, const void* x, const void* go, const void* w_large, const void* w_dyn,
-               const void* b_dyn, const BackwardWs& w, float* g_lk, float* g_w, float* g_b, cudaStream_t st) {
+int backward_t(const Problem& p, const void* x, const void* go, const void* w_large, const Estimator& est,
+               const BackwardWs& w, const BackwardGrads& g, cudaStream_t st) {
     // bf16 NHWC with whole groups of 16 channels: the tensor-core kernel
     int tiles_done = 0;
     if (g_engine_policy != ESC_ENGINE_FP32) {
@@ -513,11 +522,26 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
     if (tiles_done == 0) ++g_last_launches;
     esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), esc::bwd::kSumThreads, 0, st>>>(w.part, tiles_done > 0 ? tiles_done : tiles_x * tiles_y, w.gtap);
     ESC_CUDA(cudaGetLastError());
-    esc::bwd::finish<T><<<esc::bwd::kFinishBlocks, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, static_cast<const T*>(w_large),
-                                            static_cast<const T*>(w_dyn), static_cast<const T*>(b_dyn), g_lk, g_w, g_b,
-                                            static_cast<T*>(w.w_flip), w.dk_flip, w.bias);
+    if (est.hidden == 0) {
+        esc::bwd::finish<T><<<esc::bwd::kFinishBlocks, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, static_cast<const T*>(w_large),
+                                                static_cast<const T*>(est.w_last), static_cast<const T*>(est.b_last), g.g_lk,
+                                                g.g_w_last, g.g_b_last, static_cast<T*>(w.w_flip), w.dk_flip, w.bias);
+        ESC_CUDA(cudaGetLastError());
+        g_last_launches += 2;
+        return ESC_OK;
+    }
+    // two-layer estimator: what belongs to one image, then the sums over images
+    const size_t smem = (size_t)(10 * p.Ca + 3 * est.hidden) * sizeof(float);
+    if (smem > 48 * 1024) return ESC_ERR_UNSUPPORTED;
+    esc::bwd::mlp_image<T><<<(unsigned)p.B, 256, smem, st>>>(w.gtap, p.Ca, est.hidden, p.H, p.W, static_cast<const T*>(est.w_down),
+                                                             static_cast<const T*>(est.b_down), static_cast<const T*>(est.w_last),
+                                                             static_cast<const T*>(est.b_last), w.act, w.gt, w.dk_flip, w.bias);
     ESC_CUDA(cudaGetLastError());
-    g_last_launches += 2;
+    esc::bwd::mlp_weights<T><<<esc::bwd::kMlpBlocks, 256, 0, st>>>(w.gtap, w.act, w.gt, p.B, p.Ca, est.hidden, p.H, p.W,
+                                                                  static_cast<const T*>(w_large), g.g_lk, g.g_w_down, g.g_b_down,
+                                                                  g.g_w_last, g.g_b_last, static_cast<T*>(w.w_flip));
+    ESC_CUDA(cudaGetLastError());
+    g_last_launches += 3;
     return ESC_OK;
 }
 
@@ -919,17 +943,19 @@ size_t esc_convattn_backward_workspace_bytes(int B, int C_a, int H, int W, int K
     return carve_backward(nullptr, p).bytes;
 }
 
-int esc_convattn_backward(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
-                          const void* w_large, const void* w_dyn, const void* b_dyn, void* grad_x,
-                          float* grad_w_large, float* grad_w_dyn, float* grad_b_dyn, int dtype, int layout,
-                          void* workspace, size_t workspace_bytes_, void* stream) {
+namespace {
+int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K, const void* w_large,
+                   const Estimator& est, void* grad_x, const BackwardGrads& g, int dtype, int layout, void* workspace,
+                   size_t workspace_bytes_, void* stream) {
     g_last_launches = 0;
     Problem p{B, C, C_a, H, W, K, dtype, layout};
     int rc = check_shape(p);
     if (rc != ESC_OK) return rc;
     if (K != esc::bwd::K) return ESC_ERR_UNSUPPORTED;
     if ((long long)B * C_a > 0x7fffffffLL / esc::bwd::kSlot) return ESC_ERR_UNSUPPORTED;
-    if (!x || !grad_out || !grad_x || !w_large || !w_dyn || !b_dyn) return ESC_ERR_NULL;
+    if (!x || !grad_out || !grad_x || !w_large) return ESC_ERR_NULL;
+    rc = check_estimator(p, est);
+    if (rc != ESC_OK) return rc;
     rc = check_tensors(p, grad_out, grad_x);                 // the stencil pass reads grad_out and writes grad_x
     if (rc != ESC_OK) return rc;
     if (!aligned(x, 16)) return ESC_ERR_ALIGN;
@@ -938,24 +964,44 @@ int esc_convattn_backward(const void* x, const void* grad_out, int B, int C, int
         const size_t bytes = p.elems() * p.es();
         if (xa < oa + bytes && oa < xa + bytes) return ESC_ERR_ALIAS;
     }
-    if (!aligned(w_large, p.es()) || !aligned(w_dyn, p.es()) || !aligned(b_dyn, p.es())) return ESC_ERR_ALIGN;
-    if ((grad_w_large && !aligned(grad_w_large, 4)) || (grad_w_dyn && !aligned(grad_w_dyn, 4)) ||
-        (grad_b_dyn && !aligned(grad_b_dyn, 4)))
-        return ESC_ERR_ALIGN;
+    if (!aligned(w_large, p.es())) return ESC_ERR_ALIGN;
+    for (const float* q : {g.g_lk, g.g_w_last, g.g_b_last, g.g_w_down, g.g_b_down})
+        if (q && !aligned(q, 4)) return ESC_ERR_ALIGN;
     if (!workspace || !aligned(workspace, 256)) return ESC_ERR_WORKSPACE;
     const BackwardWs w = carve_backward(workspace, p);
     if (workspace_bytes_ < w.bytes) return ESC_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (dtype == ESC_F32)
-        rc = layout == ESC_NCHW ? backward_t<float, esc::kNCHW>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st)
-                                : backward_t<float, esc::kNHWC>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st);
+        rc = layout == ESC_NCHW ? backward_t<float, esc::kNCHW>(p, x, grad_out, w_large, est, w, g, st)
+                                : backward_t<float, esc::kNHWC>(p, x, grad_out, w_large, est, w, g, st);
     else
-        rc = layout == ESC_NCHW ? backward_t<__nv_bfloat16, esc::kNCHW>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st)
-                                : backward_t<__nv_bfloat16, esc::kNHWC>(p, x, grad_out, w_large, w_dyn, b_dyn, w, grad_w_large, grad_w_dyn, grad_b_dyn, st);
+        rc = layout == ESC_NCHW ? backward_t<__nv_bfloat16, esc::kNCHW>(p, x, grad_out, w_large, est, w, g, st)
+                                : backward_t<__nv_bfloat16, esc::kNHWC>(p, x, grad_out, w_large, est, w, g, st);
     if (rc != ESC_OK) return rc;
     // grad_x: the forward stencil on grad_out with both kernels rotated by 180 degrees, plus the constants
     p.bias = w.bias;
     return launch_stencil(p, grad_out, w.w_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false);
+}
+}  // namespace
+
+int esc_convattn_backward(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                          const void* w_large, const void* w_dyn, const void* b_dyn, void* grad_x,
+                          float* grad_w_large, float* grad_w_dyn, float* grad_b_dyn, int dtype, int layout,
+                          void* workspace, size_t workspace_bytes_, void* stream) {
+    const Estimator est{w_dyn, b_dyn, nullptr, nullptr, 0};
+    const BackwardGrads g{grad_w_large, grad_w_dyn, grad_b_dyn, nullptr, nullptr};
+    return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_large, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream);
+}
+
+int esc_convattn_backward_mlp(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                              const void* w_large, const void* w_down, const void* b_down, const void* w_up,
+                              const void* b_up, int hidden, void* grad_x, float* grad_w_large, float* grad_w_down,
+                              float* grad_b_down, float* grad_w_up, float* grad_b_up, int dtype, int layout,
+                              void* workspace, size_t workspace_bytes_, void* stream) {
+    if (hidden <= 0) return ESC_ERR_SHAPE;
+    const Estimator est{w_up, b_up, w_down, b_down, hidden};
+    const BackwardGrads g{grad_w_large, grad_w_up, grad_b_up, grad_w_down, grad_b_down};
+    return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_large, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream);
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {
