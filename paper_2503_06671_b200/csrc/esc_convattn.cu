@@ -20,6 +20,7 @@
 #include "stencil_toeplitz.cuh"
 #include "stencil_toeplitz_nchw.cuh"
 #include "backward_toeplitz.cuh"
+#include "backward_toeplitz_nchw.cuh"
 #include "stencil_dense.cuh"
 #include "stencil_dense_umma.cuh"
 #include "backward.cuh"
@@ -494,6 +495,12 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
                                                   &g_last_launches, &g_last_error);
         if (rt == ESC_OK) tiles_done = esc::bwd::toep::tiles_of(p.H, p.W);
         else if (rt != esc::tma::kNotApplicable) return rt;
+        if (tiles_done == 0) {                               // the same on NCHW tensors
+            const int rn = esc::bwd::toepn::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, go, w.part, w.ctrl, st,
+                                                       &g_last_launches, &g_last_error);
+            if (rn == ESC_OK) tiles_done = esc::bwd::toep::tiles_of(p.H, p.W);
+            else if (rn != esc::tma::kNotApplicable) return rn;
+        }
     }
     // NHWC with whole octets of channels: eight channels per block, 16-byte loads; else a block per channel
     const bool oct = LAYOUT == esc::kNHWC && p.Ca % 8 == 0 && p.C % 8 == 0;

@@ -47,6 +47,7 @@ struct Params {
     const __nv_bfloat16* x;           // for the copy-through
     const __nv_bfloat16* w_large;     // [Ca][13][13]
     const float* dk;                  // [B][Ca][9]
+    const float* bias;                // [B][Ca] constant added to every output of (image, channel), or nullptr (backward pass)
     __nv_bfloat16* out;
     unsigned* ctrl;
     int wait_first;
@@ -354,6 +355,7 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
 #pragma unroll
                 for (int v = 0; v < 9; ++v) dkv[v] = __ldcg(dp + v);
             }
+            const float bias = p.bias ? __ldg(p.bias + (size_t)un.b * p.Ca + un.g * CG + c) : 0.f;
 #pragma unroll
             for (int q = 0; q < NB; ++q)
 #pragma unroll
@@ -370,7 +372,7 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
                             in[a][1] = __uint_as_float(u & 0xffff0000u);
                             in[a][2] = __uint_as_float((w1 >> sh) << 16);
                         }
-                        float s0 = 0.f, s1 = 0.f;
+                        float s0 = bias, s1 = bias;
 #pragma unroll
                         for (int a = 0; a < 3; ++a)
 #pragma unroll
@@ -448,7 +450,7 @@ inline bool applies(int C, int Ca, int H, int W, int K, int dtype, int layout, c
 }
 
 template <bool kFused>
-inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, void* out,
+inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, const float* bias, void* out,
                   unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err, const toep::Fused* fu) {
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -457,7 +459,7 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
     if (p.units > 0x7fffffffLL) return kNotApplicable;
     p.x = static_cast<const __nv_bfloat16*>(x);
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
-    p.dk = dk; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
+    p.dk = dk; p.bias = bias; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
     p.copy_bytes = (long long)(C - Ca) * H * W * 2;           // a multiple of 16: W is a multiple of 8
     p.w_last = p.b_last = p.w_down = p.b_down = nullptr; p.hidden = 0; p.gpart = nullptr; p.garr = p.gflag = nullptr;
@@ -509,8 +511,8 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
 inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
                       const float* dk, const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent,
                       int* launches, std::string* err) {
-    if (bias || !applies(C, Ca, H, W, K, dtype, layout, x, out) || sm_count() <= 0) return kNotApplicable;
-    return launch<false>(B, C, Ca, H, W, x, w_large, dk, out, ctrl, st, dependent, launches, err, nullptr);
+    if (!applies(C, Ca, H, W, K, dtype, layout, x, out) || sm_count() <= 0) return kNotApplicable;
+    return launch<false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr);
 }
 
 inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, int hidden, const void* x, const void* out) {
@@ -523,7 +525,7 @@ inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, 
 inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
                             const toep::Fused& fu, void* out, unsigned* ctrl, cudaStream_t st, int* launches, std::string* err) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden, x, out)) return kNotApplicable;
-    return launch<true>(B, C, Ca, H, W, x, w_large, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
+    return launch<true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
 }
 
 }}}  // namespace esc::tma::toepn

@@ -97,16 +97,17 @@ def _run_backward(pkg, d, go, C_a, K, dtype, layout):
     return gx, g_lk, g_w, g_b
 
 
-@pytest.mark.parametrize("shape", [(1, 64, 16, 300, 640), (6, 32, 32, 130, 200), (40, 16, 16, 64, 64)], ids=lambda s: "x".join(map(str, s)))
-def test_backward_weight_gradients_many_units(pkg, oracle, shape):
-    """bf16 NHWC, where the tap gradients run on the tensor cores: 190, 432 and 160 units of 64x16 on 148 SMs, so CTAs
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("shape", [(1, 64, 16, 300, 640), (6, 32, 32, 130, 200), (40, 16, 16, 64, 64), (2, 32, 16, 45, 72)], ids=lambda s: "x".join(map(str, s)))
+def test_backward_weight_gradients_many_units(pkg, oracle, shape, layout):
+    """bf16 (both layouts; W a multiple of 8 as the NCHW kernel wants), where the tap gradients run on the tensor cores: 190, 432 and 160 units of 64x16 on 148 SMs, so CTAs
     walk two or three units (staging buffers, planes and barriers are re-used; image and channel group change inside
     a walk); the three weight gradients against the oracle, and against the FP32-pipe kernels."""
     B, C, C_a, H, W = shape
     K = 13
     d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=sum(shape) + 3, per_image_scale=True, channel_means=True)
     go = synth.round_to(np.random.default_rng(sum(shape) + 4).standard_normal(size=d["x"].shape).astype(np.float32), synth.BF16)
-    _, g_lk, g_w, g_b = _run_backward(pkg, d, go, C_a, K, synth.BF16, synth.NHWC)
+    _, g_lk, g_w, g_b = _run_backward(pkg, d, go, C_a, K, synth.BF16, layout)
     _, rlk, rw, rb = oracle.backward(d["x"], go, C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
     _, alk, aw, ab = oracle.backward(np.abs(d["x"]), np.abs(go), C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
     for name, got, ref, scale in (("w_large", g_lk, rlk, alk), ("w_dyn", g_w, rw, aw), ("b_dyn", g_b, rb, ab)):
@@ -114,7 +115,7 @@ def test_backward_weight_gradients_many_units(pkg, oracle, shape):
         assert (err <= 1e-5 * scale + 1e-30).all(), f"grad {name}: worst {(err / np.maximum(scale, 1e-30)).max():.3e} of its scale"
     pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32)
     try:
-        _, f_lk, f_w, f_b = _run_backward(pkg, d, go, C_a, K, synth.BF16, synth.NHWC)
+        _, f_lk, f_w, f_b = _run_backward(pkg, d, go, C_a, K, synth.BF16, layout)
     finally:
         pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
     for name, a, b, scale in (("w_large", g_lk, f_lk, alk), ("w_dyn", g_w, f_w, aw), ("b_dyn", g_b, f_b, ab)):
