@@ -274,7 +274,7 @@ int esc_convattn_forward_fused(const void* x, int B, int C, int C_a, int H, int 
  *   grad_w_large  [C_a,K,K]    fp32   dL/dLK        (may be NULL)
  *   grad_w_dyn    [9*C_a,C_a]  fp32   dL/dW_dyn     (may be NULL)
  *   grad_b_dyn    [9*C_a]      fp32   dL/db_dyn     (may be NULL)
- * K must be 13 (ESC_ERR_UNSUPPORTED otherwise).  grad_x must not overlap x or grad_out.  The workspace is one of
+ * K must be odd, 3 .. 13 (ESC_ERR_UNSUPPORTED above 13).  grad_x must not overlap x or grad_out.  The workspace is one of
  * esc_convattn_backward_workspace_bytes(...) bytes, 256-byte aligned, zeroed once with
  * esc_convattn_workspace_init(); it is not the forward workspace.  All sums are added in a fixed order.
  */

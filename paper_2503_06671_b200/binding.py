@@ -289,7 +289,7 @@ def new_backward_workspace(B, C_a, H, W, K, device="cuda"):
 
     n = esc_convattn_backward_workspace_bytes(B, C_a, H, W, K)
     if n == 0:
-        raise ValueError("invalid problem size, or K is not 13")
+        raise ValueError("invalid problem size, or K is not odd in 3 .. 13")
     ws = torch.empty(n, dtype=torch.uint8, device=device)
     esc_convattn_workspace_init(ws)
     return ws

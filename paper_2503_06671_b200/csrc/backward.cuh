@@ -274,7 +274,7 @@ sum_tiles(const float* __restrict__ part, int tiles, float* __restrict__ gtap)  
 constexpr int kFinishRoles = 6, kFinishBlocks = 32 * kFinishRoles;
 template <typename T>
 __global__ void __launch_bounds__(256)
-finish(const float* __restrict__ gtap, int B, int Ca, int H, int W, const T* __restrict__ w_large,
+finish(const float* __restrict__ gtap, int B, int Ca, int H, int W, int KK, const T* __restrict__ w_large,
        const T* __restrict__ w_dyn, const T* __restrict__ b_dyn, float* __restrict__ g_lk, float* __restrict__ g_w,
        float* __restrict__ g_b, T* __restrict__ w_flip, float* __restrict__ dk_flip, float* __restrict__ bias)
 {
@@ -288,12 +288,14 @@ finish(const float* __restrict__ gtap, int B, int Ca, int H, int W, const T* __r
         return gtap[((size_t)b * Ca + c) * kSlot + (i + P - 1) * K + (j + P - 1)];
     };
     auto gmean = [&](int b, int k) { return gtap[((size_t)b * Ca + k) * kSlot + TAPS] * inv_hw; };
+    // A large kernel of size KK < 13 sits in the middle of the 13 x 13 taps whose gradients gtap holds.
+    const int off = (K - KK) / 2, taps = KK * KK;
     if (role == 0 && g_lk)
-        for (int e = tid; e < Ca * TAPS; e += nth) {
-            const int c = e / TAPS, t = e % TAPS;
+        for (int e = tid; e < Ca * taps; e += nth) {
+            const int c = e / taps, t = (e % taps) / KK + off, u = (e % taps) % KK + off;
             float s = 0.f;
 #pragma unroll 8
-            for (int b = 0; b < B; ++b) s += gtap[((size_t)b * Ca + c) * kSlot + t];
+            for (int b = 0; b < B; ++b) s += gtap[((size_t)b * Ca + c) * kSlot + t * K + u];
             g_lk[e] = s;
         }
     if (role == 1 && g_b)
@@ -312,9 +314,9 @@ finish(const float* __restrict__ gtap, int B, int Ca, int H, int W, const T* __r
             g_w[e] = s;
         }
     if (role == 3)
-    for (int e = tid; e < Ca * TAPS; e += nth) {
-        const int c = e / TAPS, t = e % TAPS;
-        w_flip[(size_t)c * TAPS + (TAPS - 1 - t)] = w_large[e];
+    for (int e = tid; e < Ca * taps; e += nth) {
+        const int c = e / taps, t = e % taps;
+        w_flip[(size_t)c * taps + (taps - 1 - t)] = w_large[e];
     }
     if (role == 4)
     for (int e = tid; e < B * Ca * 9; e += nth) {
@@ -408,7 +410,7 @@ constexpr int kMlpRoles = 6, kMlpBlocks = 32 * kMlpRoles;
 template <typename T>
 __global__ void __launch_bounds__(256)
 mlp_weights(const float* __restrict__ gtap, const float* __restrict__ act, const float* __restrict__ gt, int B, int Ca,
-            int hidden, int H, int W, const T* __restrict__ w_large, float* __restrict__ g_lk, float* __restrict__ g_wd,
+            int hidden, int H, int W, int KK, const T* __restrict__ w_large, float* __restrict__ g_lk, float* __restrict__ g_wd,
             float* __restrict__ g_bd, float* __restrict__ g_wu, float* __restrict__ g_bu, T* __restrict__ w_flip)
 {
     const int per_role = gridDim.x / kMlpRoles, role = blockIdx.x / per_role;
@@ -418,18 +420,19 @@ mlp_weights(const float* __restrict__ gtap, const float* __restrict__ act, const
         const int c = o / 9, i = (o % 9) / 3, j = o % 3;
         return gtap[((size_t)b * Ca + c) * kSlot + (i + P - 1) * K + (j + P - 1)];
     };
+    const int off = (K - KK) / 2, taps = KK * KK;      // a smaller large kernel sits in the middle of the 13 x 13 taps
     if (role == 0 && g_lk)
-        for (int e = tid; e < Ca * TAPS; e += nth) {
-            const int c = e / TAPS, t = e % TAPS;
+        for (int e = tid; e < Ca * taps; e += nth) {
+            const int c = e / taps, t = (e % taps) / KK + off, u = (e % taps) % KK + off;
             float s = 0.f;
 #pragma unroll 8
-            for (int b = 0; b < B; ++b) s += gtap[((size_t)b * Ca + c) * kSlot + t];
+            for (int b = 0; b < B; ++b) s += gtap[((size_t)b * Ca + c) * kSlot + t * K + u];
             g_lk[e] = s;
         }
     if (role == 1)
-        for (int e = tid; e < Ca * TAPS; e += nth) {
-            const int c = e / TAPS, t = e % TAPS;
-            w_flip[(size_t)c * TAPS + (TAPS - 1 - t)] = w_large[e];
+        for (int e = tid; e < Ca * taps; e += nth) {
+            const int c = e / taps, t = e % taps;
+            w_flip[(size_t)c * taps + (taps - 1 - t)] = w_large[e];
         }
     if (role == 2 && g_bu)
         for (int o = tid; o < 9 * Ca; o += nth) {

@@ -488,15 +488,16 @@ struct BackwardGrads {
 template <typename T, int LAYOUT>
 int backward_t(const Problem& p, const void* x, const void* go, const void* w_large, const Estimator& est,
                const BackwardWs& w, const BackwardGrads& g, cudaStream_t st) {
-    // bf16 NHWC with whole groups of 16 channels: the tensor-core kernel
+    // bf16 NHWC with whole groups of 16 channels: the tensor-core kernel (all tap-gradient kernels form the 13 x 13 taps'
+    // gradients, whatever the large kernel's size: a smaller one is their middle)
     int tiles_done = 0;
     if (g_engine_policy != ESC_ENGINE_FP32) {
-        const int rt = esc::bwd::toep::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, go, w.part, w.ctrl, st,
+        const int rt = esc::bwd::toep::try_launch(p.B, p.C, p.Ca, p.H, p.W, esc::bwd::K, p.dtype, p.layout, x, go, w.part, w.ctrl, st,
                                                   &g_last_launches, &g_last_error);
         if (rt == ESC_OK) tiles_done = esc::bwd::toep::tiles_of(p.H, p.W);
         else if (rt != esc::tma::kNotApplicable) return rt;
         if (tiles_done == 0) {                               // the same on NCHW tensors
-            const int rn = esc::bwd::toepn::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, go, w.part, w.ctrl, st,
+            const int rn = esc::bwd::toepn::try_launch(p.B, p.C, p.Ca, p.H, p.W, esc::bwd::K, p.dtype, p.layout, x, go, w.part, w.ctrl, st,
                                                        &g_last_launches, &g_last_error);
             if (rn == ESC_OK) tiles_done = esc::bwd::toep::tiles_of(p.H, p.W);
             else if (rn != esc::tma::kNotApplicable) return rn;
@@ -530,7 +531,7 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
     esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), esc::bwd::kSumThreads, 0, st>>>(w.part, tiles_done > 0 ? tiles_done : tiles_x * tiles_y, w.gtap);
     ESC_CUDA(cudaGetLastError());
     if (est.hidden == 0) {
-        esc::bwd::finish<T><<<esc::bwd::kFinishBlocks, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, static_cast<const T*>(w_large),
+        esc::bwd::finish<T><<<esc::bwd::kFinishBlocks, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large),
                                                 static_cast<const T*>(est.w_last), static_cast<const T*>(est.b_last), g.g_lk,
                                                 g.g_w_last, g.g_b_last, static_cast<T*>(w.w_flip), w.dk_flip, w.bias);
         ESC_CUDA(cudaGetLastError());
@@ -544,7 +545,7 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
                                                              static_cast<const T*>(est.b_down), static_cast<const T*>(est.w_last),
                                                              static_cast<const T*>(est.b_last), w.act, w.gt, w.dk_flip, w.bias);
     ESC_CUDA(cudaGetLastError());
-    esc::bwd::mlp_weights<T><<<esc::bwd::kMlpBlocks, 256, 0, st>>>(w.gtap, w.act, w.gt, p.B, p.Ca, est.hidden, p.H, p.W,
+    esc::bwd::mlp_weights<T><<<esc::bwd::kMlpBlocks, 256, 0, st>>>(w.gtap, w.act, w.gt, p.B, p.Ca, est.hidden, p.H, p.W, p.K,
                                                                   static_cast<const T*>(w_large), g.g_lk, g.g_w_down, g.g_b_down,
                                                                   g.g_w_last, g.g_b_last, static_cast<T*>(w.w_flip));
     ESC_CUDA(cudaGetLastError());
@@ -945,7 +946,7 @@ int esc_convattn_forward_fused(const void* x, int B, int C, int C_a, int H, int 
 }
 
 size_t esc_convattn_backward_workspace_bytes(int B, int C_a, int H, int W, int K) {
-    if (B <= 0 || C_a <= 0 || H <= 0 || W <= 0 || K != esc::bwd::K) return 0;
+    if (B <= 0 || C_a <= 0 || H <= 0 || W <= 0 || K < 3 || K > esc::bwd::K || (K & 1) == 0) return 0;
     const Problem p{B, C_a, C_a, H, W, K, ESC_F32, ESC_NCHW};
     return carve_backward(nullptr, p).bytes;
 }
@@ -958,7 +959,7 @@ int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, i
     Problem p{B, C, C_a, H, W, K, dtype, layout};
     int rc = check_shape(p);
     if (rc != ESC_OK) return rc;
-    if (K != esc::bwd::K) return ESC_ERR_UNSUPPORTED;
+    if (K > esc::bwd::K) return ESC_ERR_UNSUPPORTED;         // the tap-gradient kernels hold 13 x 13 taps; a smaller LK is their middle
     if ((long long)B * C_a > 0x7fffffffLL / esc::bwd::kSlot) return ESC_ERR_UNSUPPORTED;
     if (!x || !grad_out || !grad_x || !w_large) return ESC_ERR_NULL;
     rc = check_estimator(p, est);

@@ -62,7 +62,8 @@ struct Params {
     int tiles_x, tiles_y, groups;
     long long units;
     int copy_cc, copy_cw, copy_cr, slot_stride;
-    const __nv_bfloat16* w_large;     // [Ca][13][13]
+    int K;                            // large kernel's size, odd, 3 .. 13: it sits in the middle of the 13 x 13 taps the kernel applies
+    const __nv_bfloat16* w_large;     // [Ca][K][K]
     const __nv_bfloat16* w_point;     // kMix: [16][16] point-wise filter LK^c of the decomposed form (Eq. 5), row = output channel
     const float* dk;                  // [B][Ca][9]
     const float* bias;                // [B][Ca] or nullptr
@@ -381,15 +382,18 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         // ---- packed tap pairs of this channel group: P[c][i][d + 2] = (LK[c][i][d], LK[c][i][d + 1]), zero outside 0..12
         if (un.g != cur_g) {
             // the last reader of the old table passed the barrier that closed the previous unit
-            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * K13 * K13;
+            const int KK = p.K, off = (K13 - KK) / 2;        // a smaller kernel is the 13 x 13 one with zeros around it
+            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * KK * KK;
             constexpr int N = CG * K13 * PT, PER = N / kMmaThreads;
             static_assert(N % kMmaThreads == 0, "table entries per thread");
             unsigned lo[PER], hi[PER];
 #pragma unroll
             for (int u = 0; u < PER; ++u) {                  // all loads in flight together
                 const int e = tid + u * kMmaThreads, d = (e % PT) - 2, row = e / PT;   // row = c * 13 + i
-                lo[u] = (d >= 0 && d < K13) ? wg[row * K13 + d] : 0u;
-                hi[u] = (d + 1 >= 0 && d + 1 < K13) ? wg[row * K13 + d + 1] : 0u;
+                const int c = row / K13, i = row % K13 - off, dd = d - off;
+                const bool row_ok = i >= 0 && i < KK;
+                lo[u] = (row_ok && dd >= 0 && dd < KK) ? wg[(c * KK + i) * KK + dd] : 0u;
+                hi[u] = (row_ok && dd + 1 >= 0 && dd + 1 < KK) ? wg[(c * KK + i) * KK + dd + 1] : 0u;
             }
 #pragma unroll
             for (int u = 0; u < PER; ++u) ptab[tid + u * kMmaThreads] = lo[u] | (hi[u] << 16);
@@ -598,7 +602,7 @@ struct Fused {
 template <class S, bool kBias, bool kFused, bool kMix = false>
 inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk,
                         const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches,
-                        std::string* err, const Fused* fu = nullptr, bool skip_copy = false, const void* w_point = nullptr) {
+                        std::string* err, const Fused* fu = nullptr, bool skip_copy = false, const void* w_point = nullptr, int K = K13) {
     const int cc = skip_copy ? 0 : C - Ca;                 // skip_copy: the identity channels are consumed elsewhere (fused 1x1)
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -615,6 +619,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
         p.copy_cw = shapes[pick][0]; p.copy_cr = shapes[pick][1];
         p.slot_stride = (cc * 2 * p.copy_cw * p.copy_cr + 127) / 128 * 128;
     }
+    p.K = K;
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
     p.w_point = static_cast<const __nv_bfloat16*>(w_point);
     if (kMix && (Ca != CG || !w_point || (reinterpret_cast<uintptr_t>(w_point) & 3u) != 0)) return kNotApplicable;   // one group, 4-byte loads
@@ -676,7 +681,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
 }
 
 inline bool applies(int C, int Ca, int K, int dtype, int layout) {
-    return K == K13 && dtype == 1 /*bf16*/ && layout == kNHWC && Ca % CG == 0 && C % 8 == 0 && C - Ca <= 256;
+    return K >= 3 && K <= K13 && (K & 1) && dtype == 1 /*bf16*/ && layout == kNHWC && Ca % CG == 0 && C % 8 == 0 && C - Ca <= 256;
 }
 
 // Launches the tensor-core stencil if the problem fits it: 0 on success, kNotApplicable otherwise, or an ESC_ERR_* code.
@@ -688,9 +693,9 @@ inline int try_launch_toeplitz(int B, int C, int Ca, int H, int W, int K, int dt
     *tile_w = Shape64x16::TW;
     if (w_point)
         return bias ? kNotApplicable
-                    : launch_shape<Shape64x16, false, false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, w_point);
-    return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy)
-                : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy);
+                    : launch_shape<Shape64x16, false, false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, w_point, K);
+    return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, nullptr, K)
+                : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, nullptr, K);
 }
 
 // Whether the whole forward can be one launch of the tensor-core kernel with stage 1 inside: the kernel applies,
@@ -709,9 +714,9 @@ inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype
     *tile_w = Shape64x16::TW;
     if (w_point)
         return launch_shape<Shape64x16, false, true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
-                                                           launches, err, &fu, skip_copy, w_point);
+                                                           launches, err, &fu, skip_copy, w_point, K);
     return launch_shape<Shape64x16, false, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
-                                                 launches, err, &fu, skip_copy);
+                                                 launches, err, &fu, skip_copy, nullptr, K);
 }
 
 }}}  // namespace esc::tma::toep

@@ -45,7 +45,8 @@ struct Params {
     int tiles_x, tiles_y, groups;
     long long units;
     const __nv_bfloat16* x;           // for the copy-through
-    const __nv_bfloat16* w_large;     // [Ca][13][13]
+    int K;                            // large kernel's size, odd, 3 .. 13: it sits in the middle of the 13 x 13 taps the kernel applies
+    const __nv_bfloat16* w_large;     // [Ca][K][K]
     const float* dk;                  // [B][Ca][9]
     const float* bias;                // [B][Ca] constant added to every output of (image, channel), or nullptr (backward pass)
     __nv_bfloat16* out;
@@ -282,15 +283,18 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
         // ---- packed tap pairs of this channel group: P[c][i][d + 2] = (LK[c][i][d], LK[c][i][d + 1]), zero outside 0..12
         if (un.g != cur_g) {
             if (cur_g >= 0) mma_bar();                       // everybody is done with the old table
-            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * K13 * K13;
+            const int KK = p.K, off = (K13 - KK) / 2;        // a smaller kernel is the 13 x 13 one with zeros around it
+            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * KK * KK;
             constexpr int N = CG * K13 * PT, PER = N / kMmaThreads;
             static_assert(N % kMmaThreads == 0, "table entries per thread");
             unsigned lo[PER], hi[PER];
 #pragma unroll
             for (int u = 0; u < PER; ++u) {
                 const int e = tid + u * kMmaThreads, d = (e % PT) - 2, row = e / PT;   // row = c * 13 + i
-                lo[u] = (d >= 0 && d < K13) ? wg[row * K13 + d] : 0u;
-                hi[u] = (d + 1 >= 0 && d + 1 < K13) ? wg[row * K13 + d + 1] : 0u;
+                const int c = row / K13, i = row % K13 - off, dd = d - off;
+                const bool row_ok = i >= 0 && i < KK;
+                lo[u] = (row_ok && dd >= 0 && dd < KK) ? wg[(c * KK + i) * KK + dd] : 0u;
+                hi[u] = (row_ok && dd + 1 >= 0 && dd + 1 < KK) ? wg[(c * KK + i) * KK + dd + 1] : 0u;
             }
 #pragma unroll
             for (int u = 0; u < PER; ++u) ptab[tid + u * kMmaThreads] = lo[u] | (hi[u] << 16);
@@ -445,12 +449,12 @@ inline long long units_of(int B, int Ca, int H, int W) {
 // aligned tensors (a TMA base, and the bulk copies of the identity channels).
 inline bool applies(int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* out) {
     (void)H;
-    return K == K13 && dtype == 1 /*bf16*/ && layout == kNCHW && Ca % CG == 0 && C >= Ca && W % 8 == 0 &&
+    return K >= 3 && K <= K13 && (K & 1) && dtype == 1 /*bf16*/ && layout == kNCHW && Ca % CG == 0 && C >= Ca && W % 8 == 0 &&
            (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
 }
 
 template <bool kFused>
-inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, const float* bias, void* out,
+inline int launch(int K, int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, const float* bias, void* out,
                   unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err, const toep::Fused* fu) {
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -458,6 +462,7 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
     p.units = units_of(B, Ca, H, W);
     if (p.units > 0x7fffffffLL) return kNotApplicable;
     p.x = static_cast<const __nv_bfloat16*>(x);
+    p.K = K;
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
     p.dk = dk; p.bias = bias; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
@@ -512,7 +517,7 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
                       const float* dk, const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent,
                       int* launches, std::string* err) {
     if (!applies(C, Ca, H, W, K, dtype, layout, x, out) || sm_count() <= 0) return kNotApplicable;
-    return launch<false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr);
+    return launch<false>(K, B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr);
 }
 
 inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, int hidden, const void* x, const void* out) {
@@ -525,7 +530,7 @@ inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, 
 inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
                             const toep::Fused& fu, void* out, unsigned* ctrl, cudaStream_t st, int* launches, std::string* err) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden, x, out)) return kNotApplicable;
-    return launch<true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
+    return launch<true>(K, B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
 }
 
 }}}  // namespace esc::tma::toepn

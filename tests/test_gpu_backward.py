@@ -123,14 +123,43 @@ def test_backward_weight_gradients_many_units(pkg, oracle, shape, layout):
         assert (err <= 2e-5 * scale + 1e-30).all(), f"grad {name}: the two kernels differ by {(err / np.maximum(scale, 1e-30)).max():.3e} of its scale"
 
 
+@pytest.mark.parametrize("layout", LAYOUTS)
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("K", [9, 5, 3])
+def test_backward_smaller_large_kernels(pkg, oracle, K, dtype, layout):
+    """K < 13: the tap-gradient kernels form the 13 x 13 taps' gradients, of which the K x K in the middle are the large
+    kernel's; grad_x runs the K x K stencil.  All four gradients against the oracle at the true K."""
+    B, C, C_a, H, W = 2, 32, 16, 37, 72
+    d = synth.make_inputs(B, C, C_a, H, W, K, dtype, seed=100 + K, per_image_scale=True, channel_means=True)
+    go = synth.round_to(np.random.default_rng(200 + K).standard_normal(size=d["x"].shape).astype(np.float32), dtype)
+    gx, g_lk, g_w, g_b = _run_backward(pkg, d, go, C_a, K, dtype, layout)
+    rx, rlk, rw, rb = oracle.backward(d["x"], go, C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    _, alk, aw, ab = oracle.backward(np.abs(d["x"]), np.abs(go), C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    assert tuple(g_lk.shape) == (C_a, K, K)
+    for name, got, ref, scale in (("w_large", g_lk, rlk, alk), ("w_dyn", g_w, rw, aw), ("b_dyn", g_b, rb, ab)):
+        err = np.abs(got.cpu().numpy().astype(np.float64) - ref)
+        assert (err <= 1e-5 * scale + 1e-30).all(), f"grad {name}: worst {(err / np.maximum(scale, 1e-30)).max():.3e} of its scale"
+    got = util.to_host_nchw(gx, layout)
+    assert np.array_equal(got[:, C_a:], go[:, C_a:].astype(np.float64))
+    dk = oracle.dynkernel(oracle.gap(d["x"], C_a), d["w_dyn"], d["b_dyn"])
+    mag = oracle.stencil(np.abs(go), C_a, np.abs(d["w_large"][:, ::-1, ::-1]).copy(), np.abs(dk[:, :, ::-1, ::-1]).copy())[:, :C_a]
+    gg_scale = np.abs(np.einsum("ok,bo->bk", np.abs(d["w_dyn"].astype(np.float64)), np.abs(ab.reshape(1, -1)).repeat(B, 0))) / (H * W)
+    bar = 1e-5 * mag + 1e-5 * gg_scale[:, :, None, None] + 1e-30
+    if dtype == synth.BF16:
+        bar = bar + 2.0 ** -8 * np.abs(rx[:, :C_a]) * 1.001
+    err = np.abs(got[:, :C_a] - rx[:, :C_a])
+    assert (err <= bar).all(), f"grad x: {int((err > bar).sum())} values beyond the bound"
+
+
 def test_backward_rejections(pkg):
     import torch
 
     x = torch.zeros(1, 8, 8, 16, dtype=torch.bfloat16, device="cuda")
-    w = torch.zeros(16, 9, 9, dtype=torch.bfloat16, device="cuda")
-    assert pkg.esc_convattn_backward_workspace_bytes(1, 16, 8, 8, 9) == 0          # K = 13 only
+    w = torch.zeros(16, 15, 15, dtype=torch.bfloat16, device="cuda")
+    assert pkg.esc_convattn_backward_workspace_bytes(1, 16, 8, 8, 15) == 0         # K = 3 .. 13 only
+    assert pkg.esc_convattn_backward_workspace_bytes(1, 16, 8, 8, 9) > 0
     L = pkg.lib()
     ws = pkg.new_backward_workspace(1, 16, 8, 8, 13)
-    rc = L.esc_convattn_backward(x.data_ptr(), x.data_ptr(), 1, 16, 16, 8, 8, 9, w.data_ptr(), w.data_ptr(), w.data_ptr(),
+    rc = L.esc_convattn_backward(x.data_ptr(), x.data_ptr(), 1, 16, 16, 8, 8, 15, w.data_ptr(), w.data_ptr(), w.data_ptr(),
                                  x.data_ptr(), None, None, None, 1, 1, ws.data_ptr(), ws.numel(), None)
     assert rc == 3

@@ -137,3 +137,15 @@ def test_one_launch_forward_estimator_inputs(pkg, oracle, shape, mode):
     got = util.to_host_nchw(out, synth.NHWC)
     util.check_attention(got[:, :C_a], ref[:, :C_a], mag, synth.BF16, f"{shape} {mode}")
     assert np.array_equal(got[:, C_a:], ref[:, C_a:])
+
+
+@pytest.mark.parametrize("layout", [synth.NHWC, synth.NCHW])
+@pytest.mark.parametrize("shape", [(2, 64, 16, 45, 72, 9), (1, 48, 32, 70, 136, 5), (1, 64, 16, 300, 640, 11), (3, 32, 16, 20, 24, 3)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_smaller_large_kernels_on_the_tensor_cores(pkg, oracle, shape, layout):
+    """K = 3 .. 11 (the paper's ablation of the large kernel's size): the K x K kernel is the middle of the 13 x 13 taps
+    the tensor-core kernels apply, the rest zero; every output compared with the oracle run at the true K."""
+    B, C, C_a, H, W, K = shape
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=sum(shape) + 2, per_image_scale=True, channel_means=True)
+    compare_full(pkg, oracle, d, C_a, K, synth.BF16, layout, what=f"{shape} {layout}")
+    assert pkg.esc_convattn_last_path() == (4 if layout == synth.NHWC else 6)
