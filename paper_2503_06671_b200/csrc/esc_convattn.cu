@@ -96,6 +96,7 @@ struct Workspace {
     float* dk;
     float* partial;
     float* unit_sums;
+    void* lk_pad;                    // [Ca][13][13] elements: a smaller large kernel zero-padded for the tensor-core kernels
 };
 
 bool is_large_map(int B, long long HW) { return (long double)B * HW >= 1.5e6L; }
@@ -135,7 +136,8 @@ size_t workspace_bytes(int B, int Ca, long long HW) {
     size_t off = round_up((size_t)(esc::kCtrlHeaderWords + 2 * (size_t)B) * 4, 256);
     off += round_up((size_t)B * Ca * 9 * 4, 256);
     off += round_up((size_t)B * S * Ca * 4, 256);
-    off += round_up((size_t)2 * sms_or_nominal() * 16 * 4, 256);
+    off += round_up((size_t)esc::tma::toep::kMaxFusedUnits * sms_or_nominal() * 16 * 4, 256);   // unit sums of the one-launch form
+    off += round_up((size_t)Ca * 169 * 4, 256);            // padded large kernel
     return off;
 }
 
@@ -151,6 +153,8 @@ Workspace carve(void* ws, int B, int Ca, long long HW) {
     w.partial = reinterpret_cast<float*>(p);
     p += round_up((size_t)B * slabs_for(B, HW, true) * Ca * 4, 256);
     w.unit_sums = reinterpret_cast<float*>(p);
+    p += round_up((size_t)esc::tma::toep::kMaxFusedUnits * sms_or_nominal() * 16 * 4, 256);
+    w.lk_pad = p;
     return w;
 }
 
@@ -311,8 +315,41 @@ int launch_generic(const Problem& p, const void* x, const void* w_large, const f
     return rc;                                             // the identity channels went along as copy blocks
 }
 
-int launch_stencil(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
-                   unsigned* ctrl, cudaStream_t st, bool dependent) {
+// The tensor-core depth-wise kernels are built for 13 x 13 taps.  A large kernel of odd size K < 13 is the 13 x 13 one with
+// zeros around it -- exactly the same convolution -- so it is written, zero-padded, into the workspace once per call and
+// handed to those kernels as a 13 x 13 kernel; every other kernel gets the weights as the caller gave them.
+template <typename T>
+__global__ void pad_large_kernel(const T* __restrict__ w, int Ca, int K, T* __restrict__ out) {
+    const int off = (13 - K) / 2;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < Ca * 169; e += gridDim.x * blockDim.x) {
+        const int c = e / 169, i = (e % 169) / 13 - off, j = e % 13 - off;
+        out[e] = ((unsigned)i < (unsigned)K && (unsigned)j < (unsigned)K) ? w[((size_t)c * K + i) * K + j] : T(0.0f);
+    }
+}
+struct TensorLk {
+    const void* w;
+    int K;
+};
+TensorLk tensor_lk(const Problem& p, const void* x, const void* out, const void* w_large, void* pad, cudaStream_t st) {
+    TensorLk t{w_large, p.K};
+    if (p.dense || p.dtype != ESC_BF16 || p.K >= esc::tma::K13 || !pad || g_engine_policy == ESC_ENGINE_FP32 || g_tile_policy != 0) return t;
+    if (!esc::tma::toep::applies(p.C, p.Ca, esc::tma::K13, p.dtype, p.layout) &&
+        !esc::tma::toepn::applies(p.C, p.Ca, p.H, p.W, esc::tma::K13, p.dtype, p.layout, x, out))
+        return t;
+    pad_large_kernel<__nv_bfloat16><<<(p.Ca * 169 + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w_large), p.Ca, p.K,
+                                                                            static_cast<__nv_bfloat16*>(pad));
+    if (cudaGetLastError() != cudaSuccess) return t;
+    ++g_last_launches;
+    t.w = pad; t.K = esc::tma::K13;
+    return t;
+}
+
+int launch_stencil(const Problem& p0, const void* x, const void* w_large0, const float* dk, void* out,
+                   unsigned* ctrl, cudaStream_t st, bool dependent, const TensorLk* tl = nullptr) {
+    // the tensor-core kernels see the (possibly padded) 13 x 13 kernel, everything else the caller's
+    Problem p = p0;
+    const void* w_large = w_large0;
+    if (tl) { p.K = tl->K; w_large = tl->w; }
     // Depth-wise K = 13 on NHWC bf16: the tensor-core (Toeplitz) kernel unless the caller pinned the FP32
     // kernel (by engine or by one of its tile widths) or asked for the point-wise mix, which only the
     // FP32 kernel carries.
@@ -330,6 +367,7 @@ int launch_stencil(const Problem& p, const void* x, const void* w_large, const f
         }
     }
     if (p.skip_copy) return ESC_ERR_UNSUPPORTED;           // only the tensor-core kernel can leave the identity channels out
+    p.K = p0.K; w_large = w_large0;
     if (g_engine_policy == ESC_ENGINE_TENSOR) return launch_generic(p, x, w_large, dk, out, st, dependent);
     int tile_w = g_tile_policy;
     int rc = esc::tma::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, p.w_point, dk, p.bias, out,
@@ -419,9 +457,15 @@ int launch_stencil_dense(const Problem& p, const void* x, const void* w_dense, c
     return launch_copy(p, x, out, st);
 }
 
-int forward_impl(const Problem& p, const void* x, const void* w_large, const Estimator& est,
+int forward_impl(const Problem& p0, const void* x, const void* w_large0, const Estimator& est,
                  void* out, void* ws, cudaStream_t st) {
-    const Workspace w = carve(ws, p.B, p.Ca, (long long)p.H * p.W);
+    const Workspace w = carve(ws, p0.B, p0.Ca, (long long)p0.H * p0.W);
+    // what the tensor-core kernels see: a smaller large kernel zero-padded to 13 x 13 (launched first, so that the GAP
+    // kernel stays the stencil kernel's immediate predecessor)
+    const TensorLk tl = tensor_lk(p0, x, out, w_large0, w.lk_pad, st);
+    Problem p = p0;
+    p.K = tl.K;
+    const void* w_large = tl.w;
     // Small problems on the tensor-core kernel: one launch, stage 1 inside the stencil kernel.
     if (g_fuse_stage1 && tensor_stencil_follows(p)) {
         const esc::tma::toep::Fused fu{est.w_last, est.b_last, est.w_down, est.b_down, est.hidden, w.unit_sums, w.arrivals, w.flags};
@@ -444,10 +488,10 @@ int forward_impl(const Problem& p, const void* x, const void* w_large, const Est
     }
     const bool tensor_nchw = !p.dense && !p.w_point && !p.bias && !p.skip_copy && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
                              esc::tma::toepn::applies(p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, out);
-    int rc = launch_gap(p, x, est, w, w.dk, st, tensor_stencil_follows(p) || tensor_nchw);
+    int rc = launch_gap(p0, x, est, w, w.dk, st, tensor_stencil_follows(p) || tensor_nchw);
     if (rc != ESC_OK) return rc;
-    if (p.dense) return launch_stencil_dense(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
-    return launch_stencil(p, x, w_large, w.dk, out, w.ctrl, st, /*dependent=*/true);
+    if (p0.dense) return launch_stencil_dense(p0, x, w_large0, w.dk, out, w.ctrl, st, /*dependent=*/true);
+    return launch_stencil(p0, x, w_large0, w.dk, out, w.ctrl, st, /*dependent=*/true, &tl);
 }
 
 // ---- backward pass -------------------------------------------------------------------------
@@ -457,6 +501,7 @@ struct BackwardWs {
     unsigned* ctrl;
     float *part, *gtap, *dk_flip, *bias;
     float *act, *gt;                 // two-layer estimator: activations and g_t, [B][kMaxHidden] each
+    void* lk_pad;                    // the rotated large kernel zero-padded to 13 x 13 for the tensor-core kernels
     void* w_flip;
     size_t bytes;
 };
@@ -475,6 +520,7 @@ BackwardWs carve_backward(void* ws, const Problem& p) {
     w.bias = reinterpret_cast<float*>(base + off);  off += round_up((size_t)p.B * p.Ca * 4, 256);
     w.act = reinterpret_cast<float*>(base + off);   off += round_up((size_t)p.B * esc::kMaxHidden * 4, 256);
     w.gt = reinterpret_cast<float*>(base + off);    off += round_up((size_t)p.B * esc::kMaxHidden * 4, 256);
+    w.lk_pad = base + off;                          off += round_up((size_t)p.Ca * esc::bwd::TAPS * 4, 256);
     w.bytes = off;
     return w;
 }
@@ -778,12 +824,15 @@ int esc_convattn_stencil(const void* x, int B, int C, int C_a, int H, int W, int
     if (rc != ESC_OK) return rc;
     if (!aligned(w_large, p.es()) || !aligned(dk, 4)) return ESC_ERR_ALIGN;
     unsigned* ctrl = nullptr;
+    void* pad = nullptr;
     if (workspace) {
         rc = check_workspace(p, workspace, workspace_bytes_);
         if (rc != ESC_OK) return rc;
-        ctrl = carve(workspace, B, C_a, (long long)H * W).ctrl;
+        const Workspace w = carve(workspace, B, C_a, (long long)H * W);
+        ctrl = w.ctrl; pad = w.lk_pad;
     }
-    return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
+    const TensorLk tl = tensor_lk(p, x, out, w_large, pad, static_cast<cudaStream_t>(stream));
+    return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false, &tl);
 }
 
 int esc_convattn_stencil_pw(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
@@ -799,12 +848,15 @@ int esc_convattn_stencil_pw(const void* x, int B, int C, int C_a, int H, int W, 
     if (!aligned(w_large, p.es()) || !aligned(w_point, p.es()) || !aligned(dk, 4)) return ESC_ERR_ALIGN;
     p.w_point = w_point;
     unsigned* ctrl = nullptr;
+    void* pad = nullptr;
     if (workspace) {
         rc = check_workspace(p, workspace, workspace_bytes_);
         if (rc != ESC_OK) return rc;
-        ctrl = carve(workspace, B, C_a, (long long)H * W).ctrl;
+        const Workspace w = carve(workspace, B, C_a, (long long)H * W);
+        ctrl = w.ctrl; pad = w.lk_pad;
     }
-    return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false);
+    const TensorLk tl = tensor_lk(p, x, out, w_large, pad, static_cast<cudaStream_t>(stream));
+    return launch_stencil(p, x, w_large, dk, out, ctrl, static_cast<cudaStream_t>(stream), /*dependent=*/false, &tl);
 }
 
 int esc_convattn_forward_pw(const void* x, int B, int C, int C_a, int H, int W, int K, const void* w_large,
@@ -988,7 +1040,8 @@ int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, i
     if (rc != ESC_OK) return rc;
     // grad_x: the forward stencil on grad_out with both kernels rotated by 180 degrees, plus the constants
     p.bias = w.bias;
-    return launch_stencil(p, grad_out, w.w_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false);
+    const TensorLk tl = tensor_lk(p, grad_out, grad_x, w.w_flip, w.lk_pad, st);
+    return launch_stencil(p, grad_out, w.w_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false, &tl);
 }
 }  // namespace
 

@@ -62,8 +62,7 @@ struct Params {
     int tiles_x, tiles_y, groups;
     long long units;
     int copy_cc, copy_cw, copy_cr, slot_stride;
-    int K;                            // large kernel's size, odd, 3 .. 13: it sits in the middle of the 13 x 13 taps the kernel applies
-    const __nv_bfloat16* w_large;     // [Ca][K][K]
+    const __nv_bfloat16* w_large;     // [Ca][13][13]
     const __nv_bfloat16* w_point;     // kMix: [16][16] point-wise filter LK^c of the decomposed form (Eq. 5), row = output channel
     const float* dk;                  // [B][Ca][9]
     const float* bias;                // [B][Ca] or nullptr
@@ -80,7 +79,8 @@ struct Params {
 };
 constexpr int kFusedMaxCa = 128;      // channels the fused estimator keeps in shared memory
 // scratch of the fused stage 1, a multiple of 128 bytes (the copy ring behind it is a TMA destination)
-constexpr int FUSED_SMEM_FLOATS = (kMmaThreads + kFusedMaxCa + kMaxHidden + CG * 9 + kWarps * CG + 31) / 32 * 32;
+constexpr int FUSED_SMEM_FLOATS = (kMmaThreads + kFusedMaxCa + kMaxHidden + CG * 9 + 2 * kWarps * CG + 31) / 32 * 32;
+constexpr int kMaxFusedUnits = 8;     // units a CTA may walk in the one-launch form (kMany: more than two)
 constexpr unsigned kFlagPolls = 1u << 22;   // polls of another CTA's flag before a wait gives up (about half a second)
 
 __device__ __forceinline__ Unit decode(long long u64v, const Params& p) {
@@ -133,7 +133,11 @@ __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
 // kMix: the decomposed large kernel of Eq. 5 -- the staged tile's 16 attention channels are replaced, pixel by pixel
 // and in place, by LK^c applied to them (tensor cores, one rounding to bf16) before the tile is transposed; the pooled
 // means of stage 1 are taken from the unmixed tile.
-template <class S, bool kBias, bool kFused, bool kMix = false>
+// kMany: the one-launch form for CTAs that walk three to kMaxFusedUnits units.  The interiors of all later units pass,
+// half a tile at a time, through the two halves of the buffer that otherwise holds the second unit's interior, and are
+// added up before the first unit's products, so that every image's flag advances early; the attention channels (a few
+// tens of MB at most) are then in L2 for the tiles' loads.
+template <class S, bool kBias, bool kFused, bool kMix = false, bool kMany = false>
 __global__ void __launch_bounds__(kThreads, 1)
 stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __grid_constant__ CUtensorMap map_cin,
                            const __grid_constant__ CUtensorMap map_cout, const __grid_constant__ CUtensorMap map_box,
@@ -149,7 +153,12 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
     unsigned char* sumbuf = reinterpret_cast<unsigned char*>(fsm) + FUSED_SMEM_FLOATS * 4;       // fused: interior of the second unit's tile
     unsigned char* ring = reinterpret_cast<unsigned char*>(fsm) + (kFused ? FUSED_SMEM_FLOATS * 4 + S::BOX_BYTES : 0);
     u64* bars = reinterpret_cast<u64*>(ring + NSLOT * p.slot_stride);
-    const uint32_t full = smem_u32(bars), empty = full + 8, cfull0 = full + 16, sumdone = cfull0 + 8 * NSLOT, boxfull = sumdone + 8;
+    const uint32_t full = smem_u32(bars), empty = full + 8, cfull0 = full + 16, sumdone = cfull0 + 8 * NSLOT, boxfull = sumdone + 8,
+                   boxfull1 = boxfull + 8, boxfree0 = boxfull1 + 8,     // kMany: two half-tile slots, full and free
+                   sumdone_more = boxfree0 + 16;                         // units 1 .. 7: one barrier per unit, each used once
+    // (a barrier per unit, not the phases of one: the producer lane may fall several units behind the working warps,
+    //  and a wait on a phase's parity is only meaningful one phase back)
+    auto sumdone_of = [&](int k) -> uint32_t { return k == 0 ? sumdone : sumdone_more + 8 * (uint32_t)(k - 1); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -158,6 +167,9 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         for (int s = 0; s < NSLOT; ++s) mbar_init(cfull0 + 8 * s, 1);
         mbar_init(sumdone, CG);
         mbar_init(boxfull, 1);
+        if (kMany) { mbar_init(boxfull1, 1); mbar_init(boxfree0, 1); mbar_init(boxfree0 + 8, 1); }
+        if (kFused)
+            for (int k = 1; k < (kMany ? kMaxFusedUnits : 2); ++k) mbar_init(sumdone_of(k), CG);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -169,6 +181,33 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
 
     if (warp >= kWarps) {
         if (lane != 0) return;
+        if (warp == kWarps && kFused && kMany) {
+            // ---- stage 1 fused, three or more units: the first unit's halo tile, then the later units' interiors half a
+            //      tile at a time through two slots, then the arrivals on the images' counters
+            bool alive = true;
+            const int n = (int)my_units;
+            const Unit u0 = decode(first, p);
+            mbar_expect_tx(full, S::STAGE_BYTES);
+            tma_load_4d(smem_u32(stage), &map_att, full, u0.g * CG, u0.tx * TW - P6, u0.ty * TH - P6, u0.b);
+            unsigned seen[kMaxFusedUnits];
+            for (int k = 0; k < n; ++k) seen[k] = ld_acquire(p.gflag + decode(first + k * stride, p).b);
+            for (int h = 0; h < 2 * (n - 1); ++h) {
+                const int slot = h & 1;
+                const Unit un = decode(first + (1 + (h >> 1)) * stride, p);
+                if (h >= 2 && alive) alive = mbar_wait(boxfree0 + 8 * slot, (unsigned)(((h >> 1) - 1) & 1), p.ctrl, 0xBA000000u);
+                mbar_expect_tx(boxfull + 8 * slot, S::BOX_BYTES / 2);
+                tma_load_4d(smem_u32(sumbuf + slot * (S::BOX_BYTES / 2)), &map_box, boxfull + 8 * slot, un.g * CG, un.tx * TW,
+                            un.ty * TH + slot * (TH / 2), un.b);
+            }
+            for (int k = 0; k < n; ++k) {
+                const Unit un = decode(first + k * stride, p);
+                if (alive) alive = mbar_wait(sumdone_of(k), 0u, p.ctrl, 0xB9000000u | (unsigned)k);
+                unsigned old;
+                asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.garr + un.b), "r"((unsigned)(p.upi - 1)) : "memory");
+                if (old == (unsigned)(p.upi - 1)) st_release(p.gflag + un.b, seen[k] + 1u);
+            }
+            return;
+        }
         if (warp == kWarps && kFused) {
             // ---- stage 1 fused: this lane starts the loads -- the first unit's halo tile and, for its sum alone, the
             //      interior of the second unit's tile -- and performs the arrivals on the images' counters once the
@@ -186,7 +225,7 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
             const unsigned seen[2] = {ld_acquire(p.gflag + u0.b), ld_acquire(p.gflag + u1.b)};
             for (int k = 0; k < (int)my_units; ++k) {
                 const Unit& un = k == 0 ? u0 : u1;
-                if (alive) alive = mbar_wait(sumdone, (unsigned)(k & 1), p.ctrl, 0xB9000000u);
+                if (alive) alive = mbar_wait(sumdone_of(k), 0u, p.ctrl, 0xB9000000u | (unsigned)k);
                 // release: the 16 sums (seen through the barrier) are visible to whoever reads the counter or the flag
                 unsigned old;
                 asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.garr + un.b), "r"((unsigned)(p.upi - 1)) : "memory");
@@ -275,16 +314,16 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
     float* f_mean = fsm + kMmaThreads;                       // [Ca] pooled means of the current image
     float* f_act = f_mean + kFusedMaxCa;                     // [hidden] activations of the two-layer estimator
     float* f_dk = f_act + kMaxHidden;                        // [16][9] dynamic taps of the current (image, group)
-    float* f_red = f_dk + CG * 9;                            // [8 warps][16] tile sums
-    unsigned flag0[2] = {0u, 0u};                            // the images' flags as they stood before this launch
+    float* f_red = f_dk + CG * 9;                            // [2][8 warps][16] tile sums: consecutive sums alternate between the two
+    unsigned flag0[kMany ? kMaxFusedUnits : 2] = {};         // the images' flags as they stood before this launch
     int dk_b = -1, dk_g = -1;
     if (kFused) {
         // read before this CTA arrives anywhere: the flag cannot have advanced yet
-        for (int k = 0; k < (int)my_units && k < 2; ++k) flag0[k] = ld_acquire(p.gflag + decode(first + k * stride, p).b);
+        for (int k = 0; k < (int)my_units && k < (kMany ? kMaxFusedUnits : 2); ++k) flag0[k] = ld_acquire(p.gflag + decode(first + k * stride, p).b);
     }
     // Sum of the staged tile's interior per channel (the tiles' interiors partition the image; pixels outside
     // it are zero-filled), in a fixed order; 16 sums to the unit's slot, then the producer lane is told.
-    auto tile_sum = [&](const long long unit_index, const unsigned char* src, const int pitch, const int origin) {
+    auto tile_sum = [&](const long long unit_index, const unsigned char* src, const int pitch, const int origin, float* const fr, const int k_of_cta) {
         const int gsub = lane >> 3, pr = lane & 7;           // pixel 4i + gsub of a row, channel pair pr: conflict-free
         const uint32_t* st32 = reinterpret_cast<const uint32_t*>(src) + origin * NPAIR;
         float s0 = 0.f, s1 = 0.f;
@@ -298,14 +337,14 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
             }
         s0 += __shfl_xor_sync(0xffffffffu, s0, 8);  s1 += __shfl_xor_sync(0xffffffffu, s1, 8);
         s0 += __shfl_xor_sync(0xffffffffu, s0, 16); s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
-        if (lane < 8) { f_red[warp * CG + 2 * lane] = s0; f_red[warp * CG + 2 * lane + 1] = s1; }
+        if (lane < 8) { fr[warp * CG + 2 * lane] = s0; fr[warp * CG + 2 * lane + 1] = s1; }
         mma_bar();
         if (tid < CG) {
             float tsum = 0.f;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) tsum += f_red[w * CG + tid];
+            for (int w = 0; w < kWarps; ++w) tsum += fr[w * CG + tid];
             p.gpart[unit_index * CG + tid] = tsum;
-            mbar_arrive(sumdone);
+            mbar_arrive(sumdone_of(k_of_cta));
         }
     };
     // dk of (image, group) of `un` into f_dk: wait for the image's flag, add the image's partial sums in a fixed
@@ -382,18 +421,15 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         // ---- packed tap pairs of this channel group: P[c][i][d + 2] = (LK[c][i][d], LK[c][i][d + 1]), zero outside 0..12
         if (un.g != cur_g) {
             // the last reader of the old table passed the barrier that closed the previous unit
-            const int KK = p.K, off = (K13 - KK) / 2;        // a smaller kernel is the 13 x 13 one with zeros around it
-            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * KK * KK;
+            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * K13 * K13;
             constexpr int N = CG * K13 * PT, PER = N / kMmaThreads;
             static_assert(N % kMmaThreads == 0, "table entries per thread");
             unsigned lo[PER], hi[PER];
 #pragma unroll
             for (int u = 0; u < PER; ++u) {                  // all loads in flight together
                 const int e = tid + u * kMmaThreads, d = (e % PT) - 2, row = e / PT;   // row = c * 13 + i
-                const int c = row / K13, i = row % K13 - off, dd = d - off;
-                const bool row_ok = i >= 0 && i < KK;
-                lo[u] = (row_ok && dd >= 0 && dd < KK) ? wg[(c * KK + i) * KK + dd] : 0u;
-                hi[u] = (row_ok && dd + 1 >= 0 && dd + 1 < KK) ? wg[(c * KK + i) * KK + dd + 1] : 0u;
+                lo[u] = (d >= 0 && d < K13) ? wg[row * K13 + d] : 0u;
+                hi[u] = (d + 1 >= 0 && d + 1 < K13) ? wg[row * K13 + d + 1] : 0u;
             }
 #pragma unroll
             for (int u = 0; u < PER; ++u) ptab[tid + u * kMmaThreads] = lo[u] | (hi[u] << 16);
@@ -406,10 +442,46 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         if (kFused && k == 0) {
             // both of this CTA's tiles are added up now, at the start, so that every image's flag advances long before
             // any CTA needs dk: the first from the staging buffer, the second from the copy of its interior
-            tile_sum(first, stage, SW, P6 * SW + P6);
-            if (my_units > 1) {
+            tile_sum(first, stage, SW, P6 * SW + P6, f_red, 0);
+            if (!kMany && my_units > 1) {
                 if (alive) alive = mbar_wait(boxfull, 0u, p.ctrl, 0xA9000000u);
-                tile_sum(first + stride, sumbuf, TW, 0);
+                tile_sum(first + stride, sumbuf, TW, 0, f_red + kWarps * CG, 1);
+            }
+            if (kMany) {
+                // the later units' interiors, eight rows (one per warp) at a time; a unit's two halves are added in order
+                const int gsub = lane >> 3, pr = lane & 7;
+                for (int u = 1; u < (int)my_units; ++u) {
+                    float keep = 0.f;
+#pragma unroll 1
+                    for (int half = 0; half < 2; ++half) {
+                        const int h = 2 * (u - 1) + half, slot = h & 1;
+                        if (alive) alive = mbar_wait(boxfull + 8 * slot, (unsigned)((h >> 1) & 1), p.ctrl, 0xA9000000u);
+                        const uint32_t* st32 = reinterpret_cast<const uint32_t*>(sumbuf + slot * (S::BOX_BYTES / 2));
+                        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                        for (int i = 0; i < TW / 4; ++i) {
+                            const uint32_t v = st32[(warp * TW + 4 * i + gsub) * NPAIR + pr];
+                            s0 += __uint_as_float(v << 16);
+                            s1 += __uint_as_float(v & 0xffff0000u);
+                        }
+                        s0 += __shfl_xor_sync(0xffffffffu, s0, 8);  s1 += __shfl_xor_sync(0xffffffffu, s1, 8);
+                        s0 += __shfl_xor_sync(0xffffffffu, s0, 16); s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+                        float* fr = f_red + (1 - slot) * (kWarps * CG);      // the first half follows the first tile's sum, which used f_red
+                        if (lane < 8) { fr[warp * CG + 2 * lane] = s0; fr[warp * CG + 2 * lane + 1] = s1; }
+                        mma_bar();
+                        if (tid == 0) mbar_arrive(boxfree0 + 8 * slot);       // everybody is done with the slot
+                        if (tid < CG) {
+                            float tsum = 0.f;
+#pragma unroll
+                            for (int w = 0; w < kWarps; ++w) tsum += fr[w * CG + tid];
+                            if (half == 0) keep = tsum;
+                            else {
+                                p.gpart[(first + u * stride) * CG + tid] = keep + tsum;
+                                mbar_arrive(sumdone_of(u));
+                            }
+                        }
+                    }
+                }
             }
         }
         if (kMix) {                                          // Eq. 5: the depth-wise stage sees F_att * LK^c
@@ -438,8 +510,8 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
         __syncwarp();
         if (!kFused && lane == 0) mbar_arrive(empty);        // staging may be refilled
         mma_bar();                                           // planes (and the tap table) complete
-        if (kFused && k == 0 && my_units > 1 && tid == 0) {  // every warp is past the staging buffer: the second unit's tile
-            const Unit nx = decode(first + stride, p);
+        if (kFused && k + 1 < my_units && tid == 0) {        // every warp is past the staging buffer: the next unit's tile
+            const Unit nx = decode(first + (k + 1) * stride, p);
             mbar_expect_tx(full, S::STAGE_BYTES);
             tma_load_4d(smem_u32(stage), &map_att, full, nx.g * CG, nx.tx * TW - P6, nx.ty * TH - P6, nx.b);
         }
@@ -551,7 +623,7 @@ stencil_toeplitz_nhwc_bf16(const __grid_constant__ CUtensorMap map_att, const __
             float acc1[NB][NA][4];
             mma_all(acc, warp * 2);
             mma_all(acc1, warp * 2 + 1);
-            if (kFused) obtain_dk(un, flag0[k == 0 ? 0 : 1]);
+            if (kFused) obtain_dk(un, flag0[kMany ? k : (k == 0 ? 0 : 1)]);
             else if (!dk_ready) { pdl_wait_primary(); dk_ready = true; }
             dk_all(dacc, warp * 2);
             write_back(acc, dacc, warp * 2);
@@ -599,10 +671,10 @@ struct Fused {
     unsigned *garr, *gflag;
 };
 
-template <class S, bool kBias, bool kFused, bool kMix = false>
+template <class S, bool kBias, bool kFused, bool kMix = false, bool kMany = false>
 inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk,
                         const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent, int* launches,
-                        std::string* err, const Fused* fu = nullptr, bool skip_copy = false, const void* w_point = nullptr, int K = K13) {
+                        std::string* err, const Fused* fu = nullptr, bool skip_copy = false, const void* w_point = nullptr) {
     const int cc = skip_copy ? 0 : C - Ca;                 // skip_copy: the identity channels are consumed elsewhere (fused 1x1)
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -619,7 +691,6 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
         p.copy_cw = shapes[pick][0]; p.copy_cr = shapes[pick][1];
         p.slot_stride = (cc * 2 * p.copy_cw * p.copy_cr + 127) / 128 * 128;
     }
-    p.K = K;
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
     p.w_point = static_cast<const __nv_bfloat16*>(w_point);
     if (kMix && (Ca != CG || !w_point || (reinterpret_cast<uintptr_t>(w_point) & 3u) != 0)) return kNotApplicable;   // one group, 4-byte loads
@@ -635,7 +706,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
 
     CUtensorMap m_att, m_cin, m_cout, m_box;
     if (!make_map(&m_att, x, B, C, H, W, CG, S::SW, S::ROWS, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
-    if (!make_map(&m_box, x, B, C, H, W, CG, S::TW, S::TH, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
+    if (!make_map(&m_box, x, B, C, H, W, CG, S::TW, kMany ? S::TH / 2 : S::TH, CU_TENSOR_MAP_L2_PROMOTION_L2_64B)) return kNotApplicable;
     if (cc > 0) {
         if (!make_map(&m_cin, x, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
         if (!make_map(&m_cout, out, B, C, H, W, cc, p.copy_cw, p.copy_cr)) return kNotApplicable;
@@ -645,13 +716,13 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     static_assert((S::STAGE_BYTES + CG * S::PLANE_BYTES + PTAB_BYTES) % 128 == 0 && (FUSED_SMEM_FLOATS * 4) % 128 == 0,
                   "the copy ring is a TMA destination: 128-byte aligned");
     const size_t smem = (size_t)S::STAGE_BYTES + (size_t)CG * S::PLANE_BYTES + PTAB_BYTES + (kFused ? FUSED_SMEM_FLOATS * 4 + S::BOX_BYTES : 0) +
-                        (size_t)NSLOT * p.slot_stride + 64;   // 64: the mbarriers
+                        (size_t)NSLOT * p.slot_stride + 128;  // 128: the mbarriers
     if (smem > 227 * 1024) return kNotApplicable;
     static bool attr_set[kMaxDevices] = {};
     const int dev = current_device();
     if (dev < 0) return kNotApplicable;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nhwc_bf16<S, kBias, kFused, kMix>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nhwc_bf16<S, kBias, kFused, kMix, kMany>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
         attr_set[dev] = true;
     }
@@ -668,8 +739,8 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
     attr[1].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = kFused ? 2 : 1;
-    if (kFused && (grid > sm_count() || p.units > 2 * grid)) return kNotApplicable;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias, kFused, kMix>, m_att, m_cin, m_cout, m_box, p);
+    if (kFused && (grid > sm_count() || p.units > (kMany ? kMaxFusedUnits : 2) * grid)) return kNotApplicable;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nhwc_bf16<S, kBias, kFused, kMix, kMany>, m_att, m_cin, m_cout, m_box, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_toeplitz_nhwc_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -681,7 +752,7 @@ inline int launch_shape(int B, int C, int Ca, int H, int W, const void* x, const
 }
 
 inline bool applies(int C, int Ca, int K, int dtype, int layout) {
-    return K >= 3 && K <= K13 && (K & 1) && dtype == 1 /*bf16*/ && layout == kNHWC && Ca % CG == 0 && C % 8 == 0 && C - Ca <= 256;
+    return K == K13 && dtype == 1 /*bf16*/ && layout == kNHWC && Ca % CG == 0 && C % 8 == 0 && C - Ca <= 256;
 }
 
 // Launches the tensor-core stencil if the problem fits it: 0 on success, kNotApplicable otherwise, or an ESC_ERR_* code.
@@ -693,9 +764,9 @@ inline int try_launch_toeplitz(int B, int C, int Ca, int H, int W, int K, int dt
     *tile_w = Shape64x16::TW;
     if (w_point)
         return bias ? kNotApplicable
-                    : launch_shape<Shape64x16, false, false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, w_point, K);
-    return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, nullptr, K)
-                : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, nullptr, K);
+                    : launch_shape<Shape64x16, false, false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy, w_point);
+    return bias ? launch_shape<Shape64x16, true, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy)
+                : launch_shape<Shape64x16, false, false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, skip_copy);
 }
 
 // Whether the whole forward can be one launch of the tensor-core kernel with stage 1 inside: the kernel applies,
@@ -703,7 +774,7 @@ inline int try_launch_toeplitz(int B, int C, int Ca, int H, int W, int K, int dt
 inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, int hidden) {
     if (!applies(C, Ca, K, dtype, layout) || sm_count() <= 0) return false;
     if (Ca > kFusedMaxCa || hidden > kMaxHidden) return false;
-    return units_of<Shape64x16>(B, Ca, H, W) <= 2LL * sm_count();
+    return units_of<Shape64x16>(B, Ca, H, W) <= (long long)kMaxFusedUnits * sm_count();
 }
 
 // The whole forward (stage 1 fused) as one launch; same return convention as try_launch_toeplitz.
@@ -712,11 +783,16 @@ inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype
                             int* launches, std::string* err, int* tile_w, bool skip_copy = false, const void* w_point = nullptr) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden)) return kNotApplicable;
     *tile_w = Shape64x16::TW;
+    const bool many = units_of<Shape64x16>(B, Ca, H, W) > 2LL * sm_count();   // some CTA walks three units or more
     if (w_point)
-        return launch_shape<Shape64x16, false, true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
-                                                           launches, err, &fu, skip_copy, w_point, K);
-    return launch_shape<Shape64x16, false, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
-                                                 launches, err, &fu, skip_copy, nullptr, K);
+        return many ? launch_shape<Shape64x16, false, true, true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
+                                                                        launches, err, &fu, skip_copy, w_point)
+                    : launch_shape<Shape64x16, false, true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
+                                                                  launches, err, &fu, skip_copy, w_point);
+    return many ? launch_shape<Shape64x16, false, true, false, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
+                                                                     launches, err, &fu, skip_copy)
+                : launch_shape<Shape64x16, false, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false,
+                                                        launches, err, &fu, skip_copy);
 }
 
 }}}  // namespace esc::tma::toep

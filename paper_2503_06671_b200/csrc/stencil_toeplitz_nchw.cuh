@@ -45,8 +45,7 @@ struct Params {
     int tiles_x, tiles_y, groups;
     long long units;
     const __nv_bfloat16* x;           // for the copy-through
-    int K;                            // large kernel's size, odd, 3 .. 13: it sits in the middle of the 13 x 13 taps the kernel applies
-    const __nv_bfloat16* w_large;     // [Ca][K][K]
+    const __nv_bfloat16* w_large;     // [Ca][13][13]
     const float* dk;                  // [B][Ca][9]
     const float* bias;                // [B][Ca] constant added to every output of (image, channel), or nullptr (backward pass)
     __nv_bfloat16* out;
@@ -95,7 +94,8 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, kWarps); }
         for (int s = 0; s < kCopySlots; ++s) mbar_init(cfull0 + 8 * s, 1);
-        mbar_init(sumdone, kWarps);
+        mbar_init(sumdone, kWarps);                          // one barrier per unit (the producer lane may fall behind by more
+        mbar_init(sumdone + 8, kWarps);                      // than the one phase a parity wait can tell apart)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -125,7 +125,7 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
                 // round trip stays off their path
                 for (int k = 0; k < (int)my_units && k < 2; ++k) {
                     const Unit un = decode(first + k * stride, p);
-                    if (alive) alive = mbar_wait(sumdone, (unsigned)(k & 1), p.ctrl, 0xB9000000u);
+                    if (alive) alive = mbar_wait(sumdone + 8 * k, 0u, p.ctrl, 0xB9000000u);
                     unsigned old;
                     asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(old) : "l"(p.garr + un.b), "r"((unsigned)(p.upi - 1)) : "memory");
                     if (old == (unsigned)(p.upi - 1)) st_release(p.gflag + un.b, seen[k] + 1u);   // the counter has wrapped back to 0
@@ -188,7 +188,7 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
     }
     // Sum of a tile's interior (the tiles' interiors partition the image; pixels outside it are zero-filled): this
     // warp's two channels, a row of 64 pixels per load, rows in order, then a fixed butterfly over the lanes.
-    auto tile_sum = [&](const long long unit_index, const unsigned char* buf) {
+    auto tile_sum = [&](const long long unit_index, const unsigned char* buf, const int k_of_cta) {
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
             const uint32_t* pl = reinterpret_cast<const uint32_t*>(buf + (size_t)(warp * 2 + cc) * PLANE) + (P6 * PP + XS) / 2 + lane;
@@ -204,7 +204,7 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
             for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             if (lane == 0) p.gpart[unit_index * CG + warp * 2 + cc] = s;
         }
-        if (lane == 0) mbar_arrive(sumdone);
+        if (lane == 0) mbar_arrive(sumdone + 8 * k_of_cta);
     };
     auto obtain_dk = [&](const Unit& un, const unsigned seen) {
         if (un.b == dk_b && un.g == dk_g) return;
@@ -283,18 +283,15 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
         // ---- packed tap pairs of this channel group: P[c][i][d + 2] = (LK[c][i][d], LK[c][i][d + 1]), zero outside 0..12
         if (un.g != cur_g) {
             if (cur_g >= 0) mma_bar();                       // everybody is done with the old table
-            const int KK = p.K, off = (K13 - KK) / 2;        // a smaller kernel is the 13 x 13 one with zeros around it
-            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * KK * KK;
+            const unsigned short* wg = reinterpret_cast<const unsigned short*>(p.w_large) + (size_t)un.g * CG * K13 * K13;
             constexpr int N = CG * K13 * PT, PER = N / kMmaThreads;
             static_assert(N % kMmaThreads == 0, "table entries per thread");
             unsigned lo[PER], hi[PER];
 #pragma unroll
             for (int u = 0; u < PER; ++u) {
                 const int e = tid + u * kMmaThreads, d = (e % PT) - 2, row = e / PT;   // row = c * 13 + i
-                const int c = row / K13, i = row % K13 - off, dd = d - off;
-                const bool row_ok = i >= 0 && i < KK;
-                lo[u] = (row_ok && dd >= 0 && dd < KK) ? wg[(c * KK + i) * KK + dd] : 0u;
-                hi[u] = (row_ok && dd + 1 >= 0 && dd + 1 < KK) ? wg[(c * KK + i) * KK + dd + 1] : 0u;
+                lo[u] = (d >= 0 && d < K13) ? wg[row * K13 + d] : 0u;
+                hi[u] = (d + 1 >= 0 && d + 1 < K13) ? wg[row * K13 + d + 1] : 0u;
             }
 #pragma unroll
             for (int u = 0; u < PER; ++u) ptab[tid + u * kMmaThreads] = lo[u] | (hi[u] << 16);
@@ -307,10 +304,10 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
         if (kFused && k == 0) {
             // both of this CTA's tiles are added up now, at the start, so that every image's flag advances long before
             // any CTA needs dk
-            tile_sum(first, planes);
+            tile_sum(first, planes, 0);
             if (my_units > 1) {
                 if (alive) alive = mbar_wait(full0 + 8, 0u, p.ctrl, 0xA9000000u);
-                tile_sum(first + stride, bufs + BUF_BYTES);
+                tile_sum(first + stride, bufs + BUF_BYTES, 1);
             }
         }
 
@@ -449,12 +446,12 @@ inline long long units_of(int B, int Ca, int H, int W) {
 // aligned tensors (a TMA base, and the bulk copies of the identity channels).
 inline bool applies(int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* out) {
     (void)H;
-    return K >= 3 && K <= K13 && (K & 1) && dtype == 1 /*bf16*/ && layout == kNCHW && Ca % CG == 0 && C >= Ca && W % 8 == 0 &&
+    return K == K13 && dtype == 1 /*bf16*/ && layout == kNCHW && Ca % CG == 0 && C >= Ca && W % 8 == 0 &&
            (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
 }
 
 template <bool kFused>
-inline int launch(int K, int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, const float* bias, void* out,
+inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, const float* bias, void* out,
                   unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err, const toep::Fused* fu) {
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
@@ -462,7 +459,6 @@ inline int launch(int K, int B, int C, int Ca, int H, int W, const void* x, cons
     p.units = units_of(B, Ca, H, W);
     if (p.units > 0x7fffffffLL) return kNotApplicable;
     p.x = static_cast<const __nv_bfloat16*>(x);
-    p.K = K;
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
     p.dk = dk; p.bias = bias; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
@@ -477,8 +473,8 @@ inline int launch(int K, int B, int C, int Ca, int H, int W, const void* x, cons
     CUtensorMap m_att;
     if (!make_map_nchw(&m_att, x, B, C, H, W)) return kNotApplicable;
     static_assert((2 * BUF_BYTES + PTAB_BYTES + FUSED_SMEM_FLOATS * 4) % 128 == 0, "the copy ring is a bulk-copy destination");
-    const size_t smem = (size_t)2 * BUF_BYTES + PTAB_BYTES + FUSED_SMEM_FLOATS * 4 + (size_t)kCopySlots * kCopySlotBytes + 64;   // 64: the mbarriers
-    static_assert((size_t)2 * BUF_BYTES + PTAB_BYTES + FUSED_SMEM_FLOATS * 4 + (size_t)kCopySlots * kCopySlotBytes + 64 <= 227 * 1024, "shared memory");
+    const size_t smem = (size_t)2 * BUF_BYTES + PTAB_BYTES + FUSED_SMEM_FLOATS * 4 + (size_t)kCopySlots * kCopySlotBytes + 128;  // 128: the mbarriers
+    static_assert((size_t)2 * BUF_BYTES + PTAB_BYTES + FUSED_SMEM_FLOATS * 4 + (size_t)kCopySlots * kCopySlotBytes + 128 <= 227 * 1024, "shared memory");
     static bool attr_set[kMaxDevices] = {};
     const int dev = current_device();
     if (dev < 0) return kNotApplicable;
@@ -517,7 +513,7 @@ inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int 
                       const float* dk, const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent,
                       int* launches, std::string* err) {
     if (!applies(C, Ca, H, W, K, dtype, layout, x, out) || sm_count() <= 0) return kNotApplicable;
-    return launch<false>(K, B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr);
+    return launch<false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr);
 }
 
 inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, int hidden, const void* x, const void* out) {
@@ -530,7 +526,7 @@ inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, 
 inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
                             const toep::Fused& fu, void* out, unsigned* ctrl, cudaStream_t st, int* launches, std::string* err) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden, x, out)) return kNotApplicable;
-    return launch<true>(K, B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
+    return launch<true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
 }
 
 }}}  // namespace esc::tma::toepn

@@ -97,7 +97,7 @@ def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True, engine=None):
 @pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
 def test_forward_pw(pkg, oracle, shape, dtype, layout):
     path, _ = _run(pkg, oracle, shape, dtype, layout)
-    fast = dtype == synth.BF16 and layout == synth.NHWC and shape[5] == 13 and shape[2] == 16
+    fast = dtype == synth.BF16 and layout == synth.NHWC and shape[5] <= 13 and shape[2] == 16     # any odd K up to 13
     assert path == (4 if fast else 1)                      # the mix inside the tensor-core depth-wise kernel
 
 

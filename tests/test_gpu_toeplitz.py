@@ -98,7 +98,8 @@ def test_stencil_stage_explicit_dk_and_determinism(pkg, oracle):
     assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16)) and torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
 
 
-@pytest.mark.parametrize("shape", [(1, 64, 16, 300, 640), (70, 32, 16, 40, 64), (16, 64, 32, 33, 70), (14, 48, 48, 30, 90), (1, 64, 16, 100, 150)],
+@pytest.mark.parametrize("shape", [(1, 64, 16, 300, 640), (70, 32, 16, 40, 64), (16, 64, 32, 33, 70), (14, 48, 48, 30, 90), (1, 64, 16, 100, 150),
+                                   (1, 64, 16, 540, 960), (100, 32, 16, 64, 64), (3, 64, 32, 200, 400), (1, 48, 16, 700, 1000)],
                          ids=lambda s: "x".join(map(str, s)))
 @pytest.mark.parametrize("mode", ["one_launch", "unaligned", "two_launches"])
 def test_one_launch_forward_estimator_inputs(pkg, oracle, shape, mode):
@@ -106,7 +107,8 @@ def test_one_launch_forward_estimator_inputs(pkg, oracle, shape, mode):
     units at once), the same with the estimator's weights at an address that is only 2-byte aligned, and
     "two_launches": the same forward with stage 1 as its own kernel.
     Shapes: one image with two units per CTA (190 units), 210 / 192 / 168 units whose image and channel group change
-    between a CTA's two units (one, two, three groups), and a launch with fewer units than SMs.  All outputs compared with the oracle, twice (the counters and flags are re-used)."""
+    between a CTA's two units (one, two, three groups), a launch with fewer units than SMs, and 510 / 400 / 546 / 704
+    units: CTAs walk three to five units, whose interiors pass through the two half-tile slots before the first products.  All outputs compared with the oracle, twice (the counters and flags are re-used)."""
     import torch
 
     B, C, C_a, H, W = shape
