@@ -314,9 +314,11 @@ int esc_convattn_device_status(void* workspace, void* stream);
  * 6 = the tensor-core (banded Toeplitz) kernel on NCHW tensors.  For tests and benchmarks. */
 int esc_convattn_last_path(void);
 
-/* Which arithmetic units evaluate the depth-wise 13x13 stage of Eq. 4 line 3 on NHWC bf16 tensors, for
- * later calls on this thread.  ESC_ENGINE_AUTO (default): the tensor-core kernel where it applies
- * (K = 13, C_a a multiple of 16, C a multiple of 8, no point-wise LK^c), else the FP32 kernels.
+/* Which arithmetic units evaluate the depth-wise large-kernel stage of Eq. 4 line 3 on bf16 tensors (and the tap
+ * gradients of the backward pass), for later calls on this thread.  ESC_ENGINE_AUTO (default): the tensor-core
+ * kernels where they apply -- odd K up to 13 (a smaller kernel is zero-padded to 13 x 13 in the workspace), C_a a
+ * multiple of 16; NHWC with C a multiple of 8 (also with the point-wise LK^c when C_a = 16), or NCHW with W a
+ * multiple of 8 and 16-byte aligned tensors -- else the FP32 kernels.
  * ESC_ENGINE_FP32: never the tensor-core kernel.  ESC_ENGINE_TENSOR: the tensor-core kernel or, where
  * it does not apply, the guarded generic kernel.  Both engines multiply exactly (bf16 x bf16 in fp32) and
  * accumulate in fp32; they differ in the order of the 169 additions, i.e. by fp32 rounding before
