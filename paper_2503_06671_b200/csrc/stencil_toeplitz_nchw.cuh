@@ -46,6 +46,7 @@ struct Params {
     long long units;
     const __nv_bfloat16* x;           // for the copy-through
     const __nv_bfloat16* w_large;     // [Ca][13][13]
+    const __nv_bfloat16* w_point;     // kMix: [16][16] point-wise filter LK^c of the decomposed form (Eq. 5), row = output channel
     const float* dk;                  // [B][Ca][9]
     const float* bias;                // [B][Ca] constant added to every output of (image, channel), or nullptr (backward pass)
     __nv_bfloat16* out;
@@ -78,7 +79,16 @@ __device__ __forceinline__ Unit decode(long long u64v, const Params& p) {
     return r;
 }
 
-template <bool kFused>
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+
+// kMix: the decomposed large kernel of Eq. 5 -- after a tile has landed (and, with stage 1 inside, after its sum has been
+// taken from the unmixed values) the 16 planes are replaced, eight pixels at a time and in place, by LK^c applied across
+// them: D (16 output channels x 8 pixels) = LK^c (16 x 16) x B (16 channels x 8 pixels), B straight from the planes by
+// ldmatrix.trans, one rounding to bf16; then one block-wide barrier before the depth-wise products.
+template <bool kFused, bool kMix = false>
 __global__ void __launch_bounds__(kThreads, 1)
 stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Params p)
 {
@@ -311,6 +321,37 @@ stencil_toeplitz_nchw_bf16(const __grid_constant__ CUtensorMap map_att, const Pa
             }
         }
 
+        if (kMix) {
+            // A = LK^c: a0 = (row g, columns 2t, 2t + 1), a1 = (row g + 8, ...), a2 / a3 = the same rows, columns + 8
+            const uint32_t* wp = reinterpret_cast<const uint32_t*>(p.w_point);
+            const uint32_t a0 = __ldg(wp + g * 8 + t), a1 = __ldg(wp + (g + 8) * 8 + t);
+            const uint32_t a2 = __ldg(wp + g * 8 + 4 + t), a3 = __ldg(wp + (g + 8) * 8 + 4 + t);
+            constexpr int BPR = PP / 8, NBLK = ROWS * BPR;   // blocks of 8 pixels per row, per plane
+            for (int pb = 2 * warp; pb < NBLK; pb += 2 * kWarps) {
+                // matrix mi: channels 8 (mi & 1) .. + 7 of pixel block pb + (mi >> 1); row mr of it = one channel's 8 pixels
+                const int blk = min(pb + (mi >> 1), NBLK - 1);
+                const uint32_t at = (uint32_t)(((mi & 1) * 8 + mr) * PLANE + ((blk / BPR) * PP + (blk % BPR) * 8) * 2);
+                uint32_t b[4];
+                ldsm_x4_trans(planes_a + at, b);
+                float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_bf16(d0, a0, a1, a2, a3, b[0], b[1]);
+                mma_bf16(d1, a0, a1, a2, a3, b[2], b[3]);
+                __syncwarp();                                // every lane has its inputs before any plane is overwritten
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int bk = pb + h;
+                    if (bk < NBLK) {
+                        const float* d = h ? d1 : d0;
+                        unsigned char* px = planes + ((size_t)(bk / BPR) * PP + (bk % BPR) * 8 + 2 * t) * 2;
+                        const __nv_bfloat162 lo = __floats2bfloat162_rn(d[0], d[1]), hi = __floats2bfloat162_rn(d[2], d[3]);
+                        *reinterpret_cast<__nv_bfloat162*>(px + (size_t)g * PLANE) = lo;
+                        *reinterpret_cast<__nv_bfloat162*>(px + (size_t)(g + 8) * PLANE) = hi;
+                    }
+                }
+            }
+            fence_async_smem();                              // these stores before the next tile's TMA load into the same buffer
+            mma_bar();                                       // every plane is mixed before any warp multiplies
+        }
         const unsigned sh = (g & 1) ? 0u : 16u;
         float acc[NB][NA][4], acc1[NB][NA][4], dacc[NB][NA][4];
         float dkv[9];
@@ -450,9 +491,10 @@ inline bool applies(int C, int Ca, int H, int W, int K, int dtype, int layout, c
            (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
 }
 
-template <bool kFused>
+template <bool kFused, bool kMix = false>
 inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, const float* bias, void* out,
-                  unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err, const toep::Fused* fu) {
+                  unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err, const toep::Fused* fu,
+                  const void* w_point = nullptr) {
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
     p.tiles_x = (W + TW - 1) / TW; p.tiles_y = (H + TH - 1) / TH; p.groups = Ca / CG;
@@ -460,6 +502,8 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
     if (p.units > 0x7fffffffLL) return kNotApplicable;
     p.x = static_cast<const __nv_bfloat16*>(x);
     p.w_large = static_cast<const __nv_bfloat16*>(w_large);
+    p.w_point = static_cast<const __nv_bfloat16*>(w_point);
+    if (kMix && (Ca != CG || !w_point || (reinterpret_cast<uintptr_t>(w_point) & 3u) != 0)) return kNotApplicable;   // one group, 4-byte loads
     p.dk = dk; p.bias = bias; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
     p.copy_bytes = (long long)(C - Ca) * H * W * 2;           // a multiple of 16: W is a multiple of 8
@@ -479,7 +523,7 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
     const int dev = current_device();
     if (dev < 0) return kNotApplicable;
     if (!attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nchw_bf16<kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stencil_toeplitz_nchw_bf16<kFused, kMix>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return kNotApplicable; }
         attr_set[dev] = true;
     }
@@ -497,7 +541,7 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
     cfg.attrs = attr;
     cfg.numAttrs = kFused ? 2 : 1;
     if (kFused && (grid > sm_count() || p.units > 2 * grid)) return kNotApplicable;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nchw_bf16<kFused>, m_att, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, stencil_toeplitz_nchw_bf16<kFused, kMix>, m_att, p);
     if (e != cudaSuccess) {
         char buf[256];
         snprintf(buf, sizeof buf, "stencil_toeplitz_nchw_bf16 launch: %s (%s)", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -511,8 +555,11 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
 // Launches the NCHW tensor-core stencil if the problem fits it: 0 on success, kNotApplicable otherwise, or an ESC_ERR_* code.
 inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
                       const float* dk, const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent,
-                      int* launches, std::string* err) {
+                      int* launches, std::string* err, const void* w_point = nullptr) {
     if (!applies(C, Ca, H, W, K, dtype, layout, x, out) || sm_count() <= 0) return kNotApplicable;
+    if (w_point)
+        return bias ? kNotApplicable
+                    : launch<false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, w_point);
     return launch<false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr);
 }
 
@@ -524,8 +571,11 @@ inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, 
 
 // The whole forward (stage 1 inside) as one launch.
 inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
-                            const toep::Fused& fu, void* out, unsigned* ctrl, cudaStream_t st, int* launches, std::string* err) {
+                            const toep::Fused& fu, void* out, unsigned* ctrl, cudaStream_t st, int* launches, std::string* err,
+                            const void* w_point = nullptr) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden, x, out)) return kNotApplicable;
+    if (w_point)
+        return launch<true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu, w_point);
     return launch<true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
 }
 

@@ -65,7 +65,7 @@ def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True, engine=None):
     assert pkg.esc_convattn_device_status(ws) == 0
     got = util.to_host_nchw(out, layout)
     path = pkg.esc_convattn_last_path()
-    if dtype == synth.BF16 and path in (2, 4):
+    if dtype == synth.BF16 and path in (2, 4, 6):
         # The fast kernels keep the mixed features in its bf16 tile: one rounding of F_att * LK^c, as a
         # bf16 network stores that tensor.  (a) Against the exact oracle the error is bounded by the two
         # roundings: 2^-9 * sum|w||mixed| for the intermediate plus 2^-9 * |out| for the result, both
@@ -97,8 +97,19 @@ def _run(pkg, oracle, shape, dtype, layout, width=0, forward=True, engine=None):
 @pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
 def test_forward_pw(pkg, oracle, shape, dtype, layout):
     path, _ = _run(pkg, oracle, shape, dtype, layout)
-    fast = dtype == synth.BF16 and layout == synth.NHWC and shape[5] <= 13 and shape[2] == 16     # any odd K up to 13
-    assert path == (4 if fast else 1)                      # the mix inside the tensor-core depth-wise kernel
+    fast = dtype == synth.BF16 and shape[5] <= 13 and shape[2] == 16                              # any odd K up to 13
+    fast_nchw = fast and layout == synth.NCHW and shape[4] % 8 == 0
+    assert path == (4 if fast and layout == synth.NHWC else 6 if fast_nchw else 1)   # the mix inside the tensor-core kernels
+
+
+@pytest.mark.parametrize("forward", [True, False], ids=["forward", "stencil"])
+@pytest.mark.parametrize("shape", [(2, 48, 16, 64, 64, 13), (1, 64, 16, 45, 72, 13), (1, 64, 16, 300, 640, 13), (70, 32, 16, 40, 64, 13),
+                                   (1, 16, 16, 5, 8, 13), (2, 64, 16, 37, 88, 9)], ids=lambda s: "x".join(map(str, s)))
+def test_pw_nchw_tensor_kernel(pkg, oracle, shape, forward):
+    """The mix inside the NCHW tensor-core kernel (LK^c applied across the 16 planes, eight pixels at a time): one and two
+    units per CTA, of one image and of two, a map smaller than the kernel, and K = 9."""
+    path, _ = _run(pkg, oracle, shape, synth.BF16, synth.NCHW, forward=forward)
+    assert path == 6
 
 
 @pytest.mark.parametrize("forward", [True, False], ids=["forward", "stencil"])
