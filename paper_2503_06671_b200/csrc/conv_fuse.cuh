@@ -15,6 +15,7 @@
 #pragma once
 #include "common.cuh"
 #include "stencil_toeplitz.cuh"
+#include "stencil_toeplitz_nchw.cuh"
 
 namespace esc { namespace fuse {
 
@@ -183,6 +184,175 @@ conv_fuse_nhwc_bf16(const Params p)
         }
     }
 }
+
+// ---- NCHW bf16, C in {32, 48, 64}: the same product with the roles of the operands exchanged ---------------------------
+//   out[n][px] = b[n] + sum_k W[n][k] cat[k][px] (+ residual[n][px]):  D (16 output channels x 8 pixels) = A (W, 16 x 16) x
+//   B (16 channels x 8 pixels).  A tile is C channel rows of 128 pixels (256 contiguous bytes each; rows k < Ca from `att`,
+//   the rest from `idt`) and the residual's rows, staged with 16-byte asynchronous copies three tiles deep; B comes from the
+//   tile by ldmatrix.trans (row pitch 272 bytes: conflict-free), W sits in registers as A fragments; a warp owns 16 pixels
+//   and all C output channels, adds bias and residual in fp32, rounds once and writes the results over the residual's tile,
+//   from where the block stores whole 256-byte rows.
+namespace nchw {
+constexpr int kPixN = 128, kThreadsN = 256, kPitchN = kPixN * 2 + 16;
+struct Params {
+    const __nv_bfloat16* att;         // [B][C][HW]: planes 0 .. Ca-1 are F_res
+    const __nv_bfloat16* idt;         // [B][C][HW]: planes Ca .. C-1 are F_idt
+    const __nv_bfloat16* w;           // [C][C], row = output channel
+    const __nv_bfloat16* bias;        // [C] or nullptr
+    const __nv_bfloat16* residual;    // [B][C][HW] or nullptr
+    __nv_bfloat16* out;               // [B][C][HW]
+    long long HW;                     // a multiple of 8
+    int B, C, Ca;
+};
+
+template <int C>
+__global__ void __launch_bounds__(kThreadsN, 2)
+conv_fuse_nchw_bf16(const Params p)
+{
+    constexpr int MT = C / 16, KS = C / 16, STAGE = 2 * C * kPitchN, NS = 3, WP = C * 2 + 16;
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* wsm = smem + (NS - 1) * STAGE;            // w_fuse passes through the last stage on its way to registers
+    static_assert(C * WP <= STAGE, "w_fuse fits a stage");
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int mi = lane >> 3, mr = lane & 7;
+    for (int e = tid; e < C * (C / 8); e += kThreadsN) {
+        const int r = e / (C / 8), q = e % (C / 8);
+        *reinterpret_cast<uint4*>(wsm + r * WP + q * 16) = __ldg(reinterpret_cast<const uint4*>(p.w + (size_t)r * C) + q);
+    }
+    __syncthreads();
+    uint32_t aw[MT][KS][4];                                  // A fragments: rows 16 mt + (0-7 | 8-15), columns 16 ks + (0-7 | 8-15)
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+            tma::toep::ldsm_x4(tma::smem_u32(wsm) + (uint32_t)((16 * mt + (mi & 1) * 8 + mr) * WP + (16 * ks + (mi >> 1) * 8) * 2), aw[mt][ks]);
+    float bs[MT][2];                                         // bias of this lane's output channels 16 mt + g, + 8
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        bs[mt][0] = p.bias ? __bfloat162float(p.bias[16 * mt + g]) : 0.f;
+        bs[mt][1] = p.bias ? __bfloat162float(p.bias[16 * mt + g + 8]) : 0.f;
+    }
+    pdl_wait_primary();                                      // the attention planes come from the kernel before this one
+
+    const long long tiles_per_img = (p.HW + kPixN - 1) / kPixN, ntiles = tiles_per_img * p.B;
+    auto stage = [&](long long tile, int buf) {
+        const long long b = tile / tiles_per_img, p0 = (tile - b * tiles_per_img) * kPixN;
+        const uint32_t xs = tma::smem_u32(smem + buf * STAGE), rs = xs + C * kPitchN;
+        const size_t img = (size_t)b * C * p.HW;
+#pragma unroll
+        for (int u = 0; u < C * (kPixN / 8) / kThreadsN; ++u) {
+            const int e = tid + u * kThreadsN, ch = e / (kPixN / 8), q = e % (kPixN / 8);
+            const bool ok = p0 + q * 8 < p.HW;
+            const size_t at = img + (size_t)ch * p.HW + (ok ? p0 + q * 8 : 0);
+            cp_async16(xs + ch * kPitchN + q * 16, (ch < p.Ca ? p.att : p.idt) + at, ok);
+            if (p.residual) cp_async16(rs + ch * kPitchN + q * 16, p.residual + at, ok);
+        }
+        cp_async_commit();
+    };
+    static_assert(C * (kPixN / 8) % kThreadsN == 0, "pieces per thread");
+    long long tile = blockIdx.x;
+    int buf = 0;
+#pragma unroll
+    for (int j = 0; j < NS - 1; ++j) {
+        if (tile + j * (long long)gridDim.x < ntiles) stage(tile + j * (long long)gridDim.x, j);
+        else cp_async_commit();
+    }
+    for (; tile < ntiles; tile += gridDim.x, buf = buf + 1 == NS ? 0 : buf + 1) {
+        const long long b = tile / tiles_per_img, p0 = (tile - b * tiles_per_img) * kPixN;
+        unsigned char* xsm = smem + buf * STAGE;
+        unsigned char* rsm = xsm + C * kPitchN;
+        cp_async_wait<NS - 2>();
+        __syncthreads();                                     // the tile is there for everybody; everybody is done with the tile before
+        {
+            const long long nx = tile + (NS - 1) * (long long)gridDim.x;
+            if (nx < ntiles) stage(nx, buf == 0 ? NS - 1 : buf - 1);
+            else cp_async_commit();
+        }
+        float acc[MT][2][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) acc[mt][nt][v] = 0.f;
+        const uint32_t b_lane = tma::smem_u32(xsm) + (uint32_t)(((mi & 1) * 8 + mr) * kPitchN + (warp * 16 + (mi >> 1) * 8) * 2);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t bfrag[4];                               // (channels 16 ks .. + 7 | + 8 .. + 15) x (pixels 0-7 | 8-15 of the warp's 16)
+            tma::toepn::ldsm_x4_trans(b_lane + (uint32_t)(16 * ks * kPitchN), bfrag);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                tma::toep::mma_bf16(acc[mt][0], aw[mt][ks][0], aw[mt][ks][1], aw[mt][ks][2], aw[mt][ks][3], bfrag[0], bfrag[1]);
+                tma::toep::mma_bf16(acc[mt][1], aw[mt][ks][0], aw[mt][ks][1], aw[mt][ks][2], aw[mt][ks][3], bfrag[2], bfrag[3]);
+            }
+        }
+        // acc[mt][nt]: [0], [1] = channel 16 mt + g, pixels 8 nt + 2t, + 1 of the warp's 16; [2], [3] = channel + 8
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t* cell = reinterpret_cast<uint32_t*>(rsm + (16 * mt + g + 8 * h) * kPitchN + (warp * 16 + 8 * nt + 2 * t) * 2);
+                    float v0 = acc[mt][nt][2 * h] + bs[mt][h], v1 = acc[mt][nt][2 * h + 1] + bs[mt][h];
+                    if (p.residual) {
+                        const uint32_t rr = *cell;
+                        v0 += __uint_as_float(rr << 16);
+                        v1 += __uint_as_float(rr & 0xffff0000u);
+                    }
+                    const __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                    *cell = *reinterpret_cast<const uint32_t*>(&h2);
+                }
+        __syncthreads();                                     // whole rows are complete
+        const size_t img = (size_t)b * C * p.HW;
+#pragma unroll
+        for (int u = 0; u < C * (kPixN / 8) / kThreadsN; ++u) {
+            const int e = tid + u * kThreadsN, ch = e / (kPixN / 8), q = e % (kPixN / 8);
+            if (p0 + q * 8 < p.HW)
+                *reinterpret_cast<uint4*>(p.out + img + (size_t)ch * p.HW + p0 + q * 8) = *reinterpret_cast<const uint4*>(rsm + ch * kPitchN + q * 16);
+        }
+    }
+}
+
+inline bool applies(int C, int Ca, long long HW, int dtype, int layout, const void* x, const void* out, const void* residual, const void* w) {
+    auto al = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; };
+    return dtype == 1 /*bf16*/ && layout == kNCHW && (C == 32 || C == 48 || C == 64) && Ca <= C && HW % 8 == 0 && al(x) && al(out) &&
+           al(residual) && al(w);
+}
+
+template <int C>
+inline cudaError_t launch_c(const Params& p, cudaStream_t st) {
+    const size_t smem = (size_t)3 * 2 * C * kPitchN;
+    static bool attr_set[tma::kMaxDevices] = {};
+    const int dev = tma::current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(conv_fuse_nchw_bf16<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const long long ntiles = ((p.HW + kPixN - 1) / kPixN) * p.B, cap = 2LL * (tma::sm_count() > 0 ? tma::sm_count() : 148);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(ntiles < cap ? ntiles : cap));
+    cfg.blockDim = dim3(kThreadsN);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, conv_fuse_nchw_bf16<C>, p);
+}
+inline cudaError_t launch(const Params& p, cudaStream_t st) {
+    switch (p.C) {
+        case 32: return launch_c<32>(p, st);
+        case 48: return launch_c<48>(p, st);
+        case 64: return launch_c<64>(p, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+}  // namespace nchw
 
 // Any type and layout: a block takes 32 pixels, reads their C values of `out` (the concatenated map written by the
 // stages before) into shared memory as fp32, then every thread computes outputs (pixel, channel) and writes them

@@ -359,9 +359,9 @@ int launch_stencil(const Problem& p0, const void* x, const void* w_large0, const
                                                            out, ctrl, st, dependent, &g_last_launches, &g_last_error, &tw, p.skip_copy, p.w_point);
         if (rc == ESC_OK) { g_last_path = 4; g_last_tile_w = tw; return ESC_OK; }
         if (rc != esc::tma::kNotApplicable) return rc;
-        if (!p.skip_copy) {                                  // the same arithmetic on NCHW tensors
+        {                                                    // the same arithmetic on NCHW tensors
             const int rn = esc::tma::toepn::try_launch(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, dk, p.bias, out,
-                                                       ctrl, st, dependent, &g_last_launches, &g_last_error, p.w_point);
+                                                       ctrl, st, dependent, &g_last_launches, &g_last_error, p.w_point, p.skip_copy);
             if (rn == ESC_OK) { g_last_path = 6; g_last_tile_w = esc::tma::toepn::TW; return ESC_OK; }
             if (rn != esc::tma::kNotApplicable) return rn;
         }
@@ -479,15 +479,15 @@ int forward_impl(const Problem& p0, const void* x, const void* w_large0, const E
             g_last_error.clear();
         }
     }
-    if (g_fuse_stage1 && !p.dense && (!p.w_point || p.Ca == esc::tma::CG) && !p.bias && !p.skip_copy && g_engine_policy != ESC_ENGINE_FP32 &&
+    if (g_fuse_stage1 && !p.dense && (!p.w_point || p.Ca == esc::tma::CG) && !p.bias && g_engine_policy != ESC_ENGINE_FP32 &&
         g_tile_policy == 0) {
         const esc::tma::toep::Fused fu{est.w_last, est.b_last, est.w_down, est.b_down, est.hidden, w.unit_sums, w.arrivals, w.flags};
         const int rc = esc::tma::toepn::try_launch_fused(p.B, p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, w_large, fu, out, w.ctrl, st,
-                                                         &g_last_launches, &g_last_error, p.w_point);
+                                                         &g_last_launches, &g_last_error, p.w_point, p.skip_copy);
         if (rc == ESC_OK) { g_last_path = 6; g_last_tile_w = esc::tma::toepn::TW; return ESC_OK; }
         if (rc != esc::tma::kNotApplicable) { (void)cudaGetLastError(); g_last_error.clear(); }
     }
-    const bool tensor_nchw = !p.dense && (!p.w_point || p.Ca == esc::tma::CG) && !p.bias && !p.skip_copy && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
+    const bool tensor_nchw = !p.dense && (!p.w_point || p.Ca == esc::tma::CG) && !p.bias && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
                              esc::tma::toepn::applies(p.C, p.Ca, p.H, p.W, p.K, p.dtype, p.layout, x, out);
     int rc = launch_gap(p0, x, est, w, w.dk, st, tensor_stencil_follows(p) || tensor_nchw);
     if (rc != ESC_OK) return rc;
@@ -980,6 +980,22 @@ int esc_convattn_forward_fused(const void* x, int B, int C, int C_a, int H, int 
         fp.residual = static_cast<const __nv_bfloat16*>(residual); fp.out = static_cast<__nv_bfloat16*>(out);
         fp.pixels = pixels; fp.C = C; fp.Ca = C_a;
         ESC_CUDA(esc::fuse::launch_fast(fp, st));
+        ++g_last_launches;
+        return ESC_OK;
+    }
+    // The same on NCHW tensors: the NCHW tensor-core stencil without its copy of the identity planes, then the NCHW 1x1 kernel.
+    if (K == esc::tma::K13 && g_engine_policy != ESC_ENGINE_FP32 && g_tile_policy == 0 &&
+        esc::fuse::nchw::applies(C, C_a, (long long)H * W, dtype, layout, x, out, residual, w_fuse) &&
+        esc::tma::toepn::applies(C, C_a, H, W, K, dtype, layout, x, out)) {
+        p.skip_copy = true;
+        rc = forward_impl(p, x, w_large, est, out, workspace, st);
+        if (rc != ESC_OK) return rc;
+        esc::fuse::nchw::Params fp;
+        fp.att = static_cast<const __nv_bfloat16*>(out); fp.idt = static_cast<const __nv_bfloat16*>(x);
+        fp.w = static_cast<const __nv_bfloat16*>(w_fuse); fp.bias = static_cast<const __nv_bfloat16*>(b_fuse);
+        fp.residual = static_cast<const __nv_bfloat16*>(residual); fp.out = static_cast<__nv_bfloat16*>(out);
+        fp.HW = (long long)H * W; fp.B = B; fp.C = C; fp.Ca = C_a;
+        ESC_CUDA(esc::fuse::nchw::launch(fp, st));
         ++g_last_launches;
         return ESC_OK;
     }

@@ -494,7 +494,7 @@ inline bool applies(int C, int Ca, int H, int W, int K, int dtype, int layout, c
 template <bool kFused, bool kMix = false>
 inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void* w_large, const float* dk, const float* bias, void* out,
                   unsigned* ctrl, cudaStream_t st, bool dependent, int* launches, std::string* err, const toep::Fused* fu,
-                  const void* w_point = nullptr) {
+                  const void* w_point = nullptr, bool skip_copy = false) {
     Params p;
     p.B = B; p.C = C; p.Ca = Ca; p.H = H; p.W = W;
     p.tiles_x = (W + TW - 1) / TW; p.tiles_y = (H + TH - 1) / TH; p.groups = Ca / CG;
@@ -506,7 +506,7 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
     if (kMix && (Ca != CG || !w_point || (reinterpret_cast<uintptr_t>(w_point) & 3u) != 0)) return kNotApplicable;   // one group, 4-byte loads
     p.dk = dk; p.bias = bias; p.out = static_cast<__nv_bfloat16*>(out); p.ctrl = ctrl;
     p.wait_first = dependent ? 0 : 1;
-    p.copy_bytes = (long long)(C - Ca) * H * W * 2;           // a multiple of 16: W is a multiple of 8
+    p.copy_bytes = skip_copy ? 0 : (long long)(C - Ca) * H * W * 2;   // a multiple of 16: W is a multiple of 8; skip_copy: consumed elsewhere (fused 1x1)
     p.w_last = p.b_last = p.w_down = p.b_down = nullptr; p.hidden = 0; p.gpart = nullptr; p.garr = p.gflag = nullptr;
     p.upi = p.groups * p.tiles_x * p.tiles_y;
     if (kFused) {
@@ -555,12 +555,12 @@ inline int launch(int B, int C, int Ca, int H, int W, const void* x, const void*
 // Launches the NCHW tensor-core stencil if the problem fits it: 0 on success, kNotApplicable otherwise, or an ESC_ERR_* code.
 inline int try_launch(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
                       const float* dk, const float* bias, void* out, unsigned* ctrl, cudaStream_t st, bool dependent,
-                      int* launches, std::string* err, const void* w_point = nullptr) {
+                      int* launches, std::string* err, const void* w_point = nullptr, bool skip_copy = false) {
     if (!applies(C, Ca, H, W, K, dtype, layout, x, out) || sm_count() <= 0) return kNotApplicable;
     if (w_point)
         return bias ? kNotApplicable
-                    : launch<false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, w_point);
-    return launch<false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr);
+                    : launch<false, true>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, w_point, skip_copy);
+    return launch<false>(B, C, Ca, H, W, x, w_large, dk, bias, out, ctrl, st, dependent, launches, err, nullptr, nullptr, skip_copy);
 }
 
 inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, int hidden, const void* x, const void* out) {
@@ -572,11 +572,11 @@ inline bool fused_applies(int B, int C, int Ca, int H, int W, int K, int dtype, 
 // The whole forward (stage 1 inside) as one launch.
 inline int try_launch_fused(int B, int C, int Ca, int H, int W, int K, int dtype, int layout, const void* x, const void* w_large,
                             const toep::Fused& fu, void* out, unsigned* ctrl, cudaStream_t st, int* launches, std::string* err,
-                            const void* w_point = nullptr) {
+                            const void* w_point = nullptr, bool skip_copy = false) {
     if (!fused_applies(B, C, Ca, H, W, K, dtype, layout, fu.hidden, x, out)) return kNotApplicable;
     if (w_point)
-        return launch<true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu, w_point);
-    return launch<true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu);
+        return launch<true, true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu, w_point, skip_copy);
+    return launch<true>(B, C, Ca, H, W, x, w_large, nullptr, nullptr, out, ctrl, st, /*dependent=*/false, launches, err, &fu, nullptr, skip_copy);
 }
 
 }}}  // namespace esc::tma::toepn

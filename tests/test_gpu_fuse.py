@@ -37,6 +37,12 @@ SHAPES = [
     (1, 64, 16, 300, 500, 13, synth.BF16, synth.NHWC, True, "own"),    # many units per CTA: stage 1 as a kernel of its own
     (1, 192, 48, 20, 30, 13, synth.BF16, synth.NHWC, True, "own"),     # C beyond the fast 1x1: guarded kernel in place
     (2, 24, 8, 19, 23, 13, synth.BF16, synth.NCHW, True, "own"),
+    (2, 64, 16, 45, 72, 13, synth.BF16, synth.NCHW, True, "own"),      # NCHW fast path: NCHW tensor-core stencil + NCHW 1x1 kernel
+    (1, 64, 16, 90, 136, 13, synth.BF16, synth.NCHW, True, "x"),       # several tiles of 128 pixels and a ragged last one
+    (1, 48, 16, 33, 48, 13, synth.BF16, synth.NCHW, False, None),
+    (3, 32, 16, 40, 40, 13, synth.BF16, synth.NCHW, True, "own"),
+    (1, 64, 32, 300, 504, 13, synth.BF16, synth.NCHW, True, "own"),    # two channel groups, many units per CTA
+    (1, 64, 16, 1, 8, 13, synth.BF16, synth.NCHW, True, "own"),        # eight pixels
     (2, 20, 12, 15, 17, 9, synth.F32, synth.NCHW, True, "own"),
     (1, 64, 16, 40, 60, 13, synth.F32, synth.NHWC, False, "x"),
 ]
