@@ -36,6 +36,9 @@ SHAPES = [
     (14, 48, 48, 30, 96),     # three channel groups, nothing to copy through
     (8, 64, 32, 280, 400),    # 2,016 units: thirteen or fourteen per CTA, both buffers re-used many times, two launches
     (3, 192, 48, 70, 120),    # the larger model's channel counts: 144 identity channels
+    (1, 64, 16, 540, 960),    # 510 units: three or four per CTA, two launches
+    (100, 32, 16, 64, 64),    # 400 units: three per CTA, every one of another image
+    (3, 64, 32, 200, 400),    # 546 units: image and channel group change inside a CTA's walk of three or four
 ]
 
 
