@@ -275,8 +275,13 @@ esc::CopyJob make_copy_job(const Problem& p, const void* x, void* out, long long
 template <typename T, int LAYOUT>
 int launch_generic_t(const Problem& p, const void* x, const void* w_large, const float* dk, void* out,
                      cudaStream_t st, bool dependent) {
-    const bool regtile = p.K == esc::kRtK;             // the paper's kernel size: eight outputs per thread
-    const int TX = regtile ? esc::kRtTX : esc::kGenTX, TY = regtile ? esc::kRtTY : esc::kGenTY;
+    const bool regtile = p.K == esc::kRtK;             // the paper's kernel size: a patch of outputs per thread
+    // small launches: smaller tiles, more blocks, so that every SM has several
+    auto blocks_of = [&](int tx, int ty) { return (long long)p.B * p.Ca * ((p.W + tx - 1) / tx) * ((p.H + ty - 1) / ty); };
+    const bool small = regtile && blocks_of(esc::kRtTX, esc::kRtTY) < 4LL * sms_or_nominal();
+    const bool tiny = small && blocks_of(esc::RtSmall::TX, esc::RtSmall::TY) < 2LL * sms_or_nominal();
+    const int TX = regtile ? (tiny ? esc::RtTiny::TX : small ? esc::RtSmall::TX : esc::kRtTX) : esc::kGenTX;
+    const int TY = regtile ? (tiny ? esc::RtTiny::TY : small ? esc::RtSmall::TY : esc::kRtTY) : esc::kGenTY;
     const int tiles_x = (p.W + TX - 1) / TX, tiles_y = (p.H + TY - 1) / TY;
     const long long blocks = (long long)p.B * p.Ca * tiles_x * tiles_y;
     const esc::CopyJob job = make_copy_job(p, x, out, blocks, regtile ? esc::kRtThreads : esc::kGenTX * esc::kGenTY);
@@ -290,8 +295,16 @@ int launch_generic_t(const Problem& p, const void* x, const void* w_large, const
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    if (regtile)
-        ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT>, static_cast<const T*>(x),
+    if (regtile && tiny)
+        ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT, esc::RtTiny>, static_cast<const T*>(x),
+                                    static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk,
+                                    tiles_x, tiles_y, job, p.bias));
+    else if (regtile && small)
+        ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT, esc::RtSmall>, static_cast<const T*>(x),
+                                    static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk,
+                                    tiles_x, tiles_y, job, p.bias));
+    else if (regtile)
+        ESC_CUDA(cudaLaunchKernelEx(&cfg, esc::stencil_k13_regtile<T, LAYOUT, esc::RtLarge>, static_cast<const T*>(x),
                                     static_cast<T*>(out), p.C, p.Ca, p.H, p.W, static_cast<const T*>(w_large), static_cast<const T*>(p.w_point), dk,
                                     tiles_x, tiles_y, job, p.bias));
     else

@@ -109,17 +109,31 @@ stencil_generic(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int
 // The loop runs over the 16 input rows a patch touches: a row costs five 16-byte reads and is used by
 // up to four output rows, each with its kernel row (four broadcast 16-byte reads), 104 FMAs apiece.
 // It serves the fp32 and NCHW cases that the TMA kernel does not take.
-constexpr int kRtK = 13, kRtTX = 64, kRtTY = 64, kRtOX = 8, kRtOY = 4;
-constexpr int kRtPitch = kRtTX + kRtK - 1;            // 76 floats, a multiple of 4
-constexpr int kRtRows = kRtTY + kRtK - 1;             // 76
-constexpr int kRtThreads = (kRtTX / kRtOX) * (kRtTY / kRtOY);   // 128
+// Three geometries: 64 x 64 tiles with 4 x 8 patches (most arithmetic per load: large problems), and 64 x 32 tiles with
+// 2 x 8 patches or 32 x 32 tiles with 2 x 4 patches for launches that would otherwise leave most SMs with one block of
+// four warps or none (a 320x180 fp32 map is 240 of the large tiles: its stencil stage takes 25 us with them, 18 us with
+// 480 of the middle ones; a 64x64 map 15 us as 16 large tiles, 6 us as 64 of the smallest).
+constexpr int kRtK = 13;
+template <int TX_, int TY_, int OX_, int OY_>
+struct RtGeom {
+    static constexpr int TX = TX_, TY = TY_, OX = OX_, OY = OY_;
+    static constexpr int Pitch = TX + kRtK - 1;                 // floats per staged row, a multiple of 4
+    static constexpr int Rows = TY + kRtK - 1;
+    static constexpr int Threads = (TX / OX) * (TY / OY);       // 128
+    static_assert(Pitch % 4 == 0 && OX % 4 == 0 && Threads == 128, "geometry");
+};
+using RtLarge = RtGeom<64, 64, 8, 4>;
+using RtSmall = RtGeom<64, 32, 8, 2>;
+using RtTiny = RtGeom<32, 32, 4, 2>;
+constexpr int kRtTX = RtLarge::TX, kRtTY = RtLarge::TY, kRtThreads = 128;
 
-template <typename T, int LAYOUT>
-__global__ void __launch_bounds__(kRtThreads)
+template <typename T, int LAYOUT, class G>
+__global__ void __launch_bounds__(128)
 stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca, int H, int W,
                     const T* __restrict__ w_large, const T* __restrict__ w_point, const float* __restrict__ dk,
                     int tiles_x, int tiles_y, const CopyJob job, const float* __restrict__ bias)
 {
+    constexpr int kRtTX = G::TX, kRtTY = G::TY, kRtOX = G::OX, kRtOY = G::OY, kRtPitch = G::Pitch, kRtRows = G::Rows, kRtThreads = G::Threads;
     __shared__ __align__(16) float tile[kRtRows * kRtPitch];
     __shared__ __align__(16) float wm[kRtK * 16];      // merged kernel, rows padded to 16 taps
     if (job.blocks != 0 && blockIdx.x >= job.first_block) {
@@ -136,9 +150,19 @@ stencil_k13_regtile(const T* __restrict__ x, T* __restrict__ out, int C, int Ca,
     const int tid = threadIdx.x;
     const int y0 = ty * kRtTY - P, x0 = tx * kRtTX - P;
 
-    for (int t = tid; t < kRtRows * kRtPitch; t += kRtThreads) {
-        const int r = t / kRtPitch, q = t % kRtPitch;
-        tile[t] = staged_value<T, LAYOUT>(x, w_point, b, c, y0 + r, x0 + q, C, Ca, H, W);
+    // eight loads of a thread are in flight before the first is stored: the staging is a chain of round trips otherwise
+    for (int t0 = tid; t0 < kRtRows * kRtPitch; t0 += 8 * kRtThreads) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int t = t0 + u * kRtThreads, r = t / kRtPitch, q = t % kRtPitch;
+            v[u] = t < kRtRows * kRtPitch ? staged_value<T, LAYOUT>(x, w_point, b, c, y0 + r, x0 + q, C, Ca, H, W) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int t = t0 + u * kRtThreads;
+            if (t < kRtRows * kRtPitch) tile[t] = v[u];
+        }
     }
     pdl_wait_primary();   // dk comes from the preceding kernel when launched as its dependent
     for (int t = tid; t < kRtK * 16; t += kRtThreads) {
