@@ -120,6 +120,33 @@ def test_host_side_rejections_launch_nothing(L):
     assert L.esc_convattn_device_status(None, None) == 6
 
 
+def test_backward_entries_reject_on_the_host(L):
+    """Both backward entries check shapes, pointers and the workspace before anything could be launched (fake addresses)."""
+    X, GO, GX, Wl, Wa, Wb, Wc, Wd, WS = (0x10000000, 0x18000000, 0x20000000, 0x30000000, 0x30100000, 0x30200000, 0x30300000,
+                                         0x30400000, 0x40000000)
+    L.esc_convattn_backward_workspace_bytes.restype = ctypes.c_size_t
+    need = L.esc_convattn_backward_workspace_bytes(1, 16, 32, 32, 13)
+    assert need > 0 and need % 256 == 0
+    assert L.esc_convattn_backward_workspace_bytes(1, 16, 32, 32, 9) > 0           # odd K up to 13
+    for K in (15, 17, 12, 1):
+        assert L.esc_convattn_backward_workspace_bytes(1, 16, 32, 32, K) == 0
+
+    def bwd(x=X, go=GO, K=13, gx=GX, ws=WS, wsb=None, C=64, Ca=16):
+        return L.esc_convattn_backward(x, go, 1, C, Ca, 32, 32, K, Wl, Wa, Wb, gx, None, None, None, 1, 1, ws, need if wsb is None else wsb, None)
+
+    def bwd_mlp(hidden=8, gx=GX, K=13, wd=Wa, wsb=None):
+        return L.esc_convattn_backward_mlp(X, GO, 1, 64, 16, 32, 32, K, Wl, wd, Wb, Wc, Wd, hidden, gx, None, None, None, None, None, 1, 1,
+                                           WS, need if wsb is None else wsb, None)
+
+    assert bwd(K=15) == 3 and bwd(K=12) == 2                                        # unsupported size; even size
+    assert bwd(x=None) == 1 and bwd(go=None) == 1 and bwd(gx=None) == 1             # null tensors
+    assert bwd(gx=X) == 5                                                           # grad_x over x
+    assert bwd(ws=None) == 6 and bwd(wsb=need - 256) == 6 and bwd(ws=WS + 8) == 6   # workspace missing, short, misaligned
+    assert bwd(Ca=80) == 2                                                          # C_a > C
+    assert bwd_mlp(hidden=0) == 2 and bwd_mlp(hidden=-3) == 2 and bwd_mlp(hidden=129) == 2
+    assert bwd_mlp(wd=None) == 1 and bwd_mlp(gx=X) == 5 and bwd_mlp(K=15) == 3 and bwd_mlp(wsb=0) == 6
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     from paper_2503_06671_b200 import binding
 
