@@ -13,6 +13,7 @@ from .convattn_oracle import (  # noqa: F401
     stencil,
     backward,
     backward_mlp,
+    backward_pw,
     stencil_dense,
     forward_dense,
     pointwise,

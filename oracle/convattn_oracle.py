@@ -247,6 +247,30 @@ def backward_mlp(x, grad_out, C_a, w_large, w_down, b_down, w_up, b_up):
     return gx, glk, gwd, gbd, gwu, gbu
 
 
+def backward_pw(x, grad_out, C_a, w_large, w_point, w_dyn, b_dyn):
+    """Gradients of forward_pw(x, ...) contracted with grad_out: returns (gx [B,C,H,W], g_w_large [C_a,K,K],
+    g_w_point [C_a,C_a], g_w_dyn [9*C_a,C_a], g_b_dyn [9*C_a])."""
+    x, xp = _f32(x)
+    go, gp = _f32(grad_out)
+    assert go.shape == x.shape
+    w_large, wp = _f64(w_large)
+    K = int(w_large.shape[-1])
+    assert K >= 3
+    B, C, H, W = _dims(x, C_a, K)
+    w_point, wpp = _f64(w_point)
+    assert w_point.shape == (C_a, C_a)
+    w_dyn, wdp = _f64(w_dyn)
+    b_dyn, bdp = _f64(b_dyn)
+    gx = np.empty((B, C, H, W), dtype=np.float64)
+    glk = np.empty((C_a, K, K), dtype=np.float64)
+    gwp = np.empty((C_a, C_a), dtype=np.float64)
+    gw = np.empty((9 * C_a, C_a), dtype=np.float64)
+    gb = np.empty((9 * C_a,), dtype=np.float64)
+    _load().convattn_ref_backward_pw(xp, gp, B, C, C_a, H, W, K, wp, wpp, wdp, bdp, *(a.ctypes.data_as(_f64p)
+                                     for a in (gx, glk, gwp, gw, gb)))
+    return gx, glk, gwp, gw, gb
+
+
 def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
     """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
     x, xp = _f32(x)

@@ -34,6 +34,7 @@
  * convattn_ref_backward is the gradient of the first form above with respect to x, LK, W_dyn and
  * b_dyn, by the chain rule written out; convattn_ref_backward_mlp the same with the two-layer estimator
  * (gradients with respect to x, LK, W_down, b_down, W_up, b_up).
+ * convattn_ref_backward_pw is the gradient of the decomposed form (x, LK^s, LK^c, W_dyn, b_dyn).
  *
  * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
  * Everything is accumulated in double precision with direct nested loops in
@@ -60,7 +61,9 @@
  * function, which is quadratic in x and bilinear in weights and x) and the
  * adjoint identity; the backward pass with the two-layer estimator by central differences of
  * the pinned forward and by its linear limit, where it must equal the pinned one-layer backward
- * with composed weights.
+ * with composed weights; the backward pass of the decomposed form by central differences of the pinned
+ * decomposed forward (also exact), by the identity mix, where it must equal the pinned depth-wise backward,
+ * and by the adjoint identity of its linear part.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -591,6 +594,137 @@ void convattn_ref_backward_mlp(const float *x, const float *go, int B, int C, in
                     }
     }
     free(g); free(t); free(a); free(dk); free(gtap); free(gdk); free(gt); free(gg);
+}
+
+/* Backward pass of the decomposed form of Eq. 5 (point-wise LK^c in front of the depth-wise stage, one-layer
+ * estimator), by the chain rule written out.  With m[b,n] = sum_k w_point[n,k] * x[b,k] (the mixed features, exact),
+ * g = GAP(x) of the UNMIXED features, dk = W g + b, Wm[b,n] = LK[n] + ZP(dk[b,n]) and m~, go~ zero-padded:
+ *   g_tap[b,n,i,j] = sum_{y,x} go[b,n,y,x] * m~[b,n,y+i-P,x+j-P]
+ *   g_lk[n,i,j]    = sum_b g_tap[b,n,i,j]         g_dk[b,n,i,j] = g_tap[b,n,i+P-1,j+P-1]
+ *   g_b[o]         = sum_b g_dk[b,o]              g_W[o,k]      = sum_b g_dk[b,o] * g[b,k]
+ *   g_g[b,k]       = sum_o W[o,k] * g_dk[b,o]
+ *   g_m[b,n,y,x]   = sum_{i,j} Wm[b,n,i,j] * go~[b,n,y-(i-P),x-(j-P)]         (dL/dm)
+ *   g_P[n,k]       = sum_{b,y,x} g_m[b,n,y,x] * x[b,k,y,x]                    (dL/dLK^c)
+ *   g_x[b,k,y,x]   = sum_n w_point[n,k] * g_m[b,n,y,x] + g_g[b,k] / (H*W)     k < C_a
+ *   g_x[b,c]       = go[b,c]                                                  c >= C_a
+ * Outputs: gx [B,C,H,W], glk [C_a,K,K], gwp [C_a,C_a], gw [9*C_a,C_a], gb [9*C_a]; any may be NULL.  K >= 3. */
+void convattn_ref_backward_pw(const float *x, const float *go, int B, int C, int C_a, int H, int W, int K,
+                              const double *w_large, const double *w_point, const double *w_dyn, const double *b_dyn,
+                              double *gx, double *glk, double *gwp, double *gw, double *gb)
+{
+    const int P = (K - 1) / 2;
+    const size_t HW = (size_t)H * W;
+    double *g = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    double *dk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    double *m = (double *)malloc(sizeof(double) * (size_t)B * C_a * HW);
+    double *gm = (double *)malloc(sizeof(double) * (size_t)B * C_a * HW);
+    double *gtap = (double *)malloc(sizeof(double) * (size_t)B * C_a * K * K);
+    double *gdk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    double *gg = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    convattn_ref_gap(x, B, C, C_a, H, W, g);
+    convattn_ref_dynkernel(g, B, C_a, w_dyn, b_dyn, dk);
+    /* the mixed features */
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < C_a; ++n)
+            for (size_t q = 0; q < HW; ++q) {
+                double s = 0.0;
+                for (int k = 0; k < C_a; ++k)
+                    s += w_point[(size_t)n * C_a + k] * (double)x[((size_t)b * C + k) * HW + q];
+                m[((size_t)b * C_a + n) * HW + q] = s;
+            }
+    /* tap gradients against the mixed features */
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < C_a; ++n)
+            for (int i = 0; i < K; ++i)
+                for (int j = 0; j < K; ++j) {
+                    double s = 0.0;
+                    for (int y = 0; y < H; ++y)
+                        for (int xx = 0; xx < W; ++xx) {
+                            int yy = y + i - P, xc = xx + j - P;
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                s += (double)go[IDX4(b, n, y, xx, C, H, W)] * m[((size_t)b * C_a + n) * HW + (size_t)yy * W + xc];
+                        }
+                    gtap[(((size_t)b * C_a + n) * K + i) * K + j] = s;
+                }
+    if (glk)
+        for (int n = 0; n < C_a; ++n)
+            for (int t = 0; t < K * K; ++t) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gtap[((size_t)b * C_a + n) * K * K + t];
+                glk[(size_t)n * K * K + t] = s;
+            }
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < C_a; ++n)
+            for (int i = 0; i < 3; ++i)
+                for (int j = 0; j < 3; ++j)
+                    gdk[((size_t)b * C_a + n) * 9 + i * 3 + j] = gtap[(((size_t)b * C_a + n) * K + i + P - 1) * K + j + P - 1];
+    if (gb)
+        for (int o = 0; o < 9 * C_a; ++o) {
+            double s = 0.0;
+            for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o];
+            gb[o] = s;
+        }
+    if (gw)
+        for (int o = 0; o < 9 * C_a; ++o)
+            for (int k = 0; k < C_a; ++k) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o] * g[(size_t)b * C_a + k];
+                gw[(size_t)o * C_a + k] = s;
+            }
+    for (int b = 0; b < B; ++b)
+        for (int k = 0; k < C_a; ++k) {
+            double s = 0.0;
+            for (int o = 0; o < 9 * C_a; ++o) s += w_dyn[(size_t)o * C_a + k] * gdk[(size_t)b * 9 * C_a + o];
+            gg[(size_t)b * C_a + k] = s;
+        }
+    /* dL/dm: the depth-wise stage's adjoint */
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int b = 0; b < B; ++b)
+        for (int n = 0; n < C_a; ++n)
+            for (int y = 0; y < H; ++y)
+                for (int xx = 0; xx < W; ++xx) {
+                    double s = 0.0;
+                    for (int i = 0; i < K; ++i)
+                        for (int j = 0; j < K; ++j) {
+                            int yy = y - (i - P), xc = xx - (j - P);
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                s += w_large[((size_t)n * K + i) * K + j] * (double)go[IDX4(b, n, yy, xc, C, H, W)];
+                        }
+                    for (int i = 0; i < 3; ++i)
+                        for (int j = 0; j < 3; ++j) {
+                            int yy = y - (i - 1), xc = xx - (j - 1);
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                s += dk[((size_t)b * C_a + n) * 9 + i * 3 + j] * (double)go[IDX4(b, n, yy, xc, C, H, W)];
+                        }
+                    gm[((size_t)b * C_a + n) * HW + (size_t)y * W + xx] = s;
+                }
+    if (gwp)
+        for (int n = 0; n < C_a; ++n)
+            for (int k = 0; k < C_a; ++k) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b)
+                    for (size_t q = 0; q < HW; ++q)
+                        s += gm[((size_t)b * C_a + n) * HW + q] * (double)x[((size_t)b * C + k) * HW + q];
+                gwp[(size_t)n * C_a + k] = s;
+            }
+    if (gx) {
+#pragma omp parallel for collapse(2) schedule(static)
+        for (int b = 0; b < B; ++b)
+            for (int c = 0; c < C; ++c)
+                for (size_t q = 0; q < HW; ++q) {
+                    if (c >= C_a) {
+                        gx[((size_t)b * C + c) * HW + q] = (double)go[((size_t)b * C + c) * HW + q];
+                        continue;
+                    }
+                    double s = 0.0;
+                    for (int n = 0; n < C_a; ++n)
+                        s += w_point[(size_t)n * C_a + c] * gm[((size_t)b * C_a + n) * HW + q];
+                    gx[((size_t)b * C + c) * HW + q] = s + gg[(size_t)b * C_a + c] / ((double)H * (double)W);
+                }
+    }
+    free(g); free(dk); free(m); free(gm); free(gtap); free(gdk); free(gg);
 }
 
 /* Selected outputs, one by one: idx[n] are flat indices into out[B,C,H,W]; dk is
