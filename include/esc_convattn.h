@@ -303,6 +303,24 @@ int esc_convattn_backward_mlp(const void* x, const void* grad_out, int B, int C,
                               float* grad_w_up, float* grad_b_up, int dtype, int layout,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Backward pass of esc_convattn_forward_pw, the decomposed form of Eq. 5: the point-wise filter LK^c (w_point [C_a,C_a],
+ * row = output channel, element type of x) in front of the depth-wise stage, one-layer estimator fed by the GAP of the
+ * unmixed features.  With m = LK^c x_att and g_m = dL/dm (grad_out through the rotated depth-wise kernels):
+ *   grad_w_point [C_a,C_a]  fp32   dL/dLK^c[n,k] = sum over images and pixels of g_m[n] x[k]   (may be NULL)
+ *   grad_x attention channels = LK^c transposed applied to g_m, plus the estimator's path; identity channels = grad_out
+ *   grad_w_large, grad_w_dyn, grad_b_dyn as in esc_convattn_backward, with m in the place of x_att (grad_w_dyn still
+ *   multiplies the mean of the unmixed features).
+ * m and g_m are kept in the element type of x (one rounding each for bf16), in grad_x's attention channels, so grad_x
+ * is also scratch while the call runs.  C_a must be 4, 8, 16 or 32 (ESC_ERR_UNSUPPORTED otherwise).  Same workspace,
+ * restrictions and error codes as esc_convattn_backward.  All device memory; asynchronous on `stream`.
+ */
+int esc_convattn_backward_pw(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                             const void* w_large, const void* w_point, const void* w_dyn, const void* b_dyn,
+                             void* grad_x, float* grad_w_large, float* grad_w_point, float* grad_w_dyn,
+                             float* grad_b_dyn, int dtype, int layout,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

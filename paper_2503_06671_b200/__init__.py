@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     ESC_LK_DEPTHWISE, ESC_LK_DECOMPOSED, ESC_LK_DENSE,
     esc_convattn_backward,
     esc_convattn_backward_mlp,
+    esc_convattn_backward_pw,
     esc_convattn_backward_workspace_bytes,
     new_backward_workspace,
     esc_convattn_forward_mlp,

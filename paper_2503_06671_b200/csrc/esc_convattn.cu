@@ -24,6 +24,7 @@
 #include "stencil_dense.cuh"
 #include "stencil_dense_umma.cuh"
 #include "backward.cuh"
+#include "backward_pw.cuh"
 #include "conv_fuse.cuh"
 
 namespace {
@@ -86,7 +87,8 @@ int check_tensors(const Problem& p, const void* x, const void* out) {
 
 // ---- workspace layout -------------------------------------------------------------------
 //   [ctrl words: header + B arrival counters + B launch flags][pad to 256][dk: B*Ca*9 floats][pad]
-//   [partials: B*S*Ca floats][pad][per-unit sums of the fused stage 1: 2 * SMs * 16 floats]
+//   [partials: B*S*Ca floats][pad][per-unit sums of the one-launch form: kMaxFusedUnits * SMs * 16 floats][pad]
+//   [large kernel padded to 13 x 13]
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Workspace {
@@ -517,6 +519,9 @@ struct BackwardWs {
     float *act, *gt;                 // two-layer estimator: activations and g_t, [B][kMaxHidden] each
     void* lk_pad;                    // the rotated large kernel zero-padded to 13 x 13 for the tensor-core kernels
     void* w_flip;
+    float *xs_part, *gp_part;        // decomposed form: per-chunk sums of x_att [B][chunks][Ca] and of g_P [B * chunks][Ca * Ca]
+    int chunks;                      // chunks of pixels per image in those
+    bool patch_xsum;                 // the tap-gradient kernels ran on the mixed features: take the sums of x_att from xs_part
     size_t bytes;
 };
 BackwardWs carve_backward(void* ws, const Problem& p) {
@@ -535,6 +540,11 @@ BackwardWs carve_backward(void* ws, const Problem& p) {
     w.act = reinterpret_cast<float*>(base + off);   off += round_up((size_t)p.B * esc::kMaxHidden * 4, 256);
     w.gt = reinterpret_cast<float*>(base + off);    off += round_up((size_t)p.B * esc::kMaxHidden * 4, 256);
     w.lk_pad = base + off;                          off += round_up((size_t)p.Ca * esc::bwd::TAPS * 4, 256);
+    w.chunks = esc::bwd::pw::chunks_of((long long)p.H * p.W);
+    w.patch_xsum = false;
+    w.xs_part = reinterpret_cast<float*>(base + off); off += round_up((size_t)p.B * w.chunks * p.Ca * 4, 256);
+    w.gp_part = reinterpret_cast<float*>(base + off);
+    if (esc::bwd::pw::supported(p.Ca)) off += round_up((size_t)p.B * w.chunks * p.Ca * p.Ca * 4, 256);
     w.bytes = off;
     return w;
 }
@@ -590,6 +600,13 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
     if (tiles_done == 0) ++g_last_launches;
     esc::bwd::sum_tiles<<<(unsigned)(p.B * p.Ca), esc::bwd::kSumThreads, 0, st>>>(w.part, tiles_done > 0 ? tiles_done : tiles_x * tiles_y, w.gtap);
     ESC_CUDA(cudaGetLastError());
+    if (w.patch_xsum) {
+        // decomposed form: the sums the tap-gradient kernels took are those of the mixed features; g_W wants the unmixed ones
+        const int warps = p.B * p.Ca;
+        esc::bwd::pw::sum_x<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(w.xs_part, warps, p.Ca, w.chunks, w.gtap);
+        ESC_CUDA(cudaGetLastError());
+        ++g_last_launches;
+    }
     if (est.hidden == 0) {
         esc::bwd::finish<T><<<esc::bwd::kFinishBlocks, 256, 0, st>>>(w.gtap, p.B, p.Ca, p.H, p.W, p.K, static_cast<const T*>(w_large),
                                                 static_cast<const T*>(est.w_last), static_cast<const T*>(est.b_last), g.g_lk,
@@ -611,6 +628,67 @@ int backward_t(const Problem& p, const void* x, const void* go, const void* w_la
     ESC_CUDA(cudaGetLastError());
     g_last_launches += 3;
     return ESC_OK;
+}
+
+// Decomposed form: the two per-pixel kernels around the depth-wise backward pass.
+bool pw_vec(const Problem& p) { return p.layout == ESC_NHWC && ((size_t)p.C * p.es()) % 16 == 0 && ((size_t)p.Ca * p.es()) % 16 == 0; }
+
+template <typename T, int LAYOUT, int CA>
+int pw_mix_ca(const Problem& p, const void* x, const void* w_point, void* m, const BackwardWs& w, cudaStream_t st) {
+    const unsigned blocks = (unsigned)((long long)p.B * w.chunks);
+    esc::bwd::pw::mix<T, LAYOUT, CA><<<blocks, esc::bwd::pw::kThreads, 0, st>>>(
+        static_cast<const T*>(x), static_cast<const T*>(w_point), static_cast<T*>(m), p.C, (long long)p.H * p.W, w.chunks,
+        pw_vec(p) ? 1 : 0, w.xs_part);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
+}
+template <typename T, int LAYOUT>
+int pw_mix_t(const Problem& p, const void* x, const void* w_point, void* m, const BackwardWs& w, cudaStream_t st) {
+    switch (p.Ca) {
+        case 4: return pw_mix_ca<T, LAYOUT, 4>(p, x, w_point, m, w, st);
+        case 8: return pw_mix_ca<T, LAYOUT, 8>(p, x, w_point, m, w, st);
+        case 16: return pw_mix_ca<T, LAYOUT, 16>(p, x, w_point, m, w, st);
+        case 32: return pw_mix_ca<T, LAYOUT, 32>(p, x, w_point, m, w, st);
+    }
+    return ESC_ERR_UNSUPPORTED;
+}
+
+template <typename T, int LAYOUT, int CA>
+int pw_back_ca(const Problem& p, const void* x, const void* w_point, void* gx, const BackwardWs& w, float* g_wp, cudaStream_t st) {
+    constexpr size_t smem = esc::bwd::pw::back_smem_bytes<CA>();
+    if (smem > 48 * 1024) {
+        static bool attr_set[esc::tma::kMaxDevices] = {};
+        const int dev = esc::tma::current_device();
+        if (dev < 0) return ESC_ERR_UNSUPPORTED;
+        if (!attr_set[dev]) {
+            ESC_CUDA(cudaFuncSetAttribute(esc::bwd::pw::back<T, LAYOUT, CA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            attr_set[dev] = true;
+        }
+    }
+    const unsigned blocks = (unsigned)((long long)p.B * w.chunks);
+    esc::bwd::pw::back<T, LAYOUT, CA><<<blocks, esc::bwd::pw::kThreads, smem, st>>>(
+        static_cast<const T*>(x), static_cast<const T*>(w_point), static_cast<T*>(gx), w.bias, p.C, (long long)p.H * p.W,
+        w.chunks, pw_vec(p) ? 1 : 0, w.gp_part);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    if (g_wp) {
+        const int elems = CA * CA;
+        esc::bwd::pw::sum_gp<<<(unsigned)((elems + 7) / 8), 256, 0, st>>>(w.gp_part, elems, (int)blocks, g_wp);
+        ESC_CUDA(cudaGetLastError());
+        ++g_last_launches;
+    }
+    return ESC_OK;
+}
+template <typename T, int LAYOUT>
+int pw_back_t(const Problem& p, const void* x, const void* w_point, void* gx, const BackwardWs& w, float* g_wp, cudaStream_t st) {
+    switch (p.Ca) {
+        case 4: return pw_back_ca<T, LAYOUT, 4>(p, x, w_point, gx, w, g_wp, st);
+        case 8: return pw_back_ca<T, LAYOUT, 8>(p, x, w_point, gx, w, g_wp, st);
+        case 16: return pw_back_ca<T, LAYOUT, 16>(p, x, w_point, gx, w, g_wp, st);
+        case 32: return pw_back_ca<T, LAYOUT, 32>(p, x, w_point, gx, w, g_wp, st);
+    }
+    return ESC_ERR_UNSUPPORTED;
 }
 
 // ---- fixed scratch for the entry point that must not allocate ------------------------------
@@ -1036,7 +1114,7 @@ size_t esc_convattn_backward_workspace_bytes(int B, int C_a, int H, int W, int K
 namespace {
 int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K, const void* w_large,
                    const Estimator& est, void* grad_x, const BackwardGrads& g, int dtype, int layout, void* workspace,
-                   size_t workspace_bytes_, void* stream) {
+                   size_t workspace_bytes_, void* stream, const void* w_point = nullptr, float* g_wp = nullptr) {
     g_last_launches = 0;
     Problem p{B, C, C_a, H, W, K, dtype, layout};
     int rc = check_shape(p);
@@ -1055,23 +1133,46 @@ int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, i
         if (xa < oa + bytes && oa < xa + bytes) return ESC_ERR_ALIAS;
     }
     if (!aligned(w_large, p.es())) return ESC_ERR_ALIGN;
-    for (const float* q : {g.g_lk, g.g_w_last, g.g_b_last, g.g_w_down, g.g_b_down})
+    for (const float* q : {g.g_lk, g.g_w_last, g.g_b_last, g.g_w_down, g.g_b_down, g_wp})
         if (q && !aligned(q, 4)) return ESC_ERR_ALIGN;
+    if (w_point) {
+        if (!aligned(w_point, p.es())) return ESC_ERR_ALIGN;
+        if (!esc::bwd::pw::supported(C_a) || est.hidden != 0) return ESC_ERR_UNSUPPORTED;
+        if ((long long)B * esc::bwd::pw::chunks_of((long long)H * W) > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
+    }
     if (!workspace || !aligned(workspace, 256)) return ESC_ERR_WORKSPACE;
-    const BackwardWs w = carve_backward(workspace, p);
+    BackwardWs w = carve_backward(workspace, p);
     if (workspace_bytes_ < w.bytes) return ESC_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (w_point) {
+        // decomposed form (Eq. 5): the mixed features go into grad_x's attention channels, where the tap-gradient kernels
+        // read them; grad_x is rewritten by the stencil pass and the last kernel below
+        rc = dtype == ESC_F32 ? (layout == ESC_NCHW ? pw_mix_t<float, esc::kNCHW>(p, x, w_point, grad_x, w, st)
+                                                    : pw_mix_t<float, esc::kNHWC>(p, x, w_point, grad_x, w, st))
+                              : (layout == ESC_NCHW ? pw_mix_t<__nv_bfloat16, esc::kNCHW>(p, x, w_point, grad_x, w, st)
+                                                    : pw_mix_t<__nv_bfloat16, esc::kNHWC>(p, x, w_point, grad_x, w, st));
+        if (rc != ESC_OK) return rc;
+        w.patch_xsum = true;
+    }
+    const void* x_taps = w_point ? grad_x : x;             // what the depth-wise stage saw
     if (dtype == ESC_F32)
-        rc = layout == ESC_NCHW ? backward_t<float, esc::kNCHW>(p, x, grad_out, w_large, est, w, g, st)
-                                : backward_t<float, esc::kNHWC>(p, x, grad_out, w_large, est, w, g, st);
+        rc = layout == ESC_NCHW ? backward_t<float, esc::kNCHW>(p, x_taps, grad_out, w_large, est, w, g, st)
+                                : backward_t<float, esc::kNHWC>(p, x_taps, grad_out, w_large, est, w, g, st);
     else
-        rc = layout == ESC_NCHW ? backward_t<__nv_bfloat16, esc::kNCHW>(p, x, grad_out, w_large, est, w, g, st)
-                                : backward_t<__nv_bfloat16, esc::kNHWC>(p, x, grad_out, w_large, est, w, g, st);
+        rc = layout == ESC_NCHW ? backward_t<__nv_bfloat16, esc::kNCHW>(p, x_taps, grad_out, w_large, est, w, g, st)
+                                : backward_t<__nv_bfloat16, esc::kNHWC>(p, x_taps, grad_out, w_large, est, w, g, st);
     if (rc != ESC_OK) return rc;
-    // grad_x: the forward stencil on grad_out with both kernels rotated by 180 degrees, plus the constants
-    p.bias = w.bias;
+    // grad_x: the forward stencil on grad_out with both kernels rotated by 180 degrees, plus the constants (in the
+    // decomposed form the constants belong behind the transposed mix: the last kernel adds them)
+    p.bias = w_point ? nullptr : w.bias;
     const TensorLk tl = tensor_lk(p, grad_out, grad_x, w.w_flip, w.lk_pad, st);
-    return launch_stencil(p, grad_out, w.w_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false, &tl);
+    rc = launch_stencil(p, grad_out, w.w_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false, &tl);
+    if (rc != ESC_OK || !w_point) return rc;
+    rc = dtype == ESC_F32 ? (layout == ESC_NCHW ? pw_back_t<float, esc::kNCHW>(p, x, w_point, grad_x, w, g_wp, st)
+                                                : pw_back_t<float, esc::kNHWC>(p, x, w_point, grad_x, w, g_wp, st))
+                          : (layout == ESC_NCHW ? pw_back_t<__nv_bfloat16, esc::kNCHW>(p, x, w_point, grad_x, w, g_wp, st)
+                                                : pw_back_t<__nv_bfloat16, esc::kNHWC>(p, x, w_point, grad_x, w, g_wp, st));
+    return rc;
 }
 }  // namespace
 
@@ -1093,6 +1194,17 @@ int esc_convattn_backward_mlp(const void* x, const void* grad_out, int B, int C,
     const Estimator est{w_up, b_up, w_down, b_down, hidden};
     const BackwardGrads g{grad_w_large, grad_w_up, grad_b_up, grad_w_down, grad_b_down};
     return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_large, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream);
+}
+
+int esc_convattn_backward_pw(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                             const void* w_large, const void* w_point, const void* w_dyn, const void* b_dyn, void* grad_x,
+                             float* grad_w_large, float* grad_w_point, float* grad_w_dyn, float* grad_b_dyn, int dtype,
+                             int layout, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!w_point) return ESC_ERR_NULL;
+    const Estimator est{w_dyn, b_dyn, nullptr, nullptr, 0};
+    const BackwardGrads g{grad_w_large, grad_w_dyn, grad_b_dyn, nullptr, nullptr};
+    return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_large, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream,
+                          w_point, grad_w_point);
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {
