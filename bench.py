@@ -588,6 +588,13 @@ def main():
             extras["backward"] = {"ms_per_step": st["median_ms"], "launches": pkg.esc_convattn_last_launches(),
                                   "frac_of_fp32_roofline": t_fma / (st["median_ms"] * 1e-3),
                                   "note": "roofline: 2 x K x K multiply-adds per attention pixel-channel on the FP32 pipe"}
+            if wl.C_a in (4, 8, 16, 32):
+                # the same for the decomposed form of Eq. 5 (also the gradient of LK^c): two per-pixel kernels around it
+                g_wp = torch.zeros(wl.C_a, wl.C_a, device="cuda")
+                st, _ = timer.measure(lambda i: pkg.esc_convattn_backward_pw(xs[i % n_rot], go_d, wl.C_a, wl.K, wl_d, wp_d, wd_d, bd_d, gx_d, g_lk,
+                                                                             g_wp, g_w, g_b, lay_code, bws), samples=5)
+                extras["backward"]["decomposed_large_kernel_ms_per_step"] = st["median_ms"]
+                extras["backward"]["decomposed_large_kernel_launches"] = pkg.esc_convattn_last_launches()
         except Exception as exc:
             extras["backward"] = {"error": f"{type(exc).__name__}: {exc}"}
         # with the dense large kernel of the main model (Section 3.2): an implicit GEMM on the tensor cores

@@ -20,13 +20,12 @@
 namespace esc { namespace bwd { namespace pw {
 
 constexpr int kThreads = 256;                 // one pixel per thread and pass
-constexpr int kPasses = 4;
+constexpr int kPasses = 2;
 constexpr int kChunk = kThreads * kPasses;    // pixels of one image per block
 constexpr int kPitch = kThreads + 4;          // floats per staged channel row (16-byte rows, banks shifted by four)
 
 inline int chunks_of(long long HW) { return (int)((HW + kChunk - 1) / kChunk); }
 inline bool supported(int Ca) { return Ca == 4 || Ca == 8 || Ca == 16 || Ca == 32; }
-template <int CA> constexpr size_t back_smem_bytes() { return (size_t)(CA * CA + CA + 2 * CA * kPitch) * sizeof(float); }
 
 template <typename T> __device__ __forceinline__ uint4 pack16(const float* f);
 template <> __device__ __forceinline__ uint4 pack16<float>(const float* f) {
@@ -59,21 +58,22 @@ __device__ __forceinline__ void load_px(const T* __restrict__ t, size_t b, int C
         for (int k = 0; k < CA; ++k) v[k] = Elem<T>::to_f32(t[(b * C + k) * HW + q]);
     }
 }
-template <typename T, int LAYOUT, int CA>
-__device__ __forceinline__ void store_px(T* __restrict__ t, size_t b, int C, size_t HW, size_t q, bool vec, const float (&v)[CA]) {
+// Channels k0 .. k0+G-1 of one pixel (G = 8, or 4 where C_a = 4; k0 a multiple of G).
+template <typename T, int LAYOUT, int G>
+__device__ __forceinline__ void store_group(T* __restrict__ t, size_t b, int C, size_t HW, size_t q, bool vec, int k0, const float (&v)[G]) {
     constexpr int V = Elem<T>::kVec;
     if (LAYOUT == kNHWC) {
-        T* p = t + (b * HW + q) * C;
-        if (CA % V == 0 && vec) {
+        T* p = t + (b * HW + q) * C + k0;
+        if (G % V == 0 && vec) {
 #pragma unroll
-            for (int k = 0; k < CA / V * V; k += V) *reinterpret_cast<uint4*>(p + k) = pack16<T>(&v[k]);
+            for (int k = 0; k < G / V * V; k += V) *reinterpret_cast<uint4*>(p + k) = pack16<T>(&v[k]);
         } else {
 #pragma unroll
-            for (int k = 0; k < CA; ++k) p[k] = Elem<T>::from_f32(v[k]);
+            for (int k = 0; k < G; ++k) p[k] = Elem<T>::from_f32(v[k]);
         }
     } else {
 #pragma unroll
-        for (int k = 0; k < CA; ++k) t[(b * C + k) * HW + q] = Elem<T>::from_f32(v[k]);
+        for (int k = 0; k < G; ++k) t[(b * C + k0 + k) * HW + q] = Elem<T>::from_f32(v[k]);
     }
 }
 
@@ -81,7 +81,7 @@ __device__ __forceinline__ void store_px(T* __restrict__ t, size_t b, int C, siz
 // Block = (image, chunk of kChunk pixels).  P sits in shared memory (read as broadcast 16-byte rows), a pixel's
 // channels in registers.
 template <typename T, int LAYOUT, int CA>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, CA <= 16 ? 4 : 2)
 mix(const T* __restrict__ x, const T* __restrict__ w_point, T* __restrict__ m, int C, long long HW_, int chunks, int vec_,
     float* __restrict__ xs_part)              // [B][chunks][CA]
 {
@@ -99,18 +99,24 @@ mix(const T* __restrict__ x, const T* __restrict__ w_point, T* __restrict__ m, i
     for (int pass = 0; pass < kPasses; ++pass) {
         const size_t q = (size_t)ch * kChunk + (size_t)pass * kThreads + tid;
         if (q >= HW) break;
-        float v[CA], o[CA];
+        float v[CA];
         load_px<T, LAYOUT, CA>(x, b, C, HW, q, vec, v);
 #pragma unroll
         for (int k = 0; k < CA; ++k) sx[k] += v[k];
+        // a group of outputs at a time, stored at once: a rolled loop, so that P is not read ahead into a hundred registers
+        constexpr int G = CA >= 8 ? 8 : 4;
+#pragma unroll 1
+        for (int n0 = 0; n0 < CA; n0 += G) {
+            float o[G];
 #pragma unroll
-        for (int n = 0; n < CA; ++n) {
-            float s = 0.f;
+            for (int j = 0; j < G; ++j) {
+                float s = 0.f;
 #pragma unroll
-            for (int k = 0; k < CA; ++k) s = fmaf(ps[n * CA + k], v[k], s);
-            o[n] = s;
+                for (int k = 0; k < CA; ++k) s = fmaf(ps[(n0 + j) * CA + k], v[k], s);
+                o[j] = s;
+            }
+            store_group<T, LAYOUT, G>(m, b, C, HW, q, vec, n0, o);
         }
-        store_px<T, LAYOUT, CA>(m, b, C, HW, q, vec, o);
     }
 #pragma unroll
     for (int k = 0; k < CA; ++k) {
@@ -144,75 +150,127 @@ sum_x(const float* __restrict__ xs_part, int BCa, int Ca, int chunks, float* __r
 
 // ---- g_x = P^T g_m + constant, in place; per-chunk partial sums of g_P ---------------------------------------------
 // Block = (image, chunk).  Per pass a thread turns its pixel's g_m into g_x (P's rows broadcast from shared memory) and
-// stages g_m and x_att of the pass channel-major; then thread (n, k) adds the pass's 256 products g_m[n] x[k].
-// Dynamic shared memory: P [CA][CA] | constants [CA] | g_m [CA][kPitch] | x [CA][kPitch].
+// stages g_m and x_att of the pass channel-major.  The outer products g_m[n] x[k] are then register-tiled: the CA x CA
+// pairs are cut into 4x4 tiles, the pass's 256 pixels into `kSlices` interleaved slices, thread (tile, slice) reads
+// four pixels of its four g_m rows and four x rows at a time (eight 16-byte reads per 64 FMAs; lanes of a slice group
+// read adjacent 16-byte words).  At the end the slices' sums are added per pair in slice order.
+// Dynamic shared memory: P [CA][CA] | constants [CA] | g_m [CA][kPitch] | x [CA][kPitch]  (re-used for the slices' sums).
+template <int CA> struct BackGeom {
+    static constexpr int kTiles = CA * CA / 16;                 // 4x4 tiles of (n, k) pairs
+    static constexpr int kSlices = kThreads / kTiles;           // pixel slices per pass
+    static constexpr int kPx = kThreads / kSlices;              // pixels per slice and pass
+    static constexpr int kStage = 2 * CA * kPitch > kSlices * CA * CA ? 2 * CA * kPitch : kSlices * CA * CA;
+    static_assert(CA % 4 == 0 && kTiles >= 1 && kTiles <= kThreads && kThreads % kTiles == 0, "tiling");
+};
+template <int CA> constexpr size_t back_smem_bytes() { return (size_t)(CA * CA + CA + BackGeom<CA>::kStage) * sizeof(float); }
+
 template <typename T, int LAYOUT, int CA>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, CA <= 16 ? 3 : 2)
 back(const T* __restrict__ x, const T* __restrict__ w_point, T* __restrict__ gx, const float* __restrict__ bias, int C,
      long long HW_, int chunks, int vec_, float* __restrict__ gp_part)          // [B * chunks][CA * CA]
 {
+    using G = BackGeom<CA>;
     extern __shared__ __align__(16) float sm[];
     float* ps = sm;
     float* bs = ps + CA * CA;
     float* gs = bs + CA;
     float* xs = gs + CA * kPitch;
-    constexpr int NP = (CA * CA + kThreads - 1) / kThreads;     // (n, k) pairs per thread
     const int tid = threadIdx.x;
     const size_t HW = (size_t)HW_, b = blockIdx.x / chunks;
     const int ch = blockIdx.x % chunks;
     const bool vec = vec_ != 0;
+    const int tile = tid / G::kSlices, slice = tid % G::kSlices;
+    const int n0 = (tile / (CA / 4)) * 4, k0 = (tile % (CA / 4)) * 4;
     for (int e = tid; e < CA * CA; e += kThreads) ps[e] = Elem<T>::to_f32(w_point[e]);
     if (tid < CA) bs[tid] = bias[b * CA + tid];
-    float acc[NP];
+    float acc[4][4];
 #pragma unroll
-    for (int e = 0; e < NP; ++e) acc[e] = 0.f;
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
     for (int pass = 0; pass < kPasses; ++pass) {
         const size_t q0 = (size_t)ch * kChunk + (size_t)pass * kThreads;
         if (q0 >= HW) break;
         const size_t q = q0 + tid;
         __syncthreads();                                         // P and the constants are there; the last pass's staged rows are read
-        float gm[CA], xv[CA];
-        if (q < HW) {
-            load_px<T, LAYOUT, CA>(gx, b, C, HW, q, vec, gm);
-            load_px<T, LAYOUT, CA>(x, b, C, HW, q, vec, xv);
-            float o[CA];
+        {
+            float gm[CA];
+            {
+                float xv[CA];
+                if (q < HW) {
+                    load_px<T, LAYOUT, CA>(gx, b, C, HW, q, vec, gm);
+                    load_px<T, LAYOUT, CA>(x, b, C, HW, q, vec, xv);
+                } else {
 #pragma unroll
-            for (int k = 0; k < CA; ++k) o[k] = bs[k];
+                    for (int k = 0; k < CA; ++k) gm[k] = xv[k] = 0.f;
+                }
 #pragma unroll
-            for (int n = 0; n < CA; ++n)
+                for (int k = 0; k < CA; ++k) {
+                    gs[k * kPitch + tid] = gm[k];
+                    xs[k * kPitch + tid] = xv[k];
+                }
+            }
+            if (q < HW) {
+                // a group of channels at a time (rolled, as in `mix`)
+                constexpr int G = CA >= 8 ? 8 : 4;
+#pragma unroll 1
+                for (int k0 = 0; k0 < CA; k0 += G) {
+                    float o[G];
 #pragma unroll
-                for (int k = 0; k < CA; ++k) o[k] = fmaf(ps[n * CA + k], gm[n], o[k]);
-            store_px<T, LAYOUT, CA>(gx, b, C, HW, q, vec, o);
-        } else {
+                    for (int j = 0; j < G; ++j) o[j] = bs[k0 + j];
 #pragma unroll
-            for (int k = 0; k < CA; ++k) gm[k] = xv[k] = 0.f;
-        }
+                    for (int n = 0; n < CA; ++n)
 #pragma unroll
-        for (int k = 0; k < CA; ++k) {
-            gs[k * kPitch + tid] = gm[k];
-            xs[k * kPitch + tid] = xv[k];
+                        for (int j = 0; j < G; ++j) o[j] = fmaf(ps[n * CA + k0 + j], gm[n], o[j]);
+                    store_group<T, LAYOUT, G>(gx, b, C, HW, q, vec, k0, o);
+                }
+            }
         }
         __syncthreads();
+        if (G::kPx >= 4) {
+            // pixels slice*4 + i*(4*kSlices) .. +3
+#pragma unroll 2
+            for (int i = 0; i < G::kPx / 4; ++i) {
+                const int px = slice * 4 + i * 4 * G::kSlices;
+                float4 u[4], w[4];
 #pragma unroll
-        for (int e = 0; e < NP; ++e) {
-            const int pair = e * kThreads + tid;
-            if (pair < CA * CA) {
-                const float4* a = reinterpret_cast<const float4*>(gs + (pair / CA) * kPitch);
-                const float4* c = reinterpret_cast<const float4*>(xs + (pair % CA) * kPitch);
-                float s = acc[e];
-#pragma unroll 4
-                for (int i = 0; i < kThreads / 4; ++i) {
-                    const float4 u = a[i], w = c[i];
-                    s = fmaf(u.x, w.x, s); s = fmaf(u.y, w.y, s); s = fmaf(u.z, w.z, s); s = fmaf(u.w, w.w, s);
+                for (int r = 0; r < 4; ++r) {
+                    u[r] = *reinterpret_cast<const float4*>(gs + (n0 + r) * kPitch + px);
+                    w[r] = *reinterpret_cast<const float4*>(xs + (k0 + r) * kPitch + px);
                 }
-                acc[e] = s;
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float t = acc[r][c];
+                        t = fmaf(u[r].x, w[c].x, t); t = fmaf(u[r].y, w[c].y, t);
+                        t = fmaf(u[r].z, w[c].z, t); t = fmaf(u[r].w, w[c].w, t);
+                        acc[r][c] = t;
+                    }
+            }
+        } else {
+            // fewer than four pixels per slice (C_a = 4: one tile, a pixel per thread)
+#pragma unroll
+            for (int i = 0; i < G::kPx; ++i) {
+                const int px = slice * G::kPx + i;
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(gs[(n0 + r) * kPitch + px], xs[(k0 + c) * kPitch + px], acc[r][c]);
             }
         }
     }
+    __syncthreads();
+    float* red = gs;                                             // [kSlices][CA * CA]
 #pragma unroll
-    for (int e = 0; e < NP; ++e) {
-        const int pair = e * kThreads + tid;
-        if (pair < CA * CA) gp_part[(size_t)blockIdx.x * (CA * CA) + pair] = acc[e];
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) red[slice * (CA * CA) + (n0 + r) * CA + k0 + c] = acc[r][c];
+    __syncthreads();
+    for (int e = tid; e < CA * CA; e += kThreads) {
+        float t = red[e];
+        for (int sl = 1; sl < G::kSlices; ++sl) t += red[sl * (CA * CA) + e];
+        gp_part[(size_t)blockIdx.x * (CA * CA) + e] = t;
     }
 }
 
