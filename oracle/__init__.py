@@ -14,6 +14,7 @@ from .convattn_oracle import (  # noqa: F401
     backward,
     backward_mlp,
     backward_pw,
+    backward_dense,
     stencil_dense,
     forward_dense,
     pointwise,

@@ -271,6 +271,27 @@ def backward_pw(x, grad_out, C_a, w_large, w_point, w_dyn, b_dyn):
     return gx, glk, gwp, gw, gb
 
 
+def backward_dense(x, grad_out, C_a, w_dense, w_dyn, b_dyn):
+    """Gradients of forward_dense(x, ...) contracted with grad_out: returns (gx [B,C,H,W], g_w_dense [C_a,C_a,K,K],
+    g_w_dyn [9*C_a,C_a], g_b_dyn [9*C_a])."""
+    x, xp = _f32(x)
+    go, gp = _f32(grad_out)
+    assert go.shape == x.shape
+    w_dense, wp = _f64(w_dense)
+    K = int(w_dense.shape[-1])
+    B, C, H, W = _dims(x, C_a, K)
+    assert w_dense.shape == (C_a, C_a, K, K)
+    w_dyn, wdp = _f64(w_dyn)
+    b_dyn, bdp = _f64(b_dyn)
+    gx = np.empty((B, C, H, W), dtype=np.float64)
+    gwd = np.empty((C_a, C_a, K, K), dtype=np.float64)
+    gw = np.empty((9 * C_a, C_a), dtype=np.float64)
+    gb = np.empty((9 * C_a,), dtype=np.float64)
+    _load().convattn_ref_backward_dense(xp, gp, B, C, C_a, H, W, K, wp, wdp, bdp, *(a.ctypes.data_as(_f64p)
+                                        for a in (gx, gwd, gw, gb)))
+    return gx, gwd, gw, gb
+
+
 def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
     """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
     x, xp = _f32(x)

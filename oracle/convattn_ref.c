@@ -35,6 +35,7 @@
  * b_dyn, by the chain rule written out; convattn_ref_backward_mlp the same with the two-layer estimator
  * (gradients with respect to x, LK, W_down, b_down, W_up, b_up).
  * convattn_ref_backward_pw is the gradient of the decomposed form (x, LK^s, LK^c, W_dyn, b_dyn).
+ * convattn_ref_backward_dense is the gradient of the dense form (x, the dense LK, W_dyn, b_dyn).
  *
  * (*) is cross-correlation (no kernel flip) with zero 'same' padding.
  * Everything is accumulated in double precision with direct nested loops in
@@ -63,7 +64,9 @@
  * the pinned forward and by its linear limit, where it must equal the pinned one-layer backward
  * with composed weights; the backward pass of the decomposed form by central differences of the pinned
  * decomposed forward (also exact), by the identity mix, where it must equal the pinned depth-wise backward,
- * and by the adjoint identity of its linear part.
+ * and by the adjoint identity of its linear part; the backward pass with the dense large kernel by exact
+ * differences of the pinned dense forward and by its diagonal case, where it must equal the pinned depth-wise
+ * backward.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -725,6 +728,106 @@ void convattn_ref_backward_pw(const float *x, const float *go, int B, int C, int
                 }
     }
     free(g); free(dk); free(m); free(gm); free(gtap); free(gdk); free(gg);
+}
+
+/* Backward pass of the forward with the dense large kernel of Section 3.2 (w_dense[n,k,i,j]: output channel n sums
+ * over every attention input channel k; the dynamic 3x3 kernel stays depth-wise; one-layer estimator), by the chain rule
+ * written out.  With go = dL/dout, x~ and go~ zero-padded, g = GAP(x), dk = W g + b:
+ *   g_wd[n,k,i,j] = sum_{b,y,x} go[b,n,y,x] * x~[b,k,y+i-P,x+j-P]                         (dL/dw_dense)
+ *   g_dk[b,c,i,j] = sum_{y,x} go[b,c,y,x] * x~[b,c,y+i-1,x+j-1]                           (dL/ddk, depth-wise)
+ *   g_b[o] = sum_b g_dk[b,o]     g_W[o,k] = sum_b g_dk[b,o] * g[b,k]     g_g[b,k] = sum_o W[o,k] * g_dk[b,o]
+ *   g_x[b,k,y,x]  = sum_n sum_{i,j} w_dense[n,k,i,j] * go~[b,n,y-(i-P),x-(j-P)]
+ *                 + sum_{i,j} dk[b,k,i,j] * go~[b,k,y-(i-1),x-(j-1)] + g_g[b,k] / (H*W)     k < C_a
+ *   g_x[b,c]      = go[b,c]                                                                c >= C_a
+ * Outputs: gx [B,C,H,W], gwd [C_a,C_a,K,K], gw [9*C_a,C_a], gb [9*C_a]; any may be NULL. */
+void convattn_ref_backward_dense(const float *x, const float *go, int B, int C, int C_a, int H, int W, int K,
+                                 const double *w_dense, const double *w_dyn, const double *b_dyn,
+                                 double *gx, double *gwd, double *gw, double *gb)
+{
+    const int P = (K - 1) / 2;
+    double *g = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    double *dk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    double *gdk = (double *)malloc(sizeof(double) * (size_t)B * C_a * 9);
+    double *gg = (double *)malloc(sizeof(double) * (size_t)B * C_a);
+    convattn_ref_gap(x, B, C, C_a, H, W, g);
+    convattn_ref_dynkernel(g, B, C_a, w_dyn, b_dyn, dk);
+    if (gwd) {
+#pragma omp parallel for collapse(2) schedule(static)
+        for (int n = 0; n < C_a; ++n)
+            for (int k = 0; k < C_a; ++k)
+                for (int i = 0; i < K; ++i)
+                    for (int j = 0; j < K; ++j) {
+                        double s = 0.0;
+                        for (int b = 0; b < B; ++b)
+                            for (int y = 0; y < H; ++y)
+                                for (int xx = 0; xx < W; ++xx) {
+                                    int yy = y + i - P, xc = xx + j - P;
+                                    if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                        s += (double)go[IDX4(b, n, y, xx, C, H, W)] * (double)x[IDX4(b, k, yy, xc, C, H, W)];
+                                }
+                        gwd[(((size_t)n * C_a + k) * K + i) * K + j] = s;
+                    }
+    }
+    for (int b = 0; b < B; ++b)
+        for (int c = 0; c < C_a; ++c)
+            for (int i = 0; i < 3; ++i)
+                for (int j = 0; j < 3; ++j) {
+                    double s = 0.0;
+                    for (int y = 0; y < H; ++y)
+                        for (int xx = 0; xx < W; ++xx) {
+                            int yy = y + i - 1, xc = xx + j - 1;
+                            if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                s += (double)go[IDX4(b, c, y, xx, C, H, W)] * (double)x[IDX4(b, c, yy, xc, C, H, W)];
+                        }
+                    gdk[((size_t)b * C_a + c) * 9 + i * 3 + j] = s;
+                }
+    if (gb)
+        for (int o = 0; o < 9 * C_a; ++o) {
+            double s = 0.0;
+            for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o];
+            gb[o] = s;
+        }
+    if (gw)
+        for (int o = 0; o < 9 * C_a; ++o)
+            for (int k = 0; k < C_a; ++k) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b) s += gdk[(size_t)b * 9 * C_a + o] * g[(size_t)b * C_a + k];
+                gw[(size_t)o * C_a + k] = s;
+            }
+    for (int b = 0; b < B; ++b)
+        for (int k = 0; k < C_a; ++k) {
+            double s = 0.0;
+            for (int o = 0; o < 9 * C_a; ++o) s += w_dyn[(size_t)o * C_a + k] * gdk[(size_t)b * 9 * C_a + o];
+            gg[(size_t)b * C_a + k] = s;
+        }
+    if (gx) {
+#pragma omp parallel for collapse(3) schedule(static)
+        for (int b = 0; b < B; ++b)
+            for (int c = 0; c < C; ++c)
+                for (int y = 0; y < H; ++y)
+                    for (int xx = 0; xx < W; ++xx) {
+                        if (c >= C_a) {
+                            gx[IDX4(b, c, y, xx, C, H, W)] = (double)go[IDX4(b, c, y, xx, C, H, W)];
+                            continue;
+                        }
+                        double s = 0.0;
+                        for (int n = 0; n < C_a; ++n)
+                            for (int i = 0; i < K; ++i)
+                                for (int j = 0; j < K; ++j) {
+                                    int yy = y - (i - P), xc = xx - (j - P);
+                                    if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                        s += w_dense[(((size_t)n * C_a + c) * K + i) * K + j] * (double)go[IDX4(b, n, yy, xc, C, H, W)];
+                                }
+                        for (int i = 0; i < 3; ++i)
+                            for (int j = 0; j < 3; ++j) {
+                                int yy = y - (i - 1), xc = xx - (j - 1);
+                                if (yy >= 0 && yy < H && xc >= 0 && xc < W)
+                                    s += dk[((size_t)b * C_a + c) * 9 + i * 3 + j] * (double)go[IDX4(b, c, yy, xc, C, H, W)];
+                            }
+                        gx[IDX4(b, c, y, xx, C, H, W)] = s + gg[(size_t)b * C_a + c] / ((double)H * (double)W);
+                    }
+    }
+    free(g); free(dk); free(gdk); free(gg);
 }
 
 /* Selected outputs, one by one: idx[n] are flat indices into out[B,C,H,W]; dk is
