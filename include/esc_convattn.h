@@ -321,6 +321,23 @@ int esc_convattn_backward_pw(const void* x, const void* grad_out, int B, int C, 
                              float* grad_b_dyn, int dtype, int layout,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Backward pass of esc_convattn_forward_dense, the dense large kernel of Section 3.2 (w_dense [C_a,C_a,K,K]: output
+ * channel, input channel, row, column; element type of x), depth-wise dynamic kernel, one-layer estimator:
+ *   grad_w_dense [C_a,C_a,K,K]  fp32   dL/dw_dense[n,k,i,j] = sum over images and pixels of grad_out[n,y,x] x~[k,y+i-P,x+j-P]  (may be NULL)
+ *   grad_x, grad_w_dyn, grad_b_dyn as in esc_convattn_backward (grad_x's large-kernel term sums over the output channels).
+ * C_a must be 16 (ESC_ERR_UNSUPPORTED otherwise); K odd, 3 .. 13.  The workspace is one of
+ * esc_convattn_backward_dense_workspace_bytes(...) bytes (larger than the depth-wise one: every block of the tap-gradient
+ * kernel keeps 16 x 16 x 169 sums there), 256-byte aligned, zeroed once with esc_convattn_workspace_init().  Same
+ * restrictions and error codes as esc_convattn_backward.  All device memory; asynchronous on `stream`.
+ */
+size_t esc_convattn_backward_dense_workspace_bytes(int B, int C_a, int H, int W, int K);
+int esc_convattn_backward_dense(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                                const void* w_dense, const void* w_dyn, const void* b_dyn,
+                                void* grad_x, float* grad_w_dense, float* grad_w_dyn, float* grad_b_dyn,
+                                int dtype, int layout,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

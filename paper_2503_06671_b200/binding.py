@@ -57,6 +57,9 @@ def lib():
         L.esc_convattn_backward.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_backward_mlp.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, i, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_backward_pw.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_backward_dense_workspace_bytes.argtypes = [i, i, i, i, i]
+        L.esc_convattn_backward_dense_workspace_bytes.restype = sz
+        L.esc_convattn_backward_dense.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -71,7 +74,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_forward_fused", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_backward_mlp", "esc_convattn_backward_pw", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_backward_mlp", "esc_convattn_backward_pw", "esc_convattn_backward_dense", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_set_stencil_engine", "esc_convattn_set_fused_stage1", "esc_convattn_set_dense_engine", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -330,6 +333,33 @@ def esc_convattn_backward_pw(x, grad_out, C_a, K, w_large, w_point, w_dyn, b_dyn
                                           _ptr(grad_b_dyn), _dtype_code(x), layout, _ptr(workspace),
                                           workspace.numel() * workspace.element_size(), _stream(stream)),
            "esc_convattn_backward_pw")
+    return grad_x
+
+
+def esc_convattn_backward_dense_workspace_bytes(B, C_a, H, W, K) -> int:
+    return int(lib().esc_convattn_backward_dense_workspace_bytes(B, C_a, H, W, K))
+
+
+def new_backward_dense_workspace(B, C_a, H, W, K, device="cuda"):
+    """Allocate (with torch) and zero a workspace for esc_convattn_backward_dense."""
+    import torch
+
+    n = esc_convattn_backward_dense_workspace_bytes(B, C_a, H, W, K)
+    if n == 0:
+        raise ValueError("invalid problem size, C_a is not 16, or K is not odd in 3 .. 13")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    esc_convattn_workspace_init(ws)
+    return ws
+
+
+def esc_convattn_backward_dense(x, grad_out, C_a, K, w_dense, w_dyn, b_dyn, grad_x, grad_w_dense, grad_w_dyn, grad_b_dyn, layout,
+                                workspace, stream=None):
+    """Gradients of esc_convattn_forward_dense: grad_x like x; the three weight gradients are fp32 tensors or None."""
+    B, C, H, W = _dims(x, layout)
+    _check(lib().esc_convattn_backward_dense(_ptr(x), _ptr(grad_out), B, C, C_a, H, W, K, _ptr(w_dense), _ptr(w_dyn), _ptr(b_dyn),
+                                             _ptr(grad_x), _ptr(grad_w_dense), _ptr(grad_w_dyn), _ptr(grad_b_dyn), _dtype_code(x),
+                                             layout, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_backward_dense")
     return grad_x
 
 

@@ -25,6 +25,7 @@
 #include "stencil_dense_umma.cuh"
 #include "backward.cuh"
 #include "backward_pw.cuh"
+#include "backward_dense.cuh"
 #include "conv_fuse.cuh"
 
 namespace {
@@ -523,6 +524,10 @@ struct BackwardWs {
     int chunks;                      // chunks of pixels per image in those
     bool patch_xsum;                 // the tap-gradient kernels ran on the mixed features: take the sums of x_att from xs_part
     size_t bytes;
+    float* dense_part;               // dense large kernel: the blocks' tap sums [blocks][16][16][169]
+    void* wd_flip;                   // the dense kernel with swapped channel axes and rotated taps
+    int dense_blocks;
+    size_t bytes_dense;              // bytes with those two behind the rest
 };
 BackwardWs carve_backward(void* ws, const Problem& p) {
     // sized for whichever tiling of the tap-gradient kernels has more tiles (32x32, or 64x16 on the tensor cores)
@@ -546,6 +551,10 @@ BackwardWs carve_backward(void* ws, const Problem& p) {
     w.gp_part = reinterpret_cast<float*>(base + off);
     if (esc::bwd::pw::supported(p.Ca)) off += round_up((size_t)p.B * w.chunks * p.Ca * p.Ca * 4, 256);
     w.bytes = off;
+    w.dense_blocks = sms_or_nominal();
+    w.dense_part = reinterpret_cast<float*>(base + off); off += round_up((size_t)w.dense_blocks * esc::bwd::dense::kPartFloats * 4, 256);
+    w.wd_flip = base + off;                              off += round_up((size_t)esc::bwd::dense::CA * esc::bwd::dense::CA * esc::bwd::TAPS * 4, 256);
+    w.bytes_dense = off;
     return w;
 }
 
@@ -689,6 +698,46 @@ int pw_back_t(const Problem& p, const void* x, const void* w_point, void* gx, co
         case 32: return pw_back_ca<T, LAYOUT, 32>(p, x, w_point, gx, w, g_wp, st);
     }
     return ESC_ERR_UNSUPPORTED;
+}
+
+// Dense large kernel: tap gradients of every channel pair, the rotated kernel for the stencil pass, and the constants
+// added behind it.
+template <typename T, int LAYOUT>
+int dense_tap_grad_t(const Problem& p, const void* x, const void* go, const void* w_dense, const BackwardWs& w, float* g_wd,
+                     cudaStream_t st) {
+    namespace D = esc::bwd::dense;
+    static bool attr_set[esc::tma::kMaxDevices] = {};
+    const int dev = esc::tma::current_device();
+    if (dev < 0) return ESC_ERR_UNSUPPORTED;
+    if (!attr_set[dev]) {
+        ESC_CUDA(cudaFuncSetAttribute(D::tap_grad_dense<T, LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)D::kSmemBytes));
+        attr_set[dev] = true;
+    }
+    const int tiles_x = (p.W + D::TX - 1) / D::TX, tiles_y = (p.H + D::TY - 1) / D::TY;
+    if (g_wd) {
+        D::tap_grad_dense<T, LAYOUT><<<(unsigned)w.dense_blocks, D::kThreads, D::kSmemBytes, st>>>(
+            static_cast<const T*>(x), static_cast<const T*>(go), p.B, p.C, p.H, p.W, tiles_x, tiles_y, w.dense_part);
+        ESC_CUDA(cudaGetLastError());
+        const int elems = D::CA * D::CA * p.K * p.K;
+        D::sum_dense<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(w.dense_part, w.dense_blocks, p.K, g_wd);
+        ESC_CUDA(cudaGetLastError());
+        g_last_launches += 2;
+    }
+    const int elems = D::CA * D::CA * p.K * p.K;
+    D::flip_dense<T><<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(static_cast<const T*>(w_dense), p.K, static_cast<T*>(w.wd_flip));
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
+}
+template <typename T, int LAYOUT>
+int dense_add_const_t(const Problem& p, void* gx, const BackwardWs& w, cudaStream_t st) {
+    const long long total = (long long)p.B * p.Ca * p.H * p.W;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 16LL * sms_or_nominal()) blocks = 16LL * sms_or_nominal();
+    esc::bwd::dense::add_const<T, LAYOUT><<<(unsigned)blocks, 256, 0, st>>>(static_cast<T*>(gx), w.bias, p.B, p.C, p.Ca, (long long)p.H * p.W);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
 }
 
 // ---- fixed scratch for the entry point that must not allocate ------------------------------
@@ -1114,7 +1163,8 @@ size_t esc_convattn_backward_workspace_bytes(int B, int C_a, int H, int W, int K
 namespace {
 int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K, const void* w_large,
                    const Estimator& est, void* grad_x, const BackwardGrads& g, int dtype, int layout, void* workspace,
-                   size_t workspace_bytes_, void* stream, const void* w_point = nullptr, float* g_wp = nullptr) {
+                   size_t workspace_bytes_, void* stream, const void* w_point = nullptr, float* g_wp = nullptr,
+                   bool dense = false, float* g_wd = nullptr) {
     g_last_launches = 0;
     Problem p{B, C, C_a, H, W, K, dtype, layout};
     int rc = check_shape(p);
@@ -1141,8 +1191,10 @@ int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, i
         if ((long long)B * esc::bwd::pw::chunks_of((long long)H * W) > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
     }
     if (!workspace || !aligned(workspace, 256)) return ESC_ERR_WORKSPACE;
+    if (dense && (C_a != esc::bwd::dense::CA || est.hidden != 0 || w_point)) return ESC_ERR_UNSUPPORTED;
+    if (g_wd && !aligned(g_wd, 4)) return ESC_ERR_ALIGN;
     BackwardWs w = carve_backward(workspace, p);
-    if (workspace_bytes_ < w.bytes) return ESC_ERR_WORKSPACE;
+    if (workspace_bytes_ < (dense ? w.bytes_dense : w.bytes)) return ESC_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (w_point) {
         // decomposed form (Eq. 5): the mixed features go into grad_x's attention channels, where the tap-gradient kernels
@@ -1155,6 +1207,15 @@ int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, i
         w.patch_xsum = true;
     }
     const void* x_taps = w_point ? grad_x : x;             // what the depth-wise stage saw
+    if (dense) {
+        // w_large is the dense kernel [16][16][K][K]: its gradient and its rotated form here; the depth-wise kernels
+        // below give g_dk (the middle 3 x 3 of their tap gradients) and what follows from it
+        rc = dtype == ESC_F32 ? (layout == ESC_NCHW ? dense_tap_grad_t<float, esc::kNCHW>(p, x, grad_out, w_large, w, g_wd, st)
+                                                    : dense_tap_grad_t<float, esc::kNHWC>(p, x, grad_out, w_large, w, g_wd, st))
+                              : (layout == ESC_NCHW ? dense_tap_grad_t<__nv_bfloat16, esc::kNCHW>(p, x, grad_out, w_large, w, g_wd, st)
+                                                    : dense_tap_grad_t<__nv_bfloat16, esc::kNHWC>(p, x, grad_out, w_large, w, g_wd, st));
+        if (rc != ESC_OK) return rc;
+    }
     if (dtype == ESC_F32)
         rc = layout == ESC_NCHW ? backward_t<float, esc::kNCHW>(p, x_taps, grad_out, w_large, est, w, g, st)
                                 : backward_t<float, esc::kNHWC>(p, x_taps, grad_out, w_large, est, w, g, st);
@@ -1164,6 +1225,15 @@ int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, i
     if (rc != ESC_OK) return rc;
     // grad_x: the forward stencil on grad_out with both kernels rotated by 180 degrees, plus the constants (in the
     // decomposed form the constants belong behind the transposed mix: the last kernel adds them)
+    if (dense) {
+        p.dense = true;
+        rc = launch_stencil_dense(p, grad_out, w.wd_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false);
+        if (rc != ESC_OK) return rc;
+        return dtype == ESC_F32 ? (layout == ESC_NCHW ? dense_add_const_t<float, esc::kNCHW>(p, grad_x, w, st)
+                                                      : dense_add_const_t<float, esc::kNHWC>(p, grad_x, w, st))
+                                : (layout == ESC_NCHW ? dense_add_const_t<__nv_bfloat16, esc::kNCHW>(p, grad_x, w, st)
+                                                      : dense_add_const_t<__nv_bfloat16, esc::kNHWC>(p, grad_x, w, st));
+    }
     p.bias = w_point ? nullptr : w.bias;
     const TensorLk tl = tensor_lk(p, grad_out, grad_x, w.w_flip, w.lk_pad, st);
     rc = launch_stencil(p, grad_out, w.w_flip, w.dk_flip, grad_x, w.ctrl, st, /*dependent=*/false, &tl);
@@ -1205,6 +1275,22 @@ int esc_convattn_backward_pw(const void* x, const void* grad_out, int B, int C, 
     const BackwardGrads g{grad_w_large, grad_w_dyn, grad_b_dyn, nullptr, nullptr};
     return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_large, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream,
                           w_point, grad_w_point);
+}
+
+size_t esc_convattn_backward_dense_workspace_bytes(int B, int C_a, int H, int W, int K) {
+    if (B <= 0 || C_a != esc::bwd::dense::CA || H <= 0 || W <= 0 || K < 3 || K > esc::bwd::K || (K & 1) == 0) return 0;
+    const Problem p{B, C_a, C_a, H, W, K, ESC_F32, ESC_NCHW};
+    return carve_backward(nullptr, p).bytes_dense;
+}
+
+int esc_convattn_backward_dense(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                                const void* w_dense, const void* w_dyn, const void* b_dyn, void* grad_x,
+                                float* grad_w_dense, float* grad_w_dyn, float* grad_b_dyn, int dtype, int layout,
+                                void* workspace, size_t workspace_bytes_, void* stream) {
+    const Estimator est{w_dyn, b_dyn, nullptr, nullptr, 0};
+    const BackwardGrads g{nullptr, grad_w_dyn, grad_b_dyn, nullptr, nullptr};
+    return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_dense, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream,
+                          nullptr, nullptr, /*dense=*/true, grad_w_dense);
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {
