@@ -595,6 +595,18 @@ def main():
                                                                              g_wp, g_w, g_b, lay_code, bws), samples=5)
                 extras["backward"]["decomposed_large_kernel_ms_per_step"] = st["median_ms"]
                 extras["backward"]["decomposed_large_kernel_launches"] = pkg.esc_convattn_last_launches()
+            if wl.C_a == 16:
+                # the same with the dense large kernel (Section 3.2): 2 x 16 x 16 x K x K multiply-adds per pixel for the
+                # kernel's gradient on the FP32 pipe, grad_x on the forward's tensor-core kernel
+                wdn_b = torch.from_numpy(synth.make_dense_kernel(wl.C_a, wl.K, wl.dtype, wl.seed)).to(tdt).cuda()
+                g_wdn = torch.zeros(wl.C_a, wl.C_a, wl.K, wl.K, device="cuda")
+                dws = pkg.new_backward_dense_workspace(wl.B, wl.C_a, wl.H, wl.W, wl.K)
+                st, _ = timer.measure(lambda i: pkg.esc_convattn_backward_dense(xs[i % n_rot], go_d, wl.C_a, wl.K, wdn_b, wd_d, bd_d, gx_d, g_wdn,
+                                                                                g_w, g_b, lay_code, dws), samples=5)
+                t_fma_d = 2.0 * wl.C_a * wl.C_a * wl.K * wl.K * wl.pixels / (sms * FMA_LANES_PER_SM * 2 * pk["sm_max_mhz"] * 1e6)
+                extras["backward"]["dense_large_kernel_ms_per_step"] = st["median_ms"]
+                extras["backward"]["dense_large_kernel_launches"] = pkg.esc_convattn_last_launches()
+                extras["backward"]["dense_large_kernel_frac_of_fp32_roofline_of_its_weight_gradient"] = t_fma_d / (st["median_ms"] * 1e-3)
         except Exception as exc:
             extras["backward"] = {"error": f"{type(exc).__name__}: {exc}"}
         # with the dense large kernel of the main model (Section 3.2): an implicit GEMM on the tensor cores
