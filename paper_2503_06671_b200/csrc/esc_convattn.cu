@@ -23,6 +23,7 @@
 #include "backward_toeplitz_nchw.cuh"
 #include "stencil_dense.cuh"
 #include "stencil_dense_umma.cuh"
+#include <type_traits>
 #include "backward.cuh"
 #include "backward_pw.cuh"
 #include "backward_dense.cuh"
@@ -715,8 +716,22 @@ int dense_tap_grad_t(const Problem& p, const void* x, const void* go, const void
     }
     const int tiles_x = (p.W + D::TX - 1) / D::TX, tiles_y = (p.H + D::TY - 1) / D::TY;
     if (g_wd) {
-        D::tap_grad_dense<T, LAYOUT><<<(unsigned)w.dense_blocks, D::kThreads, D::kSmemBytes, st>>>(
-            static_cast<const T*>(x), static_cast<const T*>(go), p.B, p.C, p.H, p.W, tiles_x, tiles_y, w.dense_part);
+        if (std::is_same<T, __nv_bfloat16>::value && g_engine_policy != ESC_ENGINE_FP32) {
+            // bf16: a matrix product per tap on the tensor cores
+            static bool attr_mma[esc::tma::kMaxDevices] = {};
+            if (!attr_mma[dev]) {
+                ESC_CUDA(cudaFuncSetAttribute(D::mma::tap_grad_dense_bf16<LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)D::mma::kSmemBytes));
+                attr_mma[dev] = true;
+            }
+            const int vec = LAYOUT == esc::kNHWC && p.C % 8 == 0 ? 1 : 0;
+            D::mma::tap_grad_dense_bf16<LAYOUT><<<(unsigned)w.dense_blocks, D::mma::kThreads, D::mma::kSmemBytes, st>>>(
+                static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(go), p.B, p.C, p.H, p.W, tiles_x, tiles_y, vec,
+                w.dense_part);
+        } else {
+            D::tap_grad_dense<T, LAYOUT><<<(unsigned)w.dense_blocks, D::kThreads, D::kSmemBytes, st>>>(
+                static_cast<const T*>(x), static_cast<const T*>(go), p.B, p.C, p.H, p.W, tiles_x, tiles_y, w.dense_part);
+        }
         ESC_CUDA(cudaGetLastError());
         const int elems = D::CA * D::CA * p.K * p.K;
         D::sum_dense<<<(unsigned)((elems + 255) / 256), 256, 0, st>>>(w.dense_part, w.dense_blocks, p.K, g_wd);

@@ -101,7 +101,8 @@ def test_backward_dense(pkg, oracle, shape, dtype, layout):
 
 def test_backward_dense_many_tiles(pkg, oracle):
     """More tiles than blocks: 3 x 13 x 7 = 273 tiles of 32 x 16 on one block per SM, so blocks add up two tiles, some of
-    them of two images, in their registers; bf16 NHWC, where grad_x runs on the tcgen05 kernel."""
+    them of two images, in their registers; bf16 NHWC, where the weight gradient is a matrix product per tap on the tensor
+    cores and grad_x runs on the tcgen05 kernel."""
     shape = (3, 32, 16, 200, 200, 13)
     B, C, C_a, H, W, K = shape
     d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=91, per_image_scale=True, channel_means=True)
@@ -109,6 +110,14 @@ def test_backward_dense_many_tiles(pkg, oracle):
     go = synth.round_to(np.random.default_rng(92).standard_normal(size=d["x"].shape).astype(np.float32), synth.BF16)
     gx, g = _run(pkg, d, wdn, go, C_a, K, synth.BF16, synth.NHWC)
     _check(oracle, d, wdn, go, C_a, synth.BF16, gx, g)
+    # the FP32-pipe kernel on the same bf16 tensors (what fp32 tensors always use): the same sums in another order
+    pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_FP32)
+    try:
+        _, g2 = _run(pkg, d, wdn, go, C_a, K, synth.BF16, synth.NHWC)
+    finally:
+        pkg.esc_convattn_set_stencil_engine(pkg.ESC_ENGINE_AUTO)
+    mag = oracle.backward_dense(np.abs(d["x"]), np.abs(go), C_a, np.abs(wdn), np.abs(d["w_dyn"]), np.abs(d["b_dyn"]))[1]
+    assert (np.abs(g2["w_dense"] - g["w_dense"]) <= 2e-5 * mag).all()
 
 
 def test_diagonal_kernel_equals_the_depthwise_backward(pkg):
