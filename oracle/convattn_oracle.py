@@ -292,6 +292,60 @@ def backward_dense(x, grad_out, C_a, w_dense, w_dyn, b_dyn):
     return gx, gwd, gw, gb
 
 
+def backward_variant(x, grad_out, C_a, large_kernel, w_large, w_point, w_down, b_down, w_up, b_up):
+    """Gradients of a forward with any large-kernel form ("depthwise", "pw", "dense") and the two-layer estimator of
+    Eq. 4 line 2, by the chain rule in two steps.  (1) Per image, with the generator frozen at that image's dk
+    (W_dyn = 0, b_dyn = dk[b]) the one-layer backward of the form gives the stencil stage's part of gx, the large
+    kernel's gradients (summed over images) and, as its g_b_dyn, dL/ddk[b].  (2) Through the estimator,
+    t = W_down g + b_down, a = phi(t), dk = W_up a + b_up:
+        g_bu = sum_b g_dk      g_Wu = sum_b g_dk a^T      g_a = W_up^T g_dk      g_t = g_a * phi'(t)
+        g_bd = sum_b g_t       g_Wd = sum_b g_t g^T       g_g = W_down^T g_t     gx[b, :C_a] += g_g[b] / (H W)
+    with phi'(t) = Phi(t) + t n(t).  Returns (gx, g_w_large, g_w_point or None, g_w_down, g_b_down, g_w_up, g_b_up)."""
+    import math
+
+    xa = np.ascontiguousarray(x, dtype=np.float32)
+    go = np.ascontiguousarray(grad_out, dtype=np.float32)
+    B, C, H, W = xa.shape
+    w_down = np.asarray(w_down, dtype=np.float64); b_down = np.asarray(b_down, dtype=np.float64)
+    w_up = np.asarray(w_up, dtype=np.float64); b_up = np.asarray(b_up, dtype=np.float64)
+    g = gap(xa, C_a)
+    dk = dynkernel_mlp(g, w_down, b_down, w_up, b_up).reshape(B, 9 * C_a)
+    zero_w = np.zeros((9 * C_a, C_a))
+    gx = np.empty((B, C, H, W), dtype=np.float64)
+    g_large = None
+    g_point = None
+    g_dk = np.empty((B, 9 * C_a))
+    for b in range(B):
+        xb, gb_ = xa[b:b + 1], go[b:b + 1]
+        if large_kernel == "depthwise":
+            r = backward(xb, gb_, C_a, w_large, zero_w, dk[b])
+            gxb, glb, gdkb = r[0], r[1], r[3]
+        elif large_kernel == "pw":
+            r = backward_pw(xb, gb_, C_a, w_large, w_point, zero_w, dk[b])
+            gxb, glb, gdkb = r[0], r[1], r[4]
+            g_point = r[2] if g_point is None else g_point + r[2]
+        elif large_kernel == "dense":
+            r = backward_dense(xb, gb_, C_a, w_large, zero_w, dk[b])
+            gxb, glb, gdkb = r[0], r[1], r[3]
+        else:
+            raise ValueError(large_kernel)
+        gx[b] = gxb[0]
+        g_large = glb if g_large is None else g_large + glb
+        g_dk[b] = gdkb
+    t = g @ w_down.T + b_down                                           # [B, h]
+    Phi = np.vectorize(lambda v: 0.5 * math.erfc(-v / math.sqrt(2.0)))(t)
+    a = t * Phi
+    dphi = Phi + t * np.exp(-0.5 * t * t) / math.sqrt(2.0 * math.pi)
+    g_bu = g_dk.sum(axis=0)
+    g_wu = g_dk.T @ a
+    g_t = (g_dk @ w_up) * dphi
+    g_bd = g_t.sum(axis=0)
+    g_wd = g_t.T @ g
+    g_g = g_t @ w_down                                                  # [B, C_a]
+    gx[:, :C_a] += (g_g / (float(H) * float(W)))[:, :, None, None]
+    return gx, g_large, g_point, g_wd, g_bd, g_wu, g_bu
+
+
 def stencil(x, C_a, w_large, dk, rows=None, want_mag=False):
     """Stencil stage with an explicit dk[B,C_a,3,3]; rows=(y0,y1) restricts the output rows."""
     x, xp = _f32(x)
