@@ -338,6 +338,24 @@ int esc_convattn_backward_dense(const void* x, const void* grad_out, int B, int 
                                 int dtype, int layout,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Backward pass of esc_convattn_forward_variant: any large-kernel form (ESC_LK_*) with either estimator -- the
+ * configurations the paper's models use are the dense and the decomposed large kernel with the two-layer estimator of
+ * Eq. 4 line 2.  Arguments as in esc_convattn_forward_variant (hidden = 0: one linear layer w_up [9*C_a,C_a], b_up; w_down,
+ * b_down and their gradients ignored), gradients as in esc_convattn_backward_mlp, _pw and _dense:
+ *   grad_w_large  [C_a,K,K], or [C_a,C_a,K,K] for ESC_LK_DENSE   fp32 (may be NULL)
+ *   grad_w_point  [C_a,C_a] for ESC_LK_DECOMPOSED                 fp32 (may be NULL; ignored otherwise)
+ *   grad_w_down [hidden,C_a], grad_b_down [hidden], grad_w_up [9*C_a,hidden or C_a], grad_b_up [9*C_a]   fp32 (may be NULL)
+ * Restrictions of the form's own entry apply (ESC_LK_DECOMPOSED: C_a 4, 8, 16 or 32; ESC_LK_DENSE: C_a = 16 and the
+ * workspace of esc_convattn_backward_dense_workspace_bytes; otherwise esc_convattn_backward_workspace_bytes).
+ */
+int esc_convattn_backward_variant(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                                  int large_kernel, const void* w_large, const void* w_point, const void* w_down,
+                                  const void* b_down, const void* w_up, const void* b_up, int hidden, void* grad_x,
+                                  float* grad_w_large, float* grad_w_point, float* grad_w_down, float* grad_b_down,
+                                  float* grad_w_up, float* grad_b_up, int dtype, int layout,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

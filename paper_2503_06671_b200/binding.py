@@ -60,6 +60,7 @@ def lib():
         L.esc_convattn_backward_dense_workspace_bytes.argtypes = [i, i, i, i, i]
         L.esc_convattn_backward_dense_workspace_bytes.restype = sz
         L.esc_convattn_backward_dense.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_convattn_backward_variant.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -74,7 +75,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_forward_fused", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_backward_mlp", "esc_convattn_backward_pw", "esc_convattn_backward_dense", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_backward_mlp", "esc_convattn_backward_pw", "esc_convattn_backward_dense", "esc_convattn_backward_variant", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_set_stencil_engine", "esc_convattn_set_fused_stage1", "esc_convattn_set_dense_engine", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -360,6 +361,22 @@ def esc_convattn_backward_dense(x, grad_out, C_a, K, w_dense, w_dyn, b_dyn, grad
                                              _ptr(grad_x), _ptr(grad_w_dense), _ptr(grad_w_dyn), _ptr(grad_b_dyn), _dtype_code(x),
                                              layout, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "esc_convattn_backward_dense")
+    return grad_x
+
+
+def esc_convattn_backward_variant(x, grad_out, C_a, K, large_kernel, w_large, w_point, w_down, b_down, w_up, b_up, grad_x,
+                                  grad_w_large, grad_w_point, grad_w_down, grad_b_down, grad_w_up, grad_b_up, layout, workspace,
+                                  stream=None):
+    """Gradients of esc_convattn_forward_variant: any large-kernel form (ESC_LK_*) with either estimator (w_down None
+    means one linear layer w_up, b_up).  Weight gradients are fp32 tensors or None."""
+    B, C, H, W = _dims(x, layout)
+    hidden = 0 if w_down is None else int(w_down.shape[0])
+    _check(lib().esc_convattn_backward_variant(_ptr(x), _ptr(grad_out), B, C, C_a, H, W, K, int(large_kernel), _ptr(w_large),
+                                               _ptr(w_point), _ptr(w_down), _ptr(b_down), _ptr(w_up), _ptr(b_up), hidden,
+                                               _ptr(grad_x), _ptr(grad_w_large), _ptr(grad_w_point), _ptr(grad_w_down),
+                                               _ptr(grad_b_down), _ptr(grad_w_up), _ptr(grad_b_up), _dtype_code(x), layout,
+                                               _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_convattn_backward_variant")
     return grad_x
 
 

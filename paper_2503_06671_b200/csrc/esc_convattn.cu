@@ -1202,11 +1202,11 @@ int backward_entry(const void* x, const void* grad_out, int B, int C, int C_a, i
         if (q && !aligned(q, 4)) return ESC_ERR_ALIGN;
     if (w_point) {
         if (!aligned(w_point, p.es())) return ESC_ERR_ALIGN;
-        if (!esc::bwd::pw::supported(C_a) || est.hidden != 0) return ESC_ERR_UNSUPPORTED;
+        if (!esc::bwd::pw::supported(C_a)) return ESC_ERR_UNSUPPORTED;
         if ((long long)B * esc::bwd::pw::chunks_of((long long)H * W) > 0x7fffffffLL) return ESC_ERR_UNSUPPORTED;
     }
     if (!workspace || !aligned(workspace, 256)) return ESC_ERR_WORKSPACE;
-    if (dense && (C_a != esc::bwd::dense::CA || est.hidden != 0 || w_point)) return ESC_ERR_UNSUPPORTED;
+    if (dense && (C_a != esc::bwd::dense::CA || w_point)) return ESC_ERR_UNSUPPORTED;
     if (g_wd && !aligned(g_wd, 4)) return ESC_ERR_ALIGN;
     BackwardWs w = carve_backward(workspace, p);
     if (workspace_bytes_ < (dense ? w.bytes_dense : w.bytes)) return ESC_ERR_WORKSPACE;
@@ -1306,6 +1306,25 @@ int esc_convattn_backward_dense(const void* x, const void* grad_out, int B, int 
     const BackwardGrads g{nullptr, grad_w_dyn, grad_b_dyn, nullptr, nullptr};
     return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_dense, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream,
                           nullptr, nullptr, /*dense=*/true, grad_w_dense);
+}
+
+int esc_convattn_backward_variant(const void* x, const void* grad_out, int B, int C, int C_a, int H, int W, int K,
+                                  int large_kernel, const void* w_large, const void* w_point, const void* w_down,
+                                  const void* b_down, const void* w_up, const void* b_up, int hidden, void* grad_x,
+                                  float* grad_w_large, float* grad_w_point, float* grad_w_down, float* grad_b_down,
+                                  float* grad_w_up, float* grad_b_up, int dtype, int layout, void* workspace,
+                                  size_t workspace_bytes_, void* stream) {
+    if (large_kernel != ESC_LK_DEPTHWISE && large_kernel != ESC_LK_DECOMPOSED && large_kernel != ESC_LK_DENSE)
+        return ESC_ERR_UNSUPPORTED;
+    if (hidden < 0) return ESC_ERR_SHAPE;
+    if (large_kernel == ESC_LK_DECOMPOSED && !w_point) return ESC_ERR_NULL;
+    const Estimator est{w_up, b_up, hidden > 0 ? w_down : nullptr, hidden > 0 ? b_down : nullptr, hidden};
+    const bool dense = large_kernel == ESC_LK_DENSE;
+    const BackwardGrads g{dense ? nullptr : grad_w_large, grad_w_up, grad_b_up, hidden > 0 ? grad_w_down : nullptr,
+                          hidden > 0 ? grad_b_down : nullptr};
+    return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_large, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream,
+                          large_kernel == ESC_LK_DECOMPOSED ? w_point : nullptr,
+                          large_kernel == ESC_LK_DECOMPOSED ? grad_w_point : nullptr, dense, dense ? grad_w_large : nullptr);
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {
