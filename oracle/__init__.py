@@ -24,6 +24,7 @@ from .convattn_oracle import (  # noqa: F401
     points,
     fuse,
     forward_fused,
+    fuse_backward,
     set_threads,
     max_threads,
 )

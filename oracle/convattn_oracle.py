@@ -432,6 +432,24 @@ def fuse(cat, w_fuse, b_fuse=None, residual=None, want_mag=False):
     return (out, mag) if want_mag else out
 
 
+def fuse_backward(cat, grad_out, w_fuse, want_mag=False):
+    """Gradients of fuse(cat, w_fuse, b_fuse, residual) contracted with grad_out: returns (g_cat [B,C,H,W],
+    g_w_fuse [C,C], g_b_fuse [C]); the residual's gradient is grad_out itself."""
+    cat, cp = _f32(cat)
+    go, gp = _f32(grad_out)
+    assert go.shape == cat.shape
+    B, C, H, W = (int(v) for v in cat.shape)
+    w_fuse, wp = _f64(w_fuse)
+    assert w_fuse.shape == (C, C)
+    g_cat = np.empty((B, C, H, W), dtype=np.float64)
+    g_w = np.empty((C, C), dtype=np.float64)
+    g_b = np.empty((C,), dtype=np.float64)
+    mag = np.empty((B, C, H, W), dtype=np.float64) if want_mag else None
+    _load().convattn_ref_fuse_backward(cp, gp, B, C, H, W, wp, g_cat.ctypes.data_as(_f64p), g_w.ctypes.data_as(_f64p),
+                                       g_b.ctypes.data_as(_f64p), mag.ctypes.data_as(_f64p) if want_mag else None)
+    return (g_cat, g_w, g_b, mag) if want_mag else (g_cat, g_w, g_b)
+
+
 def forward_fused(x, C_a, w_large, w_dyn, b_dyn, w_fuse, b_fuse=None, residual=None, want_mag=False, want_cat=False):
     """The whole module of Eq. 4 including its last line: ConvAttn stages, then Conv_fuse (+ residual)."""
     cat = forward(x, C_a, w_large, w_dyn, b_dyn)

@@ -66,7 +66,8 @@
  * decomposed forward (also exact), by the identity mix, where it must equal the pinned depth-wise backward,
  * and by the adjoint identity of its linear part; the backward pass with the dense large kernel by exact
  * differences of the pinned dense forward and by its diagonal case, where it must equal the pinned depth-wise
- * backward.
+ * backward; the backward pass of Conv_fuse by exact differences of the pinned convattn_ref_fuse (linear in its
+ * input and in each weight) and by the identity matrix.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -229,6 +230,52 @@ void convattn_ref_fuse(const double *cat, int B, int C, int H, int W, const doub
                     out[IDX4(b, n, y, xx, C, H, W)] = s;
                     if (mag) mag[IDX4(b, n, y, xx, C, H, W)] = m;
                 }
+}
+
+/* Backward pass of convattn_ref_fuse.  With go = dL/dout [B,C,H,W] (float values) and cat the forward's input:
+ *   g_cat[b,c,y,x] = sum_n w_fuse[n,c] * go[b,n,y,x]
+ *   g_w[n,c]       = sum_{b,y,x} go[b,n,y,x] * cat[b,c,y,x]
+ *   g_b[n]         = sum_{b,y,x} go[b,n,y,x]
+ * (the residual's gradient is go itself).  mag_cat (optional) receives sum_n |w_fuse[n,c] * go|; any output may be NULL. */
+void convattn_ref_fuse_backward(const float *cat, const float *go, int B, int C, int H, int W, const double *w_fuse,
+                                double *g_cat, double *g_w, double *g_b, double *mag_cat)
+{
+    if (g_cat) {
+#pragma omp parallel for collapse(3) schedule(static)
+        for (int b = 0; b < B; ++b)
+            for (int c = 0; c < C; ++c)
+                for (int y = 0; y < H; ++y)
+                    for (int xx = 0; xx < W; ++xx) {
+                        double s = 0.0, m = 0.0;
+                        for (int n = 0; n < C; ++n) {
+                            double t = w_fuse[(size_t)n * C + c] * (double)go[IDX4(b, n, y, xx, C, H, W)];
+                            s += t;
+                            m += fabs(t);
+                        }
+                        g_cat[IDX4(b, c, y, xx, C, H, W)] = s;
+                        if (mag_cat) mag_cat[IDX4(b, c, y, xx, C, H, W)] = m;
+                    }
+    }
+    if (g_w) {
+#pragma omp parallel for collapse(2) schedule(static)
+        for (int n = 0; n < C; ++n)
+            for (int c = 0; c < C; ++c) {
+                double s = 0.0;
+                for (int b = 0; b < B; ++b)
+                    for (int y = 0; y < H; ++y)
+                        for (int xx = 0; xx < W; ++xx)
+                            s += (double)go[IDX4(b, n, y, xx, C, H, W)] * (double)cat[IDX4(b, c, y, xx, C, H, W)];
+                g_w[(size_t)n * C + c] = s;
+            }
+    }
+    if (g_b)
+        for (int n = 0; n < C; ++n) {
+            double s = 0.0;
+            for (int b = 0; b < B; ++b)
+                for (int y = 0; y < H; ++y)
+                    for (int xx = 0; xx < W; ++xx) s += (double)go[IDX4(b, n, y, xx, C, H, W)];
+            g_b[n] = s;
+        }
 }
 
 /* Point-wise large-kernel filter LK^c of the decomposed form (Eq. 5, first factor F_att (*) LK^c):
