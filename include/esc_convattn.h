@@ -356,6 +356,23 @@ int esc_convattn_backward_variant(const void* x, const void* grad_out, int B, in
                                   float* grad_w_up, float* grad_b_up, int dtype, int layout,
                                   void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Backward pass of the module's closing 1x1 convolution with the block's residual (Eq. 4 line 4, Eq. 3 line 3:
+ * out = W_fuse cat + b_fuse + residual per pixel; what esc_convattn_forward_fused adds behind the ConvAttn stages).
+ *   cat           [B,C,H,W]  the convolution's input (the concatenated map, i.e. esc_convattn_forward's output), device
+ *   grad_out      [B,C,H,W]  dL/dout, element type and layout of cat; it is also the residual's gradient
+ *   grad_cat      [B,C,H,W]  written: W_fuse transposed applied to grad_out -- the grad_out of esc_convattn_backward*
+ *   grad_w_fuse   [C,C] fp32  sum over images and pixels of grad_out[n] cat[c]   (may be NULL)
+ *   grad_b_fuse   [C]   fp32  sum over images and pixels of grad_out[n]          (may be NULL)
+ * C must be 16, 32, 48 or 64 (ESC_ERR_UNSUPPORTED otherwise).  grad_cat must not overlap cat or grad_out.  The workspace
+ * is one of esc_conv_fuse_backward_workspace_bytes(...) bytes, 256-byte aligned; it needs no initialisation.  All sums
+ * are added in a fixed order.  All device memory; asynchronous on `stream`.
+ */
+size_t esc_conv_fuse_backward_workspace_bytes(int B, int C, int H, int W);
+int esc_conv_fuse_backward(const void* cat, const void* grad_out, int B, int C, int H, int W, const void* w_fuse,
+                           void* grad_cat, float* grad_w_fuse, float* grad_b_fuse, int dtype, int layout,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

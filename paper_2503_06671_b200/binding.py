@@ -61,6 +61,9 @@ def lib():
         L.esc_convattn_backward_dense_workspace_bytes.restype = sz
         L.esc_convattn_backward_dense.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_backward_variant.argtypes = [vp, vp, i, i, i, i, i, i, i, vp, vp, vp, vp, vp, vp, i, vp, vp, vp, vp, vp, vp, vp, i, i, vp, sz, vp]
+        L.esc_conv_fuse_backward_workspace_bytes.argtypes = [i, i, i, i]
+        L.esc_conv_fuse_backward_workspace_bytes.restype = sz
+        L.esc_conv_fuse_backward.argtypes = [vp, vp, i, i, i, i, vp, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_dynkernel_static.argtypes = [vp, i, i, i, i, i, vp, vp, vp, i, i, vp]
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
@@ -75,7 +78,7 @@ def lib():
         L.esc_status_string.restype = ctypes.c_char_p
         L.esc_last_error.restype = ctypes.c_char_p
         for name in ("esc_convattn_forward", "esc_convattn_forward_ex", "esc_convattn_forward_fused", "esc_convattn_workspace_init",
-                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_backward_mlp", "esc_convattn_backward_pw", "esc_convattn_backward_dense", "esc_convattn_backward_variant", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
+                     "esc_convattn_dynkernel", "esc_convattn_dynkernel_static", "esc_convattn_forward_mlp", "esc_convattn_dynkernel_mlp", "esc_convattn_forward_pw", "esc_convattn_stencil_pw", "esc_convattn_forward_dense", "esc_convattn_stencil_dense", "esc_convattn_forward_variant", "esc_convattn_backward", "esc_convattn_backward_mlp", "esc_convattn_backward_pw", "esc_convattn_backward_dense", "esc_convattn_backward_variant", "esc_conv_fuse_backward", "esc_convattn_stencil", "esc_convattn_forward_host", "esc_convattn_forward_host_submit", "esc_convattn_forward_host_wait",
                      "esc_convattn_device_status", "esc_convattn_last_path", "esc_convattn_last_tile_width", "esc_convattn_set_tile_width", "esc_convattn_set_stencil_engine", "esc_convattn_set_fused_stage1", "esc_convattn_set_dense_engine", "esc_convattn_last_launches",
                      "esc_version"):
             getattr(L, name).restype = i
@@ -378,6 +381,28 @@ def esc_convattn_backward_variant(x, grad_out, C_a, K, large_kernel, w_large, w_
                                                _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
            "esc_convattn_backward_variant")
     return grad_x
+
+
+def esc_conv_fuse_backward_workspace_bytes(B, C, H, W) -> int:
+    return int(lib().esc_conv_fuse_backward_workspace_bytes(B, C, H, W))
+
+
+def esc_conv_fuse_backward(cat, grad_out, w_fuse, grad_cat, grad_w_fuse, grad_b_fuse, layout, workspace=None, stream=None):
+    """Gradients of the closing 1x1 convolution: grad_cat like cat; grad_w_fuse [C,C] and grad_b_fuse [C] are fp32 tensors
+    or None.  Without a workspace one is allocated with torch for the call."""
+    import torch
+
+    B, C, H, W = _dims(cat, layout)
+    if workspace is None:
+        n = esc_conv_fuse_backward_workspace_bytes(B, C, H, W)
+        if n == 0:
+            raise EscError(3, "esc_conv_fuse_backward_workspace_bytes")
+        workspace = torch.empty(n, dtype=torch.uint8, device=cat.device)
+    _check(lib().esc_conv_fuse_backward(_ptr(cat), _ptr(grad_out), B, C, H, W, _ptr(w_fuse), _ptr(grad_cat), _ptr(grad_w_fuse),
+                                        _ptr(grad_b_fuse), _dtype_code(cat), layout, _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream(stream)),
+           "esc_conv_fuse_backward")
+    return grad_cat
 
 
 def esc_convattn_forward_variant(x, C_a, K, large_kernel, w_large, w_point, w_down, b_down, w_up, b_up, out, layout,

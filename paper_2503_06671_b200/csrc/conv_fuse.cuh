@@ -320,8 +320,9 @@ inline bool applies(int C, int Ca, long long HW, int dtype, int layout, const vo
            al(residual) && al(w);
 }
 
+// `early`: the kernel may start, and read w, while the kernel before it in the stream still runs (w must then be older than that kernel)
 template <int C>
-inline cudaError_t launch_c(const Params& p, cudaStream_t st) {
+inline cudaError_t launch_c(const Params& p, cudaStream_t st, bool early) {
     const size_t smem = (size_t)3 * 2 * C * kPitchN;
     static bool attr_set[tma::kMaxDevices] = {};
     const int dev = tma::current_device();
@@ -341,14 +342,14 @@ inline cudaError_t launch_c(const Params& p, cudaStream_t st) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = early ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, conv_fuse_nchw_bf16<C>, p);
 }
-inline cudaError_t launch(const Params& p, cudaStream_t st) {
+inline cudaError_t launch(const Params& p, cudaStream_t st, bool early = true) {
     switch (p.C) {
-        case 32: return launch_c<32>(p, st);
-        case 48: return launch_c<48>(p, st);
-        case 64: return launch_c<64>(p, st);
+        case 32: return launch_c<32>(p, st, early);
+        case 48: return launch_c<48>(p, st, early);
+        case 64: return launch_c<64>(p, st, early);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -393,7 +394,7 @@ inline bool fast_applies(int C, int Ca, int dtype, int layout) {
 }
 
 template <int C>
-inline cudaError_t launch_fast_c(const Params& p, cudaStream_t st) {
+inline cudaError_t launch_fast_c(const Params& p, cudaStream_t st, bool early) {
     constexpr int PITCH = C * 2 + 16;
     const size_t smem = (size_t)(2 * Stages<C>::N * kPix + (C <= 64 ? 0 : C)) * PITCH;   // stages of (cat, residual); w_fuse where it is not in registers
     static bool attr_set[tma::kMaxDevices] = {};
@@ -414,17 +415,17 @@ inline cudaError_t launch_fast_c(const Params& p, cudaStream_t st) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = early ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, conv_fuse_nhwc_bf16<C>, p);
 }
 
-inline cudaError_t launch_fast(const Params& p, cudaStream_t st) {
+inline cudaError_t launch_fast(const Params& p, cudaStream_t st, bool early = true) {
     switch (p.C) {
-        case 32: return launch_fast_c<32>(p, st);
-        case 48: return launch_fast_c<48>(p, st);
-        case 64: return launch_fast_c<64>(p, st);
-        case 96: return launch_fast_c<96>(p, st);
-        case 128: return launch_fast_c<128>(p, st);
+        case 32: return launch_fast_c<32>(p, st, early);
+        case 48: return launch_fast_c<48>(p, st, early);
+        case 64: return launch_fast_c<64>(p, st, early);
+        case 96: return launch_fast_c<96>(p, st, early);
+        case 128: return launch_fast_c<128>(p, st, early);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -28,6 +28,7 @@
 #include "backward_pw.cuh"
 #include "backward_dense.cuh"
 #include "conv_fuse.cuh"
+#include "conv_fuse_backward.cuh"
 
 namespace {
 
@@ -755,6 +756,55 @@ int dense_add_const_t(const Problem& p, void* gx, const BackwardWs& w, cudaStrea
     return ESC_OK;
 }
 
+// ---- backward pass of Conv_fuse -------------------------------------------------------------------------------
+struct FuseBackwardWs {
+    void* wt;                        // W_fuse transposed, element type of the tensors
+    float* part;                     // [blocks][C * C + C]
+    int passes, blocks;
+    size_t bytes;
+};
+FuseBackwardWs carve_fuse_backward(void* ws, int C, long long pixels) {
+    FuseBackwardWs w;
+    const long long runs = (pixels + esc::fuse::bwd::kThreads - 1) / esc::fuse::bwd::kThreads, cap = 4LL * sms_or_nominal();
+    w.passes = (int)std::max(2LL, (runs + cap - 1) / cap);
+    w.blocks = (int)((runs + w.passes - 1) / w.passes);
+    char* base = static_cast<char*>(ws);
+    size_t off = 0;
+    w.wt = base + off;                              off += round_up((size_t)C * C * 4, 256);
+    w.part = reinterpret_cast<float*>(base + off);  off += round_up((size_t)w.blocks * ((size_t)C * C + C) * 4, 256);
+    w.bytes = off;
+    return w;
+}
+
+template <typename T, int LAYOUT, int C>
+int fuse_wgrad_c(const void* cat, const void* go, long long HW, long long pixels, const FuseBackwardWs& w, cudaStream_t st) {
+    using G = esc::fuse::bwd::Geom<C>;
+    if (G::kSmemBytes > 48 * 1024) {
+        static bool attr_set[esc::tma::kMaxDevices] = {};
+        const int dev = esc::tma::current_device();
+        if (dev < 0) return ESC_ERR_UNSUPPORTED;
+        if (!attr_set[dev]) {
+            ESC_CUDA(cudaFuncSetAttribute(esc::fuse::bwd::wgrad<T, LAYOUT, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)G::kSmemBytes));
+            attr_set[dev] = true;
+        }
+    }
+    esc::fuse::bwd::wgrad<T, LAYOUT, C><<<(unsigned)w.blocks, esc::fuse::bwd::kThreads, G::kSmemBytes, st>>>(
+        static_cast<const T*>(cat), static_cast<const T*>(go), HW, pixels, w.passes, w.part);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
+}
+template <typename T, int LAYOUT>
+int fuse_wgrad_t(int C, const void* cat, const void* go, long long HW, long long pixels, const FuseBackwardWs& w, cudaStream_t st) {
+    switch (C) {
+        case 16: return fuse_wgrad_c<T, LAYOUT, 16>(cat, go, HW, pixels, w, st);
+        case 32: return fuse_wgrad_c<T, LAYOUT, 32>(cat, go, HW, pixels, w, st);
+        case 48: return fuse_wgrad_c<T, LAYOUT, 48>(cat, go, HW, pixels, w, st);
+        case 64: return fuse_wgrad_c<T, LAYOUT, 64>(cat, go, HW, pixels, w, st);
+    }
+    return ESC_ERR_UNSUPPORTED;
+}
+
 // ---- fixed scratch for the entry point that must not allocate ------------------------------
 // Layout: [kStaticMaxImages arrival counters][kStaticMaxPartials partial sums].  The array lives in
 // the library's device image: every GPU that loads the library holds these 64 KiB until exit.
@@ -1325,6 +1375,89 @@ int esc_convattn_backward_variant(const void* x, const void* grad_out, int B, in
     return backward_entry(x, grad_out, B, C, C_a, H, W, K, w_large, est, grad_x, g, dtype, layout, workspace, workspace_bytes_, stream,
                           large_kernel == ESC_LK_DECOMPOSED ? w_point : nullptr,
                           large_kernel == ESC_LK_DECOMPOSED ? grad_w_point : nullptr, dense, dense ? grad_w_large : nullptr);
+}
+
+size_t esc_conv_fuse_backward_workspace_bytes(int B, int C, int H, int W) {
+    if (B <= 0 || H <= 0 || W <= 0 || !esc::fuse::bwd::supported(C)) return 0;
+    return carve_fuse_backward(nullptr, C, (long long)B * H * W).bytes;
+}
+
+int esc_conv_fuse_backward(const void* cat, const void* grad_out, int B, int C, int H, int W, const void* w_fuse,
+                           void* grad_cat, float* grad_w_fuse, float* grad_b_fuse, int dtype, int layout,
+                           void* workspace, size_t workspace_bytes_, void* stream) {
+    g_last_launches = 0;
+    const Problem p{B, C, C, H, W, 3, dtype, layout};
+    int rc = check_shape(p);
+    if (rc != ESC_OK) return rc;
+    if (!esc::fuse::bwd::supported(C)) return ESC_ERR_UNSUPPORTED;
+    if (!cat || !grad_out || !w_fuse || !grad_cat) return ESC_ERR_NULL;
+    rc = check_tensors(p, grad_out, grad_cat);
+    if (rc != ESC_OK) return rc;
+    if (!aligned(cat, 16) || !aligned(w_fuse, p.es())) return ESC_ERR_ALIGN;
+    {
+        const uintptr_t xa = reinterpret_cast<uintptr_t>(cat), oa = reinterpret_cast<uintptr_t>(grad_cat);
+        const size_t bytes = p.elems() * p.es();
+        if (xa < oa + bytes && oa < xa + bytes) return ESC_ERR_ALIAS;
+    }
+    for (const float* q : {grad_w_fuse, grad_b_fuse})
+        if (q && !aligned(q, 4)) return ESC_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256)) return ESC_ERR_WORKSPACE;
+    const long long HW = (long long)H * W, pixels = (long long)B * HW;
+    const FuseBackwardWs w = carve_fuse_backward(workspace, C, pixels);
+    if (workspace_bytes_ < w.bytes) return ESC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the weight's and the bias's gradients
+    if (grad_w_fuse || grad_b_fuse) {
+        if (dtype == ESC_F32)
+            rc = layout == ESC_NCHW ? fuse_wgrad_t<float, esc::kNCHW>(C, cat, grad_out, HW, pixels, w, st)
+                                    : fuse_wgrad_t<float, esc::kNHWC>(C, cat, grad_out, HW, pixels, w, st);
+        else
+            rc = layout == ESC_NCHW ? fuse_wgrad_t<__nv_bfloat16, esc::kNCHW>(C, cat, grad_out, HW, pixels, w, st)
+                                    : fuse_wgrad_t<__nv_bfloat16, esc::kNHWC>(C, cat, grad_out, HW, pixels, w, st);
+        if (rc != ESC_OK) return rc;
+        const int elems = C * C + C;
+        esc::fuse::bwd::sum_wgrad<<<(unsigned)((elems + 7) / 8), 256, 0, st>>>(w.part, C, w.blocks, grad_w_fuse, grad_b_fuse);
+        ESC_CUDA(cudaGetLastError());
+        ++g_last_launches;
+    }
+    // grad_cat = W_fuse^T grad_out per pixel: the forward's 1x1 kernels with the transposed matrix, no bias, no residual
+    const unsigned tb = (unsigned)((C * C + 255) / 256);
+    if (dtype == ESC_F32) esc::fuse::bwd::transpose_w<float><<<tb, 256, 0, st>>>(static_cast<const float*>(w_fuse), C, static_cast<float*>(w.wt));
+    else esc::fuse::bwd::transpose_w<__nv_bfloat16><<<tb, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(w_fuse), C, static_cast<__nv_bfloat16*>(w.wt));
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    if (esc::fuse::fast_applies(C, 8, dtype, layout)) {
+        esc::fuse::Params fp;
+        fp.att = static_cast<const __nv_bfloat16*>(grad_out); fp.idt = static_cast<const __nv_bfloat16*>(grad_out);
+        fp.w = static_cast<const __nv_bfloat16*>(w.wt); fp.bias = nullptr; fp.residual = nullptr;
+        fp.out = static_cast<__nv_bfloat16*>(grad_cat);
+        fp.pixels = pixels; fp.C = C; fp.Ca = 8;
+        ESC_CUDA(esc::fuse::launch_fast(fp, st, /*early=*/false));   // its matrix was written by the kernel before it
+        ++g_last_launches;
+        return ESC_OK;
+    }
+    if (esc::fuse::nchw::applies(C, 8, HW, dtype, layout, grad_out, grad_cat, nullptr, w.wt)) {
+        esc::fuse::nchw::Params fp;
+        fp.att = static_cast<const __nv_bfloat16*>(grad_out); fp.idt = static_cast<const __nv_bfloat16*>(grad_out);
+        fp.w = static_cast<const __nv_bfloat16*>(w.wt); fp.bias = nullptr; fp.residual = nullptr;
+        fp.out = static_cast<__nv_bfloat16*>(grad_cat);
+        fp.HW = HW; fp.B = B; fp.C = C; fp.Ca = 8;
+        ESC_CUDA(esc::fuse::nchw::launch(fp, st, /*early=*/false));
+        ++g_last_launches;
+        return ESC_OK;
+    }
+    // any type and layout: the generic kernel works in place on a copy of grad_out
+    ESC_CUDA(cudaMemcpyAsync(grad_cat, grad_out, p.elems() * p.es(), cudaMemcpyDeviceToDevice, st));
+    const size_t smem = (size_t)esc::fuse::kGenPix * C * sizeof(float);
+    const unsigned blocks = (unsigned)((pixels + esc::fuse::kGenPix - 1) / esc::fuse::kGenPix);
+#define ESC_FUSE_GENERIC(T, L) esc::fuse::conv_fuse_generic<T, L><<<blocks, esc::fuse::kGenThreads, smem, st>>>( \
+        static_cast<T*>(grad_cat), static_cast<const T*>(w.wt), static_cast<const T*>(nullptr), static_cast<const T*>(nullptr), B, C, H, W)
+    if (dtype == ESC_F32) { if (layout == ESC_NCHW) ESC_FUSE_GENERIC(float, esc::kNCHW); else ESC_FUSE_GENERIC(float, esc::kNHWC); }
+    else { if (layout == ESC_NCHW) ESC_FUSE_GENERIC(__nv_bfloat16, esc::kNCHW); else ESC_FUSE_GENERIC(__nv_bfloat16, esc::kNHWC); }
+#undef ESC_FUSE_GENERIC
+    ESC_CUDA(cudaGetLastError());
+    g_last_launches += 2;
+    return ESC_OK;
 }
 
 int esc_convattn_device_status(void* workspace, void* stream) {
