@@ -607,6 +607,15 @@ def main():
                 extras["backward"]["dense_large_kernel_ms_per_step"] = st["median_ms"]
                 extras["backward"]["dense_large_kernel_launches"] = pkg.esc_convattn_last_launches()
                 extras["backward"]["dense_large_kernel_frac_of_fp32_roofline_of_its_weight_gradient"] = t_fma_d / (st["median_ms"] * 1e-3)
+            if wl.C in (16, 32, 48, 64):
+                # the closing 1x1 convolution's backward (grad_cat, grad W_fuse, grad b_fuse): 2 x 2 x C x C flops per pixel
+                wfb = torch.from_numpy(synth.make_fuse(wl.C, wl.dtype, wl.seed)["w_fuse"]).to(tdt).cuda()
+                g_wf = torch.zeros(wl.C, wl.C, device="cuda")
+                g_bf = torch.zeros(wl.C, device="cuda")
+                fws = torch.empty(pkg.esc_conv_fuse_backward_workspace_bytes(wl.B, wl.C, wl.H, wl.W), dtype=torch.uint8, device="cuda")
+                st, _ = timer.measure(lambda i: pkg.esc_conv_fuse_backward(xs[i % n_rot], go_d, wfb, gx_d, g_wf, g_bf, lay_code, fws), samples=5)
+                extras["backward"]["conv_fuse_ms_per_step"] = st["median_ms"]
+                extras["backward"]["conv_fuse_launches"] = pkg.esc_convattn_last_launches()
         except Exception as exc:
             extras["backward"] = {"error": f"{type(exc).__name__}: {exc}"}
         # with the dense large kernel of the main model (Section 3.2): an implicit GEMM on the tensor cores

@@ -765,7 +765,8 @@ struct FuseBackwardWs {
 };
 FuseBackwardWs carve_fuse_backward(void* ws, int C, long long pixels) {
     FuseBackwardWs w;
-    const long long runs = (pixels + esc::fuse::bwd::kThreads - 1) / esc::fuse::bwd::kThreads, cap = 4LL * sms_or_nominal();
+    // one block per SM at most (both kernels fill an SM), each with a run of pixels long enough to pay for its final sums
+    const long long runs = (pixels + esc::fuse::bwd::kThreads - 1) / esc::fuse::bwd::kThreads, cap = sms_or_nominal();
     w.passes = (int)std::max(2LL, (runs + cap - 1) / cap);
     w.blocks = (int)((runs + w.passes - 1) / w.passes);
     char* base = static_cast<char*>(ws);
@@ -794,8 +795,33 @@ int fuse_wgrad_c(const void* cat, const void* go, long long HW, long long pixels
     ++g_last_launches;
     return ESC_OK;
 }
+template <int C>
+int fuse_wgrad_mma_c(const void* cat, const void* go, long long pixels, const FuseBackwardWs& w, cudaStream_t st) {
+    namespace M = esc::fuse::bwd::mma;
+    static bool attr_set[esc::tma::kMaxDevices] = {};
+    const int dev = esc::tma::current_device();
+    if (dev < 0) return ESC_ERR_UNSUPPORTED;
+    if (!attr_set[dev]) {
+        ESC_CUDA(cudaFuncSetAttribute(M::wgrad_bf16_nhwc<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::MGeom<C>::kSmemBytes));
+        attr_set[dev] = true;
+    }
+    M::wgrad_bf16_nhwc<C><<<(unsigned)w.blocks, esc::fuse::bwd::kThreads, M::MGeom<C>::kSmemBytes, st>>>(
+        static_cast<const __nv_bfloat16*>(cat), static_cast<const __nv_bfloat16*>(go), pixels, w.passes, w.part);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
+}
+
 template <typename T, int LAYOUT>
 int fuse_wgrad_t(int C, const void* cat, const void* go, long long HW, long long pixels, const FuseBackwardWs& w, cudaStream_t st) {
+    if (std::is_same<T, __nv_bfloat16>::value && LAYOUT == esc::kNHWC && g_engine_policy != ESC_ENGINE_FP32) {
+        // bf16 NHWC: one matrix product over the pixels on the tensor cores
+        switch (C) {
+            case 32: return fuse_wgrad_mma_c<32>(cat, go, pixels, w, st);
+            case 48: return fuse_wgrad_mma_c<48>(cat, go, pixels, w, st);
+            case 64: return fuse_wgrad_mma_c<64>(cat, go, pixels, w, st);
+        }
+    }
     switch (C) {
         case 16: return fuse_wgrad_c<T, LAYOUT, 16>(cat, go, HW, pixels, w, st);
         case 32: return fuse_wgrad_c<T, LAYOUT, 32>(cat, go, HW, pixels, w, st);
