@@ -147,6 +147,46 @@ def test_backward_entries_reject_on_the_host(L):
     assert bwd_mlp(wd=None) == 1 and bwd_mlp(gx=X) == 5 and bwd_mlp(K=15) == 3 and bwd_mlp(wsb=0) == 6
 
 
+def test_other_backward_entries_reject_on_the_host(L):
+    """The decomposed, dense, any-form and Conv_fuse backward entries: the same checks, before anything could be launched."""
+    X, GO, GX, Wl, Wp, Wa, Wb, Wc, Wd, WS = (0x10000000, 0x18000000, 0x20000000, 0x30000000, 0x30100000, 0x30200000, 0x30300000,
+                                             0x30400000, 0x30500000, 0x40000000)
+    for f in (L.esc_convattn_backward_workspace_bytes, L.esc_convattn_backward_dense_workspace_bytes, L.esc_conv_fuse_backward_workspace_bytes):
+        f.restype = ctypes.c_size_t
+    need = L.esc_convattn_backward_workspace_bytes(1, 16, 32, 32, 13)
+    need_d = L.esc_convattn_backward_dense_workspace_bytes(1, 16, 32, 32, 13)
+    assert need_d > need and need_d % 256 == 0
+    assert L.esc_convattn_backward_dense_workspace_bytes(1, 8, 32, 32, 13) == 0     # the dense kernel is 16 x 16 channels
+    assert L.esc_convattn_backward_dense_workspace_bytes(1, 16, 32, 32, 15) == 0
+
+    def pw(wp=Wp, Ca=16, C=64, gx=GX, wsb=need, K=13):
+        return L.esc_convattn_backward_pw(X, GO, 1, C, Ca, 32, 32, K, Wl, wp, Wa, Wb, gx, None, None, None, None, 1, 1, WS, wsb, None)
+
+    assert pw(wp=None) == 1 and pw(Ca=12, C=48) == 3 and pw(gx=GO) == 5 and pw(wsb=256) == 6 and pw(K=15) == 3
+
+    def dense(Ca=16, gx=GX, wsb=need_d, go=GO):
+        return L.esc_convattn_backward_dense(X, go, 1, 64, Ca, 32, 32, 13, Wl, Wa, Wb, gx, None, None, None, 1, 1, WS, wsb, None)
+
+    assert dense(Ca=8) == 3 and dense(gx=X) == 5 and dense(go=None) == 1
+    assert dense(wsb=need) == 6                                                     # the depth-wise workspace is too small for it
+
+    def variant(form, wp=Wp, hidden=8, wsb=need_d, wdown=Wc):
+        return L.esc_convattn_backward_variant(X, GO, 1, 64, 16, 32, 32, 13, form, Wl, wp, wdown, Wd, Wa, Wb, hidden, GX,
+                                               None, None, None, None, None, None, 1, 1, WS, wsb, None)
+
+    assert variant(7) == 3 and variant(1, wp=None) == 1 and variant(0, hidden=-1) == 2 and variant(0, hidden=200) == 2
+    assert variant(0, wdown=None) == 1 and variant(2, wsb=need) == 6 and variant(0, wsb=0) == 6
+
+    need_f = L.esc_conv_fuse_backward_workspace_bytes(1, 64, 32, 32)
+    assert need_f > 0 and need_f % 256 == 0 and L.esc_conv_fuse_backward_workspace_bytes(1, 40, 32, 32) == 0
+
+    def fuse(C=64, cat=X, go=GO, gc=GX, w=Wl, ws=WS, wsb=need_f):
+        return L.esc_conv_fuse_backward(cat, go, 1, C, 32, 32, w, gc, None, None, 1, 1, ws, wsb, None)
+
+    assert fuse(C=40) == 3 and fuse(cat=None) == 1 and fuse(w=None) == 1 and fuse(gc=GO) == 5 and fuse(gc=X) == 5
+    assert fuse(ws=None) == 6 and fuse(wsb=need_f - 256) == 6 and fuse(go=GO + 2) == 4
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     from paper_2503_06671_b200 import binding
 
