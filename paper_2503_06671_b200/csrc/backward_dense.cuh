@@ -16,6 +16,7 @@
 #include "common.cuh"
 #include "backward.cuh"
 #include "stencil_toeplitz.cuh"
+#include "conv_fuse.cuh"
 
 namespace esc { namespace bwd { namespace dense {
 
@@ -105,14 +106,17 @@ tap_grad_dense(const T* __restrict__ x, const T* __restrict__ go, int B, int C, 
 // conflicts).  Per 16 pixels of a go row a warp loads the A fragments once (ldmatrix.trans: channel x pixel from
 // pixel-major storage) and, for each of its taps, the B fragments of x at the shifted position the same way, then two
 // mma.sync.m16n8k16 (x channels 0-7, 8-15).  The 169 taps are dealt to the eight warps (22 or 21 each, 8 accumulator
-// registers per tap) and stay in registers across all tiles of the block.
+// registers per tap) and stay in registers across all tiles of the block.  NHWC tensors: the next tile is fetched with
+// cp.async into a second buffer while this one is multiplied.
 namespace mma {
 using tma::toep::ldsm_x4_trans; using tma::toep::mma_bf16;
 constexpr int kWarps = 8, kThreads = kWarps * 32;
 constexpr int kTapsPerWarp = (TAPS + kWarps - 1) / kWarps;          // 22
-constexpr int XHALF = XH * XW * 16;                                  // bytes per plane of eight channels
-constexpr int GHALF = TY * TX * 16;
-constexpr size_t kSmemBytes = 2 * (size_t)XHALF + 2 * (size_t)GHALF; // 55,808 bytes
+constexpr int TYM = 8, XHM = TYM + K - 1;                            // tiles of 32 x 8 pixels here: 920 of them at 640x360 balance better over 148 blocks than 460
+constexpr int XHALF = XHM * XW * 16;                                 // bytes per plane of eight channels
+constexpr int GHALF = TYM * TX * 16;
+constexpr int kBufBytes = 2 * XHALF + 2 * GHALF;                      // 36,352 bytes: one tile of x and of go
+constexpr size_t kSmemBytes = 2 * (size_t)kBufBytes;                 // two of them
 static_assert(TX % 16 == 0, "whole MMA pixel blocks per row");
 
 template <int LAYOUT>
@@ -120,14 +124,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 tap_grad_dense_bf16(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ go, int B, int C, int H, int W,
                     int tiles_x, int tiles_y, int vec, float* __restrict__ part)   // [gridDim.x][CA][CA][13][13]
 {
-    extern __shared__ __align__(128) unsigned char smb[];
-    unsigned char* xs = smb;                      // [2][XH][XW] x 16 bytes
-    unsigned char* gs = smb + 2 * XHALF;          // [2][TY][TX] x 16 bytes
+    extern __shared__ __align__(128) unsigned char smb[];          // two buffers of [x: 2 planes][go: 2 planes]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int mi = lane >> 3, mr = lane & 7;      // ldmatrix: lane -> (matrix, row)
     // matrix mi: pixels 8 * (mi >> 1) + mr of the 16, channel half mi & 1
-    const uint32_t x_lane = tma::smem_u32(xs) + (uint32_t)((mi & 1) * XHALF + ((mi >> 1) * 8 + mr) * 16);
-    const uint32_t g_lane = tma::smem_u32(gs) + (uint32_t)((mi & 1) * GHALF + ((mi >> 1) * 8 + mr) * 16);
+    const uint32_t sm0 = tma::smem_u32(smb);
+    const uint32_t x_lane = (uint32_t)((mi & 1) * XHALF + ((mi >> 1) * 8 + mr) * 16);
+    const uint32_t g_lane = (uint32_t)(2 * XHALF + (mi & 1) * GHALF + ((mi >> 1) * 8 + mr) * 16);
     uint32_t toff[kTapsPerWarp];                  // byte offset of tap warp + 8 s inside the x tile
 #pragma unroll
     for (int s = 0; s < kTapsPerWarp; ++s) {
@@ -142,56 +145,76 @@ tap_grad_dense_bf16(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
 #pragma unroll
             for (int v = 0; v < 4; ++v) acc[s][h][v] = 0.f;
     const long long items = (long long)B * tiles_x * tiles_y;
-    for (long long it = blockIdx.x; it < items; it += gridDim.x) {
+    const bool async = LAYOUT == kNHWC && vec != 0;               // a pixel's 16 channels are two aligned 16-byte words
+    // NHWC: the next tile is fetched with cp.async (zero fill outside the image) while this one is multiplied
+    auto stage_async = [&](long long it, int buf) {
         const int b = (int)(it / ((long long)tiles_x * tiles_y));
         const int tr = (int)(it % ((long long)tiles_x * tiles_y));
-        const int y0 = (tr / tiles_x) * TY, x0 = (tr % tiles_x) * TX;
-        __syncthreads();                                          // the previous tile is read
-        if (LAYOUT == kNHWC && vec) {
-            // a pixel's 16 channels are two 16-byte words
-            for (int e = tid; e < 2 * XH * XW; e += kThreads) {
-                const int h = e & 1, col = (e >> 1) % XW, r = (e >> 1) / XW;
-                const int gy = y0 + r - P, gxx = x0 + col - P;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (gy >= 0 && gy < H && gxx >= 0 && gxx < W)
-                    v = *reinterpret_cast<const uint4*>(x + (((size_t)b * H + gy) * W + gxx) * C + 8 * h);
-                *reinterpret_cast<uint4*>(xs + h * XHALF + (r * XW + col) * 16) = v;
-            }
-            for (int e = tid; e < 2 * TY * TX; e += kThreads) {
-                const int h = e & 1, col = (e >> 1) % TX, r = (e >> 1) / TX;
-                const int gy = y0 + r, gxx = x0 + col;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (gy < H && gxx < W) v = *reinterpret_cast<const uint4*>(go + (((size_t)b * H + gy) * W + gxx) * C + 8 * h);
-                *reinterpret_cast<uint4*>(gs + h * GHALF + (r * TX + col) * 16) = v;
-            }
-        } else {
-            const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
-            for (int e = tid; e < CA * XH * XW; e += kThreads) {
-                int c, r, col;
-                if (LAYOUT == kNHWC) { c = e % CA; col = (e / CA) % XW; r = e / (CA * XW); }
-                else { col = e % XW; r = (e / XW) % XH; c = e / (XW * XH); }
-                const int gy = y0 + r - P, gxx = x0 + col - P;
-                __nv_bfloat16 v = zero;
-                if (gy >= 0 && gy < H && gxx >= 0 && gxx < W) v = x[elem_index<LAYOUT>(b, c, gy, gxx, C, H, W)];
-                *reinterpret_cast<__nv_bfloat16*>(xs + (c >> 3) * XHALF + (r * XW + col) * 16 + (c & 7) * 2) = v;
-            }
-            for (int e = tid; e < CA * TY * TX; e += kThreads) {
-                int c, r, col;
-                if (LAYOUT == kNHWC) { c = e % CA; col = (e / CA) % TX; r = e / (CA * TX); }
-                else { col = e % TX; r = (e / TX) % TY; c = e / (TX * TY); }
-                const int gy = y0 + r, gxx = x0 + col;
-                __nv_bfloat16 v = zero;
-                if (gy < H && gxx < W) v = go[elem_index<LAYOUT>(b, c, gy, gxx, C, H, W)];
-                *reinterpret_cast<__nv_bfloat16*>(gs + (c >> 3) * GHALF + (r * TX + col) * 16 + (c & 7) * 2) = v;
-            }
+        const int y0 = (tr / tiles_x) * TYM, x0 = (tr % tiles_x) * TX;
+        const uint32_t xb = sm0 + (uint32_t)(buf * kBufBytes), gb = xb + 2 * XHALF;
+        for (int e = tid; e < 2 * XHM * XW; e += kThreads) {
+            const int h = e & 1, col = (e >> 1) % XW, r = (e >> 1) / XW;
+            const int gy = y0 + r - P, gxx = x0 + col - P;
+            const bool valid = gy >= 0 && gy < H && gxx >= 0 && gxx < W;
+            fuse::cp_async16(xb + (uint32_t)(h * XHALF + (r * XW + col) * 16),
+                             x + (valid ? (((size_t)b * H + gy) * W + gxx) * C + 8 * h : 0), valid);
         }
-        __syncthreads();
-        for (int y = 0; y < TY; ++y)
+        for (int e = tid; e < 2 * TYM * TX; e += kThreads) {
+            const int h = e & 1, col = (e >> 1) % TX, r = (e >> 1) / TX;
+            const int gy = y0 + r, gxx = x0 + col;
+            const bool valid = gy < H && gxx < W;
+            fuse::cp_async16(gb + (uint32_t)(h * GHALF + (r * TX + col) * 16),
+                             go + (valid ? (((size_t)b * H + gy) * W + gxx) * C + 8 * h : 0), valid);
+        }
+        fuse::cp_async_commit();
+    };
+    auto stage_sync = [&](long long it) {                         // any layout: element by element into buffer 0
+        const int b = (int)(it / ((long long)tiles_x * tiles_y));
+        const int tr = (int)(it % ((long long)tiles_x * tiles_y));
+        const int y0 = (tr / tiles_x) * TYM, x0 = (tr % tiles_x) * TX;
+        unsigned char* xs = smb;
+        unsigned char* gs = smb + 2 * XHALF;
+        const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+        for (int e = tid; e < CA * XHM * XW; e += kThreads) {
+            int c, r, col;
+            if (LAYOUT == kNHWC) { c = e % CA; col = (e / CA) % XW; r = e / (CA * XW); }
+            else { col = e % XW; r = (e / XW) % XHM; c = e / (XW * XHM); }
+            const int gy = y0 + r - P, gxx = x0 + col - P;
+            __nv_bfloat16 v = zero;
+            if (gy >= 0 && gy < H && gxx >= 0 && gxx < W) v = x[elem_index<LAYOUT>(b, c, gy, gxx, C, H, W)];
+            *reinterpret_cast<__nv_bfloat16*>(xs + (c >> 3) * XHALF + (r * XW + col) * 16 + (c & 7) * 2) = v;
+        }
+        for (int e = tid; e < CA * TYM * TX; e += kThreads) {
+            int c, r, col;
+            if (LAYOUT == kNHWC) { c = e % CA; col = (e / CA) % TX; r = e / (CA * TX); }
+            else { col = e % TX; r = (e / TX) % TYM; c = e / (TX * TYM); }
+            const int gy = y0 + r, gxx = x0 + col;
+            __nv_bfloat16 v = zero;
+            if (gy < H && gxx < W) v = go[elem_index<LAYOUT>(b, c, gy, gxx, C, H, W)];
+            *reinterpret_cast<__nv_bfloat16*>(gs + (c >> 3) * GHALF + (r * TX + col) * 16 + (c & 7) * 2) = v;
+        }
+    };
+    if (async && (long long)blockIdx.x < items) stage_async(blockIdx.x, 0);
+    int k = 0;
+    for (long long it = blockIdx.x; it < items; it += gridDim.x, ++k) {
+        const int buf = async ? (k & 1) : 0;
+        if (async) {
+            const long long nx = it + gridDim.x;
+            if (nx < items) stage_async(nx, buf ^ 1);
+            else fuse::cp_async_commit();
+            fuse::cp_async_wait<1>();
+        } else {
+            __syncthreads();                                      // the previous tile is read
+            stage_sync(it);
+        }
+        __syncthreads();                                          // the tile is there for every warp
+        const uint32_t base = sm0 + (uint32_t)(buf * kBufBytes);
+        for (int y = 0; y < TYM; ++y)
 #pragma unroll 1
             for (int xb = 0; xb < TX / 16; ++xb) {
                 uint32_t a[4];                                    // go: (channels 0-7 | 8-15) x (pixels 0-7 | 8-15)
-                ldsm_x4_trans(g_lane + (uint32_t)((y * TX + xb * 16) * 16), a);
-                const uint32_t xrow = x_lane + (uint32_t)((y * XW + xb * 16) * 16);
+                ldsm_x4_trans(base + g_lane + (uint32_t)((y * TX + xb * 16) * 16), a);
+                const uint32_t xrow = base + x_lane + (uint32_t)((y * XW + xb * 16) * 16);
 #pragma unroll
                 for (int s = 0; s < kTapsPerWarp; ++s) {
                     if (s < kTapsPerWarp - 1 || warp + kWarps * s < TAPS) {
@@ -202,7 +225,9 @@ tap_grad_dense_bf16(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __
                     }
                 }
             }
+        if (async) __syncthreads();                               // this buffer may be refilled
     }
+    if (async) fuse::cp_async_wait<0>();
     // acc[s][h]: [0], [1] = go channel g, x channels 8 h + 2t, + 1; [2], [3] = go channel g + 8
     const int g = lane >> 2, t = lane & 3;
     float* out = part + (size_t)blockIdx.x * kPartFloats;

@@ -726,8 +726,9 @@ int dense_tap_grad_t(const Problem& p, const void* x, const void* go, const void
                 attr_mma[dev] = true;
             }
             const int vec = LAYOUT == esc::kNHWC && p.C % 8 == 0 ? 1 : 0;
+            const int tiles_ym = (p.H + D::mma::TYM - 1) / D::mma::TYM;
             D::mma::tap_grad_dense_bf16<LAYOUT><<<(unsigned)w.dense_blocks, D::mma::kThreads, D::mma::kSmemBytes, st>>>(
-                static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(go), p.B, p.C, p.H, p.W, tiles_x, tiles_y, vec,
+                static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(go), p.B, p.C, p.H, p.W, tiles_x, tiles_ym, vec,
                 w.dense_part);
         } else {
             D::tap_grad_dense<T, LAYOUT><<<(unsigned)w.dense_blocks, D::kThreads, D::kSmemBytes, st>>>(
