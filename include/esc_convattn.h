@@ -373,6 +373,15 @@ int esc_conv_fuse_backward(const void* cat, const void* grad_out, int B, int C, 
                            void* grad_cat, float* grad_w_fuse, float* grad_b_fuse, int dtype, int layout,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Self-test of the error path that every device-side wait of this library shares: launches one thread that waits, with
+ * the kernels' own bounded wait, on a barrier that nothing signals.  The wait gives up after its poll limit (about one
+ * second), records ESC_DEV_TIMEOUT in the status word of `workspace` (any initialised forward or backward workspace, device)
+ * and the kernel returns normally: no trap, no fault, the context stays usable.  esc_convattn_device_status() then returns
+ * ESC_DEV_TIMEOUT once and clears the word.  Asynchronous on `stream`.
+ */
+int esc_convattn_selftest_bounded_wait(void* workspace, void* stream);
+
 /* Synchronises `stream`, returns the workspace status word (ESC_OK or ESC_DEV_TIMEOUT) and
  * clears it. */
 int esc_convattn_device_status(void* workspace, void* stream);

@@ -68,6 +68,7 @@ def lib():
         L.esc_convattn_stencil.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, i, i, vp, sz, vp]
         L.esc_convattn_forward_host.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
         L.esc_convattn_device_status.argtypes = [vp, vp]
+        L.esc_convattn_selftest_bounded_wait.argtypes = [vp, vp]
         L.esc_convattn_forward_host_submit.argtypes = [i, vp, i, i, i, i, i, i, vp, vp, vp, vp, i, i]
         L.esc_convattn_forward_host_wait.argtypes = [i]
         L.esc_convattn_set_tile_width.argtypes = [i]
@@ -403,6 +404,12 @@ def esc_conv_fuse_backward(cat, grad_out, w_fuse, grad_cat, grad_w_fuse, grad_b_
                                         workspace.numel() * workspace.element_size(), _stream(stream)),
            "esc_conv_fuse_backward")
     return grad_cat
+
+
+def esc_convattn_selftest_bounded_wait(workspace, stream=None):
+    """Runs the library's bounded device-side wait on a barrier nothing signals (about a second): afterwards
+    esc_convattn_device_status(workspace) returns 8 (ESC_DEV_TIMEOUT) once."""
+    _check(lib().esc_convattn_selftest_bounded_wait(_ptr(workspace), _stream(stream)), "esc_convattn_selftest_bounded_wait")
 
 
 def esc_convattn_forward_variant(x, C_a, K, large_kernel, w_large, w_point, w_down, b_down, w_up, b_up, out, layout,

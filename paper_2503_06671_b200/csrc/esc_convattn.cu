@@ -832,6 +832,19 @@ int fuse_wgrad_t(int C, const void* cat, const void* go, long long HW, long long
     return ESC_ERR_UNSUPPORTED;
 }
 
+// ---- the bounded wait, run on purpose -----------------------------------------------------------------------
+// One thread waits, with the kernels' own bounded wait, on a barrier that nothing signals: the wait gives up after its
+// poll limit (about a second), records the status and the kernel returns normally.
+__global__ void bounded_wait_probe(unsigned* ctrl) {
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        const uint32_t b = esc::tma::smem_u32(&bar);
+        esc::tma::mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        esc::tma::mbar_wait(b, 0, ctrl, 0x5E1F0000u);
+    }
+}
+
 // ---- fixed scratch for the entry point that must not allocate ------------------------------
 // Layout: [kStaticMaxImages arrival counters][kStaticMaxPartials partial sums].  The array lives in
 // the library's device image: every GPU that loads the library holds these 64 KiB until exit.
@@ -1484,6 +1497,13 @@ int esc_conv_fuse_backward(const void* cat, const void* grad_out, int B, int C, 
 #undef ESC_FUSE_GENERIC
     ESC_CUDA(cudaGetLastError());
     g_last_launches += 2;
+    return ESC_OK;
+}
+
+int esc_convattn_selftest_bounded_wait(void* workspace, void* stream) {
+    if (!workspace || !aligned(workspace, 256)) return ESC_ERR_WORKSPACE;
+    bounded_wait_probe<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<unsigned*>(workspace));
+    ESC_CUDA(cudaGetLastError());
     return ESC_OK;
 }
 
