@@ -267,6 +267,109 @@ wgrad_bf16_nhwc(const __nv_bfloat16* __restrict__ cat, const __nv_bfloat16* __re
         out[e] = v;
     }
 }
+
+// The same for bf16 NCHW tensors (H W a multiple of 8, so that eight consecutive pixels of the flattened list lie in one
+// image): rows of a staged tile are channels, 128 pixels long plus 16 bytes; both operands are then the instruction's
+// native arrangement (A row-major channel x pixel, B pixel-contiguous per channel): ldmatrix without transposition.
+template <int C> struct NGeom {
+    static constexpr int PITCH = kPiece * 2 + 16;                  // bytes per staged channel row
+    static constexpr int TILE = C * PITCH;
+    static constexpr size_t kStageBytes = (size_t)4 * TILE;
+    static constexpr size_t kSmemBytes = kStageBytes > MGeom<C>::kSumBytes ? kStageBytes : MGeom<C>::kSumBytes;
+};
+
+template <int C>
+__global__ void __launch_bounds__(kThreads, 1)
+wgrad_bf16_nchw(const __nv_bfloat16* __restrict__ cat, const __nv_bfloat16* __restrict__ go, long long HW, long long pixels,
+                int passes, float* __restrict__ part)              // [gridDim.x][C * C + C]
+{
+    using G = NGeom<C>;
+    constexpr int MT = C / 16, NT = C / 8;
+    extern __shared__ __align__(128) unsigned char smb[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int mi = lane >> 3, mr = lane & 7;
+    // ldmatrix lane address inside a tile: channel 8 (mi & 1) + mr of a 16-channel group, pixels 16 warp + 8 (mi >> 1) ..
+    const uint32_t lane_off = (uint32_t)((8 * (mi & 1) + mr) * G::PITCH + (16 * warp + 8 * (mi >> 1)) * 2);
+    const uint32_t sm0 = tma::smem_u32(smb);
+    float acc[MT][NT][4], accb[MT][4];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[m][n][v] = 0.f;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) accb[m][v] = 0.f;
+    }
+    const long long first = (long long)blockIdx.x * passes * kThreads;
+    const long long last = first + (long long)passes * kThreads < pixels ? first + (long long)passes * kThreads : pixels;
+    const int pieces = first < last ? (int)((last - first + kPiece - 1) / kPiece) : 0;
+    auto stage = [&](int s) {
+        const long long p0 = first + (long long)s * kPiece;
+        const uint32_t gbuf = sm0 + (uint32_t)((s & 1) * 2 * G::TILE), cbuf = gbuf + G::TILE;
+        for (int e = tid; e < C * (kPiece / 8); e += kThreads) {
+            const int c = e / (kPiece / 8), q = e % (kPiece / 8);
+            const long long px = p0 + q * 8;
+            const bool valid = px < last;                          // pieces of eight pixels never straddle `last` or an image
+            const long long b = valid ? px / HW : 0, r = valid ? px - b * HW : 0;
+            const size_t src = ((size_t)b * C + c) * HW + r;
+            fuse::cp_async16(gbuf + (uint32_t)(c * G::PITCH + q * 16), go + src, valid);
+            fuse::cp_async16(cbuf + (uint32_t)(c * G::PITCH + q * 16), cat + src, valid);
+        }
+        fuse::cp_async_commit();
+    };
+    if (pieces > 0) stage(0);
+    for (int s = 0; s < pieces; ++s) {
+        if (s + 1 < pieces) stage(s + 1);
+        else fuse::cp_async_commit();
+        fuse::cp_async_wait<1>();
+        __syncthreads();
+        const uint32_t gbuf = sm0 + (uint32_t)((s & 1) * 2 * G::TILE) + lane_off, cbuf = gbuf + G::TILE;
+        uint32_t a[MT][4];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            tma::toep::ldsm_x4(gbuf + (uint32_t)(m * 16 * G::PITCH), a[m]);   // go: (channels 0-7 | 8-15 of group m) x (pixels 0-7 | 8-15)
+            mma_bf16(accb[m], a[m][0], a[m][1], a[m][2], a[m][3], 0x3F803F80u, 0x3F803F80u);
+        }
+#pragma unroll
+        for (int n2 = 0; n2 < MT; ++n2) {
+            uint32_t b[4];
+            tma::toep::ldsm_x4(cbuf + (uint32_t)(n2 * 16 * G::PITCH), b);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                mma_bf16(acc[m][2 * n2], a[m][0], a[m][1], a[m][2], a[m][3], b[0], b[2]);
+                mma_bf16(acc[m][2 * n2 + 1], a[m][0], a[m][1], a[m][2], a[m][3], b[1], b[3]);
+            }
+        }
+        __syncthreads();
+    }
+    fuse::cp_async_wait<0>();
+    __syncthreads();
+    constexpr int kPart = C * C + C;
+    float* sum = reinterpret_cast<float*>(smb) + warp * kPart;
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int v = 0; v < 4; v += 2)
+                *reinterpret_cast<float2*>(sum + (16 * m + g + 8 * (v >> 1)) * C + 8 * n + 2 * t) = make_float2(acc[m][n][v], acc[m][n][v + 1]);
+        if (t == 0) {
+            sum[C * C + 16 * m + g] = accb[m][0];
+            sum[C * C + 16 * m + g + 8] = accb[m][2];
+        }
+    }
+    __syncthreads();
+    const float* all = reinterpret_cast<const float*>(smb);
+    float* out = part + (size_t)blockIdx.x * kPart;
+    for (int e = tid; e < kPart; e += kThreads) {
+        float v = all[e];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) v += all[w * kPart + e];
+        out[e] = v;
+    }
+}
 }  // namespace mma
 
 // g_W [C*C] and g_b [C]: a warp per element, lanes over blocks in order, fixed butterfly.

@@ -813,8 +813,33 @@ int fuse_wgrad_mma_c(const void* cat, const void* go, long long pixels, const Fu
     return ESC_OK;
 }
 
+template <int C>
+int fuse_wgrad_mma_nchw_c(const void* cat, const void* go, long long HW, long long pixels, const FuseBackwardWs& w, cudaStream_t st) {
+    namespace M = esc::fuse::bwd::mma;
+    static bool attr_set[esc::tma::kMaxDevices] = {};
+    const int dev = esc::tma::current_device();
+    if (dev < 0) return ESC_ERR_UNSUPPORTED;
+    if (!attr_set[dev]) {
+        ESC_CUDA(cudaFuncSetAttribute(M::wgrad_bf16_nchw<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)M::NGeom<C>::kSmemBytes));
+        attr_set[dev] = true;
+    }
+    M::wgrad_bf16_nchw<C><<<(unsigned)w.blocks, esc::fuse::bwd::kThreads, M::NGeom<C>::kSmemBytes, st>>>(
+        static_cast<const __nv_bfloat16*>(cat), static_cast<const __nv_bfloat16*>(go), HW, pixels, w.passes, w.part);
+    ESC_CUDA(cudaGetLastError());
+    ++g_last_launches;
+    return ESC_OK;
+}
+
 template <typename T, int LAYOUT>
 int fuse_wgrad_t(int C, const void* cat, const void* go, long long HW, long long pixels, const FuseBackwardWs& w, cudaStream_t st) {
+    if (std::is_same<T, __nv_bfloat16>::value && LAYOUT == esc::kNCHW && HW % 8 == 0 && g_engine_policy != ESC_ENGINE_FP32) {
+        // bf16 NCHW with whole 16-byte pieces per image: the same matrix product, operands without transposition
+        switch (C) {
+            case 32: return fuse_wgrad_mma_nchw_c<32>(cat, go, HW, pixels, w, st);
+            case 48: return fuse_wgrad_mma_nchw_c<48>(cat, go, HW, pixels, w, st);
+            case 64: return fuse_wgrad_mma_nchw_c<64>(cat, go, HW, pixels, w, st);
+        }
+    }
     if (std::is_same<T, __nv_bfloat16>::value && LAYOUT == esc::kNHWC && g_engine_policy != ESC_ENGINE_FP32) {
         // bf16 NHWC: one matrix product over the pixels on the tensor cores
         switch (C) {
