@@ -163,3 +163,25 @@ def test_backward_rejections(pkg):
     rc = L.esc_convattn_backward(x.data_ptr(), x.data_ptr(), 1, 16, 16, 8, 8, 15, w.data_ptr(), w.data_ptr(), w.data_ptr(),
                                  x.data_ptr(), None, None, None, 1, 1, ws.data_ptr(), ws.numel(), None)
     assert rc == 3
+
+@pytest.mark.parametrize("layout", LAYOUTS)
+def test_backward_full_size_640x360(pkg, oracle, layout):
+    """The size bench.py times (1 x 64 x 360 x 640, C_a = 16, K = 13, bf16), every gradient element against the oracle:
+    230 units of 64x16 on 148 SMs for the tap gradients and the stencil pass."""
+    B, C, C_a, H, W, K = 1, 64, 16, 360, 640, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=640360, per_image_scale=True, channel_means=True)
+    go = synth.round_to(np.random.default_rng(640361).standard_normal(size=d["x"].shape).astype(np.float32), synth.BF16)
+    gx, g_lk, g_w, g_b = _run_backward(pkg, d, go, C_a, K, synth.BF16, layout)
+    rx, rlk, rw, rb = oracle.backward(d["x"], go, C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    _, alk, aw, ab = oracle.backward(np.abs(d["x"]), np.abs(go), C_a, d["w_large"], d["w_dyn"], d["b_dyn"])
+    for name, got, ref, scale in (("w_large", g_lk, rlk, alk), ("w_dyn", g_w, rw, aw), ("b_dyn", g_b, rb, ab)):
+        err = np.abs(got.cpu().numpy().astype(np.float64) - ref)
+        assert (err <= 1e-5 * scale + 1e-30).all(), f"grad {name}: worst {(err / np.maximum(scale, 1e-30)).max():.3e} of its scale"
+    got = util.to_host_nchw(gx, layout)
+    assert np.array_equal(got[:, C_a:], go[:, C_a:].astype(np.float64))
+    dk = oracle.dynkernel(oracle.gap(d["x"], C_a), d["w_dyn"], d["b_dyn"])
+    mag = oracle.stencil(np.abs(go), C_a, np.abs(d["w_large"][:, ::-1, ::-1]).copy(), np.abs(dk[:, :, ::-1, ::-1]).copy())[:, :C_a]
+    gg_scale = np.abs(np.einsum("ok,bo->bk", np.abs(d["w_dyn"].astype(np.float64)), np.abs(ab.reshape(1, -1)).repeat(B, 0))) / (H * W)
+    err = np.abs(got[:, :C_a] - rx[:, :C_a])
+    bar = 1e-5 * mag + 1e-5 * gg_scale[:, :, None, None] + 2.0 ** -8 * np.abs(rx[:, :C_a]) * 1.001 + 1e-30
+    assert (err <= bar).all(), f"grad x: {int((err > bar).sum())} values beyond the bound"
