@@ -165,3 +165,13 @@ def test_backward_pw_rejections(pkg):
     with pytest.raises(pkg.EscError) as e:
         pkg.esc_convattn_backward_pw(x, x.clone(), C_a, K, wl, wp, wd, bd, gx, None, None, None, None, util.layout_code(synth.NHWC), ws)
     assert e.value.status == 3
+
+def test_backward_pw_full_size_640x360(pkg, oracle):
+    """The size bench.py times (1 x 64 x 360 x 640, C_a = 16, K = 13, bf16 NHWC): 450 chunks of pixels per per-pixel kernel."""
+    shape = (1, 64, 16, 360, 640, 13)
+    B, C, C_a, H, W, K = shape
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=640360, per_image_scale=True, channel_means=True)
+    wp = synth.make_pointwise(C_a, synth.BF16, seed=640360)
+    go = synth.round_to(np.random.default_rng(640361).standard_normal(size=d["x"].shape).astype(np.float32), synth.BF16)
+    gx, g = _run(pkg, d, wp, go, C_a, K, synth.BF16, synth.NHWC)
+    _check(oracle, d, wp, go, C_a, synth.BF16, gx, g)

@@ -36,6 +36,7 @@ SHAPES = [
     (3, 32, 9, 11),       # less than one pass of pixels per image; runs cross images
     (1, 16, 20, 24),      # the narrow case: 16 tiles x 16 slices
     (1, 64, 130, 200),    # several passes per block
+    (1, 64, 360, 640),    # the size bench.py times: seven runs of 256 pixels per block, 129 blocks
 ]
 
 
