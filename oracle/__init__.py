@@ -15,6 +15,7 @@ from .convattn_oracle import (  # noqa: F401
     backward_mlp,
     backward_pw,
     backward_dense,
+    backward_dense_points,
     backward_variant,
     stencil_dense,
     forward_dense,

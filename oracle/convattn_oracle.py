@@ -292,6 +292,22 @@ def backward_dense(x, grad_out, C_a, w_dense, w_dyn, b_dyn):
     return gx, gwd, gw, gb
 
 
+def backward_dense_points(x, grad_out, C_a, K, idx):
+    """Selected entries of the dense kernel's gradient (flat indices into [C_a,C_a,K,K]): returns (values, magnitudes)."""
+    x, xp = _f32(x)
+    go, gp = _f32(grad_out)
+    assert go.shape == x.shape
+    B, C, H, W = _dims(x, C_a, K)
+    idx = np.ascontiguousarray(idx, dtype=np.int64)
+    assert idx.ndim == 1 and (idx >= 0).all() and (idx < C_a * C_a * K * K).all()
+    vals = np.empty(idx.shape, dtype=np.float64)
+    mags = np.empty(idx.shape, dtype=np.float64)
+    _load().convattn_ref_backward_dense_points(xp, gp, B, C, C_a, H, W, K, ctypes.c_int64(idx.size),
+                                               idx.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)),
+                                               vals.ctypes.data_as(_f64p), mags.ctypes.data_as(_f64p))
+    return vals, mags
+
+
 def backward_variant(x, grad_out, C_a, large_kernel, w_large, w_point, w_down, b_down, w_up, b_up):
     """Gradients of a forward with any large-kernel form ("depthwise", "pw", "dense") and the two-layer estimator of
     Eq. 4 line 2, by the chain rule in two steps.  (1) Per image, with the generator frozen at that image's dk

@@ -877,6 +877,36 @@ void convattn_ref_backward_dense(const float *x, const float *go, int B, int C, 
     free(g); free(dk); free(gdk); free(gg);
 }
 
+/* Selected entries of the dense kernel's gradient, one by one (for sizes where the whole of convattn_ref_backward_dense
+ * takes too long): idx[t] is a flat index into g_wd[C_a,C_a,K,K];
+ *   vals[t] = sum_{b,y,x} go[b,n,y,x] * x~[b,k,y+i-P,x+j-P],   mags[t] (optional) the same sum of magnitudes. */
+void convattn_ref_backward_dense_points(const float *x, const float *go, int B, int C, int C_a, int H, int W, int K,
+                                        int64_t n_idx, const int64_t *idx, double *vals, double *mags)
+{
+    const int P = (K - 1) / 2;
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t t = 0; t < n_idx; ++t) {
+        int64_t f = idx[t];
+        int j = (int)(f % K); f /= K;
+        int i = (int)(f % K); f /= K;
+        int k = (int)(f % C_a); f /= C_a;
+        int n = (int)f;
+        double s = 0.0, m = 0.0;
+        for (int b = 0; b < B; ++b)
+            for (int y = 0; y < H; ++y)
+                for (int xx = 0; xx < W; ++xx) {
+                    int yy = y + i - P, xc = xx + j - P;
+                    if (yy >= 0 && yy < H && xc >= 0 && xc < W) {
+                        double v = (double)go[IDX4(b, n, y, xx, C, H, W)] * (double)x[IDX4(b, k, yy, xc, C, H, W)];
+                        s += v;
+                        m += fabs(v);
+                    }
+                }
+        vals[t] = s;
+        if (mags) mags[t] = m;
+    }
+}
+
 /* Selected outputs, one by one: idx[n] are flat indices into out[B,C,H,W]; dk is
  * given (from convattn_ref_gap + convattn_ref_dynkernel). */
 void convattn_ref_points(const float *x, int B, int C, int C_a, int H, int W, int K,

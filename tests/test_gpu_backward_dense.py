@@ -171,3 +171,20 @@ def test_backward_dense_rejections(pkg):
     with pytest.raises(pkg.EscError) as e:
         pkg.esc_convattn_backward_dense(x, x.clone(), C_a, K, wdn, wd, bd, gx, None, None, None, util.layout_code(synth.NHWC), ws)
     assert e.value.status == 6
+
+def test_backward_dense_weight_gradient_full_size_640x360(pkg, oracle):
+    """The size bench.py times (1 x 64 x 360 x 640, C_a = 16, K = 13, bf16 NHWC; 920 tiles on one block per SM): 400 sampled
+    entries of the 43,264 of the kernel's gradient against the oracle, entry by entry."""
+    B, C, C_a, H, W, K = 1, 64, 16, 360, 640, 13
+    d = synth.make_inputs(B, C, C_a, H, W, K, synth.BF16, seed=640360, per_image_scale=True, channel_means=True)
+    wdn = synth.make_dense_kernel(C_a, K, synth.BF16, seed=640360)
+    go = synth.round_to(np.random.default_rng(640361).standard_normal(size=d["x"].shape).astype(np.float32), synth.BF16)
+    _, g = _run(pkg, d, wdn, go, C_a, K, synth.BF16, synth.NHWC)
+    rng = np.random.default_rng(5)
+    idx = np.unique(np.concatenate([rng.integers(0, C_a * C_a * K * K, size=392),
+                                    np.array([0, K * K - 1, C_a * C_a * K * K - 1, (5 * C_a + 5) * K * K + 84,   # corners, a centre tap
+                                              (0 * C_a + 15) * K * K + 12, (15 * C_a + 0) * K * K + 156])]))
+    vals, mags = oracle.backward_dense_points(d["x"], go, C_a, K, idx)
+    got = g["w_dense"].reshape(-1)[idx]
+    err = np.abs(got - vals)
+    assert (err <= 1e-5 * mags + 1e-30).all(), f"grad w_dense: worst {(err / np.maximum(mags, 1e-30)).max():.3e} of its scale"

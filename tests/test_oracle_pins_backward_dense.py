@@ -110,3 +110,15 @@ def test_planted_channel_swap_is_caught(oracle):
     wrong = oracle.backward_dense(d["x"], d["go"], 3, d["w_dense"].transpose(1, 0, 2, 3).copy(), d["w_dyn"], d["b_dyn"])[0]
     assert float(np.sum(g["x"] * u)) == pytest.approx(numx, rel=1e-10, abs=1e-9)
     assert abs(float(np.sum(wrong * u)) - numx) > 1e-3 * abs(numx)
+
+
+def test_points_equal_the_pinned_whole_gradient(oracle):
+    """backward_dense_points (used where the whole gradient takes too long) must return the entries of the pinned
+    backward_dense, every one of them, and magnitudes that bound them."""
+    d, rng = _case(B=2, C=5, C_a=3, H=7, W=9, K=5, seed=52)
+    g = _grads(oracle, d)
+    n = g["w_dense"].size
+    vals, mags = oracle.backward_dense_points(d["x"], d["go"], 3, 5, np.arange(n))
+    np.testing.assert_allclose(vals, g["w_dense"].reshape(-1), rtol=1e-13, atol=1e-13)
+    assert (mags >= np.abs(vals) - 1e-12).all()
+
