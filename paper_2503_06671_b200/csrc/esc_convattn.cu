@@ -911,7 +911,7 @@ HostPath g_host[kHostSlots];
 
 extern "C" {
 
-int esc_version(void) { return 111; }
+int esc_version(void) { return 120; }
 
 const char* esc_last_error(void) { return g_last_error.c_str(); }
 
